@@ -1,0 +1,129 @@
+"""fp64 CPU oracle for the DiG token-mixer hot path.  TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes loader around ``dig_oracle.c`` (plain C, fp64, token-by-token).  Only the test
+suite, the smoke check and the benchmark's CPU-baseline leg may import this package; the
+product path never does.  Nothing here shares code with the CUDA library.
+
+All tensors are numpy float64, C-contiguous, layout ``[B, L, H, d]`` with ``L = grid_h*grid_w``
+in canonical row-major token order.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dig_oracle.c")
+_LIB = os.path.join(_HERE, "libdig_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+ROW_FWD, ROW_REV, COL_FWD, COL_REV = 0, 1, 2, 3
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP over (batch, head) pairs only)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fPIC", "-shared", "-fopenmp", "-std=c11",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            build()
+            lib = ctypes.CDLL(_LIB)
+            dp = ctypes.POINTER(ctypes.c_double)
+            lib.dig_oracle_perm.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                            ctypes.POINTER(ctypes.c_longlong)]
+            lib.dig_oracle_gate.argtypes = [dp, dp, dp, ctypes.c_longlong, ctypes.c_longlong,
+                                            ctypes.c_int, ctypes.c_int]
+            lib.dig_oracle_gla_fwd.argtypes = [dp] * 5 + [ctypes.c_int] * 8
+            lib.dig_oracle_gla_bwd.argtypes = [dp] * 9 + [ctypes.c_int] * 8
+            lib.dig_oracle_dwconv.argtypes = [dp] * 4 + [ctypes.c_int] * 5
+            _lib = lib
+    return _lib
+
+
+def _f64(x):
+    return np.ascontiguousarray(np.asarray(x, dtype=np.float64))
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise RuntimeError(f"oracle {what} failed with code {rc}")
+
+
+def perm(direction: int, grid_h: int, grid_w: int) -> np.ndarray:
+    """perm[p] = canonical token (y*grid_w + x) visited at scan position p."""
+    out = np.empty(grid_h * grid_w, dtype=np.int64)
+    rc = _load().dig_oracle_perm(direction, grid_h, grid_w,
+                                 out.ctypes.data_as(ctypes.POINTER(ctypes.c_longlong)))
+    _check(rc, "perm")
+    return out
+
+
+def gate(x, tau_per_head) -> np.ndarray:
+    """a = logsigmoid(x) / tau[h]  (log of Eq. gate_gla's alpha).  x: [B, L, H, d_k]."""
+    x = _f64(x)
+    B, L, H, dk = x.shape
+    tau = _f64(tau_per_head)
+    assert tau.shape == (H,)
+    out = np.empty_like(x)
+    _check(_load().dig_oracle_gate(_p(x), _p(tau), _p(out), B, L, H, dk), "gate")
+    return out
+
+
+def gla_fwd(q, k, v, a, grid_h, grid_w, direction=ROW_FWD, threads=1) -> np.ndarray:
+    """o_t = q_t S_t with S_t = diag(exp(a_t)) S_{t-1} + k_t^T v_t, scanned in `direction`."""
+    q, k, v, a = map(_f64, (q, k, v, a))
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    assert L == grid_h * grid_w and k.shape == q.shape == a.shape and v.shape == (B, L, H, dv)
+    out = np.empty_like(v)
+    _check(_load().dig_oracle_gla_fwd(_p(q), _p(k), _p(v), _p(a), _p(out), B, H, grid_h, grid_w,
+                                      dk, dv, direction, threads), "gla_fwd")
+    return out
+
+
+def gla_bwd(q, k, v, a, dout, grid_h, grid_w, direction=ROW_FWD, threads=1):
+    """Gradients (dq, dk, dv, da) of <dout, gla_fwd(q,k,v,a)>."""
+    q, k, v, a, dout = map(_f64, (q, k, v, a, dout))
+    B, L, H, dk = q.shape
+    dv_ = v.shape[-1]
+    assert L == grid_h * grid_w and dout.shape == v.shape
+    dq, dk_, da = np.empty_like(q), np.empty_like(q), np.empty_like(q)
+    dv = np.empty_like(v)
+    _check(_load().dig_oracle_gla_bwd(_p(q), _p(k), _p(v), _p(a), _p(dout), _p(dq), _p(dk_),
+                                      _p(dv), _p(da), B, H, grid_h, grid_w, dk, dv_, direction,
+                                      threads), "gla_bwd")
+    return dq, dk_, dv, da
+
+
+def dwconv(x, w, bias, grid_h, grid_w, direction=ROW_FWD) -> np.ndarray:
+    """3x3 depthwise conv of the SREM module on the re-oriented token matrix.
+    x: [B, L, D] canonical order, w: [3, 3, D], bias: [D] or None."""
+    x, w = _f64(x), _f64(w)
+    B, L, D = x.shape
+    assert L == grid_h * grid_w and w.shape == (3, 3, D)
+    bp = None
+    if bias is not None:
+        bias = _f64(bias)
+        assert bias.shape == (D,)
+        bp = _p(bias)
+    y = np.empty_like(x)
+    _check(_load().dig_oracle_dwconv(_p(x), _p(w), bp, _p(y), B, grid_h, grid_w, D, direction),
+           "dwconv")
+    return y

@@ -1,0 +1,279 @@
+/*
+ * fp64 CPU oracle for the DiG token-mixer hot path (arxiv 2405.18428).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+ * CUDA library is checked against.  It shares no code, header, table or helper
+ * with the CUDA path, and the product never calls it.
+ *
+ * What is written out here
+ *   - gate transform        alpha = sigmoid(x)^(1/tau), kept as a = log(alpha)      (Eq. gate_gla)
+ *   - GLA recurrence        S_t = diag(alpha_t) S_{t-1} + k_t^T v_t,  o_t = q_t S_t (Eq. attn_gla,
+ *                           with the value-channel gate beta fixed to 1)
+ *   - its reverse-mode derivative (not printed in the paper; derived from Eq. attn_gla)
+ *   - the four scan orders of the block-by-block scanning scheme (Algorithm 1 / Algorithm 4:
+ *     flip and transpose of the reshaped token matrix), materialised as index arrays
+ *   - the 3x3 depthwise convolution of the SREM module (Algorithm 1, "DWConv2d(reshape2d(z))"),
+ *     evaluated on the re-oriented token matrix by explicit gather / conv / scatter
+ *
+ * Everything is token-by-token and element-by-element: no chunking, no blocking, no fused forms.
+ * Tensors are dense row-major doubles with layout [B][L][H][d]; L = grid_h*grid_w and the
+ * canonical token index is y*grid_w + x.
+ *
+ * Pins (tests/test_oracle_*.py): brute-force parallel form, reduction to causal linear
+ * attention (Eq. attn_simple) when alpha == 1, constant-decay closed form, fast-decay limit,
+ * permutation bijectivity and the four-block cycle, central finite differences for the
+ * backward pass, the suffix-sum gate-gradient identity, identity-initialised convolution,
+ * convolution against hand-evaluated corner / edge / interior counts.
+ * Not pinned by the paper: whether DWConv2d carries a bias (the argument is optional).
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* direction codes: 0 row-major forward, 1 row-major reverse, 2 column-major forward,
+ * 3 column-major reverse */
+
+/* perm[p] = canonical token visited at scan position p.
+ * Built the way Algorithm 1 builds the orders: start from the row-major sequence; "flip"
+ * reverses a sequence; "transpose" reshapes to 2-D, transposes and flattens. */
+int dig_oracle_perm(int direction, int grid_h, int grid_w, long long *perm)
+{
+    const long long L = (long long)grid_h * grid_w;
+    if (direction < 0 || direction > 3 || grid_h <= 0 || grid_w <= 0) return 1;
+    long long *seq = (long long *)malloc(sizeof(long long) * (size_t)L);
+    if (!seq) return 2;
+    for (long long t = 0; t < L; ++t) seq[t] = t;           /* row-major forward */
+    if (direction == 2 || direction == 3) {
+        /* transpose(reshape2d(seq)): new matrix has grid_w rows and grid_h columns */
+        for (int x = 0; x < grid_w; ++x)
+            for (int y = 0; y < grid_h; ++y)
+                perm[(long long)x * grid_h + y] = seq[(long long)y * grid_w + x];
+        memcpy(seq, perm, sizeof(long long) * (size_t)L);
+    }
+    if (direction == 1 || direction == 3) {
+        for (long long p = 0; p < L; ++p) perm[p] = seq[L - 1 - p];  /* flip */
+    } else {
+        memcpy(perm, seq, sizeof(long long) * (size_t)L);
+    }
+    free(seq);
+    return 0;
+}
+
+/* a = log(sigmoid(x)^(1/tau)) = logsigmoid(x)/tau, per head temperature.  (Eq. gate_gla) */
+int dig_oracle_gate(const double *x, const double *tau_per_head, double *a,
+                    long long B, long long L, int H, int d_k)
+{
+    for (long long bl = 0; bl < B * L; ++bl)
+        for (int h = 0; h < H; ++h)
+            for (int c = 0; c < d_k; ++c) {
+                const size_t i = ((size_t)bl * H + h) * d_k + c;
+                const double z = x[i];
+                /* log(1/(1+e^-z)), written so that neither branch overflows */
+                const double ls = (z >= 0.0) ? -log1p(exp(-z)) : z - log1p(exp(z));
+                a[i] = ls / tau_per_head[h];
+            }
+    return 0;
+}
+
+static size_t tok_off(long long b, long long t, int h, long long L, int H, int d)
+{
+    return (((size_t)b * L + t) * H + h) * (size_t)d;
+}
+
+/* Forward recurrence (Eq. attn_gla), one (b,h) pair at a time, in scan order. */
+int dig_oracle_gla_fwd(const double *q, const double *k, const double *v, const double *a,
+                       double *out, int B, int H, int grid_h, int grid_w, int d_k, int d_v,
+                       int direction, int threads)
+{
+    const long long L = (long long)grid_h * grid_w;
+    long long *perm = (long long *)malloc(sizeof(long long) * (size_t)L);
+    if (!perm) return 2;
+    if (dig_oracle_perm(direction, grid_h, grid_w, perm)) { free(perm); return 1; }
+    int err = 0;
+    (void)threads;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(threads > 0 ? threads : 1) schedule(dynamic, 1)
+#endif
+    for (int bh = 0; bh < B * H; ++bh) {
+        const int b = bh / H, h = bh % H;
+        double *S = (double *)calloc((size_t)d_k * d_v, sizeof(double));
+        if (!S) { err = 2; continue; }
+        for (long long p = 0; p < L; ++p) {
+            const long long t = perm[p];
+            const double *qt = q + tok_off(b, t, h, L, H, d_k);
+            const double *kt = k + tok_off(b, t, h, L, H, d_k);
+            const double *at = a + tok_off(b, t, h, L, H, d_k);
+            const double *vt = v + tok_off(b, t, h, L, H, d_v);
+            double *ot = out + tok_off(b, t, h, L, H, d_v);
+            for (int c = 0; c < d_k; ++c) {
+                const double al = exp(at[c]);
+                for (int e = 0; e < d_v; ++e)           /* S'_{t-1} = G_t . S_{t-1}; S_t = S' + k^T v */
+                    S[(size_t)c * d_v + e] = al * S[(size_t)c * d_v + e] + kt[c] * vt[e];
+            }
+            for (int e = 0; e < d_v; ++e) {             /* o_t = q_t S_t */
+                double acc = 0.0;
+                for (int c = 0; c < d_k; ++c) acc += qt[c] * S[(size_t)c * d_v + e];
+                ot[e] = acc;
+            }
+        }
+        free(S);
+    }
+    free(perm);
+    return err;
+}
+
+/* Reverse-mode derivative of the recurrence above.
+ *   dS_t  = q_t^T do_t + diag(alpha_{t+1}) dS_{t+1}          (dS past the end is 0)
+ *   dq_t  = S_t do_t^T,  dk_t = dS_t v_t^T,  dv_t = k_t dS_t
+ *   da_t[c] = alpha_t[c] * sum_e dS_t[c,e] S_{t-1}[c,e]
+ * S_{t-1} and S_t are re-created from checkpoints of the forward state taken every SEG
+ * positions, so memory stays small at long L. */
+int dig_oracle_gla_bwd(const double *q, const double *k, const double *v, const double *a,
+                       const double *dout, double *dq, double *dk, double *dv, double *da,
+                       int B, int H, int grid_h, int grid_w, int d_k, int d_v,
+                       int direction, int threads)
+{
+    enum { SEG = 64 };
+    const long long L = (long long)grid_h * grid_w;
+    const size_t SZ = (size_t)d_k * d_v;
+    const long long nseg = (L + SEG - 1) / SEG;
+    long long *perm = (long long *)malloc(sizeof(long long) * (size_t)L);
+    if (!perm) return 2;
+    if (dig_oracle_perm(direction, grid_h, grid_w, perm)) { free(perm); return 1; }
+    int err = 0;
+    (void)threads;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(threads > 0 ? threads : 1) schedule(dynamic, 1)
+#endif
+    for (int bh = 0; bh < B * H; ++bh) {
+        const int b = bh / H, h = bh % H;
+        double *ckpt = (double *)malloc(sizeof(double) * SZ * (size_t)nseg);   /* state entering each segment */
+        double *seg = (double *)malloc(sizeof(double) * SZ * (SEG + 1));       /* seg[j] = state before local step j */
+        double *dS = (double *)calloc(SZ, sizeof(double));
+        if (!ckpt || !seg || !dS) { err = 2; free(ckpt); free(seg); free(dS); continue; }
+        /* forward sweep, storing checkpoints */
+        {
+            double *S = (double *)calloc(SZ, sizeof(double));
+            for (long long p = 0; p < L; ++p) {
+                if (p % SEG == 0) memcpy(ckpt + SZ * (size_t)(p / SEG), S, sizeof(double) * SZ);
+                const long long t = perm[p];
+                const double *kt = k + tok_off(b, t, h, L, H, d_k);
+                const double *at = a + tok_off(b, t, h, L, H, d_k);
+                const double *vt = v + tok_off(b, t, h, L, H, d_v);
+                for (int c = 0; c < d_k; ++c) {
+                    const double al = exp(at[c]);
+                    for (int e = 0; e < d_v; ++e)
+                        S[(size_t)c * d_v + e] = al * S[(size_t)c * d_v + e] + kt[c] * vt[e];
+                }
+            }
+            free(S);
+        }
+        for (long long s = nseg - 1; s >= 0; --s) {
+            const long long p0 = s * SEG;
+            const long long n = (L - p0 < SEG) ? (L - p0) : SEG;
+            memcpy(seg, ckpt + SZ * (size_t)s, sizeof(double) * SZ);
+            for (long long j = 0; j < n; ++j) {                     /* seg[j+1] = S_{p0+j} */
+                const long long t = perm[p0 + j];
+                const double *kt = k + tok_off(b, t, h, L, H, d_k);
+                const double *at = a + tok_off(b, t, h, L, H, d_k);
+                const double *vt = v + tok_off(b, t, h, L, H, d_v);
+                const double *Sp = seg + SZ * (size_t)j;
+                double *Sn = seg + SZ * (size_t)(j + 1);
+                for (int c = 0; c < d_k; ++c) {
+                    const double al = exp(at[c]);
+                    for (int e = 0; e < d_v; ++e)
+                        Sn[(size_t)c * d_v + e] = al * Sp[(size_t)c * d_v + e] + kt[c] * vt[e];
+                }
+            }
+            for (long long j = n - 1; j >= 0; --j) {
+                const long long t = perm[p0 + j];
+                const double *qt = q + tok_off(b, t, h, L, H, d_k);
+                const double *kt = k + tok_off(b, t, h, L, H, d_k);
+                const double *at = a + tok_off(b, t, h, L, H, d_k);
+                const double *vt = v + tok_off(b, t, h, L, H, d_v);
+                const double *dot = dout + tok_off(b, t, h, L, H, d_v);
+                double *dqt = dq + tok_off(b, t, h, L, H, d_k);
+                double *dkt = dk + tok_off(b, t, h, L, H, d_k);
+                double *dat = da + tok_off(b, t, h, L, H, d_k);
+                double *dvt = dv + tok_off(b, t, h, L, H, d_v);
+                const double *Sprev = seg + SZ * (size_t)j;         /* S_{t-1} */
+                const double *Scur = seg + SZ * (size_t)(j + 1);    /* S_t     */
+                for (int c = 0; c < d_k; ++c)
+                    for (int e = 0; e < d_v; ++e) dS[(size_t)c * d_v + e] += qt[c] * dot[e];
+                for (int e = 0; e < d_v; ++e) dvt[e] = 0.0;
+                for (int c = 0; c < d_k; ++c) {
+                    const double al = exp(at[c]);
+                    double sq = 0.0, sk = 0.0, sa = 0.0;
+                    for (int e = 0; e < d_v; ++e) {
+                        const double g = dS[(size_t)c * d_v + e];
+                        sq += Scur[(size_t)c * d_v + e] * dot[e];
+                        sk += g * vt[e];
+                        sa += g * Sprev[(size_t)c * d_v + e];
+                        dvt[e] += kt[c] * g;
+                    }
+                    dqt[c] = sq;
+                    dkt[c] = sk;
+                    dat[c] = al * sa;
+                    for (int e = 0; e < d_v; ++e) dS[(size_t)c * d_v + e] *= al;   /* hand dS to step t-1 */
+                }
+            }
+        }
+        free(ckpt); free(seg); free(dS);
+    }
+    free(perm);
+    return err;
+}
+
+/* SREM depthwise convolution (Algorithm 1: DWConv2d(reshape2d(z))).
+ * x, y: [B][grid_h*grid_w][D] at canonical token positions.  w: [3][3][D].  bias: [D] or NULL.
+ * The residual stream of a block that scans in `direction` is the sequence z[p] = x[perm[p]].
+ * reshape2d views it as R x C with (R,C) = (grid_h,grid_w) for the row-major orders and
+ * (grid_w,grid_h) for the column-major ones.  The convolution is a 3x3, stride-1,
+ * zero-padded cross-correlation on that matrix: tap (u,v) multiplies z2d[i+u-1][j+v-1].
+ * The result is scattered back to canonical positions. */
+int dig_oracle_dwconv(const double *x, const double *w, const double *bias, double *y,
+                      int B, int grid_h, int grid_w, int D, int direction)
+{
+    const long long L = (long long)grid_h * grid_w;
+    long long *perm = (long long *)malloc(sizeof(long long) * (size_t)L);
+    if (!perm) return 2;
+    if (dig_oracle_perm(direction, grid_h, grid_w, perm)) { free(perm); return 1; }
+    const int R = (direction >= 2) ? grid_w : grid_h;
+    const int C = (direction >= 2) ? grid_h : grid_w;
+    double *z = (double *)malloc(sizeof(double) * (size_t)L * D);
+    double *zo = (double *)malloc(sizeof(double) * (size_t)L * D);
+    if (!z || !zo) { free(perm); free(z); free(zo); return 2; }
+    for (int b = 0; b < B; ++b) {
+        const double *xb = x + (size_t)b * L * D;
+        double *yb = y + (size_t)b * L * D;
+        for (long long p = 0; p < L; ++p)                           /* gather into scan order */
+            memcpy(z + (size_t)p * D, xb + (size_t)perm[p] * D, sizeof(double) * (size_t)D);
+        for (int i = 0; i < R; ++i)
+            for (int j = 0; j < C; ++j)
+                for (int ch = 0; ch < D; ++ch) {
+                    double acc = bias ? bias[ch] : 0.0;
+                    for (int u = 0; u < 3; ++u)
+                        for (int vv = 0; vv < 3; ++vv) {
+                            const int ii = i + u - 1, jj = j + vv - 1;
+                            if (ii < 0 || ii >= R || jj < 0 || jj >= C) continue;
+                            acc += w[((size_t)u * 3 + vv) * D + ch] *
+                                   z[((size_t)ii * C + jj) * D + ch];
+                        }
+                    zo[((size_t)i * C + j) * D + ch] = acc;
+                }
+        for (long long p = 0; p < L; ++p)                           /* scatter back */
+            memcpy(yb + (size_t)perm[p] * D, zo + (size_t)p * D, sizeof(double) * (size_t)D);
+    }
+    free(perm); free(z); free(zo);
+    return 0;
+}
+
+int dig_oracle_has_openmp(void)
+{
+#ifdef _OPENMP
+    return 1;
+#else
+    return 0;
+#endif
+}
