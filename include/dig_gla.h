@@ -1,0 +1,120 @@
+/*
+ * dig_gla.h -- C ABI of the B200 (sm_100a) library for the hot path of DiG's token mixer
+ * (arxiv 2405.18428): gated linear attention over 2-D patch grids in four scan orders,
+ * forward and backward, plus the 3x3 depthwise convolution of the SREM module.
+ *
+ * Conventions shared by every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned, dense,
+ *     with no aliasing between inputs and outputs.  `tau_per_head` and every size are host
+ *     values.  `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - Token tensors are [B][L][H][d], L = grid_h*grid_w, canonical token index y*grid_w + x
+ *     (the row-major flattening of the patch grid, i.e. the (B, T, D) sequence of Algorithm 1
+ *     split into H heads).  Results are written at canonical positions for every direction.
+ *   - Calls only enqueue work on the given stream; they do not synchronise and allocate no
+ *     device memory.  Scratch memory is a caller-provided workspace.
+ *   - Errors are return codes.  Arguments are validated on the host before any launch; after a
+ *     non-zero return the outputs are unspecified.  Nothing traps, aborts or prints.
+ */
+#ifndef DIG_GLA_H_
+#define DIG_GLA_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DIG_OK = 0,
+    DIG_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, non-positive size, bad enum */
+    DIG_ERR_UNSUPPORTED = 2,   /* valid request outside what the kernels cover */
+    DIG_ERR_WORKSPACE = 3,     /* workspace missing or smaller than dig_gla_workspace_bytes */
+    DIG_ERR_CUDA = 4,          /* a CUDA runtime call failed (launch, attribute, ...) */
+    DIG_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up (see dig_last_device_status) */
+} dig_status;
+
+/* Storage type of q, k, v, out, d_out, dq, dk, dv, x, y, w, bias.  Gates are always fp32.
+ *   DIG_F32          fp32 storage, fp32 FMA arithmetic.
+ *   DIG_BF16         bf16 storage in and out; products on the tensor cores with operands
+ *                    carried at tf32 precision and fp32 accumulation; outputs rounded to
+ *                    nearest-even bf16.
+ *   DIG_BF16_F32OUT  as DIG_BF16 but out / dq / dk / dv are stored as fp32 (the unrounded
+ *                    accumulators).  DIG_BF16 results equal these rounded to bf16, bit for bit. */
+typedef enum { DIG_F32 = 0, DIG_BF16 = 1, DIG_BF16_F32OUT = 2 } dig_dtype;
+
+/* Scan order of the token grid (Algorithm 1 / Algorithm 4: the orders reached by alternating
+ * "flip" and "transpose" of the reshaped token matrix block by block). */
+typedef enum { DIG_ROW_FWD = 0, DIG_ROW_REV = 1, DIG_COL_FWD = 2, DIG_COL_REV = 3 } dig_dir;
+
+/* Which kernel family serves a call.  AUTO picks the tensor-core kernels when they cover the
+ * request and the fp32-FMA kernels otherwise.  Forcing a family that does not cover the request
+ * returns DIG_ERR_UNSUPPORTED.  Process-wide; meant for tests and benchmarks. */
+typedef enum { DIG_IMPL_AUTO = 0, DIG_IMPL_FMA = 1, DIG_IMPL_TENSOR = 2 } dig_impl;
+dig_status dig_set_impl(int impl);
+/* The family the next call with these parameters would use (DIG_IMPL_FMA or DIG_IMPL_TENSOR),
+ * or a negative dig_status if no family covers it. */
+int dig_gla_query_impl(int d_k, int d_v, int chunk, int dtype, int backward);
+
+/* Bytes of workspace dig_gla_fwd (backward = 0) or dig_gla_bwd (backward = 1) needs.
+ * Returns 0 for invalid arguments. */
+size_t dig_gla_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
+                               int dtype, int backward);
+
+/* Gate transform (Eq. gate_gla, key-channel gate alpha = sigmoid(x)^(1/tau)) in log space:
+ *   gate[b,l,h,c] = log(alpha) = logsigmoid(g[b,l,h,c]) / tau_per_head[h]
+ * g: [B][L][H][d_k] in `dtype` storage (bf16 for both DIG_BF16 variants); tau_per_head: HOST array
+ * of H positive floats; gate: fp32 [B][L][H][d_k]. */
+dig_status dig_gate_logsigmoid(const void *g, const float *tau_per_head, float *gate,
+                               int B, int L, int H, int d_k, int dtype, void *cuda_stream);
+
+/* Gated linear attention, forward (Eq. attn_gla with the value-channel gate fixed to 1):
+ *   S_t = diag(exp(gate_t)) S_{t-1} + k_t^T v_t,  S before the first token = 0,
+ *   out_t = q_t S_t,
+ * t running over the grid in `direction`, independently per (batch, head).  Evaluated chunk by
+ * chunk (Section 3.5: chunks of `chunk` tokens worked in on-chip memory); the result does not
+ * depend on `chunk` beyond rounding.  No 1/sqrt(d) scaling and no normaliser are applied.
+ *   q, k, gate: [B][L][H][d_k]; v, out: [B][L][H][d_v]; gate is log(alpha) <= 0, fp32.
+ *   d_k, d_v: multiples of 8, 8..128; chunk in {16, 32, 64, 128}; L need not be a multiple of chunk.
+ * The in-chunk decay is formed as exp(+-cumulative gate): the magnitude of the gate summed over
+ * one chunk must stay below 80 per channel (true with a wide margin for sigmoid gates with
+ * temperature >= 1 at the chunk sizes above); beyond it results may overflow. */
+dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float *gate, void *out,
+                       int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
+                       int direction, int dtype, void *workspace, size_t workspace_bytes,
+                       void *cuda_stream);
+
+/* Gated linear attention, backward: gradients of <d_out, out> with respect to q, k, v and gate
+ * (reverse-mode derivative of Eq. attn_gla; the paper trains through the operator but does not
+ * print it).  Nothing is saved by the forward call: chunk states are recomputed here.
+ *   d_out: [B][L][H][d_v]; dq, dk: [B][L][H][d_k]; dv: [B][L][H][d_v]; dgate: fp32 [B][L][H][d_k].
+ * The fp32-FMA family covers chunk <= 64 here. */
+dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float *gate,
+                       const void *d_out, void *dq, void *dk, void *dv, float *dgate,
+                       int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
+                       int direction, int dtype, void *workspace, size_t workspace_bytes,
+                       void *cuda_stream);
+
+/* SREM depthwise convolution (Algorithm 1: DWConv2d(reshape2d(z)), 3x3, stride 1, zero padding 1,
+ * cross-correlation, one filter per channel):
+ *   y = conv3x3(z2d, w) + bias, where z2d is the token matrix of a residual stream that is
+ *   currently laid out in scan order `direction`.
+ * x and y are nevertheless addressed canonically, [B][grid_h*grid_w][D]; the re-orientation is
+ * folded into the filter taps (reverse orders rotate the filter by 180 degrees, column orders
+ * transpose it), so no permuted copy is made.
+ *   w: [3][3][D]; bias: [D] or NULL; D a multiple of 8.  fp32 accumulation.
+ * For DIG_BF16_F32OUT y is fp32, x / w / bias are bf16. */
+dig_status dig_srem_dwconv(const void *x, const void *w, const void *bias, void *y,
+                           int B, int grid_h, int grid_w, int D, int direction, int dtype,
+                           void *cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns and clears the status recorded by device code on the
+ * current device: DIG_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last query,
+ * DIG_ERR_CUDA if the synchronisation itself failed, DIG_OK otherwise. */
+dig_status dig_last_device_status(void *cuda_stream);
+
+const char *dig_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIG_GLA_H_ */

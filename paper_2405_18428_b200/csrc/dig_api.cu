@@ -1,0 +1,182 @@
+// extern "C" entry points: argument validation, kernel-family choice, launches.
+#include <atomic>
+
+#include "dig_common.cuh"
+
+namespace dig {
+
+dig_status launch_gate(const void *g, const float *tau_host, float *gate, int B, int L, int H,
+                       int dk, int dtype, cudaStream_t stream);
+dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y, int B, int gh,
+                         int gw, int D, int dir, int dtype, cudaStream_t stream);
+
+namespace {
+
+std::atomic<int> g_impl{DIG_IMPL_AUTO};
+
+// Written by device code when a bounded wait expires; read and cleared by dig_last_device_status.
+__device__ int g_device_status = 0;
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool valid_dtype(int d) { return d == DIG_F32 || d == DIG_BF16 || d == DIG_BF16_F32OUT; }
+bool valid_chunk(int c) { return c == 16 || c == 32 || c == 64 || c == 128; }
+bool valid_dim(int d) { return d >= 8 && d <= 128 && (d % 8) == 0; }
+
+bool valid_geometry(int B, int H, int gh, int gw, int dk, int dv, int chunk, int dir, int dtype)
+{
+    if (B <= 0 || H <= 0 || gh <= 0 || gw <= 0) return false;
+    if ((long long)gh * gw > (1ll << 24)) return false;
+    if ((long long)B * H > 65535) return false;
+    return valid_dim(dk) && valid_dim(dv) && valid_chunk(chunk) && dir >= 0 && dir <= 3 &&
+           valid_dtype(dtype);
+}
+
+Geom make_geom(int B, int H, int gh, int gw, int dk, int dv, int chunk, int dir)
+{
+    Geom g;
+    g.B = B; g.H = H; g.gh = gh; g.gw = gw; g.L = gh * gw; g.dk = dk; g.dv = dv; g.C = chunk;
+    g.N = (g.L + chunk - 1) / chunk; g.dir = dir;
+    return g;
+}
+
+// DIG_IMPL_FMA / DIG_IMPL_TENSOR, or a negative status.
+int choose_impl(int dk, int dv, int chunk, int dtype, bool backward)
+{
+    const int want = g_impl.load();
+    const bool t_ok = tensor_supports(dk, dv, chunk, dtype, backward);
+    const bool f_ok = fma_supports(dk, dv, chunk, dtype, backward);
+    if (want == DIG_IMPL_TENSOR) return t_ok ? DIG_IMPL_TENSOR : -(int)DIG_ERR_UNSUPPORTED;
+    if (want == DIG_IMPL_FMA) return f_ok ? DIG_IMPL_FMA : -(int)DIG_ERR_UNSUPPORTED;
+    if (t_ok) return DIG_IMPL_TENSOR;
+    if (f_ok) return DIG_IMPL_FMA;
+    return -(int)DIG_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+int *device_status_ptr()
+{
+    int *p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_device_status) != cudaSuccess) return nullptr;
+    return p;
+}
+
+}  // namespace dig
+
+using namespace dig;
+
+extern "C" {
+
+dig_status dig_set_impl(int impl)
+{
+    if (impl < DIG_IMPL_AUTO || impl > DIG_IMPL_TENSOR) return DIG_ERR_INVALID_ARG;
+    g_impl.store(impl);
+    return DIG_OK;
+}
+
+int dig_gla_query_impl(int d_k, int d_v, int chunk, int dtype, int backward)
+{
+    if (!valid_dim(d_k) || !valid_dim(d_v) || !valid_chunk(chunk) || !valid_dtype(dtype))
+        return -(int)DIG_ERR_INVALID_ARG;
+    return choose_impl(d_k, d_v, chunk, dtype, backward != 0);
+}
+
+size_t dig_gla_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
+                               int dtype, int backward)
+{
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, 0, dtype)) return 0;
+    const Geom g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, 0);
+    return carve_workspace(nullptr, g, backward != 0).bytes;
+}
+
+dig_status dig_gate_logsigmoid(const void *g, const float *tau_per_head, float *gate, int B, int L,
+                               int H, int d_k, int dtype, void *cuda_stream)
+{
+    if (!g || !tau_per_head || !gate || !aligned16(g) || !aligned16(gate)) return DIG_ERR_INVALID_ARG;
+    if (B <= 0 || L <= 0 || H <= 0 || !valid_dim(d_k) || !valid_dtype(dtype)) return DIG_ERR_INVALID_ARG;
+    return launch_gate(g, tau_per_head, gate, B, L, H, d_k, dtype, (cudaStream_t)cuda_stream);
+}
+
+dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float *gate, void *out,
+                       int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
+                       int direction, int dtype, void *workspace, size_t workspace_bytes,
+                       void *cuda_stream)
+{
+    if (!q || !k || !v || !gate || !out) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(out))
+        return DIG_ERR_INVALID_ARG;
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, direction, dtype)) return DIG_ERR_INVALID_ARG;
+    const size_t need = dig_gla_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, 0);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    const int impl = choose_impl(d_k, d_v, chunk, dtype, false);
+    if (impl < 0) return (dig_status)(-impl);
+    GlaArgs a{};
+    a.q = q; a.k = k; a.v = v; a.gate = gate; a.out = out;
+    a.ws = reinterpret_cast<float *>(workspace);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, direction);
+    a.dtype = dtype;
+    a.stream = (cudaStream_t)cuda_stream;
+    return impl == DIG_IMPL_TENSOR ? tensor_gla_fwd(a) : fma_gla_fwd(a);
+}
+
+dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float *gate,
+                       const void *d_out, void *dq, void *dk, void *dv, float *dgate, int B, int H,
+                       int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!q || !k || !v || !gate || !d_out || !dq || !dk || !dv || !dgate) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(d_out) ||
+        !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(dgate))
+        return DIG_ERR_INVALID_ARG;
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, direction, dtype)) return DIG_ERR_INVALID_ARG;
+    const size_t need = dig_gla_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, 1);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    const int impl = choose_impl(d_k, d_v, chunk, dtype, true);
+    if (impl < 0) return (dig_status)(-impl);
+    GlaArgs a{};
+    a.q = q; a.k = k; a.v = v; a.gate = gate; a.d_out = d_out;
+    a.dq = dq; a.dk = dk; a.dv = dv; a.dgate = dgate;
+    a.ws = reinterpret_cast<float *>(workspace);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, direction);
+    a.dtype = dtype;
+    a.stream = (cudaStream_t)cuda_stream;
+    return impl == DIG_IMPL_TENSOR ? tensor_gla_bwd(a) : fma_gla_bwd(a);
+}
+
+dig_status dig_srem_dwconv(const void *x, const void *w, const void *bias, void *y, int B,
+                           int grid_h, int grid_w, int D, int direction, int dtype, void *cuda_stream)
+{
+    if (!x || !w || !y || !aligned16(x) || !aligned16(w) || !aligned16(y)) return DIG_ERR_INVALID_ARG;
+    if (bias && !aligned16(bias)) return DIG_ERR_INVALID_ARG;
+    if (B <= 0 || grid_h <= 0 || grid_w <= 0 || D <= 0 || (D % 8) != 0) return DIG_ERR_INVALID_ARG;
+    if (direction < 0 || direction > 3 || !valid_dtype(dtype)) return DIG_ERR_INVALID_ARG;
+    return launch_dwconv(x, w, bias, y, B, grid_h, grid_w, D, direction, dtype, (cudaStream_t)cuda_stream);
+}
+
+dig_status dig_last_device_status(void *cuda_stream)
+{
+    if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return DIG_ERR_CUDA;
+    int host = 0;
+    if (cudaMemcpyFromSymbol(&host, g_device_status, sizeof(int)) != cudaSuccess) return DIG_ERR_CUDA;
+    if (host != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return DIG_ERR_CUDA;
+        return DIG_ERR_TIMEOUT;
+    }
+    return DIG_OK;
+}
+
+const char *dig_status_string(int status)
+{
+    switch (status) {
+        case DIG_OK: return "ok";
+        case DIG_ERR_INVALID_ARG: return "invalid argument";
+        case DIG_ERR_UNSUPPORTED: return "unsupported configuration";
+        case DIG_ERR_WORKSPACE: return "workspace missing or too small";
+        case DIG_ERR_CUDA: return "CUDA runtime error";
+        case DIG_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,127 @@
+// Shared device/host helpers of the DiG GLA library: problem descriptor, scan-order index map,
+// storage-type conversion.  Internal; the public surface is include/dig_gla.h.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dig_gla.h"
+
+namespace dig {
+
+// Geometry of one GLA call, passed by value to every kernel.
+struct Geom {
+    int B, H, gh, gw, L, dk, dv, C, N, dir;   // N = ceil(L / C) chunks per (batch, head)
+};
+
+// Canonical token (y*gw + x) visited at scan position p.  Row orders walk the row-major
+// sequence forwards / backwards; column orders walk the transposed token matrix
+// (Algorithm 1: "flip" and "transpose" of the reshaped token matrix).
+__host__ __device__ __forceinline__ int scan_token(int p, int dir, int gh, int gw, int L)
+{
+    if (dir & 1) p = L - 1 - p;
+    if (dir & 2) {
+        const int x = p / gh, y = p - x * gh;
+        return y * gw + x;
+    }
+    return p;
+}
+
+// Element offset of token t, head h in a [B][L][H][d] tensor.
+__host__ __device__ __forceinline__ size_t tok_offset(const Geom &g, int b, int t, int h, int d)
+{
+    return (((size_t)b * g.L + t) * g.H + h) * (size_t)d;
+}
+
+// ---- storage conversion ---------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x)
+{
+    return __float2bfloat16_rn(x);
+}
+
+// Load 4 consecutive elements (16-byte aligned for float, 8-byte for bf16) as floats.
+__device__ __forceinline__ float4 load4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16 *p)
+{
+    const uint2 u = *reinterpret_cast<const uint2 *>(p);
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&u.x);
+    const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&u.y);
+    return make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
+}
+__device__ __forceinline__ void store4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+__device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v)
+{
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y);
+    __nv_bfloat162 b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t *>(&a);
+    u.y = *reinterpret_cast<uint32_t *>(&b);
+    *reinterpret_cast<uint2 *>(p) = u;
+}
+
+// ---- launch plumbing shared by the .cu files --------------------------------------------
+struct GlaArgs {
+    const void *q, *k, *v;
+    const float *gate;
+    void *out;                   // forward
+    const void *d_out;           // backward
+    void *dq, *dk, *dv;
+    float *dgate;
+    float *ws;                   // workspace base (fp32 view)
+    Geom g;
+    int dtype;
+    cudaStream_t stream;
+};
+
+// Workspace carving (all fp32, every block 256-byte aligned).
+//   states  [B*H][N][dk][dv]   chunk-local K^T V, turned in place into the state entering each chunk
+//   gamma   [B*H][N][dk]       exp(sum of the chunk's gates)
+//   dstates [B*H][N][dk][dv]   (backward) chunk-local Q^T dO, turned in place into dL/d(state leaving the chunk)
+//   carry   [B*H][N][dk]       (backward) gate-gradient carried in from later chunks
+struct Workspace {
+    float *states, *gamma, *dstates, *carry;
+    size_t bytes;
+};
+inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+inline Workspace carve_workspace(float *base, const Geom &g, bool backward)
+{
+    Workspace w{};
+    const size_t bh = (size_t)g.B * g.H;
+    const size_t st = align256(bh * g.N * g.dk * g.dv * sizeof(float));
+    const size_t gm = align256(bh * g.N * g.dk * sizeof(float));
+    char *p = reinterpret_cast<char *>(base);
+    w.states = reinterpret_cast<float *>(p);            p += st;
+    w.gamma = reinterpret_cast<float *>(p);             p += gm;
+    w.bytes = st + gm;
+    if (backward) {
+        w.dstates = reinterpret_cast<float *>(p);       p += st;
+        w.carry = reinterpret_cast<float *>(p);         p += gm;
+        w.bytes += st + gm;
+    }
+    return w;
+}
+
+// Kernel families (each returns a dig_status).
+dig_status fma_gla_fwd(const GlaArgs &a);
+dig_status fma_gla_bwd(const GlaArgs &a);
+bool fma_supports(int dk, int dv, int chunk, int dtype, bool backward);
+dig_status tensor_gla_fwd(const GlaArgs &a);
+dig_status tensor_gla_bwd(const GlaArgs &a);
+bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward);
+
+// Chunk-state scans, shared by both families (plain fp32 FMA, bandwidth-bound).
+dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s);
+dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s);
+
+// Device status word (bounded waits report here).
+void device_status_note_launch();
+int *device_status_ptr();
+
+inline dig_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? DIG_OK : DIG_ERR_CUDA; }
+
+}  // namespace dig

@@ -1,0 +1,152 @@
+// SREM depthwise 3x3 convolution (Algorithm 1: DWConv2d on the reshaped token matrix), channel-last.
+// A CTA stages a (TY+2) x (TX+2) pixel halo tile of CH channels in shared memory with 16-byte
+// coalesced loads; each thread then owns 8 channels of one tile column and slides down the rows,
+// so every staged vector is read from shared memory three times instead of nine.
+// The scan order the residual stream is in (`dir`) only permutes the filter taps:
+// reverse orders see the filter rotated by 180 degrees, column orders see it transposed.
+#include "dig_common.cuh"
+
+namespace dig {
+namespace {
+
+constexpr int TY = 8, TX = 16, VEC = 8;
+// Channels per CTA: 256 bytes of one pixel, so the halo tile stays under 48 KB of shared memory.
+template <typename T> struct Cfg {
+    static constexpr int CH = 256 / (int)sizeof(T);
+    static constexpr int kLanes = CH / VEC;          // 16-byte (bf16) / 32-byte (fp32) vectors per pixel
+    static constexpr int kThreads = kLanes * TX;
+};
+
+template <typename T> struct Vec8;
+template <> struct Vec8<float> {
+    float4 a, b;
+    __device__ static Vec8 load(const float *p) { return {load4(p), load4(p + 4)}; }
+    __device__ static Vec8 zero() { return {make_float4(0, 0, 0, 0), make_float4(0, 0, 0, 0)}; }
+    __device__ void unpack(float (&f)[8]) const { f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w; }
+};
+template <> struct Vec8<__nv_bfloat16> {
+    uint4 u;
+    __device__ static Vec8 load(const __nv_bfloat16 *p) { return {*reinterpret_cast<const uint4 *>(p)}; }
+    __device__ static Vec8 zero() { return {make_uint4(0, 0, 0, 0)}; }
+    __device__ void unpack(float (&f)[8]) const
+    {
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+};
+
+__device__ __forceinline__ void store8(float *p, const float (&f)[8])
+{
+    store4(p, make_float4(f[0], f[1], f[2], f[3]));
+    store4(p + 4, make_float4(f[4], f[5], f[6], f[7]));
+}
+__device__ __forceinline__ void store8(__nv_bfloat16 *p, const float (&f)[8])
+{
+    uint4 u;
+    __nv_bfloat162 t;
+    t = __floats2bfloat162_rn(f[0], f[1]); u.x = *reinterpret_cast<uint32_t *>(&t);
+    t = __floats2bfloat162_rn(f[2], f[3]); u.y = *reinterpret_cast<uint32_t *>(&t);
+    t = __floats2bfloat162_rn(f[4], f[5]); u.z = *reinterpret_cast<uint32_t *>(&t);
+    t = __floats2bfloat162_rn(f[6], f[7]); u.w = *reinterpret_cast<uint32_t *>(&t);
+    *reinterpret_cast<uint4 *>(p) = u;
+}
+
+template <typename T, typename TO>
+__global__ void __launch_bounds__(Cfg<T>::kThreads)
+srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__restrict__ bias,
+               TO *__restrict__ y, int gh, int gw, int D, int nchb, int dir)
+{
+    constexpr int CH = Cfg<T>::CH, kLanes = Cfg<T>::kLanes, kConvThreads = Cfg<T>::kThreads;
+    __shared__ Vec8<T> tile[TY + 2][TX + 2][kLanes];
+    const int b = blockIdx.z / nchb, chb = blockIdx.z - b * nchb;
+    const int x0 = blockIdx.x * TX, y0 = blockIdx.y * TY;
+    const int lane = threadIdx.x % kLanes, col = threadIdx.x / kLanes;
+    const int ch = chb * CH + lane * VEC;
+    const bool ch_ok = ch < D;
+    const T *xb = x + (size_t)b * gh * gw * D;
+
+    for (int idx = threadIdx.x; idx < (TY + 2) * (TX + 2) * kLanes; idx += kConvThreads) {
+        const int l = idx % kLanes, pix = idx / kLanes;
+        const int tx = pix % (TX + 2), ty = pix / (TX + 2);
+        const int gy = y0 + ty - 1, gx = x0 + tx - 1, c = chb * CH + l * VEC;
+        Vec8<T> v = Vec8<T>::zero();
+        if (gy >= 0 && gy < gh && gx >= 0 && gx < gw && c < D)
+            v = Vec8<T>::load(xb + ((size_t)gy * gw + gx) * D + c);
+        tile[ty][tx][l] = v;
+    }
+    // filter taps for this thread's channels, re-oriented: wt[u][v] multiplies x[i+u-1][j+v-1]
+    float wt[3][3][8], bs[8];
+#pragma unroll
+    for (int u = 0; u < 3; ++u)
+#pragma unroll
+        for (int v = 0; v < 3; ++v) {
+            int su = u, sv = v;
+            if (dir & 2) { su = v; sv = u; }
+            if (dir & 1) { su = 2 - su; sv = 2 - sv; }
+            if (ch_ok) Vec8<T>::load(w + (size_t)(su * 3 + sv) * D + ch).unpack(wt[u][v]);
+        }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) bs[i] = 0.f;
+    if (bias != nullptr && ch_ok) Vec8<T>::load(bias + ch).unpack(bs);
+    __syncthreads();
+    if (!ch_ok || x0 + col >= gw) return;
+
+    float win[3][3][8];      // win[r][v]: tile rows ty-1, ty, ty+1 (rolling), columns col, col+1, col+2
+#pragma unroll
+    for (int v = 0; v < 3; ++v) {
+        tile[0][col + v][lane].unpack(win[0][v]);
+        tile[1][col + v][lane].unpack(win[1][v]);
+    }
+#pragma unroll
+    for (int ty = 0; ty < TY; ++ty) {
+#pragma unroll
+        for (int v = 0; v < 3; ++v) tile[ty + 2][col + v][lane].unpack(win[(ty + 2) % 3][v]);
+        if (y0 + ty < gh) {
+            float acc[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = bs[i];
+#pragma unroll
+            for (int u = 0; u < 3; ++u)
+#pragma unroll
+                for (int v = 0; v < 3; ++v)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(wt[u][v][i], win[(ty + u) % 3][v][i], acc[i]);
+            store8(y + (((size_t)b * gh + y0 + ty) * gw + x0 + col) * D + ch, acc);
+        }
+    }
+}
+
+}  // namespace
+
+dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y, int B, int gh,
+                         int gw, int D, int dir, int dtype, cudaStream_t stream)
+{
+    const int CH = dtype == DIG_F32 ? Cfg<float>::CH : Cfg<__nv_bfloat16>::CH;
+    const int nchb = (D + CH - 1) / CH;
+    const dim3 grid((gw + TX - 1) / TX, (gh + TY - 1) / TY, B * nchb);
+    if (grid.y > 65535 || (size_t)B * nchb > 65535) return DIG_ERR_UNSUPPORTED;
+    switch (dtype) {
+        case DIG_F32:
+            srem_dwconv3x3<float, float><<<grid, Cfg<float>::kThreads, 0, stream>>>(
+                (const float *)x, (const float *)w, (const float *)bias, (float *)y, gh, gw, D, nchb, dir);
+            break;
+        case DIG_BF16:
+            srem_dwconv3x3<__nv_bfloat16, __nv_bfloat16><<<grid, Cfg<__nv_bfloat16>::kThreads, 0, stream>>>(
+                (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias,
+                (__nv_bfloat16 *)y, gh, gw, D, nchb, dir);
+            break;
+        case DIG_BF16_F32OUT:
+            srem_dwconv3x3<__nv_bfloat16, float><<<grid, Cfg<__nv_bfloat16>::kThreads, 0, stream>>>(
+                (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias,
+                (float *)y, gh, gw, D, nchb, dir);
+            break;
+        default: return DIG_ERR_INVALID_ARG;
+    }
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace dig

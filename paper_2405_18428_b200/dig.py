@@ -1,0 +1,198 @@
+"""ctypes binding of the C-ABI CUDA library (include/dig_gla.h).
+
+Argument marshalling only: every function forwards torch CUDA tensors as raw device pointers
+to the entry point of the same name, on torch's current stream.  There is no CPU path: if the
+shared library is missing, loading fails with an error that says how to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdig_gla.so")
+
+DIG_OK = 0
+DIG_ERR_INVALID_ARG, DIG_ERR_UNSUPPORTED, DIG_ERR_WORKSPACE, DIG_ERR_CUDA, DIG_ERR_TIMEOUT = 1, 2, 3, 4, 5
+DIG_F32, DIG_BF16, DIG_BF16_F32OUT = 0, 1, 2
+DIG_ROW_FWD, DIG_ROW_REV, DIG_COL_FWD, DIG_COL_REV = 0, 1, 2, 3
+DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR = 0, 1, 2
+
+EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
+           "dig_gla_fwd", "dig_gla_bwd", "dig_srem_dwconv", "dig_last_device_status",
+           "dig_status_string")
+
+_lib = None
+
+
+class DigError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (dig_status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library with argtypes set.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2405_18428_b200.build` "
+                "(needs nvcc); this package has no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.dig_set_impl.argtypes = [i]
+        L.dig_set_impl.restype = i
+        L.dig_gla_query_impl.argtypes = [i] * 5
+        L.dig_gla_query_impl.restype = i
+        L.dig_gla_workspace_bytes.argtypes = [i] * 9
+        L.dig_gla_workspace_bytes.restype = sz
+        L.dig_gate_logsigmoid.argtypes = [vp, ctypes.POINTER(ctypes.c_float), vp, i, i, i, i, i, vp]
+        L.dig_gate_logsigmoid.restype = i
+        L.dig_gla_fwd.argtypes = [vp] * 5 + [i] * 9 + [vp, sz, vp]
+        L.dig_gla_fwd.restype = i
+        L.dig_gla_bwd.argtypes = [vp] * 9 + [i] * 9 + [vp, sz, vp]
+        L.dig_gla_bwd.restype = i
+        L.dig_srem_dwconv.argtypes = [vp] * 4 + [i] * 6 + [vp]
+        L.dig_srem_dwconv.restype = i
+        L.dig_last_device_status.argtypes = [vp]
+        L.dig_last_device_status.restype = i
+        L.dig_status_string.argtypes = [i]
+        L.dig_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().dig_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != DIG_OK:
+        raise DigError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _storage(dtype: int) -> torch.dtype:
+    return torch.float32 if dtype == DIG_F32 else torch.bfloat16
+
+
+def _out_storage(dtype: int) -> torch.dtype:
+    return torch.bfloat16 if dtype == DIG_BF16 else torch.float32
+
+
+def _dtype_of(t: torch.Tensor, f32_out: bool = False) -> int:
+    if t.dtype == torch.float32:
+        return DIG_F32
+    if t.dtype == torch.bfloat16:
+        return DIG_BF16_F32OUT if f32_out else DIG_BF16
+    raise TypeError(f"unsupported storage type {t.dtype}")
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, shape=None, name="tensor"):
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise ValueError(f"{name}: need a contiguous CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: shape {tuple(t.shape)} != {tuple(shape)}")
+    return t.data_ptr()
+
+
+def dig_set_impl(impl: int) -> None:
+    _check(lib().dig_set_impl(impl), "dig_set_impl")
+
+
+def dig_gla_query_impl(d_k, d_v, chunk, dtype, backward) -> int:
+    return lib().dig_gla_query_impl(d_k, d_v, chunk, dtype, int(backward))
+
+
+def dig_gla_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, backward) -> int:
+    return lib().dig_gla_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, int(backward))
+
+
+def dig_gate_logsigmoid(g: torch.Tensor, tau_per_head, gate: torch.Tensor | None = None) -> torch.Tensor:
+    """gate = logsigmoid(g) / tau[h]; g: [B, L, H, d_k] (fp32 or bf16), returns fp32."""
+    B, L, H, dk = g.shape
+    dtype = _dtype_of(g)
+    if gate is None:
+        gate = torch.empty(g.shape, dtype=torch.float32, device=g.device)
+    tau = (ctypes.c_float * H)(*[float(x) for x in tau_per_head])
+    _check(lib().dig_gate_logsigmoid(_dev(g, _storage(dtype), name="g"), tau,
+                                     _dev(gate, torch.float32, g.shape, "gate"), B, L, H, dk, dtype,
+                                     _stream()), "dig_gate_logsigmoid")
+    return gate
+
+
+def _workspace(ws, need, device):
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+    return ws
+
+
+def dig_gla_fwd(q, k, v, gate, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD, *, f32_out=False,
+                out=None, workspace=None) -> torch.Tensor:
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st = _storage(dtype)
+    if out is None:
+        out = torch.empty((B, L, H, dv), dtype=_out_storage(dtype), device=q.device)
+    need = dig_gla_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 0)
+    workspace = _workspace(workspace, need, q.device)
+    _check(lib().dig_gla_fwd(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"),
+                             _dev(v, st, (B, L, H, dv), "v"), _dev(gate, torch.float32, q.shape, "gate"),
+                             _dev(out, _out_storage(dtype), (B, L, H, dv), "out"),
+                             B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
+                             workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                             _stream()), "dig_gla_fwd")
+    return out
+
+
+def dig_gla_bwd(q, k, v, gate, d_out, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD, *,
+                f32_out=False, grads=None, workspace=None):
+    """Returns (dq, dk, dv, dgate)."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st, ost = _storage(dtype), _out_storage(dtype)
+    if grads is None:
+        grads = (torch.empty(q.shape, dtype=ost, device=q.device),
+                 torch.empty(q.shape, dtype=ost, device=q.device),
+                 torch.empty(v.shape, dtype=ost, device=q.device),
+                 torch.empty(q.shape, dtype=torch.float32, device=q.device))
+    dq, dk_, dv_, dgate = grads
+    need = dig_gla_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 1)
+    workspace = _workspace(workspace, need, q.device)
+    _check(lib().dig_gla_bwd(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"),
+                             _dev(v, st, (B, L, H, dv), "v"), _dev(gate, torch.float32, q.shape, "gate"),
+                             _dev(d_out, st, v.shape, "d_out"),
+                             _dev(dq, ost, q.shape, "dq"), _dev(dk_, ost, q.shape, "dk"),
+                             _dev(dv_, ost, v.shape, "dv"), _dev(dgate, torch.float32, q.shape, "dgate"),
+                             B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
+                             workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                             _stream()), "dig_gla_bwd")
+    return dq, dk_, dv_, dgate
+
+
+def dig_srem_dwconv(x, w, bias, grid_h, grid_w, direction=DIG_ROW_FWD, *, f32_out=False, y=None):
+    """x: [B, L, D] canonical token order; w: [3, 3, D]; bias: [D] or None."""
+    B, L, D = x.shape
+    if L != grid_h * grid_w:
+        raise ValueError("x: L != grid_h*grid_w")
+    dtype = _dtype_of(x, f32_out)
+    st = _storage(dtype)
+    if y is None:
+        y = torch.empty(x.shape, dtype=_out_storage(dtype), device=x.device)
+    _check(lib().dig_srem_dwconv(_dev(x, st, name="x"), _dev(w, st, (3, 3, D), "w"),
+                                 None if bias is None else _dev(bias, st, (D,), "bias"),
+                                 _dev(y, _out_storage(dtype), x.shape, "y"),
+                                 B, grid_h, grid_w, D, direction, dtype, _stream()), "dig_srem_dwconv")
+    return y
+
+
+def dig_last_device_status() -> int:
+    return lib().dig_last_device_status(_stream())

@@ -1,0 +1,82 @@
+"""GPU parity of the SREM depthwise conv and the gate transform against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2405_18428_b200.inputs import CONFIGS, Workload, make_inputs, round_to_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def _conv_case(B, gh, gw, D, dtype, direction, bias, seed=0):
+    from paper_2405_18428_b200 import dig
+    from parity import rel_err
+    rng = np.random.default_rng(seed)
+    mk = (lambda a: round_to_bf16(a.astype(np.float32))) if dtype == "bf16" else (lambda a: a.astype(np.float32))
+    x = mk(rng.standard_normal((B, gh * gw, D)))
+    w = mk(rng.standard_normal((3, 3, D)) / 3)
+    bvec = mk(rng.standard_normal(D)) if bias else None
+    ref = oracle.dwconv(x, w, bvec, gh, gw, direction)
+    tt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    dev = lambda a: None if a is None else torch.from_numpy(a).cuda().to(tt)
+    y32 = dig.dig_srem_dwconv(dev(x), dev(w), dev(bvec), gh, gw, direction, f32_out=True)
+    err = rel_err(y32.float().cpu().numpy(), ref)
+    assert err <= 1e-5, err           # 9 fp32 FMAs per output
+    if dtype == "bf16":
+        y16 = dig.dig_srem_dwconv(dev(x), dev(w), dev(bvec), gh, gw, direction)
+        assert torch.equal(y16, y32.to(torch.bfloat16))
+    return err
+
+
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_conv_small_ragged(direction, dtype):
+    # grid not a multiple of the tile, channels not a multiple of the channel block
+    _conv_case(2, 11, 19, 72, dtype, direction, bias=(direction % 2 == 0), seed=direction)
+
+
+def test_conv_tiny_grids():
+    for gh, gw in [(1, 1), (1, 5), (3, 1), (2, 2)]:
+        _conv_case(1, gh, gw, 8, "f32", 3, bias=True)
+
+
+def test_conv_identity_init_is_exact():
+    from paper_2405_18428_b200 import dig
+    x = torch.randn(2, 16 * 24, 136, device="cuda").to(torch.bfloat16)
+    w = torch.zeros(3, 3, 136, device="cuda", dtype=torch.bfloat16)
+    w[1, 1] = 1
+    for d in range(4):
+        assert torch.equal(dig.dig_srem_dwconv(x, w, None, 16, 24, d), x)
+
+
+@pytest.mark.parametrize("cfg", ["C2", "C5"])
+def test_conv_benchmark_shapes(cfg):
+    from paper_2405_18428_b200 import dig
+    from parity import rel_err
+    wl = CONFIGS[cfg]
+    x = make_inputs(wl, gla=False, conv=True)
+    D = wl.H * wl.d_v
+    xs, ws = torch.from_numpy(x["conv_x"]).cuda().to(torch.bfloat16), torch.from_numpy(x["conv_w"]).cuda().to(torch.bfloat16)
+    for d in wl.directions:
+        ref = oracle.dwconv(x["conv_x"], x["conv_w"], None, wl.grid_h, wl.grid_w, d)
+        y = dig.dig_srem_dwconv(xs, ws, None, wl.grid_h, wl.grid_w, d, f32_out=True)
+        assert rel_err(y.cpu().numpy(), ref) <= 1e-5
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_gate_transform(dtype):
+    from paper_2405_18428_b200 import dig
+    from parity import rel_err, TOL_GATE
+    rng = np.random.default_rng(1)
+    g = rng.standard_normal((2, 50, 5, 24)).astype(np.float32) * 4
+    g[0, 0, 0, :6] = [-100, -30, 0, 30, 100, 88.5]
+    if dtype == "bf16":
+        g = round_to_bf16(g)
+    tau = np.array([16, 4, 1, 2, 0.5], dtype=np.float32)
+    ref = oracle.gate(g, tau)
+    t = torch.from_numpy(g).cuda()
+    got = dig.dig_gate_logsigmoid(t.to(torch.bfloat16) if dtype == "bf16" else t, tau).cpu().numpy()
+    assert np.isfinite(got).all() and (got <= 0).all()
+    assert rel_err(got, ref) <= TOL_GATE
+    np.testing.assert_allclose(got, ref, rtol=3e-6, atol=1e-30)
