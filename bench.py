@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Benchmark of the DiG token-mixer hot path on B200.
+
+A step is one pass of the whole hot path over one batch of synthetic, seeded input: for every
+scan direction of the workload (one DiG block each) the gate transform, GLA forward, GLA backward
+and, where the workload has one, the SREM depthwise conv.  Every block owns its own input and
+output buffers, so a step streams far more than the 126 MB L2 and no flush is needed.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  N > 1 (torchrun) shards nothing across ranks: every rank runs the
+same workload on its own GPU (weak scaling over independent batches, no collective in the path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "gla_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def flops_per_token_head(wl, chunk):
+    """(algorithmic, executed) flops per (token, head) for fwd+bwd: causal-useful work without the
+    backward's recomputation, and full chunk x chunk blocks with it."""
+    dk, dv, C = wl.d_k, wl.d_v, chunk
+    alg = 3 * (C + 1) * (dk + dv) + 12 * dk * dv
+    exe = 2 * C * (dk + dv) + 4 * dk * dv + 2 * C * (3 * dk + 2 * dv) + 10 * dk * dv
+    return alg, exe
+
+
+def bytes_per_token_head(wl):
+    """Algorithmic HBM bytes per (token, head): every operand touched once per pass; bf16 tensors,
+    fp32 gate and gate gradient."""
+    e = 2 if wl.dtype == "bf16" else 4
+    dk, dv = wl.d_k, wl.d_v
+    fwd = e * (2 * dk + dv) + 4 * dk + e * dv
+    bwd = e * (2 * dk + 2 * dv) + 4 * dk + e * (2 * dk + dv) + 4 * dk
+    return fwd, bwd
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read only)."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.stop_flag, self.thread, self.max_mhz = [], set(), False, None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+                 "hw_thermal_slowdown": 0x40, "hw_power_brake": 0x80}
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def start(self):
+        if self.nv is not None:
+            self.thread = threading.Thread(target=self._loop, daemon=True)
+            self.thread.start()
+
+    def stop(self):
+        self.stop_flag = True
+        if self.thread is not None:
+            self.thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+class Block:
+    """Device buffers of one DiG block (one scan direction) of the workload."""
+
+    def __init__(self, wl, direction, x, torch, dig):
+        dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(
+            torch.bfloat16 if wl.dtype == "bf16" else torch.float32)
+        self.wl, self.direction = wl, direction
+        self.q, self.k, self.v, self.g, self.dO = (dev(x[n]) for n in ("q", "k", "v", "g", "dO"))
+        ost = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+        self.gate = torch.empty(self.q.shape, dtype=torch.float32, device="cuda")
+        self.out = torch.empty(self.v.shape, dtype=ost, device="cuda")
+        self.grads = (torch.empty(self.q.shape, dtype=ost, device="cuda"), torch.empty(self.q.shape, dtype=ost, device="cuda"),
+                      torch.empty(self.v.shape, dtype=ost, device="cuda"), torch.empty(self.q.shape, dtype=torch.float32, device="cuda"))
+        dt = dig.DIG_BF16 if wl.dtype == "bf16" else dig.DIG_F32
+        need = dig.dig_gla_workspace_bytes(wl.B, wl.H, wl.grid_h, wl.grid_w, wl.d_k, wl.d_v, wl.chunk, dt, 1)
+        self.ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        self.tau = x["tau"]
+        if wl.conv:
+            self.cx, self.cw = dev(x["conv_x"]), dev(x["conv_w"])
+            self.cy = torch.empty_like(self.cx)
+
+    def run(self, dig):
+        wl = self.wl
+        dig.dig_gate_logsigmoid(self.g, self.tau, self.gate)
+        dig.dig_gla_fwd(self.q, self.k, self.v, self.gate, wl.grid_h, wl.grid_w, wl.chunk, self.direction,
+                        out=self.out, workspace=self.ws)
+        if wl.backward:
+            dig.dig_gla_bwd(self.q, self.k, self.v, self.gate, self.dO, wl.grid_h, wl.grid_w, wl.chunk,
+                            self.direction, grads=self.grads, workspace=self.ws)
+        if wl.conv:
+            dig.dig_srem_dwconv(self.cx, self.cw, None, wl.grid_h, wl.grid_w, self.direction, y=self.cy)
+
+    def host_io(self, torch):
+        """Pinned host mirrors for the end-to-end leg."""
+        ins = [self.q, self.k, self.v, self.g, self.dO] + ([self.cx] if self.wl.conv else [])
+        outs = [self.out, *self.grads] + ([self.cy] if self.wl.conv else [])
+        self.h_in = [torch.empty(t.shape, dtype=t.dtype).pin_memory().copy_(t) for t in ins]
+        self.h_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in outs]
+        self.d_in, self.d_out_t = ins, outs
+        return (sum(t.numel() * t.element_size() for t in ins), sum(t.numel() * t.element_size() for t in outs))
+
+    def run_e2e(self, dig):
+        for h, d in zip(self.h_in, self.d_in):
+            d.copy_(h, non_blocking=True)
+        self.run(dig)
+        for h, d in zip(self.h_out, self.d_out_t):
+            h.copy_(d, non_blocking=True)
+
+
+def make_blocks(wl, torch, dig):
+    from paper_2405_18428_b200.inputs import make_inputs
+    blocks = []
+    for i, d in enumerate(wl.directions):
+        x = make_inputs(wl.scaled(seed=wl.seed + i))
+        blocks.append(Block(wl, d, x, torch, dig))
+    return blocks
+
+
+def time_steps(blocks, dig, torch, steps, warmup, dist, e2e=False, before_timed=None):
+    for _ in range(warmup):
+        for b in blocks:
+            b.run_e2e(dig) if e2e else b.run(dig)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    if before_timed is not None:
+        before_timed()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        for b in blocks:
+            b.run_e2e(dig) if e2e else b.run(dig)
+    t1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ms = t0.elapsed_time(t1)
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def cpu_baseline(wl, budget_s=20.0):
+    """The fp64 oracle, as it stands, on a bounded sample of the workload: whole (batch, head)
+    pairs of the first scan direction, all host cores, gate + fwd + bwd (+ conv on those batches)."""
+    import oracle
+    from paper_2405_18428_b200.inputs import make_inputs
+    cores = max(1, len(os.sched_getaffinity(0)))
+    # one (b, h) pair costs about L*dk*dv*(2 + 8) fp64 multiply-adds at ~1e9/s per core
+    per_pair = wl.L * wl.d_k * wl.d_v * 10 / 1.0e9
+    pairs_budget = max(1, int(budget_s * cores / max(per_pair, 1e-9)))
+    nb = max(1, min(wl.B, pairs_budget // wl.H))
+    sub = wl.scaled(B=nb)
+    x = make_inputs(sub)
+    d = wl.directions[0]
+    t0 = time.perf_counter()
+    a = oracle.gate(x["g"], x["tau"])
+    oracle.gla_fwd(x["q"], x["k"], x["v"], a, sub.grid_h, sub.grid_w, d, threads=cores)
+    if wl.backward:
+        oracle.gla_bwd(x["q"], x["k"], x["v"], a, x["dO"], sub.grid_h, sub.grid_w, d, threads=cores)
+    if wl.conv:
+        oracle.dwconv(x["conv_x"], x["conv_w"], None, sub.grid_h, sub.grid_w, d)
+    dt = time.perf_counter() - t0
+    tokens = nb * wl.L
+    return {"value": tokens / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{nb} of {wl.B} batches x {wl.H} heads, direction {d} of {list(wl.directions)}, "
+                      f"gate+fwd{'+bwd' if wl.backward else ''}{'+conv' if wl.conv else ''}, {dt:.2f} s"}, dt, tokens
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(max(0, min(args.warmup, 1))):
+        cpu_baseline(wl, budget_s=2.0)
+    tot_t, tot_tok, last = 0.0, 0, None
+    steps = max(1, min(args.steps, 5))
+    for _ in range(steps):
+        last, dt, tok = cpu_baseline(wl, budget_s=8.0)
+        tot_t += dt
+        tot_tok += tok
+    value = tot_tok / tot_t
+    last["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * tot_t / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "grid": [wl.grid_h, wl.grid_w], "d_k": wl.d_k,
+                   "d_v": wl.d_v, "note": "fp64 token-by-token CPU oracle on a bounded sample per step"},
+        "cpu_baseline": last,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="C2")
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--family", default="auto", choices=["auto", "fma", "tensor"])
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short tokens/s-vs-L sweep over C3, C4, C5")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    args = ap.parse_args()
+
+    from paper_2405_18428_b200.inputs import CONFIGS
+    wl = CONFIGS[args.workload]
+    if args.chunk:
+        wl = wl.scaled(chunk=args.chunk)
+    if not wl.backward:
+        wl = wl.scaled(backward=False)
+    if args.impl == "reference":
+        return run_reference(args, wl)
+
+    import torch
+    from paper_2405_18428_b200 import dig
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+    dig.lib()      # fails loudly if the CUDA library is missing
+    dig.dig_set_impl({"auto": dig.DIG_IMPL_AUTO, "fma": dig.DIG_IMPL_FMA, "tensor": dig.DIG_IMPL_TENSOR}[args.family])
+    peaks = load_peaks()
+    W = max(args.warmup, 3)
+
+    blocks = make_blocks(wl, torch, dig)
+    tokens_per_step = wl.B * wl.L * len(blocks)
+    th_per_block = wl.B * wl.L * wl.H
+
+    sampler = ClockSampler(local)
+    def before_timed():
+        dig.dig_profile_enable(True)
+        sampler.start()
+
+    ms = time_steps(blocks, dig, torch, args.steps, W, dist, before_timed=before_timed)
+    clocks = sampler.stop()
+    prof = dig.dig_profile_read()
+    dig.dig_profile_enable(False)
+    assert dig.dig_last_device_status() == dig.DIG_OK
+    launches = sum(n for n, _ in prof.values())
+    value = tokens_per_step * args.steps * world / (ms * 1e-3)
+
+    # end-to-end: pinned host -> device copies of every input, the same calls, device -> host of every result
+    h2d = d2h = 0
+    for b in blocks:
+        i, o = b.host_io(torch)
+        h2d += i
+        d2h += o
+    e2e_steps = max(3, min(args.steps, 20))
+    ms_e2e = time_steps(blocks, dig, torch, e2e_steps, 3, dist, e2e=True)
+    e2e_value = tokens_per_step * e2e_steps * world / (ms_e2e * 1e-3)
+
+    # roofline of the dominant kernel (largest share of device time), from the live event timings
+    fwd_b, bwd_b = bytes_per_token_head(wl)
+    alg_bytes = {"fma_chunk_bwd": bwd_b, "tc_chunk_bwd": bwd_b, "fma_chunk_out": fwd_b, "tc_chunk_out": fwd_b}
+    total_kernel_ms = sum(t for _, t in prof.values())
+    shares = {k: {"launches": n, "ms_per_launch": t / n, "share": t / total_kernel_ms} for k, (n, t) in prof.items()}
+    candidates = [k for k in prof if k in alg_bytes] or list(prof)
+    dom = max(candidates, key=lambda k: prof[k][1])
+    n_dom, t_dom = prof[dom]
+    roofline = None
+    if dom in alg_bytes:
+        achieved = alg_bytes[dom] * th_per_block / (t_dom / n_dom * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                    "algorithmic_bytes_per_launch": alg_bytes[dom] * th_per_block}
+    alg_f, exe_f = flops_per_token_head(wl, wl.chunk)
+    step_s = ms * 1e-3 / args.steps
+    tflops_alg = alg_f * th_per_block * len(blocks) / step_s / 1e12
+    tflops_exe = exe_f * th_per_block * len(blocks) / step_s / 1e12
+    impl = dig.dig_gla_query_impl(wl.d_k, wl.d_v, wl.chunk, dig.DIG_BF16 if wl.dtype == "bf16" else dig.DIG_F32, 1)
+
+    sweep = {}
+    if not args.no_sweep and rank == 0 and world == 1:
+        del blocks
+        torch.cuda.empty_cache()
+        for name in ("C3", "C4", "C5"):
+            w2 = CONFIGS[name].scaled(directions=(CONFIGS[name].directions[0],), conv=False)
+            bl = make_blocks(w2, torch, dig)
+            big = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+            best = None
+            for _ in range(5):
+                big.zero_()      # flush L2 between single-step timings
+                m = time_steps(bl, dig, torch, 1, 1 if best is None else 0, None)
+                best = m if best is None else min(best, m)
+            a2, e2 = flops_per_token_head(w2, w2.chunk)
+            fb, bb = bytes_per_token_head(w2)
+            th = w2.B * w2.L * w2.H
+            sweep[name] = {"L": w2.L, "B": w2.B, "H": w2.H, "d": w2.d_k, "chunk": w2.chunk, "ms": best,
+                           "tokens_per_s": w2.B * w2.L / (best * 1e-3),
+                           "tflops_alg": a2 * th / (best * 1e-3) / 1e12, "tflops_exec": e2 * th / (best * 1e-3) / 1e12,
+                           "hbm_frac_of_measured": (fb + bb) * th / (best * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+            del bl, big
+            torch.cuda.empty_cache()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu, _, _ = cpu_baseline(wl)
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": W,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": {dig.DIG_IMPL_TENSOR: "tf32", dig.DIG_IMPL_FMA: "f32"}.get(impl, "f32"), "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "grid": [wl.grid_h, wl.grid_w], "L": wl.L,
+                       "d_k": wl.d_k, "d_v": wl.d_v, "chunk": wl.chunk, "storage": wl.dtype,
+                       "directions": list(wl.directions), "conv": wl.conv, "blocks_per_step": len(wl.directions),
+                       "kernel_family": {1: "fma", 2: "tensor"}.get(impl, str(impl)),
+                       "l2": "each block has its own buffers; a step streams several times the 126 MB L2, no flush needed",
+                       "tflops_alg": tflops_alg, "tflops_exec": tflops_exe,
+                       "tensor_frac_of_sustained_bf16_peak_exec": tflops_exe / peaks["bf16_tflops_sustained"]},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / e2e_steps},
+            "gpu_launches": launches,
+            "roofline": roofline, "kernels": shares, "cpu_baseline": cpu, "sweep": sweep}))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

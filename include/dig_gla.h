@@ -114,6 +114,17 @@ dig_status dig_last_device_status(void *cuda_stream);
 
 const char *dig_status_string(int status);
 
+/* Per-kernel timing aid for benchmarks (the paper has no counterpart).  While enabled, every kernel
+ * the library launches is bracketed by two CUDA events on the launching stream (a pool of 32768
+ * pairs; launches beyond it are counted but not timed).  dig_profile_enable(1) clears the counters
+ * and starts recording, dig_profile_enable(0) stops.  dig_profile_read synchronises the recorded
+ * events and returns, for kernel number `index` (0 .. dig_profile_kernels()-1), its name (copied
+ * into `name`, NUL-terminated, at most name_bytes), the number of launches recorded and their
+ * summed device time in milliseconds.  Not thread-safe; meant for one benchmarking thread. */
+dig_status dig_profile_enable(int on);
+int dig_profile_kernels(void);
+dig_status dig_profile_read(int index, char *name, int name_bytes, int *launches, float *total_ms);
+
 #ifdef __cplusplus
 }
 #endif

@@ -1,5 +1,7 @@
 // extern "C" entry points: argument validation, kernel-family choice, launches.
 #include <atomic>
+#include <cstring>
+#include <vector>
 
 #include "dig_common.cuh"
 
@@ -53,6 +55,42 @@ int choose_impl(int dk, int dv, int chunk, int dtype, bool backward)
 }
 
 }  // namespace
+
+// ---- per-kernel timing ---------------------------------------------------------------------
+namespace {
+constexpr int kMaxTimed = 32768;
+const char *const kKernelNames[KID_COUNT] = {
+    "gate_logsigmoid", "srem_dwconv3x3", "state_scan_fwd", "state_scan_bwd",
+    "fma_chunk_state", "fma_chunk_out", "fma_chunk_bwd",
+    "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd"};
+struct Profile {
+    bool on = false;
+    std::vector<cudaEvent_t> ev;      // 2 per timed launch, created lazily and reused
+    std::vector<int> kernel_of;       // kernel id of each recorded pair
+    int launches[KID_COUNT] = {};
+};
+Profile g_prof;
+}  // namespace
+
+KernelTimer::KernelTimer(int kernel_id, cudaStream_t s) : slot(-1), stream(s)
+{
+    if (!g_prof.on) return;
+    g_prof.launches[kernel_id]++;
+    const int n = (int)g_prof.kernel_of.size();
+    if (n >= kMaxTimed) return;
+    while ((int)g_prof.ev.size() < 2 * (n + 1)) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return;
+        g_prof.ev.push_back(e);
+    }
+    g_prof.kernel_of.push_back(kernel_id);
+    slot = n;
+    cudaEventRecord(g_prof.ev[2 * slot], stream);
+}
+KernelTimer::~KernelTimer()
+{
+    if (slot >= 0) cudaEventRecord(g_prof.ev[2 * slot + 1], stream);
+}
 
 int *device_status_ptr()
 {
@@ -163,6 +201,37 @@ dig_status dig_last_device_status(void *cuda_stream)
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return DIG_ERR_CUDA;
         return DIG_ERR_TIMEOUT;
     }
+    return DIG_OK;
+}
+
+dig_status dig_profile_enable(int on)
+{
+    if (on) {
+        g_prof.kernel_of.clear();
+        for (int i = 0; i < KID_COUNT; ++i) g_prof.launches[i] = 0;
+    }
+    g_prof.on = on != 0;
+    return DIG_OK;
+}
+
+int dig_profile_kernels(void) { return KID_COUNT; }
+
+dig_status dig_profile_read(int index, char *name, int name_bytes, int *launches, float *total_ms)
+{
+    if (index < 0 || index >= KID_COUNT || !name || name_bytes <= 0 || !launches || !total_ms)
+        return DIG_ERR_INVALID_ARG;
+    std::strncpy(name, kKernelNames[index], (size_t)name_bytes - 1);
+    name[name_bytes - 1] = 0;
+    *launches = g_prof.launches[index];
+    float sum = 0.f;
+    for (size_t i = 0; i < g_prof.kernel_of.size(); ++i) {
+        if (g_prof.kernel_of[i] != index) continue;
+        if (cudaEventSynchronize(g_prof.ev[2 * i + 1]) != cudaSuccess) return DIG_ERR_CUDA;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, g_prof.ev[2 * i], g_prof.ev[2 * i + 1]) != cudaSuccess) return DIG_ERR_CUDA;
+        sum += ms;
+    }
+    *total_ms = sum;
     return DIG_OK;
 }
 

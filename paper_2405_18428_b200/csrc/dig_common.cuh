@@ -119,8 +119,22 @@ dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t
 dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s);
 
 // Device status word (bounded waits report here).
-void device_status_note_launch();
 int *device_status_ptr();
+
+// Optional per-kernel timing (dig_profile_*): when enabled, every launch site brackets its
+// kernel with two CUDA events on the launching stream.
+enum KernelId {
+    KID_GATE = 0, KID_DWCONV, KID_SCAN_FWD, KID_SCAN_BWD,
+    KID_FMA_STATE, KID_FMA_OUT, KID_FMA_BWD,
+    KID_TC_STATE, KID_TC_OUT, KID_TC_BWD,
+    KID_COUNT
+};
+struct KernelTimer {
+    KernelTimer(int kernel_id, cudaStream_t stream);
+    ~KernelTimer();
+    int slot;
+    cudaStream_t stream;
+};
 
 inline dig_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? DIG_OK : DIG_ERR_CUDA; }
 

@@ -129,6 +129,7 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
     const int nchb = (D + CH - 1) / CH;
     const dim3 grid((gw + TX - 1) / TX, (gh + TY - 1) / TY, B * nchb);
     if (grid.y > 65535 || (size_t)B * nchb > 65535) return DIG_ERR_UNSUPPORTED;
+    KernelTimer t(KID_DWCONV, stream);
     switch (dtype) {
         case DIG_F32:
             srem_dwconv3x3<float, float><<<grid, Cfg<float>::kThreads, 0, stream>>>(

@@ -46,6 +46,7 @@ dig_status launch_gate(const void *g, const float *tau_host, float *gate, int B,
     }
     const size_t n8 = (size_t)B * L * H * dk / 8;
     const int blocks = (int)((n8 + 255) / 256 < 148 * 16 ? (n8 + 255) / 256 : 148 * 16);
+    KernelTimer t(KID_GATE, stream);
     if (dtype == DIG_F32)
         gate_logsigmoid<float><<<blocks, 256, 0, stream>>>((const float *)g, gate, n8, H, dk, it);
     else

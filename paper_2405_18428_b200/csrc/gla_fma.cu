@@ -460,11 +460,13 @@ dig_status fwd_typed(const GlaArgs &a)
     dig_status st;
     auto k1 = fma_chunk_state<T, false>;
     if ((st = set_smem(k1, smem_state(g, false))) != DIG_OK) return st;
+    { KernelTimer t(KID_FMA_STATE, a.stream);
     k1<<<grid, kThreads, smem_state(g, false), a.stream>>>(
-        (const T *)a.q, (const T *)a.k, (const T *)a.v, a.gate, nullptr, w.states, w.gamma, nullptr, g);
+        (const T *)a.q, (const T *)a.k, (const T *)a.v, a.gate, nullptr, w.states, w.gamma, nullptr, g); }
     if ((st = launch_state_scan_fwd(w, g, a.stream)) != DIG_OK) return st;
     auto k3 = fma_chunk_out<T, TO>;
     if ((st = set_smem(k3, smem_out(g))) != DIG_OK) return st;
+    KernelTimer t(KID_FMA_OUT, a.stream);
     k3<<<grid, kThreads, smem_out(g), a.stream>>>((const T *)a.q, (const T *)a.k, (const T *)a.v,
                                                   a.gate, w.states, (TO *)a.out, g);
     return cuda_ok(cudaGetLastError());
@@ -481,11 +483,13 @@ dig_status bwd_typed(const GlaArgs &a)
     if ((st = set_smem(k1, smem_state(g, true))) != DIG_OK) return st;
     auto k4 = fma_chunk_bwd<T, TO>;
     if ((st = set_smem(k4, smem_bwd(g))) != DIG_OK) return st;
+    { KernelTimer t(KID_FMA_STATE, a.stream);
     k1<<<grid, kThreads, smem_state(g, true), a.stream>>>(
         (const T *)a.q, (const T *)a.k, (const T *)a.v, a.gate, (const T *)a.d_out, w.states, w.gamma,
-        w.dstates, g);
+        w.dstates, g); }
     if ((st = launch_state_scan_fwd(w, g, a.stream)) != DIG_OK) return st;
     if ((st = launch_state_scan_bwd(w, g, a.stream)) != DIG_OK) return st;
+    KernelTimer t(KID_FMA_BWD, a.stream);
     k4<<<grid, kThreads, smem_bwd(g), a.stream>>>(
         (const T *)a.q, (const T *)a.k, (const T *)a.v, a.gate, (const T *)a.d_out, w.states, w.dstates,
         w.carry, (TO *)a.dq, (TO *)a.dk, (TO *)a.dv, a.dgate, g);

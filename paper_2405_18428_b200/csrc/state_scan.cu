@@ -94,6 +94,7 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
 dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s)
 {
     const dim3 grid((g.dk * g.dv + kScanThreads - 1) / kScanThreads, g.B * g.H);
+    KernelTimer t(KID_SCAN_FWD, s);
     state_scan_fwd<<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
     return cuda_ok(cudaGetLastError());
 }
@@ -101,6 +102,7 @@ dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t
 dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s)
 {
     const dim3 grid((g.dk + kRowsPerBlock - 1) / kRowsPerBlock, g.B * g.H);
+    KernelTimer t(KID_SCAN_BWD, s);
     state_scan_bwd<<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N,
                                                        g.dk, g.dv);
     return cuda_ok(cudaGetLastError());

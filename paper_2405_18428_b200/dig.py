@@ -22,7 +22,7 @@ DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR = 0, 1, 2
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
            "dig_gla_fwd", "dig_gla_bwd", "dig_srem_dwconv", "dig_last_device_status",
-           "dig_status_string")
+           "dig_status_string", "dig_profile_enable", "dig_profile_kernels", "dig_profile_read")
 
 _lib = None
 
@@ -61,6 +61,12 @@ def lib() -> ctypes.CDLL:
         L.dig_last_device_status.restype = i
         L.dig_status_string.argtypes = [i]
         L.dig_status_string.restype = ctypes.c_char_p
+        L.dig_profile_enable.argtypes = [i]
+        L.dig_profile_enable.restype = i
+        L.dig_profile_kernels.argtypes = []
+        L.dig_profile_kernels.restype = i
+        L.dig_profile_read.argtypes = [i, ctypes.c_char_p, i, ctypes.POINTER(i), ctypes.POINTER(ctypes.c_float)]
+        L.dig_profile_read.restype = i
         _lib = L
     return _lib
 
@@ -196,3 +202,19 @@ def dig_srem_dwconv(x, w, bias, grid_h, grid_w, direction=DIG_ROW_FWD, *, f32_ou
 
 def dig_last_device_status() -> int:
     return lib().dig_last_device_status(_stream())
+
+
+def dig_profile_enable(on: bool) -> None:
+    _check(lib().dig_profile_enable(int(on)), "dig_profile_enable")
+
+
+def dig_profile_read() -> dict:
+    """{kernel name: (launches, total milliseconds)} for the launches recorded since enabling."""
+    out = {}
+    for idx in range(lib().dig_profile_kernels()):
+        name = ctypes.create_string_buffer(64)
+        n, ms = ctypes.c_int(0), ctypes.c_float(0)
+        _check(lib().dig_profile_read(idx, name, 64, ctypes.byref(n), ctypes.byref(ms)), "dig_profile_read")
+        if n.value:
+            out[name.value.decode()] = (n.value, ms.value)
+    return out
