@@ -17,7 +17,9 @@ TOL_GATE = 1e-6      # elementwise fp32 transform
 def rel_err(got, ref) -> float:
     got = np.asarray(got, dtype=np.float64)
     rms = float(np.sqrt(np.mean(ref ** 2)))
-    return float(np.abs(got - ref).max() / max(rms, 1e-300))
+    if rms == 0.0:          # an identically-zero reference (e.g. the gate gradient of a 1-token
+        rms = 1.0           # sequence): fall back to the absolute error
+    return float(np.abs(got - ref).max() / rms)
 
 
 def to_dev(x: np.ndarray, wl: Workload) -> torch.Tensor:
