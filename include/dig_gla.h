@@ -30,7 +30,8 @@ typedef enum {
     DIG_ERR_UNSUPPORTED = 2,   /* valid request outside what the kernels cover */
     DIG_ERR_WORKSPACE = 3,     /* workspace missing or smaller than dig_gla_workspace_bytes */
     DIG_ERR_CUDA = 4,          /* a CUDA runtime call failed (launch, attribute, ...) */
-    DIG_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up (see dig_last_device_status) */
+    DIG_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (see dig_last_device_status) */
+    DIG_ERR_SCRATCH_LIMIT = 6  /* dig_gla_fwd_static: the problem needs more than its built-in scratch */
 } dig_status;
 
 /* Storage type of q, k, v, out, d_out, dq, dk, dv, x, y, w, bias.  Gates are always fp32.
@@ -82,6 +83,31 @@ dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float 
                        int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
                        int direction, int dtype, void *workspace, size_t workspace_bytes,
                        void *cuda_stream);
+
+/* Forward GLA without any allocation (the paper has no counterpart; this is a packaging variant
+ * of dig_gla_fwd, same arguments minus the workspace, same results bit for bit).
+ *
+ * Who it is for: callers that cannot obtain device memory at call time -- a host application that
+ * owns every byte of the GPU and hands plugins only their inputs and outputs, a latency-critical
+ * loop in which cudaMalloc's implicit synchronisation is unacceptable, a process whose memory
+ * budget was fixed at start-up.  For them the chunk states and decay factors that dig_gla_fwd keeps
+ * in the caller's workspace live in a device array of DIG_GLA_STATIC_SCRATCH_BYTES that is part of
+ * the library image: every GPU that loads the library holds that much memory until the process
+ * exits.  The call itself allocates and frees nothing, on the host side of CUDA or through torch.
+ *
+ * Limit: requests for which dig_gla_workspace_bytes(..., backward = 0) exceeds
+ * DIG_GLA_STATIC_SCRATCH_BYTES return DIG_ERR_SCRATCH_LIMIT before anything is launched (16 MiB
+ * covers e.g. B*H = 48 sequences of 1024 tokens at d_k = d_v = 64, chunk 64).
+ *
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share the one array:
+ * it keeps whatever the previous call left there (the kernels overwrite every entry they read,
+ * so nothing needs clearing), and two calls whose kernels overlap on the GPU -- different streams,
+ * or different host threads -- race on it.  Serialise them on one stream. */
+#define DIG_GLA_STATIC_SCRATCH_BYTES ((size_t)16 << 20)
+dig_status dig_gla_fwd_static(const void *q, const void *k, const void *v, const float *gate,
+                              void *out, int B, int H, int grid_h, int grid_w, int d_k, int d_v,
+                              int chunk, int direction, int dtype, void *cuda_stream);
 
 /* Gated linear attention, backward: gradients of <d_out, out> with respect to q, k, v and gate
  * (reverse-mode derivative of Eq. attn_gla; the paper trains through the operator but does not

@@ -244,6 +244,7 @@ const char *dig_status_string(int status)
         case DIG_ERR_WORKSPACE: return "workspace missing or too small";
         case DIG_ERR_CUDA: return "CUDA runtime error";
         case DIG_ERR_TIMEOUT: return "device-side wait timed out";
+        case DIG_ERR_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of dig_gla_fwd_static";
     }
     return "unknown status";
 }

@@ -16,12 +16,14 @@ LIB_PATH = os.path.join(_PKG, "libdig_gla.so")
 
 DIG_OK = 0
 DIG_ERR_INVALID_ARG, DIG_ERR_UNSUPPORTED, DIG_ERR_WORKSPACE, DIG_ERR_CUDA, DIG_ERR_TIMEOUT = 1, 2, 3, 4, 5
+DIG_ERR_SCRATCH_LIMIT = 6
+DIG_GLA_STATIC_SCRATCH_BYTES = 16 << 20
 DIG_F32, DIG_BF16, DIG_BF16_F32OUT = 0, 1, 2
 DIG_ROW_FWD, DIG_ROW_REV, DIG_COL_FWD, DIG_COL_REV = 0, 1, 2, 3
 DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR = 0, 1, 2
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
-           "dig_gla_fwd", "dig_gla_bwd", "dig_srem_dwconv", "dig_last_device_status",
+           "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_srem_dwconv", "dig_last_device_status",
            "dig_status_string", "dig_profile_enable", "dig_profile_kernels", "dig_profile_read")
 
 _lib = None
@@ -53,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.dig_gate_logsigmoid.restype = i
         L.dig_gla_fwd.argtypes = [vp] * 5 + [i] * 9 + [vp, sz, vp]
         L.dig_gla_fwd.restype = i
+        L.dig_gla_fwd_static.argtypes = [vp] * 5 + [i] * 9 + [vp]
+        L.dig_gla_fwd_static.restype = i
         L.dig_gla_bwd.argtypes = [vp] * 9 + [i] * 9 + [vp, sz, vp]
         L.dig_gla_bwd.restype = i
         L.dig_srem_dwconv.argtypes = [vp] * 4 + [i] * 6 + [vp]
@@ -155,6 +159,22 @@ def dig_gla_fwd(q, k, v, gate, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD, 
                              B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
                              workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                              _stream()), "dig_gla_fwd")
+    return out
+
+
+def dig_gla_fwd_static(q, k, v, gate, out, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD) -> torch.Tensor:
+    """dig_gla_fwd for callers that cannot allocate: the scratch is a fixed array inside the
+    library, so `out` must be given and nothing is allocated here either.  `out` is bf16 for bf16
+    inputs unless it is an fp32 tensor, which selects the fp32-output variant."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out=(q.dtype == torch.bfloat16 and out.dtype == torch.float32))
+    st = _storage(dtype)
+    _check(lib().dig_gla_fwd_static(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"),
+                                    _dev(v, st, (B, L, H, dv), "v"), _dev(gate, torch.float32, q.shape, "gate"),
+                                    _dev(out, _out_storage(dtype), (B, L, H, dv), "out"),
+                                    B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype, _stream()),
+           "dig_gla_fwd_static")
     return out
 
 

@@ -31,8 +31,8 @@ def test_every_declared_symbol_is_exported(L):
 
 
 def test_status_strings(L):
-    seen = {L.dig_status_string(i).decode() for i in range(6)}
-    assert len(seen) == 6 and "unknown status" not in seen
+    seen = {L.dig_status_string(i).decode() for i in range(7)}
+    assert len(seen) == 7 and "unknown status" not in seen
     assert L.dig_status_string(99).decode() == "unknown status"
 
 
