@@ -99,6 +99,19 @@ int *device_status_ptr()
     return p;
 }
 
+int device_sm_count()
+{
+    static std::atomic<int> cached[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    int n = cached[dev].load();
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached[dev].store(n);
+    }
+    return n;
+}
+
 }  // namespace dig
 
 using namespace dig;

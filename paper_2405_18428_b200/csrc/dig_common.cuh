@@ -115,11 +115,21 @@ dig_status tensor_gla_bwd(const GlaArgs &a);
 bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward);
 
 // Chunk-state scans, shared by both families (plain fp32 FMA, bandwidth-bound).
-dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s);
+// `tiles`: the states are stored transposed, in swizzled operand-tile order (tensor-core forward pass).
+dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tiles = false);
 dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s);
+// Tensor-core backward pass: forward and reverse scan in one launch over states kept in tile order.
+dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s);
 
 // Device status word (bounded waits report here).
 int *device_status_ptr();
+// Streaming multiprocessors of the current device (cached per device), 0 on error.
+int device_sm_count();
+
+// Tensor-core kernels (one .cu file each).
+dig_status launch_tc_state(const GlaArgs &a, const Workspace &w, bool backward, int sm_count, int *status);
+dig_status launch_tc_out(const GlaArgs &a, const Workspace &w, int sm_count, int *status);
+dig_status launch_tc_bwd(const GlaArgs &a, const Workspace &w, int sm_count, int *status);
 
 // Optional per-kernel timing (dig_profile_*): when enabled, every launch site brackets its
 // kernel with two CUDA events on the launching stream.

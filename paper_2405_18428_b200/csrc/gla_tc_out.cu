@@ -1,0 +1,202 @@
+// Tensor-core output kernel of chunkwise gated linear attention (Eq. attn_gla, Section 3.5):
+//   out = tril(Qt Kt^T) V + Qt S,   Qt = q*exp(Lam), Kt = k*exp(-Lam),
+// S the state entering the chunk (read as S^T, [d_v][d_k], from the workspace).
+//
+// A persistent CTA of 512 threads works on two chunks at a time, stacked along the M dimension
+// of tcgen05.mma (rows 0-63 chunk a, rows 64-127 chunk b).  The B operands of the two chunks are
+// concatenated along N, so every product is 8 instructions of M = N = 128 for both chunks:
+//   scores  [Qa;Qb] [Ka;Kb]^T      -> wanted blocks (a, cols 0-63), (b, cols 64-127)
+//   inter   [Qa;Qb] [Sa^T;Sb^T]^T  -> same blocks of the output accumulator
+//   intra   [Pa;Pb] [Va | Vb]      -> accumulated on top
+// The other blocks of the accumulators hold cross terms that are never read.  While a pair is in
+// the tensor pipe the next pair's q, k, v rows are already being loaded into registers, and its gate
+// rows and incoming states arrive by bulk asynchronous copies (cp.async.bulk) in shared memory.
+#include "tc_tiles.cuh"
+
+namespace dig {
+namespace {
+
+using namespace tc;
+
+constexpr int NT = 512;
+constexpr int W = 16;                          // accumulator columns per thread
+constexpr int kTileK = 128 * 64 * 4;           // 128 rows x 64 columns, K-format
+constexpr int kTileM = T * 128 * 4;            // 64 rows x 128 columns, M-format
+
+struct OutRaw {
+    uint4 q[2], k[2], v[2];
+};
+
+__device__ __forceinline__ void load_raw(OutRaw &r, const bf16 *q, const bf16 *k, const bf16 *v, const Geom &g,
+                                         const Item (&it)[2])
+{
+    const int row = threadIdx.x >> 3, col = (threadIdx.x & 7) * 8;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        const int tok = item_token(g, it[half], row);
+        r.q[half] = ld_row8(q, g, it[half].b, tok, it[half].h, DK, col);
+        r.k[half] = ld_row8(k, g, it[half].b, tok, it[half].h, DK, col);
+        r.v[half] = ld_row8(v, g, it[half].b, tok, it[half].h, DV, col);
+    }
+}
+
+// The two chunks' incoming states (already tf32-rounded and in tile order in the workspace) go
+// straight into the stacked S^T tile: per chunk one 8 KB bulk copy per column block.
+__device__ __forceinline__ void fetch_states(char *tS, const float *states, int pair, int total, uint64_t *bar)
+{
+    fence_async_smem();
+    const uint32_t n = (2 * pair + 1 < total) ? 2u : 1u;
+    mbar_arrive_expect_tx(bar, n * (uint32_t)(DK * DV * 4));
+    for (uint32_t half = 0; half < n; ++half) {
+        const char *src = reinterpret_cast<const char *>(states + (size_t)(2 * pair + half) * (DK * DV));
+        bulk_g2s(tS + half * (T * 128), src, T * 128, bar);
+        bulk_g2s(tS + 128 * 128 + half * (T * 128), src + T * 128, T * 128, bar);
+    }
+}
+
+template <typename TO>
+__global__ void __launch_bounds__(NT)
+tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *__restrict__ v,
+            const float *__restrict__ gate, const float *__restrict__ states, TO *__restrict__ out,
+            int *status, Geom g)
+{
+    extern __shared__ char smem_raw[];
+    char *base = align1024(smem_raw);
+    char *tQ = base, *tK = base + kTileK, *tS = base + 2 * kTileK, *tP = base + 3 * kTileK;    // K-format, 128 rows
+    char *tV = base + 4 * kTileK;                                                              // M-format, 64 x 128
+    float *sLam = reinterpret_cast<float *>(tV + kTileM);
+    float *sLast = sLam + 2 * T * kLamPitch, *sTot = sLast + 128;
+    Control *ctl = reinterpret_cast<Control *>(sTot + NT);
+    constexpr uint32_t kCols = 256;
+    constexpr uint32_t aP = 0, aO = 128;
+    uint64_t *barP = &ctl->bar[0], *barO = &ctl->bar[1], *barG = &ctl->bar[2], *barS = &ctl->bar[3];
+    setup(ctl, 4, kCols, 2, 4);
+    const uint32_t tmem = ctl->tmem_base;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int R = 32 * (warp & 3) + lane, half_r = R >> 6, r = R & 63, c0 = W * (warp >> 2);
+    const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
+
+    const int total = g.B * g.H * g.N, npairs = (total + 1) / 2;
+    OutRaw raw;
+    int pair = blockIdx.x;
+    if (pair < npairs) {
+        const Item it[2] = {item_of(g, 2 * pair, total), item_of(g, 2 * pair + 1, total)};
+        load_raw(raw, q, k, v, g, it);
+        if (warp >= 4 && warp < 8) fetch_gate_rows(sLam, gate, g, it[(warp - 4) >> 1], warp - 4, barG, lane);
+        if (threadIdx.x == 0) fetch_states(tS, states, pair, total, barS);
+    }
+    uint32_t parity = 0;
+    bool ok = true;
+    for (; pair < npairs; pair += gridDim.x) {
+        const int next = pair + gridDim.x;
+        const Item nit[2] = {item_of(g, 2 * next, total), item_of(g, 2 * next + 1, total)};
+        ok = mbar_wait(barG, parity, status);
+        if (!__syncthreads_and(ok)) break;
+        gate_prefix<NT, 2>(sLam, sLast, sTot, kLog2e);
+        {
+            const int row = threadIdx.x >> 3, j = threadIdx.x & 7, col = j * 8;
+            const bool flip = j >= 4;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int id = 2 * pair + half;
+                const bool keep = id < total && (id % g.N) * T + row < g.L;
+                float lam[8], x[8];
+                read_lam8(sLam, 64 * half + row, col, lam);
+                unpack8(raw.q[half], x, keep);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) x[e] *= ex2(lam[e]);
+                st_k8<128>(tQ, 64 * half + row, col, x, flip);
+                unpack8(raw.k[half], x, keep);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) x[e] *= ex2(-lam[e]);
+                st_k8<128>(tK, 64 * half + row, col, x, flip);
+                unpack8(raw.v[half], x, keep);
+                st_m8<T, false>(tV, row, 64 * half + col, x, flip);
+            }
+        }
+        fence_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            if (mbar_wait(barS, parity, status)) {
+                tc_fence_after_sync();
+                issue<128, 128, false, false, 128, 128>(tmem + aP, kdesc<128>(tQ), kdesc<128>(tK), false);     // scores
+                mma_commit(barP);
+                issue<128, 128, false, false, 128, 128>(tmem + aO, kdesc<128>(tQ), kdesc<128>(tS), false);     // Qt S
+            }
+        }
+        if (next < npairs) {
+            if (warp >= 4 && warp < 8) fetch_gate_rows(sLam, gate, g, nit[(warp - 4) >> 1], warp - 4, barG, lane);   // the gate table is free again
+            load_raw(raw, q, k, v, g, nit);
+        }
+        ok = mbar_wait(barP, parity, status);
+        if (ok) {
+            tc_fence_after_sync();
+            float p[W];
+            tmem_ld(tmem + lane_base + aP + (uint32_t)(64 * half_r + c0), p);
+#pragma unroll
+            for (int j = 0; j < W; ++j)
+                if (c0 + j > r) p[j] = 0.f;                   // keep s <= t; the diagonal has weight 1
+#pragma unroll
+            for (int j = 0; j < W / 4; ++j)
+                st_k4<128>(tP, R, c0 + 4 * j, make_float4(p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]));
+        }
+        fence_async_smem();
+        tc_fence_before_sync();
+        ok = __syncthreads_and(ok);
+        if (!ok) break;
+        if (threadIdx.x == 0) {
+            tc_fence_after_sync();
+            issue<128, 128, false, true, 128, T>(tmem + aO, kdesc<128>(tP), mdesc<T>(tV), true);           // + P V
+            mma_commit(barO);
+        }
+        ok = mbar_wait(barO, parity, status);
+        parity ^= 1;
+        if (ok) {
+            tc_fence_after_sync();
+            if (threadIdx.x == 0 && next < npairs) fetch_states(tS, states, next, total, barS);           // S^T tile is free again
+            float o[W];
+            tmem_ld(tmem + lane_base + aO + (uint32_t)(64 * half_r + c0), o);
+            const Item it = item_of(g, 2 * pair + half_r, total);
+            const int tok = item_token(g, it, r);
+            if (tok >= 0) store16(out + tok_offset(g, it.b, tok, it.h, DV) + c0, o);
+        }
+        tc_fence_before_sync();
+        if (!__syncthreads_and(ok)) break;
+        tc_fence_after_sync();
+    }
+    if (!ok) {      // a wait gave up: let bulk copies still in flight land before the CTA's memory goes away
+        mbar_wait(barG, parity, status);
+        mbar_wait(barS, parity, status);
+    }
+    teardown(ctl, kCols);
+}
+
+constexpr size_t out_smem()
+{
+    return 1024 + 4 * (size_t)kTileK + kTileM + sizeof(float) * (2 * T * kLamPitch + 128 + NT) + sizeof(Control);
+}
+
+template <typename TO>
+dig_status launch_typed(const GlaArgs &a, const Workspace &w, int sm_count, int *status)
+{
+    const Geom &g = a.g;
+    const int total = g.B * g.H * g.N, npairs = (total + 1) / 2;
+    auto kern = tc_out_pair<TO>;
+    constexpr size_t smem = out_smem();
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
+    const int grid = npairs < sm_count ? npairs : sm_count;
+    KernelTimer t(KID_TC_OUT, a.stream);
+    kern<<<grid, NT, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate, w.states,
+                                       (TO *)a.out, status, g);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace
+
+dig_status launch_tc_out(const GlaArgs &a, const Workspace &w, int sm_count, int *status)
+{
+    return a.dtype == DIG_BF16 ? launch_typed<bf16>(a, w, sm_count, status) : launch_typed<float>(a, w, sm_count, status);
+}
+
+}  // namespace dig

@@ -13,36 +13,63 @@ namespace dig {
 namespace {
 
 constexpr int kScanThreads = 128;
-constexpr int kAhead = 4;
+constexpr int kAhead = 8;
 
+__device__ __forceinline__ float round_tf32(float x)
+{
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u);
+}
+__device__ __forceinline__ float4 round4_tf32(float4 v)
+{
+    return make_float4(round_tf32(v.x), round_tf32(v.y), round_tf32(v.z), round_tf32(v.w));
+}
+
+// One thread per 4 consecutive state elements.  TILES = false: states are [d_k][d_v] row-major,
+// decay indexed by the row.  TILES = true (tensor-core forward pass, d_k = d_v = 64): each state is
+// stored transposed ([d_v][d_k]) in the swizzled operand-tile order the output kernel copies
+// straight into shared memory (two column blocks of 64 rows x 128 bytes, 16-byte pieces of a row
+// XOR-ed with row & 7); the decay is indexed by the logical column, and the stored states are
+// rounded to tf32 (the running value is not).
+// The loads of a batch of kAhead chunks do not depend on the running value, so they are all in
+// flight before the short dependent chain of FMAs runs.
+template <bool TILES>
 __global__ void __launch_bounds__(kScanThreads)
 state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int N, int dk, int dv)
 {
-    const int elem = blockIdx.x * kScanThreads + threadIdx.x;
-    if (elem >= dk * dv) return;
-    const int c = elem / dv;
-    float *st = states + (size_t)blockIdx.y * N * dk * dv + elem;
-    const float *gm = gamma + (size_t)blockIdx.y * N * dk + c;
-    const size_t sstride = (size_t)dk * dv;
-    float run = 0.f;
-    int i = 0;
-    for (; i + kAhead <= N; i += kAhead) {
-        float u[kAhead], g[kAhead];
-#pragma unroll
-        for (int j = 0; j < kAhead; ++j) {
-            u[j] = st[(size_t)(i + j) * sstride];
-            g[j] = gm[(size_t)(i + j) * dk];
-        }
-#pragma unroll
-        for (int j = 0; j < kAhead; ++j) {
-            st[(size_t)(i + j) * sstride] = run;
-            run = fmaf(g[j], run, u[j]);
-        }
+    const int e4 = blockIdx.x * kScanThreads + threadIdx.x;          // float4 index inside one state
+    if (e4 * 4 >= dk * dv) return;
+    int row, col;
+    if (TILES) {
+        row = (e4 & 511) >> 3;
+        col = (e4 >> 9) * 32 + (((e4 & 7) ^ (row & 7)) << 2);
+    } else {
+        row = (e4 * 4) / dv;
+        col = (e4 * 4) - row * dv;
     }
-    for (; i < N; ++i) {
-        const float u = st[(size_t)i * sstride], g = gm[(size_t)i * dk];
-        st[(size_t)i * sstride] = run;
-        run = fmaf(g, run, u);
+    float4 *st = reinterpret_cast<float4 *>(states + (size_t)blockIdx.y * N * dk * dv) + e4;
+    const float *gm = gamma + (size_t)blockIdx.y * N * dk + (TILES ? col : row);
+    const size_t sstride = (size_t)dk * dv / 4;
+    float4 run = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < N; i += kAhead) {
+        float4 u[kAhead], g[kAhead];
+#pragma unroll
+        for (int j = 0; j < kAhead; ++j) {
+            if (i + j < N) {
+                u[j] = st[(size_t)(i + j) * sstride];
+                if (TILES) g[j] = *reinterpret_cast<const float4 *>(gm + (size_t)(i + j) * dk);
+                else g[j].x = g[j].y = g[j].z = g[j].w = gm[(size_t)(i + j) * dk];
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kAhead; ++j) {
+            if (i + j < N) {
+                st[(size_t)(i + j) * sstride] = TILES ? round4_tf32(run) : run;
+                run.x = fmaf(g[j].x, run.x, u[j].x);
+                run.y = fmaf(g[j].y, run.y, u[j].y);
+                run.z = fmaf(g[j].z, run.z, u[j].z);
+                run.w = fmaf(g[j].w, run.w, u[j].w);
+            }
+        }
     }
 }
 
@@ -89,13 +116,97 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
     }
 }
 
+// Both scans of the tensor-core backward pass in one launch (d_k = d_v = 64).  The per-chunk
+// matrices U (in `states`) and W (in `dstates`) are [d_k][d_v] in swizzled tile order; a thread owns
+// the same 16-byte piece of one row in both column blocks (8 floats), so the decay index is its row
+// and the order of the pieces inside the row does not matter.  It first runs the forward
+// recurrence (states <- S_[i], rounded to tf32 for the consumer), then walks back over the chunks:
+//   dstates <- diag(gamma_i) D_[i] (rounded to tf32), carry_i = row sums of S_[i+1] * D_[i],
+// reading back the S values it wrote itself.  Block = 8 rows x 8 pieces; grid (8, B*H).
+constexpr int kBack = 4;
+__device__ __forceinline__ float4 fma4(float g, float4 r, float4 u)
+{
+    return make_float4(fmaf(g, r.x, u.x), fmaf(g, r.y, u.y), fmaf(g, r.z, u.z), fmaf(g, r.w, u.w));
+}
+__global__ void __launch_bounds__(64)
+state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, const float *__restrict__ gamma,
+                     float *__restrict__ carry, int N)
+{
+    const int t = threadIdx.x, c = 8 * blockIdx.x + (t >> 3);
+    const size_t base = (size_t)blockIdx.y * N * 4096;
+    float4 *S = reinterpret_cast<float4 *>(states + base) + c * 8 + (t & 7);
+    float4 *D = reinterpret_cast<float4 *>(dstates + base) + c * 8 + (t & 7);
+    const float *gm = gamma + (size_t)blockIdx.y * N * 64 + c;
+    float *cr = carry + (size_t)blockIdx.y * N * 64 + c;
+    float4 r0 = make_float4(0.f, 0.f, 0.f, 0.f), r1 = r0;
+    for (int i = 0; i < N; i += kAhead) {
+        float4 u0[kAhead], u1[kAhead];
+        float g[kAhead];
+#pragma unroll
+        for (int j = 0; j < kAhead; ++j)
+            if (i + j < N) {
+                u0[j] = S[(size_t)(i + j) * 1024];
+                u1[j] = S[(size_t)(i + j) * 1024 + 512];
+                g[j] = gm[(size_t)(i + j) * 64];
+            }
+#pragma unroll
+        for (int j = 0; j < kAhead; ++j)
+            if (i + j < N) {
+                S[(size_t)(i + j) * 1024] = round4_tf32(r0);
+                S[(size_t)(i + j) * 1024 + 512] = round4_tf32(r1);
+                r0 = fma4(g[j], r0, u0[j]);
+                r1 = fma4(g[j], r1, u1[j]);
+            }
+    }
+    float4 d0 = make_float4(0.f, 0.f, 0.f, 0.f), d1 = d0;
+    for (int i = N - 1; i >= 0; i -= kBack) {
+        float4 w0[kBack], w1[kBack], s0[kBack], s1[kBack];
+        float g[kBack];
+#pragma unroll
+        for (int j = 0; j < kBack; ++j) {
+            const int ch = i - j;
+            if (ch >= 0) {
+                w0[j] = D[(size_t)ch * 1024];
+                w1[j] = D[(size_t)ch * 1024 + 512];
+                g[j] = gm[(size_t)ch * 64];
+                if (ch + 1 < N) {
+                    s0[j] = S[(size_t)(ch + 1) * 1024];
+                    s1[j] = S[(size_t)(ch + 1) * 1024 + 512];
+                } else {
+                    s0[j] = s1[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kBack; ++j) {
+            const int ch = i - j;
+            if (ch >= 0) {            // uniform over the block
+                float dot = s0[j].x * d0.x + s0[j].y * d0.y + s0[j].z * d0.z + s0[j].w * d0.w +
+                            s1[j].x * d1.x + s1[j].y * d1.y + s1[j].z * d1.z + s1[j].w * d1.w;
+                D[(size_t)ch * 1024] = round4_tf32(make_float4(g[j] * d0.x, g[j] * d0.y, g[j] * d0.z, g[j] * d0.w));
+                D[(size_t)ch * 1024 + 512] = round4_tf32(make_float4(g[j] * d1.x, g[j] * d1.y, g[j] * d1.z, g[j] * d1.w));
+                d0 = fma4(g[j], d0, w0[j]);
+                d1 = fma4(g[j], d1, w1[j]);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                if ((t & 7) == 0) cr[(size_t)ch * 64] = dot;
+            }
+        }
+    }
+}
+
 }  // namespace
 
-dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s)
+dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tiles)
 {
-    const dim3 grid((g.dk * g.dv + kScanThreads - 1) / kScanThreads, g.B * g.H);
+    const dim3 grid((g.dk * g.dv / 4 + kScanThreads - 1) / kScanThreads, g.B * g.H);
+    if (tiles && (g.dk != 64 || g.dv != 64)) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_SCAN_FWD, s);
-    state_scan_fwd<<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
+    if (tiles)
+        state_scan_fwd<true><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
+    else
+        state_scan_fwd<false><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
     return cuda_ok(cudaGetLastError());
 }
 
@@ -105,6 +216,14 @@ dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t
     KernelTimer t(KID_SCAN_BWD, s);
     state_scan_bwd<<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N,
                                                        g.dk, g.dv);
+    return cuda_ok(cudaGetLastError());
+}
+
+dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s)
+{
+    if (g.dk != 64 || g.dv != 64) return DIG_ERR_UNSUPPORTED;
+    KernelTimer t(KID_SCAN_BWD, s);
+    state_scan_bwd_tiles<<<dim3(8, g.B * g.H), 64, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N);
     return cuda_ok(cudaGetLastError());
 }
 

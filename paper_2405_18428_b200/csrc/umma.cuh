@@ -37,11 +37,12 @@ __device__ __forceinline__ uint32_t tile_offset_m(int row, int col)     // M-for
                       ((col & 7) << 2));
 }
 
+// Round to tf32 (10 explicit mantissa bits), nearest with ties away from zero: what
+// cvt.rna.tf32.f32 computes for finite values, done with two integer operations because the
+// conversion instruction runs at a quarter of their rate.
 __device__ __forceinline__ float to_tf32(float x)
 {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return __uint_as_float(r);
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u);
 }
 
 // 64-bit matrix descriptor: start address, leading / stride byte offsets (all >> 4), descriptor
@@ -148,6 +149,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *s
             }
         }
     }
+}
+
+// ---- bulk asynchronous copies (TMA engine, no tensor map) ------------------------------------
+// Both addresses 16-byte aligned, size a multiple of 16 bytes.  Completion is reported to an
+// mbarrier as transferred bytes.
+__device__ __forceinline__ void bulk_g2s(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// One arrival that also announces `bytes` of pending bulk-copy traffic.
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 
 // Tensor-memory allocation: one warp allocates `cols` (power of two >= 32) columns and publishes
