@@ -83,8 +83,10 @@ struct GlaArgs {
 //   gamma   [B*H][N][dk]       exp(sum of the chunk's gates)
 //   dstates [B*H][N][dk][dv]   (backward) chunk-local Q^T dO, turned in place into dL/d(state leaving the chunk)
 //   carry   [B*H][N][dk]       (backward) gate-gradient carried in from later chunks
+//   dstates_m [B*H][N][dk][dv] (backward) second copy of the decayed state gradients, in the other
+//                              operand-tile order (used by the tensor-core family only)
 struct Workspace {
-    float *states, *gamma, *dstates, *carry;
+    float *states, *gamma, *dstates, *carry, *dstates_m;
     size_t bytes;
 };
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -101,7 +103,8 @@ inline Workspace carve_workspace(float *base, const Geom &g, bool backward)
     if (backward) {
         w.dstates = reinterpret_cast<float *>(p);       p += st;
         w.carry = reinterpret_cast<float *>(p);         p += gm;
-        w.bytes += st + gm;
+        w.dstates_m = reinterpret_cast<float *>(p);     p += st;
+        w.bytes += 2 * st + gm;
     }
     return w;
 }

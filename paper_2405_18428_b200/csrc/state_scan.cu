@@ -121,7 +121,8 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
 // the same 16-byte piece of one row in both column blocks (8 floats), so the decay index is its row
 // and the order of the pieces inside the row does not matter.  It first runs the forward
 // recurrence (states <- S_[i], rounded to tf32 for the consumer), then walks back over the chunks:
-//   dstates <- diag(gamma_i) D_[i] (rounded to tf32), carry_i = row sums of S_[i+1] * D_[i],
+//   dstates, dstates_m <- diag(gamma_i) D_[i] (rounded to tf32, in the two operand-tile orders),
+//   carry_i = row sums of S_[i+1] * D_[i],
 // reading back the S values it wrote itself.  Block = 8 rows x 8 pieces; grid (8, B*H).
 constexpr int kBack = 4;
 __device__ __forceinline__ float4 fma4(float g, float4 r, float4 u)
@@ -129,13 +130,17 @@ __device__ __forceinline__ float4 fma4(float g, float4 r, float4 u)
     return make_float4(fmaf(g, r.x, u.x), fmaf(g, r.y, u.y), fmaf(g, r.z, u.z), fmaf(g, r.w, u.w));
 }
 __global__ void __launch_bounds__(64)
-state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, const float *__restrict__ gamma,
-                     float *__restrict__ carry, int N)
+state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, float *__restrict__ dstates_m,
+                     const float *__restrict__ gamma, float *__restrict__ carry, int N)
 {
     const int t = threadIdx.x, c = 8 * blockIdx.x + (t >> 3);
     const size_t base = (size_t)blockIdx.y * N * 4096;
     float4 *S = reinterpret_cast<float4 *>(states + base) + c * 8 + (t & 7);
     float4 *D = reinterpret_cast<float4 *>(dstates + base) + c * 8 + (t & 7);
+    // The same values once more in the other tile order (32-byte pieces of a row XOR-ed with row & 3):
+    // this thread's logical columns 4*p .. 4*p+3 of both column blocks, p = piece ^ (row & 7).
+    const int lp = (t & 7) ^ (c & 7);
+    float4 *DM = reinterpret_cast<float4 *>(dstates_m + base) + c * 8 + ((((lp >> 1) ^ (c & 3)) << 1) | (lp & 1));
     const float *gm = gamma + (size_t)blockIdx.y * N * 64 + c;
     float *cr = carry + (size_t)blockIdx.y * N * 64 + c;
     float4 r0 = make_float4(0.f, 0.f, 0.f, 0.f), r1 = r0;
@@ -183,8 +188,12 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, co
             if (ch >= 0) {            // uniform over the block
                 float dot = s0[j].x * d0.x + s0[j].y * d0.y + s0[j].z * d0.z + s0[j].w * d0.w +
                             s1[j].x * d1.x + s1[j].y * d1.y + s1[j].z * d1.z + s1[j].w * d1.w;
-                D[(size_t)ch * 1024] = round4_tf32(make_float4(g[j] * d0.x, g[j] * d0.y, g[j] * d0.z, g[j] * d0.w));
-                D[(size_t)ch * 1024 + 512] = round4_tf32(make_float4(g[j] * d1.x, g[j] * d1.y, g[j] * d1.z, g[j] * d1.w));
+                const float4 e0 = round4_tf32(make_float4(g[j] * d0.x, g[j] * d0.y, g[j] * d0.z, g[j] * d0.w));
+                const float4 e1 = round4_tf32(make_float4(g[j] * d1.x, g[j] * d1.y, g[j] * d1.z, g[j] * d1.w));
+                D[(size_t)ch * 1024] = e0;
+                D[(size_t)ch * 1024 + 512] = e1;
+                DM[(size_t)ch * 1024] = e0;
+                DM[(size_t)ch * 1024 + 512] = e1;
                 d0 = fma4(g[j], d0, w0[j]);
                 d1 = fma4(g[j], d1, w1[j]);
                 dot += __shfl_xor_sync(0xffffffffu, dot, 1);
@@ -223,7 +232,7 @@ dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaSt
 {
     if (g.dk != 64 || g.dv != 64) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_SCAN_BWD, s);
-    state_scan_bwd_tiles<<<dim3(8, g.B * g.H), 64, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N);
+    state_scan_bwd_tiles<<<dim3(8, g.B * g.H), 64, 0, s>>>(w.states, w.dstates, w.dstates_m, w.gamma, w.carry, g.N);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -97,18 +97,19 @@ __device__ __forceinline__ void st_m8(char *tile, int row, int col8, const float
     float4 *p0 = reinterpret_cast<float4 *>(base), *p1 = reinterpret_cast<float4 *>(base + 16);
     if (flip) { *p1 = hi; *p0 = lo; } else { *p0 = lo; *p1 = hi; }
 }
-// 4 consecutive columns starting at col4 (a multiple of 4), rounded to tf32.
-template <int ROWS>
+// 4 consecutive columns starting at col4 (a multiple of 4), rounded to tf32 unless ROUND = false.
+template <int ROWS, bool ROUND = true>
 __device__ __forceinline__ void st_k4(char *tile, int row, int col4, float4 v)
 {
     *reinterpret_cast<float4 *>(tile + (col4 >> 5) * (ROWS * 128) + row * 128 + ((((col4 & 31) >> 2) ^ (row & 7)) << 4)) =
-        tf32x4(v.x, v.y, v.z, v.w);
+        ROUND ? tf32x4(v.x, v.y, v.z, v.w) : v;
 }
-template <int ROWS>
+template <int ROWS, bool ROUND = true>
 __device__ __forceinline__ void st_m4(char *tile, int row, int col4, float4 v)
 {
     *reinterpret_cast<float4 *>(tile + (col4 >> 5) * (ROWS * 128) + row * 128 +
-                                (((((col4 & 31) >> 3)) ^ (row & 3)) << 5) + ((col4 & 4) << 2)) = tf32x4(v.x, v.y, v.z, v.w);
+                                (((((col4 & 31) >> 3)) ^ (row & 3)) << 5) + ((col4 & 4) << 2)) =
+        ROUND ? tf32x4(v.x, v.y, v.z, v.w) : v;
 }
 // 8 consecutive columns of an M-format tile back into registers.
 template <int ROWS>
@@ -124,8 +125,9 @@ __device__ __forceinline__ void ld_m8(const char *tile, int row, int col8, float
 // the table holds raw gates) is applied while reading, so the sums are in log2 units.
 // Turns every chunk's rows into inclusive prefix sums down the rows, in place; sLast[ch*64 + c]
 // receives the last row (the chunk total).  NT threads; sTot has NT floats.
-// Ends with a __syncthreads().
-template <int NT, int NCH>
+// Ends with a barrier.
+// GROUP: the NT threads are only part of the CTA and synchronise with sync_group.
+template <int NT, int NCH, bool GROUP = false>
 __device__ __forceinline__ void gate_prefix(float *sLam, float *sLast, float *sTot, float scale = 1.f)
 {
     constexpr int NSEG = NT / 64;                 // row segments over all NCH*T rows
@@ -139,7 +141,7 @@ __device__ __forceinline__ void gate_prefix(float *sLam, float *sLast, float *sT
 #pragma unroll
     for (int j = 1; j < R; ++j) a[j] += a[j - 1];
     sTot[seg * 64 + c] = a[R - 1];
-    __syncthreads();
+    if (GROUP) sync_group(NT); else __syncthreads();
     const int first = (seg / SEG_PER_CH) * SEG_PER_CH;
     float add = 0.f;
 #pragma unroll
@@ -148,7 +150,7 @@ __device__ __forceinline__ void gate_prefix(float *sLam, float *sLast, float *sT
 #pragma unroll
     for (int j = 0; j < R; ++j) sLam[(R * seg + j) * kLamPitch + c] = a[j] + add;
     if (seg - first == SEG_PER_CH - 1) sLast[(seg / SEG_PER_CH) * 64 + c] = a[R - 1] + add;
-    __syncthreads();
+    if (GROUP) sync_group(NT); else __syncthreads();
 }
 
 // Fetches 32 gate rows (rows 32*part .. 32*part+31 of the stacked table; `it` is the item those
