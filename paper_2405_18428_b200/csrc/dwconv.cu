@@ -9,7 +9,7 @@
 namespace dig {
 namespace {
 
-constexpr int TY = 8, TX = 16, VEC = 8;
+constexpr int TY = 4, TX = 8, VEC = 8;
 // Channels per CTA: 256 bytes of one pixel, so the halo tile stays under 48 KB of shared memory.
 template <typename T> struct Cfg {
     static constexpr int CH = 256 / (int)sizeof(T);

@@ -176,11 +176,11 @@ dig_status launch_tc_state(const GlaArgs &a, const Workspace &w, bool backward, 
         kern<<<grid, NT, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                            (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, status, g);
     } else {
-        constexpr int NT = 256;
+        constexpr int NT = 512;
         auto kern = tc_state_pair<NT, false>;
         constexpr size_t smem = state_smem<NT, false>();
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
-        const int grid = npairs < 2 * sm_count ? npairs : 2 * sm_count;
+        const int grid = npairs < sm_count ? npairs : sm_count;
         KernelTimer t(KID_TC_STATE, a.stream);
         kern<<<grid, NT, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                            nullptr, w.states, w.gamma, nullptr, status, g);

@@ -13,7 +13,7 @@ namespace dig {
 namespace {
 
 constexpr int kScanThreads = 128;
-constexpr int kAhead = 8;
+constexpr int kAhead = 16;
 
 __device__ __forceinline__ float round_tf32(float x)
 {
@@ -124,7 +124,7 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
 //   dstates, dstates_m <- diag(gamma_i) D_[i] (rounded to tf32, in the two operand-tile orders),
 //   carry_i = row sums of S_[i+1] * D_[i],
 // reading back the S values it wrote itself.  Block = 8 rows x 8 pieces; grid (8, B*H).
-constexpr int kBack = 4;
+constexpr int kBack = 8;
 __device__ __forceinline__ float4 fma4(float g, float4 r, float4 u)
 {
     return make_float4(fmaf(g, r.x, u.x), fmaf(g, r.y, u.y), fmaf(g, r.z, u.z), fmaf(g, r.w, u.w));
