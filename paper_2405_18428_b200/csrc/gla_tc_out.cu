@@ -9,8 +9,10 @@
 //   inter   [Qa;Qb] [Sa^T;Sb^T]^T  -> same blocks of the output accumulator
 //   intra   [Pa;Pb] [Va | Vb]      -> accumulated on top
 // The other blocks of the accumulators hold cross terms that are never read.  While a pair is in
-// the tensor pipe the next pair's q, k, v rows are already being loaded into registers, and its gate
-// rows and incoming states arrive by bulk asynchronous copies (cp.async.bulk) in shared memory.
+// the tensor pipe the next pair's q, k, v and gate rows are already being loaded into registers, and
+// its incoming states arrive by bulk asynchronous copies (cp.async.bulk) in their operand tile.  A
+// seventeenth warp issues the MMAs and the bulk copies; results leave through a staging area with
+// coalesced 16-byte stores.
 #include "tc_tiles.cuh"
 
 namespace dig {
@@ -18,18 +20,26 @@ namespace {
 
 using namespace tc;
 
-constexpr int NT = 512;
+constexpr int NT = 512;                       // threads that build operands and post-process accumulators
+constexpr int NTA = NT + 32;                  // plus one warp that issues the MMAs and the bulk loads
 constexpr int W = 16;                          // accumulator columns per thread
 constexpr int kTileK = 128 * 64 * 4;           // 128 rows x 64 columns, K-format
 constexpr int kTileM = T * 128 * 4;            // 64 rows x 128 columns, M-format
 
 struct OutRaw {
     uint4 q[2], k[2], v[2];
+    float4 g[4];
 };
 
-__device__ __forceinline__ void load_raw(OutRaw &r, const bf16 *q, const bf16 *k, const bf16 *v, const Geom &g,
-                                         const Item (&it)[2])
+__device__ __forceinline__ void load_raw(OutRaw &r, const bf16 *q, const bf16 *k, const bf16 *v, const float *gate,
+                                         const Geom &g, const Item (&it)[2])
 {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int u = threadIdx.x + NT * i, half = u >> 10;
+        const Item ci = pick(it[0], it[1], half);
+        r.g[i] = ld_row4(gate, g, ci.b, item_token(g, ci, (u >> 4) & 63), ci.h, DK, (u & 15) * 4);
+    }
     const int row = threadIdx.x >> 3, col = (threadIdx.x & 7) * 8;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
@@ -55,7 +65,7 @@ __device__ __forceinline__ void fetch_states(char *tS, const float *states, int 
 }
 
 template <typename TO>
-__global__ void __launch_bounds__(NT)
+__global__ void __launch_bounds__(NTA)
 tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *__restrict__ v,
             const float *__restrict__ gate, const float *__restrict__ states, TO *__restrict__ out,
             int *status, Geom g)
@@ -67,13 +77,18 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
     float *sLam = reinterpret_cast<float *>(tV + kTileM);
     float *sLast = sLam + 2 * T * kLamPitch, *sTot = sLast + 128;
     Control *ctl = reinterpret_cast<Control *>(sTot + NT);
+    // results are staged over the score tile's operands (Q and K tiles) once every product has completed
+    constexpr int kOutPitch = 64 * (int)sizeof(TO) + 16;
+    static_assert(128 * kOutPitch <= 2 * kTileK, "output staging must fit in the tiles it reuses");
+    char *stage = tQ;
     constexpr uint32_t kCols = 256;
     constexpr uint32_t aP = 0, aO = 128;
-    uint64_t *barP = &ctl->bar[0], *barO = &ctl->bar[1], *barG = &ctl->bar[2], *barS = &ctl->bar[3];
-    setup(ctl, 4, kCols, 2, 4);
+    uint64_t *barP = &ctl->bar[0], *barO = &ctl->bar[1], *barS = &ctl->bar[2];
+    setup(ctl, 3, kCols);
     const uint32_t tmem = ctl->tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int R = 32 * (warp & 3) + lane, half_r = R >> 6, r = R & 63, c0 = W * (warp >> 2);
+    const bool issuer = warp == NT / 32;                      // the extra warp: MMAs and bulk loads
+    const int R = 32 * (warp & 3) + lane, half_r = R >> 6, r = R & 63, c0 = W * ((warp >> 2) & 3);
     const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
 
     const int total = g.B * g.H * g.N, npairs = (total + 1) / 2;
@@ -81,25 +96,32 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
     int pair = blockIdx.x;
     if (pair < npairs) {
         const Item it[2] = {item_of(g, 2 * pair, total), item_of(g, 2 * pair + 1, total)};
-        load_raw(raw, q, k, v, g, it);
-        if (warp >= 4 && warp < 8) fetch_gate_rows(sLam, gate, g, it[(warp - 4) >> 1], warp - 4, barG, lane);
-        if (threadIdx.x == 0) fetch_states(tS, states, pair, total, barS);
+        if (!issuer) load_raw(raw, q, k, v, gate, g, it);
+        else if (lane == 0) fetch_states(tS, states, pair, total, barS);
     }
     uint32_t parity = 0;
     bool ok = true;
+    Item cur[2] = {item_of(g, 2 * pair, total), item_of(g, 2 * pair + 1, total)};
     for (; pair < npairs; pair += gridDim.x) {
         const int next = pair + gridDim.x;
         const Item nit[2] = {item_of(g, 2 * next, total), item_of(g, 2 * next + 1, total)};
-        ok = mbar_wait(barG, parity, status);
-        if (!__syncthreads_and(ok)) break;
-        gate_prefix<NT, 2>(sLam, sLast, sTot, kLog2e);
-        {
-            const int row = threadIdx.x >> 3, j = threadIdx.x & 7, col = j * 8;
-            const bool flip = j >= 4;
+        const int row = threadIdx.x >> 3, j = threadIdx.x & 7, col = j * 8;
+        const bool flip = j >= 4;
+        if (!issuer) {
+            sync_group(NT);          // the previous pair's results have left the staging area
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int u = threadIdx.x + NT * i, grow = (u >> 4) & 127;
+                const Item ci = pick(cur[0], cur[1], grow >> 6);
+                const float sc = (ci.valid && ci.chunk * T + (grow & 63) < g.L) ? kLog2e : 0.f;
+                *reinterpret_cast<float4 *>(sLam + grow * kLamPitch + (u & 15) * 4) =
+                    make_float4(raw.g[i].x * sc, raw.g[i].y * sc, raw.g[i].z * sc, raw.g[i].w * sc);
+            }
+            sync_group(NT);
+            gate_prefix<NT, 2, true>(sLam, sLast, sTot);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                const int id = 2 * pair + half;
-                const bool keep = id < total && (id % g.N) * T + row < g.L;
+                const bool keep = cur[half].valid && cur[half].chunk * T + row < g.L;
                 float lam[8], x[8];
                 read_lam8(sLam, 64 * half + row, col, lam);
                 unpack8(raw.q[half], x, keep);
@@ -113,62 +135,74 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
                 unpack8(raw.v[half], x, keep);
                 st_m8<T, false>(tV, row, 64 * half + col, x, flip);
             }
+            fence_async_smem();
         }
-        fence_async_smem();
         tc_fence_before_sync();
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            if (mbar_wait(barS, parity, status)) {
+        if (!__syncthreads_and(ok)) break;
+        if (issuer) {
+            if (lane == 0) {
+                ok = mbar_wait(barS, parity, status);
                 tc_fence_after_sync();
                 issue<128, 128, false, false, 128, 128>(tmem + aP, kdesc<128>(tQ), kdesc<128>(tK), false);     // scores
                 mma_commit(barP);
                 issue<128, 128, false, false, 128, 128>(tmem + aO, kdesc<128>(tQ), kdesc<128>(tS), false);     // Qt S
             }
-        }
-        if (next < npairs) {
-            if (warp >= 4 && warp < 8) fetch_gate_rows(sLam, gate, g, nit[(warp - 4) >> 1], warp - 4, barG, lane);   // the gate table is free again
-            load_raw(raw, q, k, v, g, nit);
-        }
-        ok = mbar_wait(barP, parity, status);
-        if (ok) {
-            tc_fence_after_sync();
-            float p[W];
-            tmem_ld(tmem + lane_base + aP + (uint32_t)(64 * half_r + c0), p);
+        } else {
+            ok = mbar_wait(barP, parity, status);
+            if (ok) {
+                tc_fence_after_sync();
+                float p[W];
+                tmem_ld(tmem + lane_base + aP + (uint32_t)(64 * half_r + c0), p);
 #pragma unroll
-            for (int j = 0; j < W; ++j)
-                if (c0 + j > r) p[j] = 0.f;                   // keep s <= t; the diagonal has weight 1
+                for (int jj = 0; jj < W; ++jj)
+                    if (c0 + jj > r) p[jj] = 0.f;                   // keep s <= t; the diagonal has weight 1
 #pragma unroll
-            for (int j = 0; j < W / 4; ++j)
-                st_k4<128>(tP, R, c0 + 4 * j, make_float4(p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]));
-        }
-        fence_async_smem();
-        tc_fence_before_sync();
-        ok = __syncthreads_and(ok);
-        if (!ok) break;
-        if (threadIdx.x == 0) {
-            tc_fence_after_sync();
-            issue<128, 128, false, true, 128, T>(tmem + aO, kdesc<128>(tP), mdesc<T>(tV), true);           // + P V
-            mma_commit(barO);
-        }
-        ok = mbar_wait(barO, parity, status);
-        parity ^= 1;
-        if (ok) {
-            tc_fence_after_sync();
-            if (threadIdx.x == 0 && next < npairs) fetch_states(tS, states, next, total, barS);           // S^T tile is free again
-            float o[W];
-            tmem_ld(tmem + lane_base + aO + (uint32_t)(64 * half_r + c0), o);
-            const Item it = item_of(g, 2 * pair + half_r, total);
-            const int tok = item_token(g, it, r);
-            if (tok >= 0) store16(out + tok_offset(g, it.b, tok, it.h, DV) + c0, o);
+                for (int jj = 0; jj < W / 4; ++jj)
+                    st_k4<128>(tP, R, c0 + 4 * jj, make_float4(p[4 * jj], p[4 * jj + 1], p[4 * jj + 2], p[4 * jj + 3]));
+            }
+            fence_async_smem();
         }
         tc_fence_before_sync();
         if (!__syncthreads_and(ok)) break;
-        tc_fence_after_sync();
+        if (issuer) {
+            if (lane == 0) {
+                tc_fence_after_sync();
+                issue<128, 128, false, true, 128, T>(tmem + aO, kdesc<128>(tP), mdesc<T>(tV), true);           // + P V
+                mma_commit(barO);
+                // once everything has completed the state tile is free for the next pair
+                if (mbar_wait(barO, parity, status) && next < npairs) fetch_states(tS, states, next, total, barS);
+            }
+        } else {
+            // the tensor pipe is busy for a while: a good moment to start the next pair's loads
+            if (next < npairs) load_raw(raw, q, k, v, gate, g, nit);
+            ok = mbar_wait(barO, parity, status);
+            if (ok) {
+                tc_fence_after_sync();
+                float o[W];
+                tmem_ld(tmem + lane_base + aO + (uint32_t)(64 * half_r + c0), o);
+                store16(reinterpret_cast<TO *>(stage + R * kOutPitch) + c0, o);
+            }
+            tc_fence_before_sync();
+            sync_group(NT);
+            if (ok) {
+                // coalesced stores of the staged rows: 16 bytes per thread
+                constexpr int PER_ROW = 64 * (int)sizeof(TO) / 16;
+#pragma unroll
+                for (int i = 0; i < PER_ROW / 4; ++i) {
+                    const int u = threadIdx.x + NT * i, rr = u / PER_ROW, piece = u % PER_ROW;
+                    const Item it = pick(cur[0], cur[1], rr >> 6);
+                    const int tr = item_token(g, it, rr & 63);
+                    if (tr >= 0)
+                        *reinterpret_cast<uint4 *>(reinterpret_cast<char *>(out) + tok_offset(g, it.b, tr, it.h, DV) * sizeof(TO) + piece * 16) =
+                            *reinterpret_cast<const uint4 *>(stage + rr * kOutPitch + piece * 16);
+                }
+            }
+        }
+        parity ^= 1;
+        cur[0] = nit[0];
+        cur[1] = nit[1];
     }
-    if (!ok) {      // a wait gave up: let bulk copies still in flight land before the CTA's memory goes away
-        mbar_wait(barG, parity, status);
-        mbar_wait(barS, parity, status);
-    }
+    if (!ok) mbar_wait(barS, parity, status);      // let a state copy still in flight land before the CTA's memory goes away
     teardown(ctl, kCols);
 }
 
@@ -187,7 +221,7 @@ dig_status launch_typed(const GlaArgs &a, const Workspace &w, int sm_count, int 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
     const int grid = npairs < sm_count ? npairs : sm_count;
     KernelTimer t(KID_TC_OUT, a.stream);
-    kern<<<grid, NT, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate, w.states,
+    kern<<<grid, NTA, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate, w.states,
                                        (TO *)a.out, status, g);
     return cuda_ok(cudaGetLastError());
 }

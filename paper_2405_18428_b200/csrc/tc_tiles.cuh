@@ -39,6 +39,16 @@ __device__ __forceinline__ Item item_of(const Geom &g, int id, int total)
     it.h = bh - it.b * g.H;
     return it;
 }
+// One of two items without indexing an array (keeps both in registers).
+__device__ __forceinline__ Item pick(const Item &a, const Item &b, bool second)
+{
+    Item it;
+    it.b = second ? b.b : a.b;
+    it.h = second ? b.h : a.h;
+    it.chunk = second ? b.chunk : a.chunk;
+    it.valid = second ? b.valid : a.valid;
+    return it;
+}
 // Canonical token of tile row r of the item, or -1 for rows past the end of the sequence.
 __device__ __forceinline__ int item_token(const Geom &g, const Item &it, int r)
 {
