@@ -186,6 +186,45 @@ def time_steps(blocks, dig, torch, steps, warmup, dist, e2e=False, before_timed=
     return ms
 
 
+def time_graph_steps(blocks, dig, torch, steps, warmup, dist):
+    """The same K steps as time_steps, with one step captured in a CUDA graph and replayed (the
+    kernels and their order are unchanged; only the host-side launch cost goes away).  Returns None
+    if the capture fails."""
+    try:
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            for b in blocks:
+                b.run(dig)          # first calls outside the capture (per-kernel attribute set-up)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                for b in blocks:
+                    b.run(dig)
+        torch.cuda.synchronize()
+    except Exception:
+        return None
+    for _ in range(warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        graph.replay()
+    t1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ms = t0.elapsed_time(t1)
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
 def cpu_baseline(wl, budget_s=20.0):
     """The fp64 oracle, as it stands, on a bounded sample of the workload: whole (batch, head)
     pairs of the first scan direction, all host cores, gate + fwd + bwd (+ conv on those batches)."""
@@ -198,19 +237,27 @@ def cpu_baseline(wl, budget_s=20.0):
     nb = max(1, min(wl.B, pairs_budget // wl.H))
     sub = wl.scaled(B=nb)
     x = make_inputs(sub)
-    d = wl.directions[0]
+    # whole steps of the sample (every scan direction of the workload), repeated until about half the
+    # budget is spent, so that the timing is not dominated by start-up effects
     t0 = time.perf_counter()
-    a = oracle.gate(x["g"], x["tau"])
-    oracle.gla_fwd(x["q"], x["k"], x["v"], a, sub.grid_h, sub.grid_w, d, threads=cores)
-    if wl.backward:
-        oracle.gla_bwd(x["q"], x["k"], x["v"], a, x["dO"], sub.grid_h, sub.grid_w, d, threads=cores)
-    if wl.conv:
-        oracle.dwconv(x["conv_x"], x["conv_w"], None, sub.grid_h, sub.grid_w, d)
+    passes = 0
+    while True:
+        for d in wl.directions:
+            a = oracle.gate(x["g"], x["tau"])
+            oracle.gla_fwd(x["q"], x["k"], x["v"], a, sub.grid_h, sub.grid_w, d, threads=cores)
+            if wl.backward:
+                oracle.gla_bwd(x["q"], x["k"], x["v"], a, x["dO"], sub.grid_h, sub.grid_w, d, threads=cores)
+            if wl.conv:
+                oracle.dwconv(x["conv_x"], x["conv_w"], None, sub.grid_h, sub.grid_w, d)
+        passes += 1
+        if time.perf_counter() - t0 >= 0.5 * budget_s:
+            break
     dt = time.perf_counter() - t0
-    tokens = nb * wl.L
+    tokens = nb * wl.L * len(wl.directions) * passes
     return {"value": tokens / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{nb} of {wl.B} batches x {wl.H} heads, direction {d} of {list(wl.directions)}, "
-                      f"gate+fwd{'+bwd' if wl.backward else ''}{'+conv' if wl.conv else ''}, {dt:.2f} s"}, dt, tokens
+            "sample": f"{nb} of {wl.B} batches x {wl.H} heads, directions {list(wl.directions)}, "
+                      f"gate+fwd{'+bwd' if wl.backward else ''}{'+conv' if wl.conv else ''}, "
+                      f"{passes} passes, {dt:.2f} s wall on {cores} threads"}, dt, tokens
 
 
 def run_reference(args, wl):
@@ -247,7 +294,8 @@ def main():
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--family", default="auto", choices=["auto", "fma", "tensor"])
-    ap.add_argument("--no-sweep", action="store_true", help="skip the short tokens/s-vs-L sweep over C3, C4, C5")
+    ap.add_argument("--eager", action="store_true", help="time plain stream launches instead of one CUDA graph per step")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short tokens/s-vs-L sweep over C3, C4 (chunk 64 and 32), C5")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     args = ap.parse_args()
 
@@ -280,13 +328,18 @@ def main():
     tokens_per_step = wl.B * wl.L * len(blocks)
     th_per_block = wl.B * wl.L * wl.H
 
+    # headline: K steps, kernels launched back to back (one CUDA graph per step unless --eager)
     sampler = ClockSampler(local)
-    def before_timed():
-        dig.dig_profile_enable(True)
+    ms_eager = time_steps(blocks, dig, torch, args.steps, W, dist, before_timed=None if not args.eager else sampler.start)
+    ms_graph = None
+    if not args.eager:
         sampler.start()
-
-    ms = time_steps(blocks, dig, torch, args.steps, W, dist, before_timed=before_timed)
+        ms_graph = time_graph_steps(blocks, dig, torch, args.steps, W, dist)
     clocks = sampler.stop()
+    ms = ms_graph if ms_graph is not None else ms_eager
+    launch_mode = "cuda_graph" if ms_graph is not None else "eager"
+    # per-kernel times: the same K steps once more with every launch bracketed by two CUDA events
+    ms_events = time_steps(blocks, dig, torch, args.steps, W, dist, before_timed=lambda: dig.dig_profile_enable(True))
     prof = dig.dig_profile_read()
     dig.dig_profile_enable(False)
     assert dig.dig_last_device_status() == dig.DIG_OK
@@ -327,8 +380,10 @@ def main():
     if not args.no_sweep and rank == 0 and world == 1:
         del blocks
         torch.cuda.empty_cache()
-        for name in ("C3", "C4", "C5"):
-            w2 = CONFIGS[name].scaled(directions=(CONFIGS[name].directions[0],), conv=False)
+        cases = [("C3", {}), ("C4", {}), ("C4_chunk32", {"chunk": 32}), ("C5", {})]
+        for name, over in cases:
+            base_wl = CONFIGS[name.split("_")[0]]
+            w2 = base_wl.scaled(directions=(base_wl.directions[0],), conv=False, **over)
             bl = make_blocks(w2, torch, dig)
             big = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
             best = None
@@ -339,12 +394,16 @@ def main():
             a2, e2 = flops_per_token_head(w2, w2.chunk)
             fb, bb = bytes_per_token_head(w2)
             th = w2.B * w2.L * w2.H
+            fam = dig.dig_gla_query_impl(w2.d_k, w2.d_v, w2.chunk, dig.DIG_BF16, 1)
             sweep[name] = {"L": w2.L, "B": w2.B, "H": w2.H, "d": w2.d_k, "chunk": w2.chunk, "ms": best,
+                           "kernel_family": {1: "fma", 2: "tensor"}.get(fam, str(fam)),
                            "tokens_per_s": w2.B * w2.L / (best * 1e-3),
                            "tflops_alg": a2 * th / (best * 1e-3) / 1e12, "tflops_exec": e2 * th / (best * 1e-3) / 1e12,
                            "hbm_frac_of_measured": (fb + bb) * th / (best * 1e-3) / 1e9 / peaks["hbm_gbs"]}
             del bl, big
             torch.cuda.empty_cache()
+        sweep["note"] = ("gate + fwd + bwd of one block, first scan direction, L2 flushed before each timing, best of 5; "
+                         "chunk 128 is left out: no kernel family runs its backward pass")
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -358,6 +417,8 @@ def main():
             "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "grid": [wl.grid_h, wl.grid_w], "L": wl.L,
                        "d_k": wl.d_k, "d_v": wl.d_v, "chunk": wl.chunk, "storage": wl.dtype,
                        "directions": list(wl.directions), "conv": wl.conv, "blocks_per_step": len(wl.directions),
+                       "launch": launch_mode, "ms_per_step_eager": ms_eager / args.steps,
+                       "ms_per_step_with_kernel_events": ms_events / args.steps,
                        "kernel_family": {1: "fma", 2: "tensor"}.get(impl, str(impl)),
                        "l2": "each block has its own buffers; a step streams several times the 126 MB L2, no flush needed",
                        "tflops_alg": tflops_alg, "tflops_exec": tflops_exe,
