@@ -26,6 +26,10 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu capture summarised
+# in profiles/; only valid for the kernel as it stood when the capture was taken (reset to None on change).
+NCU_TRAFFIC = {("C2", "tc_chunk_bwd"): 79.9e6}
+
 METRIC = "gla_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -368,7 +372,8 @@ def main():
     if dom in alg_bytes:
         achieved = alg_bytes[dom] * th_per_block / (t_dom / n_dom * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get((wl.name, dom)),
+                    "peak_source": peaks["source"],
                     "algorithmic_bytes_per_launch": alg_bytes[dom] * th_per_block}
     alg_f, exe_f = flops_per_token_head(wl, wl.chunk)
     step_s = ms * 1e-3 / args.steps
