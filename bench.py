@@ -163,6 +163,21 @@ def make_blocks(wl, torch, dig):
     return blocks
 
 
+def max_over_ranks(ms, dist, device="cuda"):
+    """Step time of the job = the slowest rank's (ranks run independent replicas of the workload)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(tokens_per_step_per_rank, steps, world, ms):
+    """Whole-job throughput: every rank processes its own copy of the workload (weak scaling)."""
+    return tokens_per_step_per_rank * steps * world / (ms * 1e-3)
+
+
 def time_steps(blocks, dig, torch, steps, warmup, dist, e2e=False, before_timed=None):
     for _ in range(warmup):
         for b in blocks:
@@ -182,12 +197,7 @@ def time_steps(blocks, dig, torch, steps, warmup, dist, e2e=False, before_timed=
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
-    ms = t0.elapsed_time(t1)
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return ms
+    return max_over_ranks(t0.elapsed_time(t1), dist)
 
 
 def time_graph_steps(blocks, dig, torch, steps, warmup, dist):
@@ -221,12 +231,7 @@ def time_graph_steps(blocks, dig, torch, steps, warmup, dist):
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
-    ms = t0.elapsed_time(t1)
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return ms
+    return max_over_ranks(t0.elapsed_time(t1), dist)
 
 
 def cpu_baseline(wl, budget_s=20.0):
@@ -348,7 +353,7 @@ def main():
     dig.dig_profile_enable(False)
     assert dig.dig_last_device_status() == dig.DIG_OK
     launches = sum(n for n, _ in prof.values())
-    value = tokens_per_step * args.steps * world / (ms * 1e-3)
+    value = job_tokens_per_s(tokens_per_step, args.steps, world, ms)
 
     # end-to-end: pinned host -> device copies of every input, the same calls, device -> host of every result
     h2d = d2h = 0
@@ -358,7 +363,7 @@ def main():
         d2h += o
     e2e_steps = max(3, min(args.steps, 20))
     ms_e2e = time_steps(blocks, dig, torch, e2e_steps, 3, dist, e2e=True)
-    e2e_value = tokens_per_step * e2e_steps * world / (ms_e2e * 1e-3)
+    e2e_value = job_tokens_per_s(tokens_per_step, e2e_steps, world, ms_e2e)
 
     # roofline of the dominant kernel (largest share of device time), from the live event timings
     fwd_b, bwd_b = bytes_per_token_head(wl)
