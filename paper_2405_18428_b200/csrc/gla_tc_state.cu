@@ -11,7 +11,8 @@
 // instruction costs the same ~60 cycles whether it is 64 or 128 wide) yields both chunks' products
 // on the diagonal blocks of a 128 x 128 accumulator; the off-diagonal blocks are never read.
 // CTAs are persistent and prefetch the next pair's rows into registers while the current pair is in
-// the tensor pipe.
+// the tensor pipe.  Results are staged in shared memory in tile order and leave as one 16 KB bulk
+// copy (cp.async.bulk) per chunk and matrix.
 #include "tc_tiles.cuh"
 
 namespace dig {
@@ -23,46 +24,53 @@ constexpr int kPairTile = T * 128 * 4;        // bytes of one 64 x 128 M-format 
 
 template <int NT, bool BWD>
 struct StateRaw {
-    static constexpr int NROW = 1024 / NT;    // 16-byte row pieces per tensor per thread (both chunks)
-    static constexpr int NG = 2048 / NT;      // float4 gate pieces per thread (both chunks)
+    static constexpr int NROW = 1024 / NT;    // (row, 8-column) pieces per thread over both chunks
     uint4 k[NROW], v[NROW], q[BWD ? NROW : 1], d[BWD ? NROW : 1];
-    float4 g[NG];
+    float4 g0[NROW], g1[NROW];                // the gates of the same 8 columns
 };
+
+// Piece i of this thread: chunk half, token row and first column (8 lanes cover one 128-byte bf16 row).
+template <int NT>
+__device__ __forceinline__ void piece_of(int i, int &half, int &row, int &col)
+{
+    const int u = threadIdx.x + NT * i;
+    half = u >> 9; row = (u >> 3) & 63; col = (u & 7) * 8;
+}
 
 template <int NT, bool BWD>
 __device__ __forceinline__ void load_raw(StateRaw<NT, BWD> &r, const bf16 *q, const bf16 *k, const bf16 *v,
-                                         const bf16 *d_out, const float *gate, const Geom &g, int pair, int total)
+                                         const bf16 *d_out, const float *gate, const Geom &g, const Item &ia, const Item &ib)
 {
-    const Item it[2] = {item_of(g, 2 * pair, total), item_of(g, 2 * pair + 1, total)};
 #pragma unroll
     for (int i = 0; i < StateRaw<NT, BWD>::NROW; ++i) {
-        const int u = threadIdx.x + NT * i, half = u >> 9, row = (u >> 3) & 63, col = (u & 7) * 8;
-        const int tok = item_token(g, it[half], row);
-        r.k[i] = ld_row8(k, g, it[half].b, tok, it[half].h, DK, col);
-        r.v[i] = ld_row8(v, g, it[half].b, tok, it[half].h, DV, col);
+        int half, row, col;
+        piece_of<NT>(i, half, row, col);
+        const size_t off = row_offset(g, pick(ia, ib, half), row) + col;
+        r.k[i] = ldg16(k + off);
+        r.v[i] = ldg16(v + off);
         if (BWD) {
-            r.q[i] = ld_row8(q, g, it[half].b, tok, it[half].h, DK, col);
-            r.d[i] = ld_row8(d_out, g, it[half].b, tok, it[half].h, DV, col);
+            r.q[i] = ldg16(q + off);
+            r.d[i] = ldg16(d_out + off);
         }
-    }
-#pragma unroll
-    for (int i = 0; i < StateRaw<NT, BWD>::NG; ++i) {
-        const int u = threadIdx.x + NT * i, half = u >> 10, row = (u >> 4) & 63, col = (u & 15) * 4;
-        const int tok = item_token(g, it[half], row);
-        r.g[i] = ld_row4(gate, g, it[half].b, tok, it[half].h, DK, col);
+        r.g0[i] = ldg16(gate + off);
+        r.g1[i] = ldg16(gate + off + 4);
     }
 }
 
 template <int NT, bool BWD>
-__global__ void __launch_bounds__(NT)
+__global__ void __launch_bounds__(NT, BWD ? 1 : 2)
 tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *__restrict__ v,
               const float *__restrict__ gate, const bf16 *__restrict__ d_out, float *__restrict__ states,
               float *__restrict__ gamma, float *__restrict__ dstates, int *status, Geom g)
 {
     constexpr int W = 64 / (NT / 128);        // accumulator columns per thread
+    constexpr int NROW = StateRaw<NT, BWD>::NROW;
     extern __shared__ char smem_raw[];
     char *base = align1024(smem_raw);
     char *tKh = base, *tV = base + kPairTile, *tQ = base + 2 * kPairTile, *tG = base + 3 * kPairTile;
+    // once the products have completed, their operand tiles stage the results: chunk a / b of U in
+    // the two halves of the first tile, of W in the second
+    char *stage = base;
     float *sLam = reinterpret_cast<float *>(base + (BWD ? 4 : 2) * kPairTile);
     float *sLast = sLam + 2 * T * kLamPitch, *sTot = sLast + 128;
     Control *ctl = reinterpret_cast<Control *>(sTot + NT);
@@ -75,17 +83,25 @@ tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16
     const int total = g.B * g.H * g.N, npairs = (total + 1) / 2;
     StateRaw<NT, BWD> raw;
     int pair = blockIdx.x;
-    if (pair < npairs) load_raw<NT, BWD>(raw, q, k, v, d_out, gate, g, pair, total);
+    Item ca = item_of(g, 2 * pair, total), cb = item_of(g, 2 * pair + 1, total);
+    if (pair < npairs) load_raw<NT, BWD>(raw, q, k, v, d_out, gate, g, ca, cb);
     uint32_t parity = 0;
     for (; pair < npairs; pair += gridDim.x) {
+        const int next = pair + gridDim.x;
+        const Item na = item_of(g, 2 * next, total), nb = item_of(g, 2 * next + 1, total);
+        // the previous pair's staged states have been read by the bulk stores
+        if (threadIdx.x == 0) bulk_wait_read();
+        __syncthreads();
         // gates -> shared memory (log2 units, zero for rows past the end), prefix sums down each chunk
 #pragma unroll
-        for (int i = 0; i < StateRaw<NT, BWD>::NG; ++i) {
-            const int u = threadIdx.x + NT * i, row = (u >> 4) & 127, col = (u & 15) * 4;
-            const int id = 2 * pair + (row >> 6);
-            const float sc = (id < total && (id % g.N) * T + (row & 63) < g.L) ? kLog2e : 0.f;
-            const float4 a = raw.g[i];
-            *reinterpret_cast<float4 *>(sLam + row * kLamPitch + col) = make_float4(a.x * sc, a.y * sc, a.z * sc, a.w * sc);
+        for (int i = 0; i < NROW; ++i) {
+            int half, row, col;
+            piece_of<NT>(i, half, row, col);
+            const Item ci = pick(ca, cb, half);
+            const float sc = (ci.valid && ci.chunk * T + row < g.L) ? kLog2e : 0.f;
+            float *dst = sLam + (64 * half + row) * kLamPitch + col;
+            *reinterpret_cast<float4 *>(dst) = make_float4(raw.g0[i].x * sc, raw.g0[i].y * sc, raw.g0[i].z * sc, raw.g0[i].w * sc);
+            *reinterpret_cast<float4 *>(dst + 4) = make_float4(raw.g1[i].x * sc, raw.g1[i].y * sc, raw.g1[i].z * sc, raw.g1[i].w * sc);
         }
         __syncthreads();
         gate_prefix<NT, 2>(sLam, sLast, sTot);
@@ -95,11 +111,12 @@ tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16
         }
         // operands
 #pragma unroll
-        for (int i = 0; i < StateRaw<NT, BWD>::NROW; ++i) {
-            const int u = threadIdx.x + NT * i, half = u >> 9, row = (u >> 3) & 63, j = u & 7, col = j * 8;
-            const bool flip = j >= 4;
-            const int id = 2 * pair + half;
-            const bool keep = id < total && (id % g.N) * T + row < g.L;
+        for (int i = 0; i < NROW; ++i) {
+            int half, row, col;
+            piece_of<NT>(i, half, row, col);
+            const bool flip = col >= 32;
+            const Item ci = pick(ca, cb, half);
+            const bool keep = ci.valid && ci.chunk * T + row < g.L;
             float lam[8], x[8];
             read_lam8(sLam, 64 * half + row, col, lam);
             unpack8(raw.k[i], x, keep);
@@ -130,25 +147,38 @@ tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16
             }
             mma_commit(&ctl->bar[0]);
         }
-        const int next = pair + gridDim.x;
-        if (next < npairs) load_raw<NT, BWD>(raw, q, k, v, d_out, gate, g, next, total);
+        if (next < npairs) load_raw<NT, BWD>(raw, q, k, v, d_out, gate, g, na, nb);
         const bool ok = mbar_wait(&ctl->bar[0], parity, status);
         parity ^= 1;
         if (ok) {
+            // accumulators -> staging, in the tile order the workspace keeps (the layout of store_swizzled)
             tc_fence_after_sync();
-            const int id = 2 * pair + half_r;
             float acc[W];
             tmem_ld(tmem + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(64 * half_r + c0), acc);
-            if (id < total) store_swizzled(states + (size_t)id * (DK * DV), r, c0, acc);
+            store_swizzled(reinterpret_cast<float *>(stage + half_r * (DK * DV * 4)), r, c0, acc);
             if (BWD) {
                 tmem_ld(tmem + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(128 + 64 * half_r + c0), acc);
-                if (id < total) store_swizzled(dstates + (size_t)id * (DK * DV), r, c0, acc);
+                store_swizzled(reinterpret_cast<float *>(stage + kPairTile + half_r * (DK * DV * 4)), r, c0, acc);
             }
         }
+        fence_async_smem();
         tc_fence_before_sync();
         if (!__syncthreads_and(ok)) break;       // a wait gave up: every thread leaves together
         tc_fence_after_sync();
+        if (threadIdx.x == 0) {
+            // one 16 KB bulk store per chunk and matrix
+            for (int half = 0; half < 2; ++half) {
+                const int id = 2 * pair + half;
+                if (id >= total) break;
+                bulk_s2g(states + (size_t)id * (DK * DV), stage + half * (DK * DV * 4), DK * DV * 4);
+                if (BWD) bulk_s2g(dstates + (size_t)id * (DK * DV), stage + kPairTile + half * (DK * DV * 4), DK * DV * 4);
+            }
+            bulk_commit();
+        }
+        ca = na;
+        cb = nb;
     }
+    if (threadIdx.x == 0) bulk_wait_all();
     teardown(ctl, kCols);
 }
 
@@ -176,11 +206,11 @@ dig_status launch_tc_state(const GlaArgs &a, const Workspace &w, bool backward, 
         kern<<<grid, NT, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                            (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, status, g);
     } else {
-        constexpr int NT = 512;
+        constexpr int NT = 256;           // 100 KB of shared memory: two CTAs per SM overlap each other's phases
         auto kern = tc_state_pair<NT, false>;
         constexpr size_t smem = state_smem<NT, false>();
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
-        const int grid = npairs < sm_count ? npairs : sm_count;
+        const int grid = npairs < 2 * sm_count ? npairs : 2 * sm_count;
         KernelTimer t(KID_TC_STATE, a.stream);
         kern<<<grid, NT, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                            nullptr, w.states, w.gamma, nullptr, status, g);

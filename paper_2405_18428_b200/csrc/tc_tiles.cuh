@@ -56,6 +56,16 @@ __device__ __forceinline__ int item_token(const Geom &g, const Item &it, int r)
     return (it.valid && p < g.L) ? scan_token(p, g.dir, g.gh, g.gw, g.L) : -1;
 }
 
+// Element offset of tile row r of the item in a [B][L][H][64] tensor; rows past the end of the
+// sequence map to token 0 (loads stay unconditional, the consumer zeroes the values).
+__device__ __forceinline__ size_t row_offset(const Geom &g, const Item &it, int r)
+{
+    const int tok = item_token(g, it, r);
+    return tok_offset(g, it.b, tok < 0 ? 0 : tok, it.h, 64);
+}
+__device__ __forceinline__ uint4 ldg16(const bf16 *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }
+__device__ __forceinline__ float4 ldg16(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+
 // 8 consecutive bf16 / 4 consecutive floats of a token row.  The load is unconditional so that it
 // can stay in flight across a loop iteration: for tok < 0 (a row past the end of the sequence)
 // token 0 is read instead and the consumer zeroes the values.
