@@ -37,17 +37,15 @@ struct BwdRaw {
 __device__ __forceinline__ void load_raw(BwdRaw &r, const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *d_out,
                                          const float *gate, const Geom &g, const Item &it)
 {
+    // 8 lanes cover one 128-byte bf16 row; the same lanes take the 8 gates of their columns
     const int row = threadIdx.x >> 3, col = (threadIdx.x & 7) * 8;
-    const int tok = item_token(g, it, row);
-    r.q = ld_row8(q, g, it.b, tok, it.h, DK, col);
-    r.k = ld_row8(k, g, it.b, tok, it.h, DK, col);
-    r.v = ld_row8(v, g, it.b, tok, it.h, DV, col);
-    r.d = ld_row8(d_out, g, it.b, tok, it.h, DV, col);
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int u = threadIdx.x + NT * i;
-        r.gt[i] = ld_row4(gate, g, it.b, item_token(g, it, u >> 4), it.h, DK, (u & 15) * 4);
-    }
+    const size_t off = row_offset(g, it, row) + col;
+    r.q = ldg16(q + off);
+    r.k = ldg16(k + off);
+    r.v = ldg16(v + off);
+    r.d = ldg16(d_out + off);
+    r.gt[0] = ldg16(gate + off);
+    r.gt[1] = ldg16(gate + off + 4);
 }
 
 // State entering the chunk, and the decayed state gradient leaving it in both tile orders:
@@ -141,12 +139,11 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
                 issue<64, 64, false, false, T, T>(tmem + aP + kUpper, kdesc<T>(tGk), kdesc<T>(tVk), false);     // dO V^T
             }
         } else {
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const int u = threadIdx.x + NT * i, grow = u >> 4;
-                const float sc = it.chunk * T + grow < g.L ? kLog2e : 0.f;
-                *reinterpret_cast<float4 *>(sLam + grow * kLamPitch + (u & 15) * 4) =
-                    make_float4(raw.gt[i].x * sc, raw.gt[i].y * sc, raw.gt[i].z * sc, raw.gt[i].w * sc);
+            {
+                const float sc = keep ? kLog2e : 0.f;
+                float *dst = sLam + row * kLamPitch + col;
+                *reinterpret_cast<float4 *>(dst) = make_float4(raw.gt[0].x * sc, raw.gt[0].y * sc, raw.gt[0].z * sc, raw.gt[0].w * sc);
+                *reinterpret_cast<float4 *>(dst + 4) = make_float4(raw.gt[1].x * sc, raw.gt[1].y * sc, raw.gt[1].z * sc, raw.gt[1].w * sc);
             }
             sync_group(NT);
             gate_prefix<NT, 1, true>(sLam, sLast, sTot);

@@ -28,25 +28,22 @@ constexpr int kTileM = T * 128 * 4;            // 64 rows x 128 columns, M-forma
 
 struct OutRaw {
     uint4 q[2], k[2], v[2];
-    float4 g[4];
+    float4 g0[2], g1[2];
 };
 
+// 8 lanes cover one 128-byte bf16 row; the same lanes take the 8 gates of their columns.
 __device__ __forceinline__ void load_raw(OutRaw &r, const bf16 *q, const bf16 *k, const bf16 *v, const float *gate,
                                          const Geom &g, const Item (&it)[2])
 {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int u = threadIdx.x + NT * i, half = u >> 10;
-        const Item ci = pick(it[0], it[1], half);
-        r.g[i] = ld_row4(gate, g, ci.b, item_token(g, ci, (u >> 4) & 63), ci.h, DK, (u & 15) * 4);
-    }
     const int row = threadIdx.x >> 3, col = (threadIdx.x & 7) * 8;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
-        const int tok = item_token(g, it[half], row);
-        r.q[half] = ld_row8(q, g, it[half].b, tok, it[half].h, DK, col);
-        r.k[half] = ld_row8(k, g, it[half].b, tok, it[half].h, DK, col);
-        r.v[half] = ld_row8(v, g, it[half].b, tok, it[half].h, DV, col);
+        const size_t off = row_offset(g, it[half], row) + col;
+        r.q[half] = ldg16(q + off);
+        r.k[half] = ldg16(k + off);
+        r.v[half] = ldg16(v + off);
+        r.g0[half] = ldg16(gate + off);
+        r.g1[half] = ldg16(gate + off + 4);
     }
 }
 
@@ -110,12 +107,13 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
         if (!issuer) {
             sync_group(NT);          // the previous pair's results have left the staging area
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int u = threadIdx.x + NT * i, grow = (u >> 4) & 127;
-                const Item ci = pick(cur[0], cur[1], grow >> 6);
-                const float sc = (ci.valid && ci.chunk * T + (grow & 63) < g.L) ? kLog2e : 0.f;
-                *reinterpret_cast<float4 *>(sLam + grow * kLamPitch + (u & 15) * 4) =
-                    make_float4(raw.g[i].x * sc, raw.g[i].y * sc, raw.g[i].z * sc, raw.g[i].w * sc);
+            for (int half = 0; half < 2; ++half) {
+                const float sc = (cur[half].valid && cur[half].chunk * T + row < g.L) ? kLog2e : 0.f;
+                float *dst = sLam + (64 * half + row) * kLamPitch + col;
+                *reinterpret_cast<float4 *>(dst) =
+                    make_float4(raw.g0[half].x * sc, raw.g0[half].y * sc, raw.g0[half].z * sc, raw.g0[half].w * sc);
+                *reinterpret_cast<float4 *>(dst + 4) =
+                    make_float4(raw.g1[half].x * sc, raw.g1[half].y * sc, raw.g1[half].z * sc, raw.g1[half].w * sc);
             }
             sync_group(NT);
             gate_prefix<NT, 2, true>(sLam, sLast, sTot);
