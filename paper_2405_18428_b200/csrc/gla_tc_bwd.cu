@@ -97,8 +97,8 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
     const int total = g.B * g.H * g.N;
     BwdRaw raw;
     int id = blockIdx.x;
+    Item it = item_of(g, id, total);
     if (id < total) {
-        const Item it = item_of(g, id, total);
         if (issuer) {
             if (lane == 0) fetch_states(tSk, tDk, tDm, states, dstates, dstates_m, id, barS);
         } else {
@@ -109,7 +109,6 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
     bool ok = true;
     for (; id < total; id += gridDim.x) {
         float *sLam = sLamBuf;
-        const Item it = item_of(g, id, total);
         const int next = id + gridDim.x;
         const Item nit = item_of(g, next, total);
         const int row = threadIdx.x >> 3, j = threadIdx.x & 7, col = j * 8;
@@ -294,6 +293,7 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
             }
         }
         parity ^= 1;
+        it = nit;
     }
     if (!ok) {      // a wait gave up: let bulk copies still in flight land before the CTA's memory goes away
         mbar_wait(barS, parity, status);

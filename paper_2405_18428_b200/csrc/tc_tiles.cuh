@@ -94,8 +94,7 @@ __device__ __forceinline__ float4 tf32x4(float a, float b, float c, float d)
 }
 
 // ---- stores into operand tiles (ROWS rows, column blocks of 32 words) -----------------------
-// 8 consecutive columns starting at col8 (a multiple of 8).  `flip` swaps the order of the two
-// 16-byte stores so that threads working on the two column blocks of a row hit different banks.
+// 8 consecutive columns starting at col8 (a multiple of 8).
 // ROUND = false is for values that are exact in tf32 already (bf16 numbers, or rounded before).
 template <int ROWS, bool ROUND = true>
 __device__ __forceinline__ void st_k8(char *tile, int row, int col8, const float (&f)[8], bool flip)
@@ -106,7 +105,9 @@ __device__ __forceinline__ void st_k8(char *tile, int row, int col8, const float
     const float4 hi = ROUND ? tf32x4(f[4], f[5], f[6], f[7]) : make_float4(f[4], f[5], f[6], f[7]);
     float4 *p0 = reinterpret_cast<float4 *>(base + ((c ^ s) << 4));
     float4 *p1 = reinterpret_cast<float4 *>(base + (((c + 1) ^ s) << 4));
-    if (flip) { *p1 = hi; *p0 = lo; } else { *p0 = lo; *p1 = hi; }
+    (void)flip;          // a lane-dependent store order would diverge the warp and costs more than the bank conflict it avoids
+    *p0 = lo;
+    *p1 = hi;
 }
 template <int ROWS, bool ROUND = true>
 __device__ __forceinline__ void st_m8(char *tile, int row, int col8, const float (&f)[8], bool flip)
@@ -115,7 +116,9 @@ __device__ __forceinline__ void st_m8(char *tile, int row, int col8, const float
     const float4 lo = ROUND ? tf32x4(f[0], f[1], f[2], f[3]) : make_float4(f[0], f[1], f[2], f[3]);
     const float4 hi = ROUND ? tf32x4(f[4], f[5], f[6], f[7]) : make_float4(f[4], f[5], f[6], f[7]);
     float4 *p0 = reinterpret_cast<float4 *>(base), *p1 = reinterpret_cast<float4 *>(base + 16);
-    if (flip) { *p1 = hi; *p0 = lo; } else { *p0 = lo; *p1 = hi; }
+    (void)flip;          // a lane-dependent store order would diverge the warp and costs more than the bank conflict it avoids
+    *p0 = lo;
+    *p1 = hi;
 }
 // 4 consecutive columns starting at col4 (a multiple of 4), rounded to tf32 unless ROUND = false.
 template <int ROWS, bool ROUND = true>
