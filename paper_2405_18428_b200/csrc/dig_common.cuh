@@ -149,6 +149,32 @@ struct KernelTimer {
     cudaStream_t stream;
 };
 
+// ---- programmatic dependent launch -------------------------------------------------------
+// Kernels launched through launch_pdl may be scheduled while the previous kernel of the stream is
+// still draining; they call pdl_wait() before their first access to global memory, which blocks
+// until that kernel has completed and its writes are visible.  pdl_launch_dependents() lets the
+// next kernel of the stream do the same with respect to this one.  Both are no-ops for a kernel
+// launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline dig_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? DIG_OK : DIG_ERR_CUDA; }
 
 }  // namespace dig

@@ -68,6 +68,8 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
     const int ch = chb * CH + lane * VEC;
     const bool ch_ok = ch < D;
     const T *xb = x + (size_t)b * gh * gw * D;
+    pdl_launch_dependents();
+    pdl_wait();
 
     for (int idx = threadIdx.x; idx < (TY + 2) * (TX + 2) * kLanes; idx += kConvThreads) {
         const int l = idx % kLanes, pix = idx / kLanes;
@@ -132,18 +134,18 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
     KernelTimer t(KID_DWCONV, stream);
     switch (dtype) {
         case DIG_F32:
-            srem_dwconv3x3<float, float><<<grid, Cfg<float>::kThreads, 0, stream>>>(
-                (const float *)x, (const float *)w, (const float *)bias, (float *)y, gh, gw, D, nchb, dir);
+            launch_pdl(srem_dwconv3x3<float, float>, grid, dim3(Cfg<float>::kThreads), 0, stream,
+                       (const float *)x, (const float *)w, (const float *)bias, (float *)y, gh, gw, D, nchb, dir);
             break;
         case DIG_BF16:
-            srem_dwconv3x3<__nv_bfloat16, __nv_bfloat16><<<grid, Cfg<__nv_bfloat16>::kThreads, 0, stream>>>(
-                (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias,
-                (__nv_bfloat16 *)y, gh, gw, D, nchb, dir);
+            launch_pdl(srem_dwconv3x3<__nv_bfloat16, __nv_bfloat16>, grid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
+                       (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias,
+                       (__nv_bfloat16 *)y, gh, gw, D, nchb, dir);
             break;
         case DIG_BF16_F32OUT:
-            srem_dwconv3x3<__nv_bfloat16, float><<<grid, Cfg<__nv_bfloat16>::kThreads, 0, stream>>>(
-                (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias,
-                (float *)y, gh, gw, D, nchb, dir);
+            launch_pdl(srem_dwconv3x3<__nv_bfloat16, float>, grid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
+                       (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias,
+                       (float *)y, gh, gw, D, nchb, dir);
             break;
         default: return DIG_ERR_INVALID_ARG;
     }

@@ -20,6 +20,8 @@ __global__ void __launch_bounds__(256)
 gate_logsigmoid(const T *__restrict__ g, float *__restrict__ gate, size_t n8, int H, int dk,
                 InvTau inv_tau)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
         const size_t e = i * 8;
@@ -48,9 +50,9 @@ dig_status launch_gate(const void *g, const float *tau_host, float *gate, int B,
     const int blocks = (int)((n8 + 255) / 256 < 148 * 16 ? (n8 + 255) / 256 : 148 * 16);
     KernelTimer t(KID_GATE, stream);
     if (dtype == DIG_F32)
-        gate_logsigmoid<float><<<blocks, 256, 0, stream>>>((const float *)g, gate, n8, H, dk, it);
+        launch_pdl(gate_logsigmoid<float>, dim3(blocks), dim3(256), 0, stream, (const float *)g, gate, n8, H, dk, it);
     else
-        gate_logsigmoid<__nv_bfloat16><<<blocks, 256, 0, stream>>>((const __nv_bfloat16 *)g, gate, n8, H, dk, it);
+        launch_pdl(gate_logsigmoid<__nv_bfloat16>, dim3(blocks), dim3(256), 0, stream, (const __nv_bfloat16 *)g, gate, n8, H, dk, it);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -87,7 +87,9 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
     uint64_t *barA = &ctl->bar[0], *barB = &ctl->bar[1], *barS = &ctl->bar[2];
     constexpr uint32_t kCols = 256;
     constexpr uint32_t aP = 0, aQK = 64, aV = 128, kUpper = 16u << 16;      // upper half of a lane quarter
+    pdl_launch_dependents();
     setup(ctl, 4, kCols);
+    pdl_wait();
     const uint32_t tmem = ctl->tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool issuer = warp == NT / 32;                                    // the extra warp: MMAs and bulk loads
@@ -316,9 +318,9 @@ dig_status launch_typed(const GlaArgs &a, const Workspace &w, int sm_count, int 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
     const int grid = total < sm_count ? total : sm_count;
     KernelTimer t(KID_TC_BWD, a.stream);
-    kern<<<grid, NTA, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
-                                       (const bf16 *)a.d_out, w.states, w.dstates, w.dstates_m, w.carry, (TO *)a.dq, (TO *)a.dk,
-                                       (TO *)a.dv, a.dgate, status, g);
+    launch_pdl(kern, dim3(grid), dim3(NTA), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
+               (const bf16 *)a.d_out, (const float *)w.states, (const float *)w.dstates, (const float *)w.dstates_m,
+               (const float *)w.carry, (TO *)a.dq, (TO *)a.dk, (TO *)a.dv, a.dgate, status, g);
     return cuda_ok(cudaGetLastError());
 }
 

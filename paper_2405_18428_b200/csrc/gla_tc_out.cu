@@ -81,7 +81,9 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
     constexpr uint32_t kCols = 256;
     constexpr uint32_t aP = 0, aO = 128;
     uint64_t *barP = &ctl->bar[0], *barO = &ctl->bar[1], *barS = &ctl->bar[2];
+    pdl_launch_dependents();
     setup(ctl, 3, kCols);
+    pdl_wait();
     const uint32_t tmem = ctl->tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool issuer = warp == NT / 32;                      // the extra warp: MMAs and bulk loads
@@ -219,8 +221,8 @@ dig_status launch_typed(const GlaArgs &a, const Workspace &w, int sm_count, int 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
     const int grid = npairs < sm_count ? npairs : sm_count;
     KernelTimer t(KID_TC_OUT, a.stream);
-    kern<<<grid, NTA, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate, w.states,
-                                       (TO *)a.out, status, g);
+    launch_pdl(kern, dim3(grid), dim3(NTA), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
+               a.gate, (const float *)w.states, (TO *)a.out, status, g);
     return cuda_ok(cudaGetLastError());
 }
 

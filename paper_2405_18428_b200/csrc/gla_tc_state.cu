@@ -75,7 +75,9 @@ tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16
     float *sLast = sLam + 2 * T * kLamPitch, *sTot = sLast + 128;
     Control *ctl = reinterpret_cast<Control *>(sTot + NT);
     constexpr uint32_t kCols = BWD ? 256 : 128;
+    pdl_launch_dependents();
     setup(ctl, 1, kCols);
+    pdl_wait();
     const uint32_t tmem = ctl->tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int R = 32 * (warp & 3) + lane, half_r = R >> 6, r = R & 63, c0 = W * (warp >> 2);
@@ -203,8 +205,8 @@ dig_status launch_tc_state(const GlaArgs &a, const Workspace &w, bool backward, 
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
         const int grid = npairs < sm_count ? npairs : sm_count;
         KernelTimer t(KID_TC_STATE, a.stream);
-        kern<<<grid, NT, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
-                                           (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, status, g);
+        launch_pdl(kern, dim3(grid), dim3(NT), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
+                   a.gate, (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, status, g);
     } else {
         constexpr int NT = 256;           // 100 KB of shared memory: two CTAs per SM overlap each other's phases
         auto kern = tc_state_pair<NT, false>;
@@ -212,8 +214,8 @@ dig_status launch_tc_state(const GlaArgs &a, const Workspace &w, bool backward, 
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
         const int grid = npairs < 2 * sm_count ? npairs : 2 * sm_count;
         KernelTimer t(KID_TC_STATE, a.stream);
-        kern<<<grid, NT, smem, a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
-                                           nullptr, w.states, w.gamma, nullptr, status, g);
+        launch_pdl(kern, dim3(grid), dim3(NT), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
+                   a.gate, (const bf16 *)nullptr, w.states, w.gamma, (float *)nullptr, status, g);
     }
     return cuda_ok(cudaGetLastError());
 }

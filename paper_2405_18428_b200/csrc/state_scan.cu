@@ -36,6 +36,8 @@ template <bool TILES>
 __global__ void __launch_bounds__(kScanThreads)
 state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int N, int dk, int dv)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int e4 = blockIdx.x * kScanThreads + threadIdx.x;          // float4 index inside one state
     if (e4 * 4 >= dk * dv) return;
     int row, col;
@@ -133,6 +135,8 @@ __global__ void __launch_bounds__(64)
 state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, float *__restrict__ dstates_m,
                      const float *__restrict__ gamma, float *__restrict__ carry, int N)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = threadIdx.x, c = 8 * blockIdx.x + (t >> 3);
     const size_t base = (size_t)blockIdx.y * N * 4096;
     float4 *S = reinterpret_cast<float4 *>(states + base) + c * 8 + (t & 7);
@@ -213,7 +217,7 @@ dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t
     if (tiles && (g.dk != 64 || g.dv != 64)) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_SCAN_FWD, s);
     if (tiles)
-        state_scan_fwd<true><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
+        launch_pdl(state_scan_fwd<true>, grid, dim3(kScanThreads), 0, s, w.states, (const float *)w.gamma, g.N, g.dk, g.dv);
     else
         state_scan_fwd<false><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
     return cuda_ok(cudaGetLastError());
@@ -232,7 +236,8 @@ dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaSt
 {
     if (g.dk != 64 || g.dv != 64) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_SCAN_BWD, s);
-    state_scan_bwd_tiles<<<dim3(8, g.B * g.H), 64, 0, s>>>(w.states, w.dstates, w.dstates_m, w.gamma, w.carry, g.N);
+    launch_pdl(state_scan_bwd_tiles, dim3(8, g.B * g.H), dim3(64), 0, s, w.states, w.dstates, w.dstates_m,
+               (const float *)w.gamma, w.carry, g.N);
     return cuda_ok(cudaGetLastError());
 }
 
