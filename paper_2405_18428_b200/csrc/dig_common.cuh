@@ -153,7 +153,8 @@ struct KernelTimer {
 // Kernels launched through launch_pdl may be scheduled while the previous kernel of the stream is
 // still draining; they call pdl_wait() before their first access to global memory, which blocks
 // until that kernel has completed and its writes are visible.  pdl_launch_dependents() lets the
-// next kernel of the stream do the same with respect to this one.  Both are no-ops for a kernel
+// next kernel of the stream do the same with respect to this one; it is called after pdl_wait(), so
+// that early launches cannot cascade past a kernel whose own predecessor is still running.  Both are no-ops for a kernel
 // launched the ordinary way.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

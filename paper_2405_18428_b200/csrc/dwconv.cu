@@ -68,8 +68,8 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
     const int ch = chb * CH + lane * VEC;
     const bool ch_ok = ch < D;
     const T *xb = x + (size_t)b * gh * gw * D;
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();      // only once this kernel's own predecessor has completed
 
     for (int idx = threadIdx.x; idx < (TY + 2) * (TX + 2) * kLanes; idx += kConvThreads) {
         const int l = idx % kLanes, pix = idx / kLanes;

@@ -20,8 +20,8 @@ __global__ void __launch_bounds__(256)
 gate_logsigmoid(const T *__restrict__ g, float *__restrict__ gate, size_t n8, int H, int dk,
                 InvTau inv_tau)
 {
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();      // only once this kernel's own predecessor has completed
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
         const size_t e = i * 8;

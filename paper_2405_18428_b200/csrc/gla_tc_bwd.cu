@@ -87,9 +87,7 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
     uint64_t *barA = &ctl->bar[0], *barB = &ctl->bar[1], *barS = &ctl->bar[2];
     constexpr uint32_t kCols = 256;
     constexpr uint32_t aP = 0, aQK = 64, aV = 128, kUpper = 16u << 16;      // upper half of a lane quarter
-    pdl_launch_dependents();
     setup(ctl, 4, kCols);
-    pdl_wait();
     const uint32_t tmem = ctl->tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool issuer = warp == NT / 32;                                    // the extra warp: MMAs and bulk loads
@@ -100,13 +98,12 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
     BwdRaw raw;
     int id = blockIdx.x;
     Item it = item_of(g, id, total);
-    if (id < total) {
-        if (issuer) {
-            if (lane == 0) fetch_states(tSk, tDk, tDm, states, dstates, dstates_m, id, barS);
-        } else {
-            load_raw(raw, q, k, v, d_out, gate, g, it);
-        }
-    }
+    // q, k, v, dO and the gates are inputs of the whole call: their loads need not wait for the scan
+    // kernel that is still finishing; the states and carries it writes do
+    if (id < total && !issuer) load_raw(raw, q, k, v, d_out, gate, g, it);
+    pdl_wait();
+    pdl_launch_dependents();          // only once this kernel's own predecessor has completed
+    if (id < total && issuer && lane == 0) fetch_states(tSk, tDk, tDm, states, dstates, dstates_m, id, barS);
     uint32_t parity = 0;
     bool ok = true;
     for (; id < total; id += gridDim.x) {

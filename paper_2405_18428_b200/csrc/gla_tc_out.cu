@@ -81,9 +81,7 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
     constexpr uint32_t kCols = 256;
     constexpr uint32_t aP = 0, aO = 128;
     uint64_t *barP = &ctl->bar[0], *barO = &ctl->bar[1], *barS = &ctl->bar[2];
-    pdl_launch_dependents();
     setup(ctl, 3, kCols);
-    pdl_wait();
     const uint32_t tmem = ctl->tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool issuer = warp == NT / 32;                      // the extra warp: MMAs and bulk loads
@@ -95,9 +93,15 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
     int pair = blockIdx.x;
     if (pair < npairs) {
         const Item it[2] = {item_of(g, 2 * pair, total), item_of(g, 2 * pair + 1, total)};
+        // q, k, v and the gates are inputs of the whole call: their loads need not wait for the scan
+        // kernel that is still finishing; the states it writes do
         if (!issuer) load_raw(raw, q, k, v, gate, g, it);
-        else if (lane == 0) fetch_states(tS, states, pair, total, barS);
+        pdl_wait();
+        if (issuer && lane == 0) fetch_states(tS, states, pair, total, barS);
+    } else {
+        pdl_wait();
     }
+    pdl_launch_dependents();          // only once this kernel's own predecessor has completed
     uint32_t parity = 0;
     bool ok = true;
     Item cur[2] = {item_of(g, 2 * pair, total), item_of(g, 2 * pair + 1, total)};

@@ -75,9 +75,9 @@ tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16
     float *sLast = sLam + 2 * T * kLamPitch, *sTot = sLast + 128;
     Control *ctl = reinterpret_cast<Control *>(sTot + NT);
     constexpr uint32_t kCols = BWD ? 256 : 128;
-    pdl_launch_dependents();
     setup(ctl, 1, kCols);
     pdl_wait();
+    pdl_launch_dependents();      // only once this kernel's own predecessor has completed
     const uint32_t tmem = ctl->tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int R = 32 * (warp & 3) + lane, half_r = R >> 6, r = R & 63, c0 = W * (warp >> 2);

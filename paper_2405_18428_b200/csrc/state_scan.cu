@@ -36,8 +36,8 @@ template <bool TILES>
 __global__ void __launch_bounds__(kScanThreads)
 state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int N, int dk, int dv)
 {
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();      // only once this kernel's own predecessor has completed
     const int e4 = blockIdx.x * kScanThreads + threadIdx.x;          // float4 index inside one state
     if (e4 * 4 >= dk * dv) return;
     int row, col;
@@ -135,8 +135,8 @@ __global__ void __launch_bounds__(64)
 state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, float *__restrict__ dstates_m,
                      const float *__restrict__ gamma, float *__restrict__ carry, int N)
 {
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();      // only once this kernel's own predecessor has completed
     const int t = threadIdx.x, c = 8 * blockIdx.x + (t >> 3);
     const size_t base = (size_t)blockIdx.y * N * 4096;
     float4 *S = reinterpret_cast<float4 *>(states + base) + c * 8 + (t & 7);
