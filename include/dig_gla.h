@@ -76,6 +76,8 @@ dig_status dig_gate_logsigmoid(const void *g, const float *tau_per_head, float *
  * depend on `chunk` beyond rounding.  No 1/sqrt(d) scaling and no normaliser are applied.
  *   q, k, gate: [B][L][H][d_k]; v, out: [B][L][H][d_v]; gate is log(alpha) <= 0, fp32.
  *   d_k, d_v: multiples of 8, 8..128; chunk in {16, 32, 64, 128}; L need not be a multiple of chunk.
+ * The tensor-core kernels work on 64-token tiles: with them a request for chunk = 128 is evaluated
+ * in 64-token tiles (dig_gla_query_impl tells which family serves a request).
  * The in-chunk decay is formed as exp(+-cumulative gate): the magnitude of the gate summed over
  * one chunk must stay below 80 per channel (true with a wide margin for sigmoid gates with
  * temperature >= 1 at the chunk sizes above); beyond it results may overflow. */
@@ -113,7 +115,8 @@ dig_status dig_gla_fwd_static(const void *q, const void *k, const void *v, const
  * (reverse-mode derivative of Eq. attn_gla; the paper trains through the operator but does not
  * print it).  Nothing is saved by the forward call: chunk states are recomputed here.
  *   d_out: [B][L][H][d_v]; dq, dk: [B][L][H][d_k]; dv: [B][L][H][d_v]; dgate: fp32 [B][L][H][d_k].
- * The fp32-FMA family covers chunk <= 64 here. */
+ * The fp32-FMA family covers chunk <= 64 here; chunk = 128 is served by the tensor-core family only
+ * (bf16 storage, d_k = d_v = 64). */
 dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float *gate,
                        const void *d_out, void *dq, void *dk, void *dv, float *dgate,
                        int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,

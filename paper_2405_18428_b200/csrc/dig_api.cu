@@ -42,6 +42,10 @@ Geom make_geom(int B, int H, int gh, int gw, int dk, int dv, int chunk, int dir)
 }
 
 // DIG_IMPL_FMA / DIG_IMPL_TENSOR, or a negative status.
+// The tensor-core kernels hold 64 tokens per tile; a request for chunks of 128 is evaluated by them
+// with 64-token tiles (the result does not depend on the chunk size beyond rounding).
+int tile_chunk(int impl, int chunk) { return (impl == DIG_IMPL_TENSOR && chunk == 128) ? 64 : chunk; }
+
 int choose_impl(int dk, int dv, int chunk, int dtype, bool backward)
 {
     const int want = g_impl.load();
@@ -136,7 +140,9 @@ size_t dig_gla_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, in
                                int dtype, int backward)
 {
     if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, 0, dtype)) return 0;
-    const Geom g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, 0);
+    // sized for whichever family may serve the call (the tensor family uses 64-token tiles for chunk 128)
+    const bool tensor_ok = tensor_supports(d_k, d_v, chunk, dtype, backward != 0);
+    const Geom g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(tensor_ok ? DIG_IMPL_TENSOR : DIG_IMPL_FMA, chunk), 0);
     return carve_workspace(nullptr, g, backward != 0).bytes;
 }
 
@@ -164,7 +170,7 @@ dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float 
     GlaArgs a{};
     a.q = q; a.k = k; a.v = v; a.gate = gate; a.out = out;
     a.ws = reinterpret_cast<float *>(workspace);
-    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, direction);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
     a.dtype = dtype;
     a.stream = (cudaStream_t)cuda_stream;
     return impl == DIG_IMPL_TENSOR ? tensor_gla_fwd(a) : fma_gla_fwd(a);
@@ -188,7 +194,7 @@ dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float 
     a.q = q; a.k = k; a.v = v; a.gate = gate; a.d_out = d_out;
     a.dq = dq; a.dk = dk; a.dv = dv; a.dgate = dgate;
     a.ws = reinterpret_cast<float *>(workspace);
-    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, direction);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
     a.dtype = dtype;
     a.stream = (cudaStream_t)cuda_stream;
     return impl == DIG_IMPL_TENSOR ? tensor_gla_bwd(a) : fma_gla_bwd(a);

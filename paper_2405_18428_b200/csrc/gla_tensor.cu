@@ -1,6 +1,7 @@
 // Tensor-core kernel family for chunkwise gated linear attention on sm_100a (Eq. attn_gla
 // evaluated chunk by chunk, Section 3.5): dispatch of the forward and backward pipelines.
-// bf16 storage, chunk = 64, d_k = d_v = 64.
+// bf16 storage, d_k = d_v = 64, 64-token tiles (chunk = 64; chunk = 128 requests are evaluated with
+// the same tiles).
 //
 // Why tf32 operands: the decayed operands q*exp(Lam), k*exp(-Lam), the masked scores and the
 // chunk states are not bf16 numbers; rounding them to bf16 (8 significant bits) puts the maximum
@@ -19,7 +20,7 @@ bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward)
 {
     (void)backward;
     if (dtype != DIG_BF16 && dtype != DIG_BF16_F32OUT) return false;
-    return dk == 64 && dv == 64 && chunk == 64;
+    return dk == 64 && dv == 64 && (chunk == 64 || chunk == 128);      // 128: served with 64-token tiles
 }
 
 dig_status tensor_gla_fwd(const GlaArgs &a)

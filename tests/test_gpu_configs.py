@@ -29,14 +29,13 @@ def test_c5_other_directions_four_heads(direction):
 @pytest.mark.parametrize("chunk", [32, 64, 128])
 def test_c4_chunk_sweep(chunk):
     """112 x 112 grid: 64 does not divide the column length, so column orders straddle columns.
-    Chunk 128 is covered in the forward direction only (no kernel family runs its backward pass)."""
+    Chunk 32 runs on the fp32-FMA kernels, 64 and 128 on the tensor-core kernels (128 in 64-token tiles)."""
     from paper_2405_18428_b200 import dig
     from parity import check_workload
     wl = CONFIGS["C4"]
     assert _family(wl, chunk, False) > 0
-    bwd = _family(wl, chunk, True) > 0
-    assert bwd or chunk == 128
-    errs = check_workload(wl, 2, chunk=chunk, backward=bwd)
+    assert _family(wl, chunk, True) > 0
+    errs = check_workload(wl, 2, chunk=chunk, backward=True)
     print("C4 chunk", chunk, {k: f"{v:.2e}" for k, v in errs.items()})
 
 
@@ -50,3 +49,14 @@ def test_chunk_size_does_not_change_the_result_beyond_rounding():
     for n in a:
         rms = np.sqrt(np.mean(a[n].astype(np.float64) ** 2))
         assert np.abs(a[n].astype(np.float64) - b[n]).max() <= 2e-2 * rms, n
+
+
+def test_chunk128_forward_on_the_fma_family_matches_too():
+    """Forcing the fp32-FMA family keeps a real 128-token chunk (forward only there)."""
+    from paper_2405_18428_b200 import dig
+    from parity import check_workload
+    dig.dig_set_impl(dig.DIG_IMPL_FMA)
+    try:
+        check_workload(CONFIGS["C4"].scaled(H=2), 1, chunk=128, backward=False)
+    finally:
+        dig.dig_set_impl(dig.DIG_IMPL_AUTO)
