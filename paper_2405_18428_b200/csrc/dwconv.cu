@@ -1,7 +1,6 @@
 // SREM depthwise 3x3 convolution (Algorithm 1: DWConv2d on the reshaped token matrix), channel-last.
 // A CTA stages a (TY+2) x (TX+2) pixel halo tile of CH channels in shared memory with 16-byte
-// coalesced loads; each thread then owns 8 channels of one tile column and slides down the rows,
-// so every staged vector is read from shared memory three times instead of nine.
+// coalesced loads; each thread then owns 8 channels of one tile column and walks down the rows.
 // The scan order the residual stream is in (`dir`) only permutes the filter taps:
 // reverse orders see the filter rotated by 180 degrees, column orders see it transposed.
 #include "dig_common.cuh"
@@ -80,8 +79,11 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
             v = Vec8<T>::load(xb + ((size_t)gy * gw + gx) * D + c);
         tile[ty][tx][l] = v;
     }
-    // filter taps for this thread's channels, re-oriented: wt[u][v] multiplies x[i+u-1][j+v-1]
-    float wt[3][3][8], bs[8];
+    // filter taps for this thread's channels, re-oriented: wt[u][v] multiplies x[i+u-1][j+v-1].  They are
+    // kept packed (and unpacked at every use) so that the kernel stays at a register count that lets
+    // six CTAs share an SM; the loads of the tile are what it waits for, not the arithmetic.
+    Vec8<T> wt[3][3];
+    float bs[8];
 #pragma unroll
     for (int u = 0; u < 3; ++u)
 #pragma unroll
@@ -89,7 +91,7 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
             int su = u, sv = v;
             if (dir & 2) { su = v; sv = u; }
             if (dir & 1) { su = 2 - su; sv = 2 - sv; }
-            if (ch_ok) Vec8<T>::load(w + (size_t)(su * 3 + sv) * D + ch).unpack(wt[u][v]);
+            wt[u][v] = ch_ok ? Vec8<T>::load(w + (size_t)(su * 3 + sv) * D + ch) : Vec8<T>::zero();
         }
 #pragma unroll
     for (int i = 0; i < 8; ++i) bs[i] = 0.f;
@@ -97,16 +99,8 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
     __syncthreads();
     if (!ch_ok || x0 + col >= gw) return;
 
-    float win[3][3][8];      // win[r][v]: tile rows ty-1, ty, ty+1 (rolling), columns col, col+1, col+2
-#pragma unroll
-    for (int v = 0; v < 3; ++v) {
-        tile[0][col + v][lane].unpack(win[0][v]);
-        tile[1][col + v][lane].unpack(win[1][v]);
-    }
 #pragma unroll
     for (int ty = 0; ty < TY; ++ty) {
-#pragma unroll
-        for (int v = 0; v < 3; ++v) tile[ty + 2][col + v][lane].unpack(win[(ty + 2) % 3][v]);
         if (y0 + ty < gh) {
             float acc[8];
 #pragma unroll
@@ -114,9 +108,13 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
 #pragma unroll
             for (int u = 0; u < 3; ++u)
 #pragma unroll
-                for (int v = 0; v < 3; ++v)
+                for (int v = 0; v < 3; ++v) {
+                    float xv[8], wv[8];
+                    tile[ty + u][col + v][lane].unpack(xv);
+                    wt[u][v].unpack(wv);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(wt[u][v][i], win[(ty + u) % 3][v][i], acc[i]);
+                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(wv[i], xv[i], acc[i]);
+                }
             store8(y + (((size_t)b * gh + y0 + ty) * gw + x0 + col) * D + ch, acc);
         }
     }

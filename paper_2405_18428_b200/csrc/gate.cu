@@ -11,8 +11,10 @@ struct InvTau { float v[kMaxHeads]; };
 
 __device__ __forceinline__ float log_sigmoid(float x)
 {
-    // log(1/(1+e^-x)) without overflow on either side
-    return x >= 0.f ? -log1pf(expf(-x)) : x - log1pf(expf(x));
+    // log(1/(1+e^-x)) = min(x, 0) - log1p(e^-|x|), without overflow on either side.  e^-|x| <= 1 comes
+    // from the fast exponential (a few ulp; its error enters the result damped by 1/(1+t)), the
+    // logarithm stays the accurate one: the result keeps an absolute error near 1e-7.
+    return fminf(x, 0.f) - log1pf(__expf(-fabsf(x)));
 }
 
 template <typename T>
