@@ -49,6 +49,7 @@ def _load():
             lib.dig_oracle_gla_fwd.argtypes = [dp] * 5 + [ctypes.c_int] * 8
             lib.dig_oracle_gla_bwd.argtypes = [dp] * 9 + [ctypes.c_int] * 8
             lib.dig_oracle_dwconv.argtypes = [dp] * 4 + [ctypes.c_int] * 5
+            lib.dig_oracle_dwconv_bwd.argtypes = [dp] * 6 + [ctypes.c_int] * 5
             _lib = lib
     return _lib
 
@@ -127,3 +128,15 @@ def dwconv(x, w, bias, grid_h, grid_w, direction=ROW_FWD) -> np.ndarray:
     _check(_load().dig_oracle_dwconv(_p(x), _p(w), bp, _p(y), B, grid_h, grid_w, D, direction),
            "dwconv")
     return y
+
+
+def dwconv_bwd(x, w, dy, grid_h, grid_w, direction=ROW_FWD, with_bias=True):
+    """Gradients (dx, dw, dbias) of <dy, dwconv(x, w, bias)>; dbias is None if with_bias is False."""
+    x, w, dy = _f64(x), _f64(w), _f64(dy)
+    B, L, D = x.shape
+    assert L == grid_h * grid_w and w.shape == (3, 3, D) and dy.shape == x.shape
+    dx, dw = np.empty_like(x), np.empty_like(w)
+    db = np.empty(D, dtype=np.float64) if with_bias else None
+    _check(_load().dig_oracle_dwconv_bwd(_p(x), _p(w), _p(dy), _p(dx), _p(dw), None if db is None else _p(db),
+                                         B, grid_h, grid_w, D, direction), "dwconv_bwd")
+    return dx, dw, db

@@ -13,7 +13,8 @@
  *   - the four scan orders of the block-by-block scanning scheme (Algorithm 1 / Algorithm 4:
  *     flip and transpose of the reshaped token matrix), materialised as index arrays
  *   - the 3x3 depthwise convolution of the SREM module (Algorithm 1, "DWConv2d(reshape2d(z))"),
- *     evaluated on the re-oriented token matrix by explicit gather / conv / scatter
+ *     evaluated on the re-oriented token matrix by explicit gather / conv / scatter, and its
+ *     reverse-mode derivative
  *
  * Everything is token-by-token and element-by-element: no chunking, no blocking, no fused forms.
  * Tensors are dense row-major doubles with layout [B][L][H][d]; L = grid_h*grid_w and the
@@ -23,7 +24,9 @@
  * attention (Eq. attn_simple) when alpha == 1, constant-decay closed form, fast-decay limit,
  * permutation bijectivity and the four-block cycle, central finite differences for the
  * backward pass, the suffix-sum gate-gradient identity, identity-initialised convolution,
- * convolution against hand-evaluated corner / edge / interior counts.
+ * convolution against hand-evaluated corner / edge / interior counts; for the convolution's
+ * derivative: central finite differences, the adjoint identity <dy, conv(x)> = <dx, x>, and
+ * dw of an identity-initialised filter on a one-pixel image.
  * Not pinned by the paper: whether DWConv2d carries a bias (the argument is optional).
  */
 #include <math.h>
@@ -266,6 +269,55 @@ int dig_oracle_dwconv(const double *x, const double *w, const double *bias, doub
             memcpy(yb + (size_t)perm[p] * D, zo + (size_t)p * D, sizeof(double) * (size_t)D);
     }
     free(perm); free(z); free(zo);
+    return 0;
+}
+
+/* Reverse mode of the SREM depthwise convolution above (the paper trains through the module but
+ * does not print its derivative): given dL/dy, returns dL/dx, dL/dw and dL/dbias of
+ *     y = DWConv2d(reshape2d(z)) + bias
+ * in the same re-oriented layout.  Written as the transpose of the forward loops: every product
+ * w[u][v][ch] * z[i+u-1][j+v-1][ch] that contributed to y[i][j][ch] sends dy[i][j][ch] * w back to
+ * that input pixel and dy * z to that tap.  dw: [3][3][D], dbias: [D] (may be NULL). */
+int dig_oracle_dwconv_bwd(const double *x, const double *w, const double *dy, double *dx, double *dw,
+                          double *dbias, int B, int grid_h, int grid_w, int D, int direction)
+{
+    const long long L = (long long)grid_h * grid_w;
+    long long *perm = (long long *)malloc(sizeof(long long) * (size_t)L);
+    if (!perm) return 2;
+    if (dig_oracle_perm(direction, grid_h, grid_w, perm)) { free(perm); return 1; }
+    const int R = (direction >= 2) ? grid_w : grid_h;
+    const int C = (direction >= 2) ? grid_h : grid_w;
+    double *z = (double *)malloc(sizeof(double) * (size_t)L * D);
+    double *g = (double *)malloc(sizeof(double) * (size_t)L * D);
+    double *dz = (double *)malloc(sizeof(double) * (size_t)L * D);
+    if (!z || !g || !dz) { free(perm); free(z); free(g); free(dz); return 2; }
+    memset(dw, 0, sizeof(double) * 9 * (size_t)D);
+    if (dbias) memset(dbias, 0, sizeof(double) * (size_t)D);
+    for (int b = 0; b < B; ++b) {
+        const double *xb = x + (size_t)b * L * D, *gb = dy + (size_t)b * L * D;
+        double *dxb = dx + (size_t)b * L * D;
+        for (long long p = 0; p < L; ++p) {                         /* gather into scan order */
+            memcpy(z + (size_t)p * D, xb + (size_t)perm[p] * D, sizeof(double) * (size_t)D);
+            memcpy(g + (size_t)p * D, gb + (size_t)perm[p] * D, sizeof(double) * (size_t)D);
+        }
+        memset(dz, 0, sizeof(double) * (size_t)L * D);
+        for (int i = 0; i < R; ++i)
+            for (int j = 0; j < C; ++j)
+                for (int ch = 0; ch < D; ++ch) {
+                    const double gy = g[((size_t)i * C + j) * D + ch];
+                    if (dbias) dbias[ch] += gy;
+                    for (int u = 0; u < 3; ++u)
+                        for (int vv = 0; vv < 3; ++vv) {
+                            const int ii = i + u - 1, jj = j + vv - 1;
+                            if (ii < 0 || ii >= R || jj < 0 || jj >= C) continue;
+                            dz[((size_t)ii * C + jj) * D + ch] += gy * w[((size_t)u * 3 + vv) * D + ch];
+                            dw[((size_t)u * 3 + vv) * D + ch] += gy * z[((size_t)ii * C + jj) * D + ch];
+                        }
+                }
+        for (long long p = 0; p < L; ++p)                           /* scatter back */
+            memcpy(dxb + (size_t)perm[p] * D, dz + (size_t)p * D, sizeof(double) * (size_t)D);
+    }
+    free(perm); free(z); free(g); free(dz);
     return 0;
 }
 

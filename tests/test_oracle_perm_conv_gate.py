@@ -150,3 +150,61 @@ def test_gate_extreme_logits_stay_finite():
     np.testing.assert_allclose(a[2], np.log(0.5) / 2)
     assert a[4] == 0.0 or abs(a[4]) < 1e-300
     assert np.isfinite(a).all()
+
+
+# ---- reverse mode of the SREM convolution --------------------------------------------------------
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+def test_conv_backward_matches_central_finite_differences(direction):
+    rng = np.random.default_rng(20 + direction)
+    gh, gw, D, B = 4, 5, 3, 2
+    x = rng.standard_normal((B, gh * gw, D))
+    w = rng.standard_normal((3, 3, D))
+    bias = rng.standard_normal(D)
+    dy = rng.standard_normal((B, gh * gw, D))
+    dx, dw, db = oracle.dwconv_bwd(x, w, dy, gh, gw, direction)
+    loss = lambda xx, ww, bb: float((dy * oracle.dwconv(xx, ww, bb, gh, gw, direction)).sum())
+    h = 1e-6
+    for arr, grad, which in ((x, dx, 0), (w, dw, 1), (bias, db, 2)):
+        for _ in range(6):
+            idx = tuple(rng.integers(0, n) for n in arr.shape)
+            plus, minus = arr.copy(), arr.copy()
+            plus[idx] += h
+            minus[idx] -= h
+            args_p = [x, w, bias]
+            args_m = [x, w, bias]
+            args_p[which], args_m[which] = plus, minus
+            fd = (loss(*args_p) - loss(*args_m)) / (2 * h)
+            assert abs(fd - grad[idx]) <= 1e-7 * max(1.0, abs(fd)), (which, idx, fd, grad[idx])
+
+
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+def test_conv_backward_is_the_adjoint_of_the_forward_map(direction):
+    """<dy, conv(x)> = <dx, x> (the map is linear in x without bias), and likewise in w."""
+    rng = np.random.default_rng(30 + direction)
+    gh, gw, D = 5, 3, 4
+    x = rng.standard_normal((1, gh * gw, D))
+    w = rng.standard_normal((3, 3, D))
+    dy = rng.standard_normal((1, gh * gw, D))
+    dx, dw, db = oracle.dwconv_bwd(x, w, dy, gh, gw, direction)
+    y = oracle.dwconv(x, w, None, gh, gw, direction)
+    assert abs((dy * y).sum() - (dx * x).sum()) <= 1e-12 * np.abs(dy * y).sum()
+    assert abs((dy * y).sum() - (dw * w).sum()) <= 1e-12 * np.abs(dy * y).sum()
+    np.testing.assert_allclose(db, dy.sum(axis=(0, 1)), rtol=1e-13)
+
+
+def test_conv_backward_of_identity_filter_and_single_pixel():
+    """Identity-initialised filter (centre tap 1): dx == dy.  A 1 x 1 image only ever touches the
+    centre tap: dw is x*dy there and 0 elsewhere."""
+    rng = np.random.default_rng(40)
+    gh, gw, D = 4, 4, 2
+    w = np.zeros((3, 3, D))
+    w[1, 1] = 1.0
+    x = rng.standard_normal((2, gh * gw, D))
+    dy = rng.standard_normal((2, gh * gw, D))
+    dx, _, _ = oracle.dwconv_bwd(x, w, dy, gh, gw, 3)
+    np.testing.assert_array_equal(dx, dy)
+    x1, dy1 = rng.standard_normal((1, 1, D)), rng.standard_normal((1, 1, D))
+    _, dw1, _ = oracle.dwconv_bwd(x1, rng.standard_normal((3, 3, D)), dy1, 1, 1, 0)
+    want = np.zeros((3, 3, D))
+    want[1, 1] = (x1 * dy1)[0, 0]
+    np.testing.assert_allclose(dw1, want, rtol=1e-15)
