@@ -136,6 +136,19 @@ dig_status dig_srem_dwconv(const void *x, const void *w, const void *bias, void 
                            int B, int grid_h, int grid_w, int D, int direction, int dtype,
                            void *cuda_stream);
 
+/* Reverse mode of dig_srem_dwconv (the paper trains through the SREM module; the derivative is not
+ * printed there): given dy = dL/dy, computes dx = dL/dx, dw = dL/dw and, if dbias is not NULL,
+ * dbias = dL/dbias of  y = conv3x3(z2d, w) + bias  in the same scan-order convention.
+ *   x, dy, dx: [B][grid_h*grid_w][D] canonical order (dx in the output storage type of `dtype`);
+ *   w: [3][3][D] in the storage type; dw: fp32 [3][3][D]; dbias: fp32 [D] or NULL.
+ * dx is the forward stencil run on dy in the opposite scan sense; dw and dbias are reductions over
+ * all pixels, summed in a fixed order (bit-identical from run to run).  Needs a workspace of
+ * dig_srem_dwconv_bwd_workspace_bytes (0 for invalid sizes) for per-slab partial sums. */
+size_t dig_srem_dwconv_bwd_workspace_bytes(int B, int grid_h, int grid_w, int D);
+dig_status dig_srem_dwconv_bwd(const void *x, const void *w, const void *dy, void *dx, float *dw, float *dbias,
+                               int B, int grid_h, int grid_w, int D, int direction, int dtype, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the status recorded by device code on the
  * current device: DIG_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last query,
  * DIG_ERR_CUDA if the synchronisation itself failed, DIG_OK otherwise. */

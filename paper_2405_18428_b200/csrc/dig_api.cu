@@ -11,6 +11,9 @@ dig_status launch_gate(const void *g, const float *tau_host, float *gate, int B,
                        int dk, int dtype, cudaStream_t stream);
 dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y, int B, int gh,
                          int gw, int D, int dir, int dtype, cudaStream_t stream);
+size_t dwconv_bwd_workspace_bytes(int B, int gh, int gw, int D);
+dig_status launch_dwconv_bwd(const void *x, const void *w, const void *dy, void *dx, float *dw, float *dbias,
+                             int B, int gh, int gw, int D, int dir, int dtype, float *partial, cudaStream_t stream);
 
 namespace {
 
@@ -64,7 +67,7 @@ int choose_impl(int dk, int dv, int chunk, int dtype, bool backward)
 namespace {
 constexpr int kMaxTimed = 32768;
 const char *const kKernelNames[KID_COUNT] = {
-    "gate_logsigmoid", "srem_dwconv3x3", "state_scan_fwd", "state_scan_bwd",
+    "gate_logsigmoid", "srem_dwconv3x3", "srem_dwconv_wgrad", "state_scan_fwd", "state_scan_bwd",
     "fma_chunk_state", "fma_chunk_out", "fma_chunk_bwd",
     "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd"};
 struct Profile {
@@ -208,6 +211,28 @@ dig_status dig_srem_dwconv(const void *x, const void *w, const void *bias, void 
     if (B <= 0 || grid_h <= 0 || grid_w <= 0 || D <= 0 || (D % 8) != 0) return DIG_ERR_INVALID_ARG;
     if (direction < 0 || direction > 3 || !valid_dtype(dtype)) return DIG_ERR_INVALID_ARG;
     return launch_dwconv(x, w, bias, y, B, grid_h, grid_w, D, direction, dtype, (cudaStream_t)cuda_stream);
+}
+
+size_t dig_srem_dwconv_bwd_workspace_bytes(int B, int grid_h, int grid_w, int D)
+{
+    if (B <= 0 || grid_h <= 0 || grid_w <= 0 || D <= 0 || (D % 8) != 0) return 0;
+    if ((long long)B * grid_h * grid_w > (1ll << 30)) return 0;
+    return dwconv_bwd_workspace_bytes(B, grid_h, grid_w, D);
+}
+
+dig_status dig_srem_dwconv_bwd(const void *x, const void *w, const void *dy, void *dx, float *dw, float *dbias,
+                               int B, int grid_h, int grid_w, int D, int direction, int dtype, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream)
+{
+    if (!x || !w || !dy || !dx || !dw) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(dy) || !aligned16(dx) || !aligned16(dw)) return DIG_ERR_INVALID_ARG;
+    if (dbias && !aligned16(dbias)) return DIG_ERR_INVALID_ARG;
+    if (direction < 0 || direction > 3 || !valid_dtype(dtype)) return DIG_ERR_INVALID_ARG;
+    const size_t need = dig_srem_dwconv_bwd_workspace_bytes(B, grid_h, grid_w, D);
+    if (need == 0) return DIG_ERR_INVALID_ARG;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    return launch_dwconv_bwd(x, w, dy, dx, dw, dbias, B, grid_h, grid_w, D, direction, dtype,
+                             reinterpret_cast<float *>(workspace), (cudaStream_t)cuda_stream);
 }
 
 dig_status dig_last_device_status(void *cuda_stream)

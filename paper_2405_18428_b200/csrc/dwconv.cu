@@ -120,6 +120,90 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
     }
 }
 
+// ---- reverse mode: filter and bias gradients ------------------------------------------------------
+// dw'[u][v][c] = sum over pixels of dy[i][j][c] * x[i+u-1][j+v-1][c] (zero outside the grid), computed
+// in canonical taps and written to the stored tap the scan order maps (u, v) to; dbias = sum of dy.
+// A CTA takes 128 consecutive pixels and one block of channels: its threads (8 channels each, 8
+// pixels in flight) read dy and the nine neighbours straight from global memory (they hit L1 / L2),
+// reduce over their pixel groups in shared memory and write one partial sum per CTA; a second kernel
+// adds the partial sums in a fixed order, so the result does not depend on scheduling.
+constexpr int kWgPixels = 128, kWgGroups = 8;
+
+template <typename T>
+__global__ void __launch_bounds__(Cfg<T>::kLanes * kWgGroups)
+srem_dwconv_wgrad(const T *__restrict__ x, const T *__restrict__ dy, float *__restrict__ partial,
+                  int npix, int gh, int gw, int D, int dir)
+{
+    constexpr int CH = Cfg<T>::CH, kLanes = Cfg<T>::kLanes;
+    __shared__ float red[kWgGroups][10][CH];
+    const int lane = threadIdx.x % kLanes, grp = threadIdx.x / kLanes;
+    const int ch = blockIdx.x * CH + lane * VEC;
+    const bool ch_ok = ch < D;
+    pdl_wait();
+    pdl_launch_dependents();
+    float acc[10][8];
+#pragma unroll
+    for (int k = 0; k < 10; ++k)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[k][i] = 0.f;
+    const int p0 = blockIdx.y * kWgPixels, p1 = min(p0 + kWgPixels, npix);
+    if (ch_ok) {
+        for (int p = p0 + grp; p < p1; p += kWgGroups) {
+            const int b = p / (gh * gw), ij = p - b * (gh * gw), i = ij / gw, j = ij - i * gw;
+            float g[8];
+            Vec8<T>::load(dy + (size_t)p * D + ch).unpack(g);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[9][e] += g[e];
+#pragma unroll
+            for (int u = 0; u < 3; ++u)
+#pragma unroll
+                for (int v = 0; v < 3; ++v) {
+                    const int ii = i + u - 1, jj = j + v - 1;
+                    if (ii < 0 || ii >= gh || jj < 0 || jj >= gw) continue;
+                    float xv[8];
+                    Vec8<T>::load(x + ((size_t)b * gh * gw + (size_t)ii * gw + jj) * D + ch).unpack(xv);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[u * 3 + v][e] = fmaf(g[e], xv[e], acc[u * 3 + v][e]);
+                }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 10; ++k)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) red[grp][k][lane * VEC + e] = acc[k][e];
+    __syncthreads();
+    // partial[slab][k][D]: k = stored tap index 0..8, 9 = bias
+    for (int idx = threadIdx.x; idx < 10 * CH; idx += kLanes * kWgGroups) {
+        const int k = idx / CH, c = idx - k * CH;
+        if (blockIdx.x * CH + c >= D) continue;
+        float sum = 0.f;
+#pragma unroll
+        for (int gidx = 0; gidx < kWgGroups; ++gidx) sum += red[gidx][k][c];
+        int ks = k;
+        if (k < 9) {
+            int su = k / 3, sv = k - 3 * su;
+            if (dir & 2) { const int t = su; su = sv; sv = t; }
+            if (dir & 1) { su = 2 - su; sv = 2 - sv; }
+            ks = su * 3 + sv;
+        }
+        partial[((size_t)blockIdx.y * 10 + ks) * D + blockIdx.x * CH + c] = sum;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+srem_dwconv_wgrad_sum(const float *__restrict__ partial, float *__restrict__ dw, float *__restrict__ dbias,
+                      int nslab, int D)
+{
+    pdl_wait();
+    pdl_launch_dependents();
+    const int idx = blockIdx.x * 256 + threadIdx.x;
+    if (idx >= 10 * D) return;
+    float sum = 0.f;
+    for (int s = 0; s < nslab; ++s) sum += partial[(size_t)s * 10 * D + idx];
+    if (idx < 9 * D) dw[idx] = sum;
+    else if (dbias != nullptr) dbias[idx - 9 * D] = sum;
+}
+
 }  // namespace
 
 dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y, int B, int gh,
@@ -147,6 +231,40 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
             break;
         default: return DIG_ERR_INVALID_ARG;
     }
+    return cuda_ok(cudaGetLastError());
+}
+
+size_t dwconv_bwd_workspace_bytes(int B, int gh, int gw, int D)
+{
+    const size_t nslab = ((size_t)B * gh * gw + kWgPixels - 1) / kWgPixels;
+    return nslab * 10 * (size_t)D * sizeof(float);
+}
+
+// dx = the forward stencil applied to dy with the filter rotated by 180 degrees, which is the forward
+// kernel in the opposite scan sense (dir ^ 1); dw, dbias by the two reduction kernels above.
+dig_status launch_dwconv_bwd(const void *x, const void *w, const void *dy, void *dx, float *dw, float *dbias,
+                             int B, int gh, int gw, int D, int dir, int dtype, float *partial, cudaStream_t stream)
+{
+    dig_status st = launch_dwconv(dy, w, nullptr, dx, B, gh, gw, D, dir ^ 1, dtype, stream);
+    if (st != DIG_OK) return st;
+    const int npix = B * gh * gw, nslab = (npix + kWgPixels - 1) / kWgPixels;
+    if (nslab > 65535) return DIG_ERR_UNSUPPORTED;
+    {
+        KernelTimer t(KID_DWCONV_WGRAD, stream);
+        if (dtype == DIG_F32) {
+            const dim3 grid((D + Cfg<float>::CH - 1) / Cfg<float>::CH, nslab);
+            launch_pdl(srem_dwconv_wgrad<float>, grid, dim3(Cfg<float>::kLanes * kWgGroups), 0, stream,
+                       (const float *)x, (const float *)dy, partial, npix, gh, gw, D, dir);
+        } else {
+            const dim3 grid((D + Cfg<__nv_bfloat16>::CH - 1) / Cfg<__nv_bfloat16>::CH, nslab);
+            launch_pdl(srem_dwconv_wgrad<__nv_bfloat16>, grid, dim3(Cfg<__nv_bfloat16>::kLanes * kWgGroups), 0, stream,
+                       (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)dy, partial, npix, gh, gw, D, dir);
+        }
+    }
+    if (cudaGetLastError() != cudaSuccess) return DIG_ERR_CUDA;
+    KernelTimer t(KID_DWCONV_WGRAD, stream);
+    launch_pdl(srem_dwconv_wgrad_sum, dim3((10 * D + 255) / 256), dim3(256), 0, stream, (const float *)partial, dw, dbias,
+               nslab, D);
     return cuda_ok(cudaGetLastError());
 }
 

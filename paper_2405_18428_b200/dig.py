@@ -23,7 +23,8 @@ DIG_ROW_FWD, DIG_ROW_REV, DIG_COL_FWD, DIG_COL_REV = 0, 1, 2, 3
 DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR = 0, 1, 2
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
-           "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_srem_dwconv", "dig_last_device_status",
+           "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
+           "dig_srem_dwconv_bwd_workspace_bytes", "dig_last_device_status",
            "dig_status_string", "dig_profile_enable", "dig_profile_kernels", "dig_profile_read")
 
 _lib = None
@@ -61,6 +62,10 @@ def lib() -> ctypes.CDLL:
         L.dig_gla_bwd.restype = i
         L.dig_srem_dwconv.argtypes = [vp] * 4 + [i] * 6 + [vp]
         L.dig_srem_dwconv.restype = i
+        L.dig_srem_dwconv_bwd_workspace_bytes.argtypes = [i] * 4
+        L.dig_srem_dwconv_bwd_workspace_bytes.restype = ctypes.c_size_t
+        L.dig_srem_dwconv_bwd.argtypes = [vp] * 6 + [i] * 6 + [vp, ctypes.c_size_t, vp]
+        L.dig_srem_dwconv_bwd.restype = i
         L.dig_last_device_status.argtypes = [vp]
         L.dig_last_device_status.restype = i
         L.dig_status_string.argtypes = [i]
@@ -218,6 +223,33 @@ def dig_srem_dwconv(x, w, bias, grid_h, grid_w, direction=DIG_ROW_FWD, *, f32_ou
                                  _dev(y, _out_storage(dtype), x.shape, "y"),
                                  B, grid_h, grid_w, D, direction, dtype, _stream()), "dig_srem_dwconv")
     return y
+
+
+def dig_srem_dwconv_bwd(x, w, dy, grid_h, grid_w, direction=DIG_ROW_FWD, *, with_bias=True, f32_out=False,
+                        workspace=None):
+    """Reverse mode of dig_srem_dwconv: returns (dx, dw, dbias); dw and dbias are fp32, dbias None
+    unless `with_bias`."""
+    B, L, D = x.shape
+    if L != grid_h * grid_w:
+        raise ValueError("x.shape[1] must equal grid_h * grid_w")
+    st = x.dtype
+    dtype = _dtype_of(x, f32_out)
+    need = lib().dig_srem_dwconv_bwd_workspace_bytes(B, grid_h, grid_w, D)
+    if need == 0:
+        raise ValueError("dig_srem_dwconv_bwd: unsupported sizes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+    dx = torch.empty(x.shape, dtype=_out_storage(dtype), device=x.device)
+    dw = torch.empty((3, 3, D), dtype=torch.float32, device=x.device)
+    db = torch.empty((D,), dtype=torch.float32, device=x.device) if with_bias else None
+    _check(lib().dig_srem_dwconv_bwd(_dev(x, st, name="x"), _dev(w, st, (3, 3, D), "w"), _dev(dy, st, x.shape, "dy"),
+                                     _dev(dx, _out_storage(dtype), x.shape, "dx"),
+                                     _dev(dw, torch.float32, (3, 3, D), "dw"),
+                                     None if db is None else _dev(db, torch.float32, (D,), "dbias"),
+                                     B, grid_h, grid_w, D, direction, dtype,
+                                     _dev(workspace, torch.uint8, name="workspace"), workspace.numel(), _stream()),
+           "dig_srem_dwconv_bwd")
+    return dx, dw, db
 
 
 def dig_last_device_status() -> int:

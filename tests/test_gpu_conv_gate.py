@@ -80,3 +80,68 @@ def test_gate_transform(dtype):
     assert np.isfinite(got).all() and (got <= 0).all()
     assert rel_err(got, ref) <= TOL_GATE
     np.testing.assert_allclose(got, ref, rtol=3e-6, atol=1e-30)
+
+
+# ---- reverse mode of the SREM convolution ----------------------------------------------------------
+def _conv_bwd_case(B, gh, gw, D, dtype, direction, with_bias, seed=0):
+    from paper_2405_18428_b200 import dig
+    from parity import rel_err
+    rng = np.random.default_rng(100 + seed)
+    mk = lambda a: round_to_bf16(a.astype(np.float32)) if dtype == "bf16" else a.astype(np.float32)
+    x = mk(rng.standard_normal((B, gh * gw, D)))
+    dy = mk(rng.standard_normal((B, gh * gw, D)))
+    w = mk(rng.standard_normal((3, 3, D)) / 3)
+    rdx, rdw, rdb = oracle.dwconv_bwd(x, w, dy, gh, gw, direction, with_bias)
+    tt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    dev = lambda a: torch.from_numpy(a).cuda().to(tt)
+    dx, dw, db = dig.dig_srem_dwconv_bwd(dev(x), dev(w), dev(dy), gh, gw, direction, with_bias=with_bias, f32_out=True)
+    assert dx.dtype == torch.float32 and dw.dtype == torch.float32
+    assert rel_err(dx.cpu().numpy(), rdx) <= 1e-5            # 9 fp32 FMAs per output
+    assert rel_err(dw.cpu().numpy(), rdw) <= 1e-5            # fp32 sums of B*gh*gw products, blocked
+    if with_bias:
+        assert rel_err(db.cpu().numpy(), rdb) <= 1e-5
+    else:
+        assert db is None and rdb is None
+    if dtype == "bf16":
+        dx16, dw2, _ = dig.dig_srem_dwconv_bwd(dev(x), dev(w), dev(dy), gh, gw, direction, with_bias=False)
+        assert torch.equal(dx16, dx.to(torch.bfloat16))
+        assert torch.equal(dw2, dw)                          # fixed summation order
+
+
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_conv_bwd_small_ragged(direction, dtype):
+    # 2*11*19 = 418 pixels: three full slabs and a ragged one; 72 channels: a partial channel block
+    _conv_bwd_case(2, 11, 19, 72, dtype, direction, with_bias=(direction % 2 == 0), seed=direction)
+
+
+def test_conv_bwd_tiny_grids():
+    for gh, gw in [(1, 1), (1, 5), (3, 1), (2, 2)]:
+        _conv_bwd_case(1, gh, gw, 8, "f32", 2, with_bias=True)
+
+
+@pytest.mark.parametrize("cfg", ["C2", "C5"])
+def test_conv_bwd_benchmark_shapes(cfg):
+    from paper_2405_18428_b200 import dig
+    from parity import rel_err
+    wl = CONFIGS[cfg]
+    x = make_inputs(wl, gla=False, conv=True)
+    D = wl.H * wl.d_v
+    rng = np.random.default_rng(7)
+    dy = round_to_bf16(rng.standard_normal(x["conv_x"].shape).astype(np.float32))
+    xs, ws, dys = (torch.from_numpy(a).cuda().to(torch.bfloat16) for a in (x["conv_x"], x["conv_w"], dy))
+    d = wl.directions[-1]
+    rdx, rdw, rdb = oracle.dwconv_bwd(x["conv_x"], x["conv_w"], dy, wl.grid_h, wl.grid_w, d, True)
+    dx, dw, db = dig.dig_srem_dwconv_bwd(xs, ws, dys, wl.grid_h, wl.grid_w, d, f32_out=True)
+    assert rel_err(dx.cpu().numpy(), rdx) <= 1e-5
+    assert rel_err(dw.cpu().numpy(), rdw) <= 1e-5
+    assert rel_err(db.cpu().numpy(), rdb) <= 1e-5
+
+
+def test_conv_bwd_rejects_short_workspace():
+    from paper_2405_18428_b200 import dig
+    x = torch.zeros(1, 16, 8, device="cuda")
+    w = torch.zeros(3, 3, 8, device="cuda")
+    ws = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(RuntimeError):
+        dig.dig_srem_dwconv_bwd(x, w, x, 4, 4, 0, workspace=ws)
