@@ -50,6 +50,8 @@ def _load():
             lib.dig_oracle_gla_bwd.argtypes = [dp] * 9 + [ctypes.c_int] * 8
             lib.dig_oracle_dwconv.argtypes = [dp] * 4 + [ctypes.c_int] * 5
             lib.dig_oracle_dwconv_bwd.argtypes = [dp] * 6 + [ctypes.c_int] * 5
+            lib.dig_oracle_outgate_fwd.argtypes = [dp] * 5 + [ctypes.c_longlong, ctypes.c_int, ctypes.c_double]
+            lib.dig_oracle_outgate_bwd.argtypes = [dp] * 9 + [ctypes.c_longlong, ctypes.c_int, ctypes.c_double]
             _lib = lib
     return _lib
 
@@ -140,3 +142,36 @@ def dwconv_bwd(x, w, dy, grid_h, grid_w, direction=ROW_FWD, with_bias=True):
     _check(_load().dig_oracle_dwconv_bwd(_p(x), _p(w), _p(dy), _p(dx), _p(dw), None if db is None else _p(db),
                                          B, grid_h, grid_w, D, direction), "dwconv_bwd")
     return dx, dw, db
+
+
+def _opt(a, d):
+    if a is None:
+        return None, None
+    a = _f64(a)
+    assert a.shape == (d,)
+    return a, _p(a)
+
+
+def outgate(o, r, ln_w=None, ln_b=None, eps=1e-5) -> np.ndarray:
+    """z = Swish(r) * LN(o) per row of the last axis (Eq. attn_gla, the line forming Y_t)."""
+    o, r = _f64(o), _f64(r)
+    assert o.shape == r.shape
+    d = o.shape[-1]
+    (_w, wp), (_b, bp) = _opt(ln_w, d), _opt(ln_b, d)
+    z = np.empty_like(o)
+    _check(_load().dig_oracle_outgate_fwd(_p(o), _p(r), wp, bp, _p(z), o.size // d, d, float(eps)), "outgate")
+    return z
+
+
+def outgate_bwd(o, r, dz, ln_w=None, ln_b=None, eps=1e-5):
+    """Gradients (do, dr, dln_w, dln_b) of <dz, outgate(o, r, ln_w, ln_b)>; the affine gradients are
+    those with respect to a weight of ones / a bias of zeros where the argument is None."""
+    o, r, dz = _f64(o), _f64(r), _f64(dz)
+    assert o.shape == r.shape == dz.shape
+    d = o.shape[-1]
+    (_w, wp), (_b, bp) = _opt(ln_w, d), _opt(ln_b, d)
+    do, dr = np.empty_like(o), np.empty_like(o)
+    dw, db = np.empty(d), np.empty(d)
+    _check(_load().dig_oracle_outgate_bwd(_p(o), _p(r), wp, bp, _p(dz), _p(do), _p(dr), _p(dw), _p(db),
+                                          o.size // d, d, float(eps)), "outgate_bwd")
+    return do, dr, dw, db

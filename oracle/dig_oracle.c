@@ -15,6 +15,8 @@
  *   - the 3x3 depthwise convolution of the SREM module (Algorithm 1, "DWConv2d(reshape2d(z))"),
  *     evaluated on the re-oriented token matrix by explicit gather / conv / scatter, and its
  *     reverse-mode derivative
+ *   - the output gate z = Swish(r) (.) LN(o) that follows the recurrence (Eq. attn_gla, the line
+ *     forming Y_t before the projection W_O), and its reverse-mode derivative
  *
  * Everything is token-by-token and element-by-element: no chunking, no blocking, no fused forms.
  * Tensors are dense row-major doubles with layout [B][L][H][d]; L = grid_h*grid_w and the
@@ -26,7 +28,10 @@
  * backward pass, the suffix-sum gate-gradient identity, identity-initialised convolution,
  * convolution against hand-evaluated corner / edge / interior counts; for the convolution's
  * derivative: central finite differences, the adjoint identity <dy, conv(x)> = <dx, x>, and
- * dw of an identity-initialised filter on a one-pixel image.
+ * dw of an identity-initialised filter on a one-pixel image; for the output gate: a library
+ * layer-norm and silu on the same rows, zero-mean / unit-variance and shift-scale invariance of
+ * the normalisation, Swish's values at 0 and far from 0, central finite differences of the
+ * derivative, and do summing to zero over a row when the affine part is absent.
  * Not pinned by the paper: whether DWConv2d carries a bias (the argument is optional).
  */
 #include <math.h>
@@ -328,4 +333,81 @@ int dig_oracle_has_openmp(void)
 #else
     return 0;
 #endif
+}
+
+/* ---- output gate of the GLA layer -------------------------------------------------------------------
+ * Eq. attn_gla, the line that forms Y_t before the output projection: per (token, head) row o of
+ * length d_v and gate pre-activation r = X_t W_r + b_r of the same length,
+ *     z = Swish(r) (.) LN(o),    Swish(r) = r * sigmoid(r),
+ *     LN(o)_e = (o_e - mean(o)) / sqrt(var(o) + eps) * ln_w[e] + ln_b[e],
+ * mean and (biased) variance over the d_v entries of the row.  The paper does not say what LN
+ * normalises over, nor whether it has an affine part or which eps: this reading takes one row per
+ * head, an optional affine part shared by all heads (NULL = weight 1 / bias 0) and eps as an
+ * argument.  rows = B * L * H. */
+int dig_oracle_outgate_fwd(const double *o, const double *r, const double *ln_w, const double *ln_b,
+                           double *z, long long rows, int d_v, double eps)
+{
+    if (rows < 0 || d_v <= 0) return 1;
+    for (long long i = 0; i < rows; ++i) {
+        const double *oi = o + (size_t)i * d_v, *ri = r + (size_t)i * d_v;
+        double mean = 0.0, var = 0.0;
+        for (int e = 0; e < d_v; ++e) mean += oi[e];
+        mean /= d_v;
+        for (int e = 0; e < d_v; ++e) var += (oi[e] - mean) * (oi[e] - mean);
+        var /= d_v;
+        const double rstd = 1.0 / sqrt(var + eps);
+        for (int e = 0; e < d_v; ++e) {
+            const double y = (oi[e] - mean) * rstd * (ln_w ? ln_w[e] : 1.0) + (ln_b ? ln_b[e] : 0.0);
+            const double sg = 1.0 / (1.0 + exp(-ri[e]));
+            z[(size_t)i * d_v + e] = ri[e] * sg * y;
+        }
+    }
+    return 0;
+}
+
+/* Reverse mode of the above (not printed in the paper): given dz, the gradients with respect to o, r
+ * and the affine part.  With n = (o - mean) * rstd, y = n * w + b, s = Swish(r):
+ *   dr = dz * y * s'(r),  s'(r) = sg + r * sg * (1 - sg);   dy = dz * s;
+ *   dln_w = sum over rows of dy * n;  dln_b = sum over rows of dy;   dn = dy * w;
+ *   do = rstd * (dn - mean(dn) - n * mean(dn * n))   (the derivative of the normalisation). */
+int dig_oracle_outgate_bwd(const double *o, const double *r, const double *ln_w, const double *ln_b,
+                           const double *dz, double *d_o, double *d_r, double *dln_w, double *dln_b,
+                           long long rows, int d_v, double eps)
+{
+    if (rows < 0 || d_v <= 0) return 1;
+    double *n = (double *)malloc(sizeof(double) * (size_t)d_v);
+    double *dn = (double *)malloc(sizeof(double) * (size_t)d_v);
+    if (!n || !dn) { free(n); free(dn); return 2; }
+    if (dln_w) memset(dln_w, 0, sizeof(double) * (size_t)d_v);
+    if (dln_b) memset(dln_b, 0, sizeof(double) * (size_t)d_v);
+    for (long long i = 0; i < rows; ++i) {
+        const double *oi = o + (size_t)i * d_v, *ri = r + (size_t)i * d_v, *gi = dz + (size_t)i * d_v;
+        double mean = 0.0, var = 0.0;
+        for (int e = 0; e < d_v; ++e) mean += oi[e];
+        mean /= d_v;
+        for (int e = 0; e < d_v; ++e) var += (oi[e] - mean) * (oi[e] - mean);
+        var /= d_v;
+        const double rstd = 1.0 / sqrt(var + eps);
+        double m1 = 0.0, m2 = 0.0;
+        for (int e = 0; e < d_v; ++e) {
+            const double w = ln_w ? ln_w[e] : 1.0, b = ln_b ? ln_b[e] : 0.0;
+            n[e] = (oi[e] - mean) * rstd;
+            const double y = n[e] * w + b;
+            const double sg = 1.0 / (1.0 + exp(-ri[e]));
+            const double s = ri[e] * sg;
+            d_r[(size_t)i * d_v + e] = gi[e] * y * (sg + ri[e] * sg * (1.0 - sg));
+            const double dy = gi[e] * s;
+            if (dln_w) dln_w[e] += dy * n[e];
+            if (dln_b) dln_b[e] += dy;
+            dn[e] = dy * w;
+            m1 += dn[e];
+            m2 += dn[e] * n[e];
+        }
+        m1 /= d_v;
+        m2 /= d_v;
+        for (int e = 0; e < d_v; ++e) d_o[(size_t)i * d_v + e] = rstd * (dn[e] - m1 - n[e] * m2);
+    }
+    free(n);
+    free(dn);
+    return 0;
 }
