@@ -149,6 +149,27 @@ dig_status dig_srem_dwconv_bwd(const void *x, const void *w, const void *dy, voi
                                int B, int grid_h, int grid_w, int D, int direction, int dtype, void *workspace,
                                size_t workspace_bytes, void *cuda_stream);
 
+/* Output gate of the GLA layer (Eq. attn_gla, the line that forms Y_t before the projection W_O):
+ *     z = Swish(r) (.) LN(o),   Swish(r) = r * sigmoid(r),
+ * per row of d_v values; `rows` = B * L * H rows of the [B][L][H][d_v] tensors o (the output of
+ * dig_gla_fwd), r (the gate pre-activation X W_r + b_r) and z, in the storage types of `dtype`.
+ * The paper does not fix LN further; here it normalises each (token, head) row over its d_v values
+ * (biased variance, `eps` added under the root) and applies an optional affine part shared by all
+ * heads: ln_w, ln_b are fp32 [d_v] device arrays or NULL (weight 1 / bias 0).
+ * d_v: a multiple of 8, at most 128.  fp32 arithmetic. */
+dig_status dig_gla_outgate_fwd(const void *o, const void *r, const float *ln_w, const float *ln_b, void *z,
+                               long long rows, int d_v, float eps, int dtype, void *cuda_stream);
+
+/* Reverse mode of dig_gla_outgate_fwd (not printed in the paper): from dz = dL/dz computes d_o and d_r
+ * (output storage type of `dtype`) and, where the pointer is not NULL, dln_w and dln_b (fp32 [d_v]; the
+ * gradients at weight 1 / bias 0 where ln_w / ln_b is NULL), summed over all rows in a fixed order.
+ * The workspace (dig_gla_outgate_bwd_workspace_bytes; 0 for invalid sizes) holds per-CTA partial sums
+ * and is needed only when dln_w or dln_b is requested. */
+size_t dig_gla_outgate_bwd_workspace_bytes(long long rows, int d_v);
+dig_status dig_gla_outgate_bwd(const void *o, const void *r, const float *ln_w, const float *ln_b, const void *dz,
+                               void *d_o, void *d_r, float *dln_w, float *dln_b, long long rows, int d_v, float eps,
+                               int dtype, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the status recorded by device code on the
  * current device: DIG_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last query,
  * DIG_ERR_CUDA if the synchronisation itself failed, DIG_OK otherwise. */

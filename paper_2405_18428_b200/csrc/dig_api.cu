@@ -11,6 +11,12 @@ dig_status launch_gate(const void *g, const float *tau_host, float *gate, int B,
                        int dk, int dtype, cudaStream_t stream);
 dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y, int B, int gh,
                          int gw, int D, int dir, int dtype, cudaStream_t stream);
+size_t outgate_bwd_workspace_bytes(long long rows, int dv);
+dig_status launch_outgate_fwd(const void *o, const void *r, const float *ln_w, const float *ln_b, void *z,
+                              long long rows, int dv, float eps, int dtype, cudaStream_t stream);
+dig_status launch_outgate_bwd(const void *o, const void *r, const void *dz, const float *ln_w, const float *ln_b,
+                              void *d_o, void *d_r, float *dln_w, float *dln_b, long long rows, int dv, float eps,
+                              int dtype, float *partial, cudaStream_t stream);
 size_t dwconv_bwd_workspace_bytes(int B, int gh, int gw, int D);
 dig_status launch_dwconv_bwd(const void *x, const void *w, const void *dy, void *dx, float *dw, float *dbias,
                              int B, int gh, int gw, int D, int dir, int dtype, float *partial, cudaStream_t stream);
@@ -67,7 +73,7 @@ int choose_impl(int dk, int dv, int chunk, int dtype, bool backward)
 namespace {
 constexpr int kMaxTimed = 32768;
 const char *const kKernelNames[KID_COUNT] = {
-    "gate_logsigmoid", "srem_dwconv3x3", "srem_dwconv_wgrad", "state_scan_fwd", "state_scan_bwd",
+    "gate_logsigmoid", "srem_dwconv3x3", "srem_dwconv_wgrad", "gla_outgate", "state_scan_fwd", "state_scan_bwd",
     "fma_chunk_state", "fma_chunk_out", "fma_chunk_bwd",
     "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd"};
 struct Profile {
@@ -233,6 +239,40 @@ dig_status dig_srem_dwconv_bwd(const void *x, const void *w, const void *dy, voi
     if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
     return launch_dwconv_bwd(x, w, dy, dx, dw, dbias, B, grid_h, grid_w, D, direction, dtype,
                              reinterpret_cast<float *>(workspace), (cudaStream_t)cuda_stream);
+}
+
+static bool outgate_sizes_ok(long long rows, int d_v, float eps)
+{
+    return rows > 0 && rows <= (1ll << 40) && d_v > 0 && d_v <= 128 && (d_v % 8) == 0 && eps >= 0.f;
+}
+
+dig_status dig_gla_outgate_fwd(const void *o, const void *r, const float *ln_w, const float *ln_b, void *z,
+                               long long rows, int d_v, float eps, int dtype, void *cuda_stream)
+{
+    if (!o || !r || !z || !aligned16(o) || !aligned16(r) || !aligned16(z)) return DIG_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype) || !outgate_sizes_ok(rows, d_v, eps)) return DIG_ERR_INVALID_ARG;
+    return launch_outgate_fwd(o, r, ln_w, ln_b, z, rows, d_v, eps, dtype, (cudaStream_t)cuda_stream);
+}
+
+size_t dig_gla_outgate_bwd_workspace_bytes(long long rows, int d_v)
+{
+    if (!outgate_sizes_ok(rows, d_v, 0.f)) return 0;
+    return outgate_bwd_workspace_bytes(rows, d_v);
+}
+
+dig_status dig_gla_outgate_bwd(const void *o, const void *r, const float *ln_w, const float *ln_b, const void *dz,
+                               void *d_o, void *d_r, float *dln_w, float *dln_b, long long rows, int d_v, float eps,
+                               int dtype, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!o || !r || !dz || !d_o || !d_r) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(o) || !aligned16(r) || !aligned16(dz) || !aligned16(d_o) || !aligned16(d_r)) return DIG_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype) || !outgate_sizes_ok(rows, d_v, eps)) return DIG_ERR_INVALID_ARG;
+    if (dln_w || dln_b) {
+        const size_t need = outgate_bwd_workspace_bytes(rows, d_v);
+        if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    }
+    return launch_outgate_bwd(o, r, dz, ln_w, ln_b, d_o, d_r, dln_w, dln_b, rows, d_v, eps, dtype,
+                              reinterpret_cast<float *>(workspace), (cudaStream_t)cuda_stream);
 }
 
 dig_status dig_last_device_status(void *cuda_stream)

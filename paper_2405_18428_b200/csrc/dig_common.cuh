@@ -137,7 +137,7 @@ dig_status launch_tc_bwd(const GlaArgs &a, const Workspace &w, int sm_count, int
 // Optional per-kernel timing (dig_profile_*): when enabled, every launch site brackets its
 // kernel with two CUDA events on the launching stream.
 enum KernelId {
-    KID_GATE = 0, KID_DWCONV, KID_DWCONV_WGRAD, KID_SCAN_FWD, KID_SCAN_BWD,
+    KID_GATE = 0, KID_DWCONV, KID_DWCONV_WGRAD, KID_OUTGATE, KID_SCAN_FWD, KID_SCAN_BWD,
     KID_FMA_STATE, KID_FMA_OUT, KID_FMA_BWD,
     KID_TC_STATE, KID_TC_OUT, KID_TC_BWD,
     KID_COUNT

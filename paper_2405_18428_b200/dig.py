@@ -24,7 +24,8 @@ DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR = 0, 1, 2
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
            "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
-           "dig_srem_dwconv_bwd_workspace_bytes", "dig_last_device_status",
+           "dig_srem_dwconv_bwd_workspace_bytes", "dig_gla_outgate_fwd", "dig_gla_outgate_bwd",
+           "dig_gla_outgate_bwd_workspace_bytes", "dig_last_device_status",
            "dig_status_string", "dig_profile_enable", "dig_profile_kernels", "dig_profile_read")
 
 _lib = None
@@ -66,6 +67,13 @@ def lib() -> ctypes.CDLL:
         L.dig_srem_dwconv_bwd_workspace_bytes.restype = ctypes.c_size_t
         L.dig_srem_dwconv_bwd.argtypes = [vp] * 6 + [i] * 6 + [vp, ctypes.c_size_t, vp]
         L.dig_srem_dwconv_bwd.restype = i
+        ll, fl = ctypes.c_longlong, ctypes.c_float
+        L.dig_gla_outgate_fwd.argtypes = [vp] * 5 + [ll, i, fl, i, vp]
+        L.dig_gla_outgate_fwd.restype = i
+        L.dig_gla_outgate_bwd_workspace_bytes.argtypes = [ll, i]
+        L.dig_gla_outgate_bwd_workspace_bytes.restype = ctypes.c_size_t
+        L.dig_gla_outgate_bwd.argtypes = [vp] * 9 + [ll, i, fl, i, vp, ctypes.c_size_t, vp]
+        L.dig_gla_outgate_bwd.restype = i
         L.dig_last_device_status.argtypes = [vp]
         L.dig_last_device_status.restype = i
         L.dig_status_string.argtypes = [i]
@@ -270,3 +278,45 @@ def dig_profile_read() -> dict:
         if n.value:
             out[name.value.decode()] = (n.value, ms.value)
     return out
+
+
+def _affine(t, d, name):
+    return None if t is None else _dev(t, torch.float32, (d,), name)
+
+
+def dig_gla_outgate_fwd(o, r, ln_w=None, ln_b=None, eps=1e-5, *, f32_out=False):
+    """z = Swish(r) * LN(o) over the last axis; o, r: [..., d_v]; ln_w, ln_b: fp32 [d_v] or None."""
+    d = o.shape[-1]
+    dtype = _dtype_of(o, f32_out)
+    z = torch.empty(o.shape, dtype=_out_storage(dtype), device=o.device)
+    _check(lib().dig_gla_outgate_fwd(_dev(o, o.dtype, name="o"), _dev(r, o.dtype, o.shape, "r"),
+                                     _affine(ln_w, d, "ln_w"), _affine(ln_b, d, "ln_b"),
+                                     _dev(z, z.dtype, name="z"), o.numel() // d, d, float(eps), dtype, _stream()),
+           "dig_gla_outgate_fwd")
+    return z
+
+
+def dig_gla_outgate_bwd(o, r, dz, ln_w=None, ln_b=None, eps=1e-5, *, affine_grads=True, f32_out=False,
+                        workspace=None):
+    """Returns (d_o, d_r, dln_w, dln_b); the last two are fp32 [d_v], or None without `affine_grads`."""
+    d = o.shape[-1]
+    rows = o.numel() // d
+    dtype = _dtype_of(o, f32_out)
+    d_o = torch.empty(o.shape, dtype=_out_storage(dtype), device=o.device)
+    d_r = torch.empty_like(d_o)
+    dw = db = None
+    wsp, wsn = None, 0
+    if affine_grads:
+        dw = torch.empty(d, dtype=torch.float32, device=o.device)
+        db = torch.empty(d, dtype=torch.float32, device=o.device)
+        if workspace is None:
+            workspace = torch.empty(lib().dig_gla_outgate_bwd_workspace_bytes(rows, d), dtype=torch.uint8,
+                                    device=o.device)
+        wsp, wsn = _dev(workspace, torch.uint8, name="workspace"), workspace.numel()
+    _check(lib().dig_gla_outgate_bwd(_dev(o, o.dtype, name="o"), _dev(r, o.dtype, o.shape, "r"),
+                                     _affine(ln_w, d, "ln_w"), _affine(ln_b, d, "ln_b"),
+                                     _dev(dz, o.dtype, o.shape, "dz"), _dev(d_o, d_o.dtype, name="d_o"),
+                                     _dev(d_r, d_r.dtype, name="d_r"),
+                                     None if dw is None else dw.data_ptr(), None if db is None else db.data_ptr(),
+                                     rows, d, float(eps), dtype, wsp, wsn, _stream()), "dig_gla_outgate_bwd")
+    return d_o, d_r, dw, db
