@@ -44,8 +44,9 @@ __device__ __forceinline__ void load_raw(BwdRaw &r, const bf16 *q, const bf16 *k
     r.k = ldg16(k + off);
     r.v = ldg16(v + off);
     r.d = ldg16(d_out + off);
-    r.gt[0] = ldg16(gate + off);
-    r.gt[1] = ldg16(gate + off + 4);
+    const int fl = col >= 32 ? 4 : 0;         // flipped lanes hold their upper four columns first
+    r.gt[0] = ldg16(gate + off + fl);
+    r.gt[1] = ldg16(gate + off + 4 - fl);
 }
 
 // State entering the chunk, and the decayed state gradient leaving it in both tile orders:
@@ -118,9 +119,9 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
             carry_in = __ldg(carry + (size_t)id * DK + (threadIdx.x & 63));
             sync_group(NT);              // the previous chunk's results have left the staging area
             float x[8];
-            unpack8(raw.v, x, keep);
+            unpack8(raw.v, x, keep, flip);
             st_k8<T, false>(tVk, row, col, x, flip);
-            unpack8(raw.d, x, keep);
+            unpack8(raw.d, x, keep, flip);
             st_k8<T, false>(tGk, row, col, x, flip);
             st_m8<T, false>(tGm, row, col, x, flip);
             fence_async_smem();
@@ -140,19 +141,20 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
             {
                 const float sc = keep ? kLog2e : 0.f;
                 float *dst = sLam + row * kLamPitch + col;
-                *reinterpret_cast<float4 *>(dst) = make_float4(raw.gt[0].x * sc, raw.gt[0].y * sc, raw.gt[0].z * sc, raw.gt[0].w * sc);
-                *reinterpret_cast<float4 *>(dst + 4) = make_float4(raw.gt[1].x * sc, raw.gt[1].y * sc, raw.gt[1].z * sc, raw.gt[1].w * sc);
+                const int fl = flip ? 4 : 0;
+                *reinterpret_cast<float4 *>(dst + fl) = make_float4(raw.gt[0].x * sc, raw.gt[0].y * sc, raw.gt[0].z * sc, raw.gt[0].w * sc);
+                *reinterpret_cast<float4 *>(dst + 4 - fl) = make_float4(raw.gt[1].x * sc, raw.gt[1].y * sc, raw.gt[1].z * sc, raw.gt[1].w * sc);
             }
             sync_group(NT);
             gate_prefix<NT, 1, true>(sLam, sLast, sTot);
             float lam[8], x[8];
-            read_lam8(sLam, row, col, lam);
-            unpack8(raw.q, x, keep);
+            read_lam8(sLam, row, col, lam, flip);
+            unpack8(raw.q, x, keep, flip);
 #pragma unroll
             for (int e = 0; e < 8; ++e) x[e] = to_tf32(x[e] * ex2(lam[e]));
             st_k8<T, false>(tQk, row, col, x, flip);
             st_m8<T, false>(tQm, row, col, x, flip);
-            unpack8(raw.k, x, keep);
+            unpack8(raw.k, x, keep, flip);
 #pragma unroll
             for (int e = 0; e < 8; ++e) x[e] = to_tf32(x[e] * ex2(-lam[e]));
             st_k8<T, false>(tKk, row, col, x, flip);

@@ -42,8 +42,9 @@ __device__ __forceinline__ void load_raw(OutRaw &r, const bf16 *q, const bf16 *k
         r.q[half] = ldg16(q + off);
         r.k[half] = ldg16(k + off);
         r.v[half] = ldg16(v + off);
-        r.g0[half] = ldg16(gate + off);
-        r.g1[half] = ldg16(gate + off + 4);
+        const int fl = col >= 32 ? 4 : 0;     // flipped lanes hold their upper four columns first
+        r.g0[half] = ldg16(gate + off + fl);
+        r.g1[half] = ldg16(gate + off + 4 - fl);
     }
 }
 
@@ -116,9 +117,10 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
             for (int half = 0; half < 2; ++half) {
                 const float sc = (cur[half].valid && cur[half].chunk * T + row < g.L) ? kLog2e : 0.f;
                 float *dst = sLam + (64 * half + row) * kLamPitch + col;
-                *reinterpret_cast<float4 *>(dst) =
+                const int fl = flip ? 4 : 0;
+                *reinterpret_cast<float4 *>(dst + fl) =
                     make_float4(raw.g0[half].x * sc, raw.g0[half].y * sc, raw.g0[half].z * sc, raw.g0[half].w * sc);
-                *reinterpret_cast<float4 *>(dst + 4) =
+                *reinterpret_cast<float4 *>(dst + 4 - fl) =
                     make_float4(raw.g1[half].x * sc, raw.g1[half].y * sc, raw.g1[half].z * sc, raw.g1[half].w * sc);
             }
             sync_group(NT);
@@ -127,16 +129,16 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
             for (int half = 0; half < 2; ++half) {
                 const bool keep = cur[half].valid && cur[half].chunk * T + row < g.L;
                 float lam[8], x[8];
-                read_lam8(sLam, 64 * half + row, col, lam);
-                unpack8(raw.q[half], x, keep);
+                read_lam8(sLam, 64 * half + row, col, lam, flip);
+                unpack8(raw.q[half], x, keep, flip);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) x[e] *= ex2(lam[e]);
                 st_k8<128>(tQ, 64 * half + row, col, x, flip);
-                unpack8(raw.k[half], x, keep);
+                unpack8(raw.k[half], x, keep, flip);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) x[e] *= ex2(-lam[e]);
                 st_k8<128>(tK, 64 * half + row, col, x, flip);
-                unpack8(raw.v[half], x, keep);
+                unpack8(raw.v[half], x, keep, flip);
                 st_m8<T, false>(tV, row, 64 * half + col, x, flip);
             }
             fence_async_smem();

@@ -52,8 +52,9 @@ __device__ __forceinline__ void load_raw(StateRaw<NT, BWD> &r, const bf16 *q, co
             r.q[i] = ldg16(q + off);
             r.d[i] = ldg16(d_out + off);
         }
-        r.g0[i] = ldg16(gate + off);
-        r.g1[i] = ldg16(gate + off + 4);
+        const int fl = col >= 32 ? 4 : 0;     // flipped lanes hold their upper four columns first
+        r.g0[i] = ldg16(gate + off + fl);
+        r.g1[i] = ldg16(gate + off + 4 - fl);
     }
 }
 
@@ -102,8 +103,9 @@ tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16
             const Item ci = pick(ca, cb, half);
             const float sc = (ci.valid && ci.chunk * T + row < g.L) ? kLog2e : 0.f;
             float *dst = sLam + (64 * half + row) * kLamPitch + col;
-            *reinterpret_cast<float4 *>(dst) = make_float4(raw.g0[i].x * sc, raw.g0[i].y * sc, raw.g0[i].z * sc, raw.g0[i].w * sc);
-            *reinterpret_cast<float4 *>(dst + 4) = make_float4(raw.g1[i].x * sc, raw.g1[i].y * sc, raw.g1[i].z * sc, raw.g1[i].w * sc);
+            const int fl = col >= 32 ? 4 : 0;
+            *reinterpret_cast<float4 *>(dst + fl) = make_float4(raw.g0[i].x * sc, raw.g0[i].y * sc, raw.g0[i].z * sc, raw.g0[i].w * sc);
+            *reinterpret_cast<float4 *>(dst + 4 - fl) = make_float4(raw.g1[i].x * sc, raw.g1[i].y * sc, raw.g1[i].z * sc, raw.g1[i].w * sc);
         }
         __syncthreads();
         gate_prefix<NT, 2>(sLam, sLast, sTot);
@@ -120,19 +122,21 @@ tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16
             const Item ci = pick(ca, cb, half);
             const bool keep = ci.valid && ci.chunk * T + row < g.L;
             float lam[8], x[8];
-            read_lam8(sLam, 64 * half + row, col, lam);
-            unpack8(raw.k[i], x, keep);
+            read_lam8(sLam, 64 * half + row, col, lam, flip);
+            float last[8];
+            read_lam8(sLast, 0, 64 * half + col, last, flip);       // chunk totals of the same columns
+            unpack8(raw.k[i], x, keep, flip);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) x[e] *= ex2(sLast[64 * half + col + e] - lam[e]);
+            for (int e = 0; e < 8; ++e) x[e] *= ex2(last[e] - lam[e]);
             st_m8<T>(tKh, row, 64 * half + col, x, flip);
-            unpack8(raw.v[i], x, keep);
+            unpack8(raw.v[i], x, keep, flip);
             st_m8<T, false>(tV, row, 64 * half + col, x, flip);
             if (BWD) {
-                unpack8(raw.q[i], x, keep);
+                unpack8(raw.q[i], x, keep, flip);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) x[e] *= ex2(lam[e]);
                 st_m8<T>(tQ, row, 64 * half + col, x, flip);
-                unpack8(raw.d[i], x, keep);
+                unpack8(raw.d[i], x, keep, flip);
                 st_m8<T, false>(tG, row, 64 * half + col, x, flip);
             }
         }

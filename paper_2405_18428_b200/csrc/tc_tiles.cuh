@@ -78,10 +78,15 @@ __device__ __forceinline__ float4 ld_row4(const float *base, const Geom &g, int 
     return __ldg(reinterpret_cast<const float4 *>(base + tok_offset(g, b, tok < 0 ? 0 : tok, h, d) + col));
 }
 // `keep` = false turns the row into zeros.
-__device__ __forceinline__ void unpack8(const uint4 &u, float (&f)[8], bool keep = true)
+// `flip`: the lanes that hold columns 32-63 of a row keep the two 4-column halves of their 8 columns
+// exchanged in registers (f[0..3] = columns col8+4..col8+7) and store the upper half first.  The 8
+// lanes that serve one 16-byte store phase then hit 8 different bank groups of an operand tile or of
+// the gate table; in natural order lane j and lane j+4 collide.  The tile stores, the gate loads and
+// read_lam8 take the same flag, so the exchange costs four selects per input vector and nothing else.
+__device__ __forceinline__ void unpack8(const uint4 &u, float (&f)[8], bool keep = true, bool flip = false)
 {
     const uint32_t m = keep ? 0xffffffffu : 0u;
-    const uint32_t w[4] = {u.x & m, u.y & m, u.z & m, u.w & m};
+    const uint32_t w[4] = {(flip ? u.z : u.x) & m, (flip ? u.w : u.y) & m, (flip ? u.x : u.z) & m, (flip ? u.y : u.w) & m};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         f[2 * i] = __uint_as_float(w[i] << 16);
@@ -103,9 +108,9 @@ __device__ __forceinline__ void st_k8(char *tile, int row, int col8, const float
     const int c = (col8 & 31) >> 2, s = row & 7;
     const float4 lo = ROUND ? tf32x4(f[0], f[1], f[2], f[3]) : make_float4(f[0], f[1], f[2], f[3]);
     const float4 hi = ROUND ? tf32x4(f[4], f[5], f[6], f[7]) : make_float4(f[4], f[5], f[6], f[7]);
-    float4 *p0 = reinterpret_cast<float4 *>(base + ((c ^ s) << 4));
-    float4 *p1 = reinterpret_cast<float4 *>(base + (((c + 1) ^ s) << 4));
-    (void)flip;          // a lane-dependent store order would diverge the warp and costs more than the bank conflict it avoids
+    const int fl = flip ? 1 : 0;          // f[0..3] belong to piece c + fl (see unpack8)
+    float4 *p0 = reinterpret_cast<float4 *>(base + (((c + fl) ^ s) << 4));
+    float4 *p1 = reinterpret_cast<float4 *>(base + (((c + 1 - fl) ^ s) << 4));
     *p0 = lo;
     *p1 = hi;
 }
@@ -115,8 +120,8 @@ __device__ __forceinline__ void st_m8(char *tile, int row, int col8, const float
     char *base = tile + (col8 >> 5) * (ROWS * 128) + row * 128 + (((((col8 & 31) >> 3)) ^ (row & 3)) << 5);
     const float4 lo = ROUND ? tf32x4(f[0], f[1], f[2], f[3]) : make_float4(f[0], f[1], f[2], f[3]);
     const float4 hi = ROUND ? tf32x4(f[4], f[5], f[6], f[7]) : make_float4(f[4], f[5], f[6], f[7]);
-    float4 *p0 = reinterpret_cast<float4 *>(base), *p1 = reinterpret_cast<float4 *>(base + 16);
-    (void)flip;          // a lane-dependent store order would diverge the warp and costs more than the bank conflict it avoids
+    const int fl = flip ? 16 : 0;         // f[0..3] belong to the upper 16 bytes of the atom in flipped lanes
+    float4 *p0 = reinterpret_cast<float4 *>(base + fl), *p1 = reinterpret_cast<float4 *>(base + 16 - fl);
     *p0 = lo;
     *p1 = hi;
 }
@@ -200,10 +205,11 @@ __device__ __forceinline__ void fetch_gate_rows(float *sLam, const float *gate, 
     }
 }
 
-__device__ __forceinline__ void read_lam8(const float *sLam, int row, int col8, float (&lam)[8])
+__device__ __forceinline__ void read_lam8(const float *sLam, int row, int col8, float (&lam)[8], bool flip = false)
 {
-    const float4 a = *reinterpret_cast<const float4 *>(sLam + row * kLamPitch + col8);
-    const float4 b = *reinterpret_cast<const float4 *>(sLam + row * kLamPitch + col8 + 4);
+    const int fl = flip ? 4 : 0;
+    const float4 a = *reinterpret_cast<const float4 *>(sLam + row * kLamPitch + col8 + fl);
+    const float4 b = *reinterpret_cast<const float4 *>(sLam + row * kLamPitch + col8 + 4 - fl);
     lam[0] = a.x; lam[1] = a.y; lam[2] = a.z; lam[3] = a.w; lam[4] = b.x; lam[5] = b.y; lam[6] = b.z; lam[7] = b.w;
 }
 
