@@ -47,12 +47,15 @@ typedef enum { DIG_F32 = 0, DIG_BF16 = 1, DIG_BF16_F32OUT = 2 } dig_dtype;
  * "flip" and "transpose" of the reshaped token matrix block by block). */
 typedef enum { DIG_ROW_FWD = 0, DIG_ROW_REV = 1, DIG_COL_FWD = 2, DIG_COL_REV = 3 } dig_dir;
 
-/* Which kernel family serves a call.  AUTO picks the tensor-core kernels when they cover the
- * request and the fp32-FMA kernels otherwise.  Forcing a family that does not cover the request
- * returns DIG_ERR_UNSUPPORTED.  Process-wide; meant for tests and benchmarks. */
-typedef enum { DIG_IMPL_AUTO = 0, DIG_IMPL_FMA = 1, DIG_IMPL_TENSOR = 2 } dig_impl;
+/* Which kernel family serves a call.  AUTO picks the tcgen05 tensor-core kernels (TENSOR) when they
+ * cover the request (bf16 storage, d_k = d_v = 64, chunks of 64 or 128), else the warp-level
+ * tensor-core kernels (MMA: bf16 storage, any supported head and chunk size that fits shared
+ * memory), else the fp32-FMA kernels (fp32 storage, whose products must be fp32-accurate).  Forcing
+ * a family that does not cover the request returns DIG_ERR_UNSUPPORTED.  Process-wide; meant for
+ * tests and benchmarks. */
+typedef enum { DIG_IMPL_AUTO = 0, DIG_IMPL_FMA = 1, DIG_IMPL_TENSOR = 2, DIG_IMPL_MMA = 3 } dig_impl;
 dig_status dig_set_impl(int impl);
-/* The family the next call with these parameters would use (DIG_IMPL_FMA or DIG_IMPL_TENSOR),
+/* The family the next call with these parameters would use (DIG_IMPL_FMA, _TENSOR or _MMA),
  * or a negative dig_status if no family covers it. */
 int dig_gla_query_impl(int d_k, int d_v, int chunk, int dtype, int backward);
 

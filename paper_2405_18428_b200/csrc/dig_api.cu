@@ -50,7 +50,7 @@ Geom make_geom(int B, int H, int gh, int gw, int dk, int dv, int chunk, int dir)
     return g;
 }
 
-// DIG_IMPL_FMA / DIG_IMPL_TENSOR, or a negative status.
+// DIG_IMPL_FMA / DIG_IMPL_TENSOR / DIG_IMPL_MMA, or a negative status.
 // The tensor-core kernels hold 64 tokens per tile; a request for chunks of 128 is evaluated by them
 // with 64-token tiles (the result does not depend on the chunk size beyond rounding).
 int tile_chunk(int impl, int chunk) { return (impl == DIG_IMPL_TENSOR && chunk == 128) ? 64 : chunk; }
@@ -60,9 +60,12 @@ int choose_impl(int dk, int dv, int chunk, int dtype, bool backward)
     const int want = g_impl.load();
     const bool t_ok = tensor_supports(dk, dv, chunk, dtype, backward);
     const bool f_ok = fma_supports(dk, dv, chunk, dtype, backward);
+    const bool m_ok = mma_supports(dk, dv, chunk, dtype, backward);
     if (want == DIG_IMPL_TENSOR) return t_ok ? DIG_IMPL_TENSOR : -(int)DIG_ERR_UNSUPPORTED;
     if (want == DIG_IMPL_FMA) return f_ok ? DIG_IMPL_FMA : -(int)DIG_ERR_UNSUPPORTED;
+    if (want == DIG_IMPL_MMA) return m_ok ? DIG_IMPL_MMA : -(int)DIG_ERR_UNSUPPORTED;
     if (t_ok) return DIG_IMPL_TENSOR;
+    if (m_ok) return DIG_IMPL_MMA;
     if (f_ok) return DIG_IMPL_FMA;
     return -(int)DIG_ERR_UNSUPPORTED;
 }
@@ -75,6 +78,7 @@ constexpr int kMaxTimed = 32768;
 const char *const kKernelNames[KID_COUNT] = {
     "gate_logsigmoid", "srem_dwconv3x3", "srem_dwconv_wgrad", "gla_outgate", "state_scan_fwd", "state_scan_bwd",
     "fma_chunk_state", "fma_chunk_out", "fma_chunk_bwd",
+    "mma_chunk_state", "mma_chunk_out", "mma_chunk_bwd",
     "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd"};
 struct Profile {
     bool on = false;
@@ -133,7 +137,7 @@ extern "C" {
 
 dig_status dig_set_impl(int impl)
 {
-    if (impl < DIG_IMPL_AUTO || impl > DIG_IMPL_TENSOR) return DIG_ERR_INVALID_ARG;
+    if (impl < DIG_IMPL_AUTO || impl > DIG_IMPL_MMA) return DIG_ERR_INVALID_ARG;
     g_impl.store(impl);
     return DIG_OK;
 }
@@ -182,7 +186,7 @@ dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float 
     a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
     a.dtype = dtype;
     a.stream = (cudaStream_t)cuda_stream;
-    return impl == DIG_IMPL_TENSOR ? tensor_gla_fwd(a) : fma_gla_fwd(a);
+    return impl == DIG_IMPL_TENSOR ? tensor_gla_fwd(a) : impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
 }
 
 dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float *gate,
@@ -206,7 +210,7 @@ dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float 
     a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
     a.dtype = dtype;
     a.stream = (cudaStream_t)cuda_stream;
-    return impl == DIG_IMPL_TENSOR ? tensor_gla_bwd(a) : fma_gla_bwd(a);
+    return impl == DIG_IMPL_TENSOR ? tensor_gla_bwd(a) : impl == DIG_IMPL_MMA ? mma_gla_bwd(a) : fma_gla_bwd(a);
 }
 
 dig_status dig_srem_dwconv(const void *x, const void *w, const void *bias, void *y, int B,

@@ -113,6 +113,9 @@ inline Workspace carve_workspace(float *base, const Geom &g, bool backward)
 dig_status fma_gla_fwd(const GlaArgs &a);
 dig_status fma_gla_bwd(const GlaArgs &a);
 bool fma_supports(int dk, int dv, int chunk, int dtype, bool backward);
+dig_status mma_gla_fwd(const GlaArgs &a);
+dig_status mma_gla_bwd(const GlaArgs &a);
+bool mma_supports(int dk, int dv, int chunk, int dtype, bool backward);
 dig_status tensor_gla_fwd(const GlaArgs &a);
 dig_status tensor_gla_bwd(const GlaArgs &a);
 bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward);
@@ -139,6 +142,7 @@ dig_status launch_tc_bwd(const GlaArgs &a, const Workspace &w, int sm_count, int
 enum KernelId {
     KID_GATE = 0, KID_DWCONV, KID_DWCONV_WGRAD, KID_OUTGATE, KID_SCAN_FWD, KID_SCAN_BWD,
     KID_FMA_STATE, KID_FMA_OUT, KID_FMA_BWD,
+    KID_MMA_STATE, KID_MMA_OUT, KID_MMA_BWD,
     KID_TC_STATE, KID_TC_OUT, KID_TC_BWD,
     KID_COUNT
 };

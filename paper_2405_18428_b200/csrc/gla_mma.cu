@@ -1,0 +1,645 @@
+// Warp-MMA kernel family for chunkwise gated linear attention (Eq. attn_gla, evaluated chunk by chunk
+// as Section 3.5 describes): serves bf16 requests whose head size or chunk size the tcgen05 family
+// does not cover (any d_k, d_v that is a multiple of 8 up to 128, chunks of 16, 32, 64 or 128 tokens
+// as far as shared memory allows), e.g. the 72-wide heads of the largest model.  Same decomposition
+// as the other families: per-chunk state contributions, a scan over the chunks, then one CTA per
+// (chunk, batch*head) for the outputs or the gradients.  Every contraction runs on the tensor cores
+// through mma.sync.m16n8k8 (tf32 operands, fp32 accumulation) with fragments read straight from
+// padded fp32 tiles in shared memory, so any multiple of 8 works as a contraction length and any
+// multiple of 16 (after zero padding) as an output extent.  Operands are rounded to tf32 when the
+// tiles are filled.
+//
+// Notation per chunk (rows j = 0..C-1 in scan order, zero rows past the end of the sequence):
+//   Lam_j = inclusive prefix sum of the gates, gamma = exp(Lam_{C-1}),
+//   Qt = q*exp(Lam), Kt = k*exp(-Lam), Kh = k*exp(Lam_{C-1}-Lam),
+//   S = state entering the chunk, Dg = diag(gamma) * dL/d(state leaving the chunk).
+#include "dig_common.cuh"
+
+namespace dig {
+namespace {
+
+constexpr int kThreads = 256, kWarps = kThreads / 32;
+constexpr int kMaxNB = 8;                    // 8-column fragments per warp tile: up to 64 columns
+
+__host__ __device__ constexpr int pad16(int d) { return (d + 15) & ~15; }
+// Row pitch (floats) of a tile whose rows hold `d` values: a multiple of 4 whose quarter is odd, so the
+// 8 rows x 4 columns a fragment load touches fall into 32 different banks.
+__host__ __device__ constexpr int pitch(int d) { return pad16(d) + 4; }
+
+// Sizes of a launch, either compile-time constants (the frequent shapes: strides fold into the
+// instructions, loops unroll, divisions become shifts) or read from the geometry (everything else).
+template <int C_, int DK_, int DV_>
+struct FixedDims {
+    __device__ explicit FixedDims(const Geom &) {}
+    __device__ constexpr int C() const { return C_; }
+    __device__ constexpr int dk() const { return DK_; }
+    __device__ constexpr int dv() const { return DV_; }
+};
+struct AnyDims {
+    int c_, dk_, dv_;
+    __device__ explicit AnyDims(const Geom &g) : c_(g.C), dk_(g.dk), dv_(g.dv) {}
+    __device__ int C() const { return c_; }
+    __device__ int dk() const { return dk_; }
+    __device__ int dv() const { return dv_; }
+};
+
+__device__ __forceinline__ float tf32r(float x)
+{
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+    return __uint_as_float(u);
+}
+
+__device__ __forceinline__ void mma8(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// One warp: acc[nb] += A(r0 .. r0+15, k) * B(k, c0 + 8 nb .. c0 + 8 nb + 7) for k in [k0, k1), nb < nbw.
+// A(m, k) = A[m*sam + k*sak], B(k, n) = Bm[k*sbk + n*sbn]; k0, k1 multiples of 8.
+// Fragment layout of m16n8k8: with g = lane / 4, t = lane % 4 a lane holds A(g | g+8, t | t+4),
+// B(t | t+4, g) and the results C(g | g+8, 2t | 2t+1).
+__device__ __forceinline__ void warp_mma(float (&acc)[kMaxNB][4], const float *A, int sam, int sak, int r0,
+                                         const float *Bm, int sbk, int sbn, int c0, int nbw, int k0, int k1)
+{
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const float *pa = A + (r0 + g) * sam + (t + k0) * sak;
+    const float *pb = Bm + (t + k0) * sbk + (c0 + g) * sbn;
+#pragma unroll 2
+    for (int k = k0; k < k1; k += 8) {
+        uint32_t a[4];
+        a[0] = __float_as_uint(pa[0]);
+        a[1] = __float_as_uint(pa[8 * sam]);
+        a[2] = __float_as_uint(pa[4 * sak]);
+        a[3] = __float_as_uint(pa[8 * sam + 4 * sak]);
+#pragma unroll
+        for (int nb = 0; nb < kMaxNB; ++nb)
+            if (nb < nbw) {
+                const uint32_t b0 = __float_as_uint(pb[8 * nb * sbn]);
+                const uint32_t b1 = __float_as_uint(pb[4 * sbk + 8 * nb * sbn]);
+                mma8(acc[nb], a, b0, b1);
+            }
+        pa += 8 * sak;
+        pb += 8 * sbk;
+    }
+}
+
+__device__ __forceinline__ void zero(float (&acc)[kMaxNB][4])
+{
+#pragma unroll
+    for (int nb = 0; nb < kMaxNB; ++nb)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nb][i] = 0.f;
+}
+
+// Calls f(row, col, v0, v1) for every pair of adjacent result columns this lane holds (col even).
+template <typename F>
+__device__ __forceinline__ void for_pairs(const float (&acc)[kMaxNB][4], int r0, int c0, int nbw, F f)
+{
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int nb = 0; nb < kMaxNB; ++nb)
+        if (nb < nbw) {
+            f(r0 + g, c0 + 8 * nb + 2 * t, acc[nb][0], acc[nb][1]);
+            f(r0 + g + 8, c0 + 8 * nb + 2 * t, acc[nb][2], acc[nb][3]);
+        }
+}
+
+// The warp tiles of an M x N result (M, N multiples of 16): 16 rows by 1/2, 1/4 or 1/8 of the columns,
+// split as far as the column count allows until every warp has a tile.
+struct Tiling {
+    int nrt, nbw, ntiles;
+    __device__ Tiling(int M, int N) : nrt(M >> 4)
+    {
+        const int nfrag = N >> 3;
+        int cs = 2;
+        while (nrt * cs < kWarps && nfrag % (2 * cs) == 0) cs *= 2;
+        nbw = nfrag / cs;
+        ntiles = nrt * cs;
+    }
+    __device__ void at(int tile, int &r0, int &c0) const
+    {
+        const int rt = tile % nrt, ct = tile / nrt;
+        r0 = 16 * rt;
+        c0 = 8 * nbw * ct;
+    }
+};
+
+__device__ __forceinline__ void store2(float *p, float a, float b) { *reinterpret_cast<float2 *>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store2(__nv_bfloat16 *p, float a, float b)
+{
+    *reinterpret_cast<__nv_bfloat162 *>(p) = __floats2bfloat162_rn(a, b);
+}
+
+// ---- tile fills -----------------------------------------------------------------------------------
+// sRow[j] = index of the chunk's row j among the (token, head) rows of a [B][L][H][.] tensor, or -1 past
+// the end of the sequence.  Every later access to global memory goes through this table.
+__device__ __forceinline__ void fill_rows(int *sRow, const Geom &g, int C, int b, int h, int chunk)
+{
+    for (int j = threadIdx.x; j < C; j += kThreads) {
+        const int p = chunk * C + j;
+        sRow[j] = p < g.L ? (b * g.L + scan_token(p, g.dir, g.gh, g.gw, g.L)) * g.H + h : -1;
+    }
+}
+// Every tile is filled in one phase at the start of a kernel so that a CTA pays the latency of global
+// memory once: fp32 sources travel by cp.async (no registers, all copies in flight together), bf16
+// sources in register batches of four 8-byte loads per thread.  Rows past the end of the sequence and
+// the padding columns become zero.  The values are rescaled / rounded in place afterwards.
+__device__ __forceinline__ void cp_async16(float *dst, const float *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void load_rows(float *dst, int ld, const __nv_bfloat16 *src, const int *sRow, int C, int d)
+{
+    constexpr int U = 4;
+    const int per_row = pad16(d) >> 2, n = C * per_row;
+    for (int base = threadIdx.x; base < n; base += U * kThreads) {
+        uint2 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int idx = base + u * kThreads;
+            raw[u] = make_uint2(0u, 0u);
+            if (idx < n) {
+                const int j = idx / per_row, c = (idx - j * per_row) << 2;
+                const int row = sRow[j];
+                if (row >= 0 && c < d) raw[u] = *reinterpret_cast<const uint2 *>(src + (size_t)row * d + c);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int idx = base + u * kThreads;
+            if (idx < n) {
+                const int j = idx / per_row, c = (idx - j * per_row) << 2;
+                *reinterpret_cast<float4 *>(dst + j * ld + c) =
+                    make_float4(__uint_as_float(raw[u].x << 16), __uint_as_float(raw[u].x & 0xffff0000u),
+                                __uint_as_float(raw[u].y << 16), __uint_as_float(raw[u].y & 0xffff0000u));
+            }
+        }
+    }
+}
+__device__ __forceinline__ void load_gates(float *dst, int ld, const float *gate, const int *sRow, int C, int dk)
+{
+    const int per_row = pad16(dk) >> 2;
+    for (int idx = threadIdx.x; idx < C * per_row; idx += kThreads) {
+        const int j = idx / per_row, c = (idx - j * per_row) << 2;
+        const int row = sRow[j];
+        if (row >= 0 && c < dk) cp_async16(dst + j * ld + c, gate + (size_t)row * dk + c);
+        else *reinterpret_cast<float4 *>(dst + j * ld + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+// A [dk][dv] state of the workspace -> [pad16(dk)][ld] tile (unrounded), padding zero.
+__device__ __forceinline__ void load_state(float *dst, int ld, const float *src, int dk, int dv)
+{
+    const int per_row = pad16(dv) >> 2;
+    for (int idx = threadIdx.x; idx < pad16(dk) * per_row; idx += kThreads) {
+        const int r = idx / per_row, c = (idx - r * per_row) << 2;
+        if (r < dk && c < dv) cp_async16(dst + r * ld + c, src + r * dv + c);
+        else *reinterpret_cast<float4 *>(dst + r * ld + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+// In place: rows of a state tile times exp(row_scale[r]) (row_scale may be null), rounded to tf32.
+__device__ __forceinline__ void round_state(float *t, int ld, int dk, int dv, const float *row_scale)
+{
+    const int per_row = pad16(dv) >> 2;
+    for (int idx = threadIdx.x; idx < dk * per_row; idx += kThreads) {
+        const int r = idx / per_row, c = (idx - r * per_row) << 2;
+        const float sc = row_scale ? __expf(row_scale[r]) : 1.f;
+        float4 val = *reinterpret_cast<const float4 *>(t + r * ld + c);
+        *reinterpret_cast<float4 *>(t + r * ld + c) = make_float4(tf32r(val.x * sc), tf32r(val.y * sc), tf32r(val.z * sc), tf32r(val.w * sc));
+    }
+}
+// In place: gates -> inclusive prefix sums down the rows of the chunk; sLast receives the last row.
+__device__ __forceinline__ void prefix_gates(float *lam, int ld, int C, int dkp, float *sLast)
+{
+    for (int c = threadIdx.x; c < dkp; c += kThreads) {
+        float run = 0.f;
+#pragma unroll 8
+        for (int j = 0; j < C; ++j) {
+            run += lam[j * ld + c];
+            lam[j * ld + c] = run;
+        }
+        sLast[c] = run;
+    }
+}
+// In place: sQ (raw q) -> Qt = q*exp(Lam), sK (raw k) -> Kt = k*exp(-Lam), or with sLast given
+// -> Kh = k*exp(Lam_{C-1}-Lam); rounded to tf32.  Either tile may be null.
+__device__ __forceinline__ void scale_qk(float *sQ, float *sK, const float *sLam, const float *sLast, int ldk, int C, int dk)
+{
+    const int per_row = pad16(dk) >> 2;
+    for (int idx = threadIdx.x; idx < C * per_row; idx += kThreads) {
+        const int j = idx / per_row, c = (idx - j * per_row) << 2;
+        const float4 lam = *reinterpret_cast<const float4 *>(sLam + j * ldk + c);
+        if (sQ) {
+            const float4 x = *reinterpret_cast<const float4 *>(sQ + j * ldk + c);
+            *reinterpret_cast<float4 *>(sQ + j * ldk + c) = make_float4(
+                tf32r(x.x * __expf(lam.x)), tf32r(x.y * __expf(lam.y)), tf32r(x.z * __expf(lam.z)), tf32r(x.w * __expf(lam.w)));
+        }
+        if (sK) {
+            float4 e = make_float4(-lam.x, -lam.y, -lam.z, -lam.w);
+            if (sLast) {
+                const float4 last = *reinterpret_cast<const float4 *>(sLast + c);
+                e = make_float4(last.x - lam.x, last.y - lam.y, last.z - lam.z, last.w - lam.w);
+            }
+            const float4 x = *reinterpret_cast<const float4 *>(sK + j * ldk + c);
+            *reinterpret_cast<float4 *>(sK + j * ldk + c) = make_float4(
+                tf32r(x.x * __expf(e.x)), tf32r(x.y * __expf(e.y)), tf32r(x.z * __expf(e.z)), tf32r(x.w * __expf(e.w)));
+        }
+    }
+}
+
+// sP[t][s] = A_t . B_s for s <= t, 0 above the diagonal, rounded to tf32 (A, B: [C][ld] tiles, contraction
+// over the first K columns).  The diagonal has weight 1: the token's own k^T v enters undecayed.
+__device__ __forceinline__ void masked_scores(float *sP, int ldp, const float *A, const float *Bm, int ld, int C, int K)
+{
+    const Tiling tl(C, C);
+    const int warp = threadIdx.x >> 5;
+    for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
+        int r0, c0;
+        tl.at(tile, r0, c0);
+        float acc[kMaxNB][4];
+        zero(acc);
+        if (c0 <= r0 + 15) warp_mma(acc, A, ld, 1, r0, Bm, 1, ld, c0, tl.nbw, 0, K);
+        for_pairs(acc, r0, c0, tl.nbw, [&](int t, int s, float v0, float v1) {
+            *reinterpret_cast<float2 *>(sP + t * ldp + s) = make_float2(s <= t ? tf32r(v0) : 0.f, s + 1 <= t ? tf32r(v1) : 0.f);
+        });
+    }
+}
+
+// ---- kernel 1: chunk-local state contributions ------------------------------------------------------
+// U = Kh^T V (and, for the backward pass, W = Qt^T dO); gamma = exp(Lam_{C-1}).
+template <bool BWD, typename DM>
+__global__ void __launch_bounds__(kThreads)
+mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
+                const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate,
+                const __nv_bfloat16 *__restrict__ d_out, float *__restrict__ states, float *__restrict__ gamma,
+                float *__restrict__ dstates, Geom g)
+{
+    extern __shared__ __align__(16) float smem[];
+    __shared__ int sRow[128];
+    const DM dm(g);
+    const int C = dm.C(), dk = dm.dk(), dv = dm.dv();
+    const int chunk = blockIdx.x, bh = blockIdx.y, b = bh / g.H, h = bh - b * g.H;
+    const int dkp = pad16(dk), dvp = pad16(dv), ldk = pitch(dk), ldv = pitch(dv);
+    float *sLam = smem;                     // gates -> Lam
+    float *sX = sLam + C * ldk;             // k -> Kh
+    float *sV = sX + C * ldk;
+    float *sLast = sV + C * ldv;            // [dkp]
+    float *sQ = sLast + dkp;                // BWD: q -> Qt
+    float *sG = sQ + (BWD ? C * ldk : 0);   // BWD: dO
+
+    fill_rows(sRow, g, C, b, h, chunk);
+    __syncthreads();
+    load_gates(sLam, ldk, gate, sRow, C, dk);
+    load_rows(sX, ldk, k, sRow, C, dk);
+    load_rows(sV, ldv, v, sRow, C, dv);
+    if (BWD) {
+        load_rows(sQ, ldk, q, sRow, C, dk);
+        load_rows(sG, ldv, d_out, sRow, C, dv);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    prefix_gates(sLam, ldk, C, dkp, sLast);
+    __syncthreads();
+    const size_t chunk_id = (size_t)bh * g.N + chunk;
+    for (int c = threadIdx.x; c < dk; c += kThreads) gamma[chunk_id * dk + c] = __expf(sLast[c]);
+    scale_qk(BWD ? sQ : nullptr, sX, sLam, sLast, ldk, C, dk);
+    __syncthreads();
+    const Tiling tl(dkp, dvp);
+    const int warp = threadIdx.x >> 5;
+    float *U = states + chunk_id * dk * dv;
+    float *W = BWD ? dstates + chunk_id * dk * dv : nullptr;
+    for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
+        int r0, c0;
+        tl.at(tile, r0, c0);
+        float acc[kMaxNB][4];
+        zero(acc);
+        warp_mma(acc, sX, 1, ldk, r0, sV, ldv, 1, c0, tl.nbw, 0, C);           // sum_t Kh[t][c] V[t][e]
+        for_pairs(acc, r0, c0, tl.nbw, [&](int c, int e, float v0, float v1) {
+            if (c < dk && e < dv) store2(U + c * dv + e, v0, v1);
+        });
+        if (BWD) {
+            zero(acc);
+            warp_mma(acc, sQ, 1, ldk, r0, sG, ldv, 1, c0, tl.nbw, 0, C);       // sum_t Qt[t][c] dO[t][e]
+            for_pairs(acc, r0, c0, tl.nbw, [&](int c, int e, float v0, float v1) {
+                if (c < dk && e < dv) store2(W + c * dv + e, v0, v1);
+            });
+        }
+    }
+}
+
+// ---- kernel 3: outputs ------------------------------------------------------------------------------
+// out = tril(Qt Kt^T) V + Qt S
+template <typename TO, typename DM>
+__global__ void __launch_bounds__(kThreads)
+mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
+              const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate, const float *__restrict__ states,
+              TO *__restrict__ out, Geom g)
+{
+    extern __shared__ __align__(16) float smem[];
+    __shared__ int sRow[128];
+    const DM dm(g);
+    const int C = dm.C(), dk = dm.dk(), dv = dm.dv();
+    const int chunk = blockIdx.x, bh = blockIdx.y, b = bh / g.H, h = bh - b * g.H;
+    const int dkp = pad16(dk), dvp = pad16(dv), ldk = pitch(dk), ldv = pitch(dv), ldp = pitch(C);
+    float *sLam = smem;
+    float *sQ = sLam + C * ldk;
+    float *sK = sQ + C * ldk;
+    float *sV = sK + C * ldk;
+    float *sS = sV + C * ldv;               // [dkp][ldv]
+    float *sLast = sS + dkp * ldv;          // [dkp]
+    float *sP = (C <= dk) ? sLam : sLast + dkp;       // the scores reuse the gate tile when they fit
+
+    fill_rows(sRow, g, C, b, h, chunk);
+    __syncthreads();
+    load_gates(sLam, ldk, gate, sRow, C, dk);
+    load_state(sS, ldv, states + ((size_t)bh * g.N + chunk) * dk * dv, dk, dv);
+    load_rows(sV, ldv, v, sRow, C, dv);
+    load_rows(sQ, ldk, q, sRow, C, dk);
+    load_rows(sK, ldk, k, sRow, C, dk);
+    cp_async_wait_all();
+    __syncthreads();
+    prefix_gates(sLam, ldk, C, dkp, sLast);
+    __syncthreads();
+    scale_qk(sQ, sK, sLam, nullptr, ldk, C, dk);
+    round_state(sS, ldv, dk, dv, nullptr);
+    __syncthreads();
+    masked_scores(sP, ldp, sQ, sK, ldk, C, dk);
+    __syncthreads();
+    const Tiling tl(C, dvp);
+    const int warp = threadIdx.x >> 5;
+    for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
+        int r0, c0;
+        tl.at(tile, r0, c0);
+        float acc[kMaxNB][4];
+        zero(acc);
+        warp_mma(acc, sP, ldp, 1, r0, sV, ldv, 1, c0, tl.nbw, 0, r0 + 16);     // columns past the diagonal are zero
+        warp_mma(acc, sQ, ldk, 1, r0, sS, ldv, 1, c0, tl.nbw, 0, dk);
+        for_pairs(acc, r0, c0, tl.nbw, [&](int j, int e, float v0, float v1) {
+            const int row = sRow[j];
+            if (row >= 0 && e < dv) store2(out + (size_t)row * dv + e, v0, v1);
+        });
+    }
+}
+
+// ---- kernel 4: gradients ----------------------------------------------------------------------------
+//   P = tril(Qt Kt^T),  dP = tril(dO V^T)
+//   dq = (dP Kt + dO S^T) * exp(Lam)
+//   dk = (dP^T Qt + V Dg^T) * exp(-Lam)
+//   dv = P^T dO + Kt Dg
+//   dgate_j = carry + sum_{r >= j in chunk} (q*dq - k*dk)_r,   q*dq = Qt*(dq accumulator), k*dk alike
+template <typename TO, typename DM>
+__global__ void __launch_bounds__(kThreads)
+mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
+              const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate,
+              const __nv_bfloat16 *__restrict__ d_out, const float *__restrict__ states,
+              const float *__restrict__ dstates, const float *__restrict__ carry, TO *__restrict__ dq,
+              TO *__restrict__ dk_out, TO *__restrict__ dv_out, float *__restrict__ dgate, Geom g)
+{
+    extern __shared__ __align__(16) float smem[];
+    __shared__ int sRow[128];
+    const DM dm(g);
+    const int C = dm.C(), dk = dm.dk(), dv = dm.dv();
+    const int chunk = blockIdx.x, bh = blockIdx.y, b = bh / g.H, h = bh - b * g.H;
+    const int dkp = pad16(dk), dvp = pad16(dv), ldk = pitch(dk), ldv = pitch(dv), ldp = pitch(C);
+    float *sLam = smem;                     // Lam, later x = q*dq - k*dk
+    float *sQ = sLam + C * ldk;
+    float *sK = sQ + C * ldk;
+    float *sV = sK + C * ldk;
+    float *sG = sV + C * ldv;               // dO
+    float *sS = sG + C * ldv;               // [dkp][ldv]
+    float *sD = sS + dkp * ldv;             // [dkp][ldv]  Dg
+    float *sP = sD + dkp * ldv;             // [C][ldp]
+    float *sdP = sP + C * ldp;              // [C][ldp]
+    float *sLast = sdP + C * ldp;           // [dkp]
+    const size_t chunk_id = (size_t)bh * g.N + chunk;
+
+    fill_rows(sRow, g, C, b, h, chunk);
+    __syncthreads();
+    load_gates(sLam, ldk, gate, sRow, C, dk);
+    load_state(sS, ldv, states + chunk_id * dk * dv, dk, dv);
+    load_state(sD, ldv, dstates + chunk_id * dk * dv, dk, dv);
+    load_rows(sV, ldv, v, sRow, C, dv);
+    load_rows(sG, ldv, d_out, sRow, C, dv);
+    load_rows(sQ, ldk, q, sRow, C, dk);
+    load_rows(sK, ldk, k, sRow, C, dk);
+    const float carry_in = threadIdx.x < dk ? carry[chunk_id * dk + threadIdx.x] : 0.f;
+    cp_async_wait_all();
+    __syncthreads();
+    prefix_gates(sLam, ldk, C, dkp, sLast);
+    __syncthreads();
+    scale_qk(sQ, sK, sLam, nullptr, ldk, C, dk);
+    round_state(sS, ldv, dk, dv, nullptr);
+    round_state(sD, ldv, dk, dv, sLast);                                         // Dg = diag(gamma) D
+    __syncthreads();
+    masked_scores(sP, ldp, sQ, sK, ldk, C, dk);
+    masked_scores(sdP, ldp, sG, sV, ldv, C, dv);
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gi = lane >> 2, ti = lane & 3;
+    {
+        // dv[s][e] = sum_{t >= s} P[t][s] dO[t][e] + sum_c Kt[s][c] Dg[c][e]
+        const Tiling tl(C, dvp);
+        for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
+            int r0, c0;
+            tl.at(tile, r0, c0);
+            float acc[kMaxNB][4];
+            zero(acc);
+            warp_mma(acc, sP, 1, ldp, r0, sG, ldv, 1, c0, tl.nbw, r0, C);
+            warp_mma(acc, sK, ldk, 1, r0, sD, ldv, 1, c0, tl.nbw, 0, dk);
+            for_pairs(acc, r0, c0, tl.nbw, [&](int j, int e, float v0, float v1) {
+                const int row = sRow[j];
+                if (row >= 0 && e < dv) store2(dv_out + (size_t)row * dv + e, v0, v1);
+            });
+        }
+    }
+    {
+        // dq and dk of the same (row, channel) tile; x = q*dq - k*dk replaces Lam, element by element
+        const Tiling tl(C, dkp);
+        for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
+            int r0, c0;
+            tl.at(tile, r0, c0);
+            float acc[kMaxNB][4], xq[kMaxNB][4];
+            zero(acc);
+            warp_mma(acc, sdP, ldp, 1, r0, sK, ldk, 1, c0, tl.nbw, 0, r0 + 16);          // sum_{s <= t} dP[t][s] Kt[s][c]
+            warp_mma(acc, sG, ldv, 1, r0, sS, 1, ldv, c0, tl.nbw, 0, dv);                // sum_e dO[t][e] S[c][e]
+#pragma unroll
+            for (int nb = 0; nb < kMaxNB; ++nb)
+                if (nb < tl.nbw) {
+#pragma unroll
+                    for (int i = 0; i < 4; i += 2) {
+                        const float2 qt = *reinterpret_cast<const float2 *>(sQ + (r0 + gi + 4 * i) * ldk + c0 + 8 * nb + 2 * ti);
+                        xq[nb][i] = qt.x * acc[nb][i];
+                        xq[nb][i + 1] = qt.y * acc[nb][i + 1];
+                    }
+                }
+            for_pairs(acc, r0, c0, tl.nbw, [&](int j, int c, float v0, float v1) {
+                const int row = sRow[j];
+                if (row >= 0 && c < dk) {
+                    const float2 lam = *reinterpret_cast<const float2 *>(sLam + j * ldk + c);
+                    store2(dq + (size_t)row * dk + c, v0 * __expf(lam.x), v1 * __expf(lam.y));
+                }
+            });
+            zero(acc);
+            warp_mma(acc, sdP, 1, ldp, r0, sQ, ldk, 1, c0, tl.nbw, r0, C);               // sum_{t >= s} dP[t][s] Qt[t][c]
+            warp_mma(acc, sV, ldv, 1, r0, sD, 1, ldv, c0, tl.nbw, 0, dv);                // sum_e V[s][e] Dg[c][e]
+#pragma unroll
+            for (int nb = 0; nb < kMaxNB; ++nb)
+                if (nb < tl.nbw) {
+#pragma unroll
+                    for (int i = 0; i < 4; i += 2) {
+                        const float2 kt = *reinterpret_cast<const float2 *>(sK + (r0 + gi + 4 * i) * ldk + c0 + 8 * nb + 2 * ti);
+                        xq[nb][i] -= kt.x * acc[nb][i];
+                        xq[nb][i + 1] -= kt.y * acc[nb][i + 1];
+                    }
+                }
+            for_pairs(acc, r0, c0, tl.nbw, [&](int j, int c, float v0, float v1) {
+                const int row = sRow[j];
+                if (row >= 0 && c < dk) {
+                    const float2 lam = *reinterpret_cast<const float2 *>(sLam + j * ldk + c);
+                    store2(dk_out + (size_t)row * dk + c, v0 * __expf(-lam.x), v1 * __expf(-lam.y));
+                }
+            });
+            __syncwarp();
+            for_pairs(xq, r0, c0, tl.nbw, [&](int j, int c, float v0, float v1) {
+                *reinterpret_cast<float2 *>(sLam + j * ldk + c) = make_float2(v0, v1);
+            });
+        }
+    }
+    __syncthreads();
+    // gate gradient: suffix sums of x down the chunk plus what later chunks carry in
+    if (threadIdx.x < dk) {             // d_k <= 128 < kThreads
+        const int c = threadIdx.x;
+        float run = carry_in;
+        for (int j = C - 1; j >= 0; --j) {
+            const int row = sRow[j];
+            if (row < 0) continue;
+            run += sLam[j * ldk + c];
+            dgate[(size_t)row * dk + c] = run;
+        }
+    }
+}
+
+size_t smem_state(const Geom &g, bool bwd)
+{
+    return sizeof(float) * ((size_t)g.C * (pitch(g.dk) * (bwd ? 3 : 2) + pitch(g.dv) * (bwd ? 2 : 1)) + pad16(g.dk));
+}
+size_t smem_out(const Geom &g)
+{
+    size_t n = (size_t)g.C * (3 * pitch(g.dk) + pitch(g.dv)) + (size_t)pad16(g.dk) * pitch(g.dv) + pad16(g.dk);
+    if (g.C > g.dk) n += (size_t)g.C * pitch(g.C);
+    return sizeof(float) * n;
+}
+size_t smem_bwd(const Geom &g)
+{
+    return sizeof(float) * ((size_t)g.C * (3 * pitch(g.dk) + 2 * pitch(g.dv) + 2 * pitch(g.C)) +
+                            2 * (size_t)pad16(g.dk) * pitch(g.dv) + pad16(g.dk));
+}
+constexpr size_t kMaxSmem = 227 * 1024 - 1024;      // the row table is static shared memory
+
+template <typename K>
+dig_status set_smem(K kernel, size_t bytes)
+{
+    if (bytes > kMaxSmem) return DIG_ERR_UNSUPPORTED;
+    return cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+}
+
+using bf16 = __nv_bfloat16;
+
+template <typename TO, typename DM>
+dig_status fwd_dims(const GlaArgs &a)
+{
+    const Geom &g = a.g;
+    const Workspace w = carve_workspace(a.ws, g, false);
+    const dim3 grid(g.N, g.B * g.H);
+    dig_status st;
+    auto k1 = mma_chunk_state<false, DM>;
+    if ((st = set_smem(k1, smem_state(g, false))) != DIG_OK) return st;
+    auto k3 = mma_chunk_out<TO, DM>;
+    if ((st = set_smem(k3, smem_out(g))) != DIG_OK) return st;
+    {
+        KernelTimer t(KID_MMA_STATE, a.stream);
+        k1<<<grid, kThreads, smem_state(g, false), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
+                                                              nullptr, w.states, w.gamma, nullptr, g);
+    }
+    if ((st = launch_state_scan_fwd(w, g, a.stream)) != DIG_OK) return st;
+    KernelTimer t(KID_MMA_OUT, a.stream);
+    k3<<<grid, kThreads, smem_out(g), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate, w.states,
+                                                  (TO *)a.out, g);
+    return cuda_ok(cudaGetLastError());
+}
+
+template <typename TO, typename DM>
+dig_status bwd_dims(const GlaArgs &a)
+{
+    const Geom &g = a.g;
+    const Workspace w = carve_workspace(a.ws, g, true);
+    const dim3 grid(g.N, g.B * g.H);
+    dig_status st;
+    auto k1 = mma_chunk_state<true, DM>;
+    if ((st = set_smem(k1, smem_state(g, true))) != DIG_OK) return st;
+    auto k4 = mma_chunk_bwd<TO, DM>;
+    if ((st = set_smem(k4, smem_bwd(g))) != DIG_OK) return st;
+    {
+        KernelTimer t(KID_MMA_STATE, a.stream);
+        k1<<<grid, kThreads, smem_state(g, true), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
+                                                             (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, g);
+    }
+    if ((st = launch_state_scan_fwd(w, g, a.stream)) != DIG_OK) return st;
+    if ((st = launch_state_scan_bwd(w, g, a.stream)) != DIG_OK) return st;
+    KernelTimer t(KID_MMA_BWD, a.stream);
+    k4<<<grid, kThreads, smem_bwd(g), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
+                                                  (const bf16 *)a.d_out, w.states, w.dstates, w.carry, (TO *)a.dq, (TO *)a.dk,
+                                                  (TO *)a.dv, a.dgate, g);
+    return cuda_ok(cudaGetLastError());
+}
+
+// The shapes of the paper's models that the tcgen05 family leaves to this one get kernels with
+// compile-time sizes: 72-wide heads with 64-token chunks, 64-wide heads with 32-token chunks.
+template <typename TO>
+dig_status fwd_typed(const GlaArgs &a)
+{
+    const Geom &g = a.g;
+    if (g.C == 64 && g.dk == 72 && g.dv == 72) return fwd_dims<TO, FixedDims<64, 72, 72>>(a);
+    if (g.C == 32 && g.dk == 64 && g.dv == 64) return fwd_dims<TO, FixedDims<32, 64, 64>>(a);
+    return fwd_dims<TO, AnyDims>(a);
+}
+template <typename TO>
+dig_status bwd_typed(const GlaArgs &a)
+{
+    const Geom &g = a.g;
+    if (g.C == 64 && g.dk == 72 && g.dv == 72) return bwd_dims<TO, FixedDims<64, 72, 72>>(a);
+    if (g.C == 32 && g.dk == 64 && g.dv == 64) return bwd_dims<TO, FixedDims<32, 64, 64>>(a);
+    return bwd_dims<TO, AnyDims>(a);
+}
+
+}  // namespace
+
+bool mma_supports(int dk, int dv, int chunk, int dtype, bool backward)
+{
+    if (dtype == DIG_F32) return false;      // one tf32 pass is not fp32-accurate
+    Geom g{};
+    g.dk = dk; g.dv = dv; g.C = chunk;
+    if (backward) return smem_bwd(g) <= kMaxSmem && smem_state(g, true) <= kMaxSmem;
+    return smem_out(g) <= kMaxSmem && smem_state(g, false) <= kMaxSmem;
+}
+
+dig_status mma_gla_fwd(const GlaArgs &a)
+{
+    if (a.dtype == DIG_BF16) return fwd_typed<__nv_bfloat16>(a);
+    if (a.dtype == DIG_BF16_F32OUT) return fwd_typed<float>(a);
+    return DIG_ERR_UNSUPPORTED;
+}
+
+dig_status mma_gla_bwd(const GlaArgs &a)
+{
+    if (a.dtype == DIG_BF16) return bwd_typed<__nv_bfloat16>(a);
+    if (a.dtype == DIG_BF16_F32OUT) return bwd_typed<float>(a);
+    return DIG_ERR_UNSUPPORTED;
+}
+
+}  // namespace dig

@@ -95,26 +95,39 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
     float run[kMaxPerLane];
 #pragma unroll
     for (int r = 0; r < kMaxPerLane; ++r) run[r] = 0.f;
-    for (int i = N - 1; i >= 0; --i) {
-        float w[kMaxPerLane], sn[kMaxPerLane];
-        const float g = gm[(size_t)i * dk];
+    // kLook chunks are loaded ahead of the recurrence, so the walk pays the latency of global memory
+    // once per kLook chunks and not once per chunk
+    constexpr int kLook = 8;
+    for (int i = N - 1; i >= 0; i -= kLook) {
+        float w[kLook][kMaxPerLane], sn[kLook][kMaxPerLane], g[kLook];
 #pragma unroll
-        for (int r = 0; r < kMaxPerLane; ++r) {
-            const int e = lane + 32 * r;
-            w[r] = (e < dv) ? D[(size_t)i * sstride + e] : 0.f;
-            sn[r] = (e < dv && i + 1 < N) ? S[(size_t)(i + 1) * sstride + e] : 0.f;
+        for (int j = 0; j < kLook; ++j) {
+            const int ch = i - j;
+            g[j] = 0.f;
+            if (ch >= 0) g[j] = gm[(size_t)ch * dk];
+#pragma unroll
+            for (int r = 0; r < kMaxPerLane; ++r) {
+                const int e = lane + 32 * r;
+                w[j][r] = (ch >= 0 && e < dv) ? D[(size_t)ch * sstride + e] : 0.f;
+                sn[j][r] = (ch >= 0 && e < dv && ch + 1 < N) ? S[(size_t)(ch + 1) * sstride + e] : 0.f;
+            }
         }
-        float dot = 0.f;
 #pragma unroll
-        for (int r = 0; r < kMaxPerLane; ++r) {
-            const int e = lane + 32 * r;
-            if (e < dv) D[(size_t)i * sstride + e] = run[r];
-            dot = fmaf(sn[r], run[r], dot);
-            run[r] = fmaf(g, run[r], w[r]);
+        for (int j = 0; j < kLook; ++j) {
+            const int ch = i - j;
+            if (ch < 0) break;          // uniform over the warp
+            float dot = 0.f;
+#pragma unroll
+            for (int r = 0; r < kMaxPerLane; ++r) {
+                const int e = lane + 32 * r;
+                if (e < dv) D[(size_t)ch * sstride + e] = run[r];
+                dot = fmaf(sn[j][r], run[r], dot);
+                run[r] = fmaf(g[j], run[r], w[j][r]);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+            if (lane == 0) cr[(size_t)ch * dk] = dot;
         }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-        if (lane == 0) cr[(size_t)i * dk] = dot;
     }
 }
 
