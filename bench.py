@@ -339,7 +339,7 @@ def main():
     ap.add_argument("--workload", default="C2")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--family", default="auto", choices=["auto", "fma", "tensor"])
+    ap.add_argument("--family", default="auto", choices=["auto", "fma", "tensor", "mma"])
     ap.add_argument("--eager", action="store_true", help="time plain stream launches instead of one CUDA graph per step")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short tokens/s-vs-L sweep over C3, C4 (chunks 32, 64, 128), C5")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
@@ -366,7 +366,7 @@ def main():
         dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
         dist = dist_mod
     dig.lib()      # fails loudly if the CUDA library is missing
-    dig.dig_set_impl({"auto": dig.DIG_IMPL_AUTO, "fma": dig.DIG_IMPL_FMA, "tensor": dig.DIG_IMPL_TENSOR}[args.family])
+    dig.dig_set_impl({"auto": dig.DIG_IMPL_AUTO, "fma": dig.DIG_IMPL_FMA, "tensor": dig.DIG_IMPL_TENSOR, "mma": dig.DIG_IMPL_MMA}[args.family])
     peaks = load_peaks()
     W = max(args.warmup, 3)
 
@@ -443,7 +443,7 @@ def main():
             th = w2.B * w2.L * w2.H
             fam = dig.dig_gla_query_impl(w2.d_k, w2.d_v, w2.chunk, dig.DIG_BF16, 1)
             sweep[name] = {"L": w2.L, "B": w2.B, "H": w2.H, "d": w2.d_k, "chunk": w2.chunk, "ms": best,
-                           "kernel_family": {1: "fma", 2: "tensor"}.get(fam, str(fam)),
+                           "kernel_family": {1: "fma", 2: "tensor", 3: "mma"}.get(fam, str(fam)),
                            "tokens_per_s": w2.B * w2.L / (best * 1e-3),
                            "tflops_alg": a2 * th / (best * 1e-3) / 1e12, "tflops_exec": e2 * th / (best * 1e-3) / 1e12,
                            "hbm_frac_of_measured": (fb + bb) * th / (best * 1e-3) / 1e9 / peaks["hbm_gbs"]}
@@ -460,13 +460,13 @@ def main():
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": W,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": {dig.DIG_IMPL_TENSOR: "tf32", dig.DIG_IMPL_FMA: "f32"}.get(impl, "f32"), "data": "synthetic",
+            "dtype": {dig.DIG_IMPL_TENSOR: "tf32", dig.DIG_IMPL_MMA: "tf32", dig.DIG_IMPL_FMA: "f32"}.get(impl, "f32"), "data": "synthetic",
             "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "grid": [wl.grid_h, wl.grid_w], "L": wl.L,
                        "d_k": wl.d_k, "d_v": wl.d_v, "chunk": wl.chunk, "storage": wl.dtype,
                        "directions": list(wl.directions), "conv": wl.conv, "blocks_per_step": len(wl.directions),
                        "launch": launch_mode, "ms_per_step_eager": ms_eager / args.steps,
                        "ms_per_step_with_kernel_events": ms_events / args.steps,
-                       "kernel_family": {1: "fma", 2: "tensor"}.get(impl, str(impl)),
+                       "kernel_family": {1: "fma", 2: "tensor", 3: "mma"}.get(impl, str(impl)),
                        "l2": "each block has its own buffers; a step streams several times the 126 MB L2, no flush needed",
                        "tflops_alg": tflops_alg, "tflops_exec": tflops_exe,
                        "tensor_frac_of_sustained_bf16_peak_exec": tflops_exe / peaks["bf16_tflops_sustained"]},

@@ -122,8 +122,8 @@ bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward);
 
 // Chunk-state scans, shared by both families (plain fp32 FMA, bandwidth-bound).
 // `tiles`: the states are stored transposed, in swizzled operand-tile order (tensor-core forward pass).
-dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tiles = false);
-dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s);
+dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tiles = false, bool tf32 = false);
+dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tf32 = false);
 // Tensor-core backward pass: forward and reverse scan in one launch over states kept in tile order.
 dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s);
 

@@ -12,13 +12,14 @@
 // Notation per chunk (rows j = 0..C-1 in scan order, zero rows past the end of the sequence):
 //   Lam_j = inclusive prefix sum of the gates, gamma = exp(Lam_{C-1}),
 //   Qt = q*exp(Lam), Kt = k*exp(-Lam), Kh = k*exp(Lam_{C-1}-Lam),
-//   S = state entering the chunk, Dg = diag(gamma) * dL/d(state leaving the chunk).
+//   S = state entering the chunk, Dg = diag(gamma) * dL/d(state leaving the chunk); the scan kernels
+//   leave both rounded to tf32 in the workspace.
 #include "dig_common.cuh"
 
 namespace dig {
 namespace {
 
-constexpr int kThreads = 256, kWarps = kThreads / 32;
+constexpr int kThreads = 512, kWarps = kThreads / 32;
 constexpr int kMaxNB = 8;                    // 8-column fragments per warp tile: up to 64 columns
 
 __host__ __device__ constexpr int pad16(int d) { return (d + 15) & ~15; }
@@ -30,12 +31,14 @@ __host__ __device__ constexpr int pitch(int d) { return pad16(d) + 4; }
 // instructions, loops unroll, divisions become shifts) or read from the geometry (everything else).
 template <int C_, int DK_, int DV_>
 struct FixedDims {
+    static constexpr int kC = C_, kDK = DK_, kDV = DV_;      // 0 = not known at compile time
     __device__ explicit FixedDims(const Geom &) {}
     __device__ constexpr int C() const { return C_; }
     __device__ constexpr int dk() const { return DK_; }
     __device__ constexpr int dv() const { return DV_; }
 };
 struct AnyDims {
+    static constexpr int kC = 0, kDK = 0, kDV = 0;
     int c_, dk_, dv_;
     __device__ explicit AnyDims(const Geom &g) : c_(g.C), dk_(g.dk), dv_(g.dv) {}
     __device__ int C() const { return c_; }
@@ -61,7 +64,8 @@ __device__ __forceinline__ void mma8(float (&c)[4], const uint32_t (&a)[4], uint
 // A(m, k) = A[m*sam + k*sak], B(k, n) = Bm[k*sbk + n*sbn]; k0, k1 multiples of 8.
 // Fragment layout of m16n8k8: with g = lane / 4, t = lane % 4 a lane holds A(g | g+8, t | t+4),
 // B(t | t+4, g) and the results C(g | g+8, 2t | 2t+1).
-__device__ __forceinline__ void warp_mma(float (&acc)[kMaxNB][4], const float *A, int sam, int sak, int r0,
+template <int NB>
+__device__ __forceinline__ void warp_mma(float (&acc)[NB][4], const float *A, int sam, int sak, int r0,
                                          const float *Bm, int sbk, int sbn, int c0, int nbw, int k0, int k1)
 {
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -75,7 +79,7 @@ __device__ __forceinline__ void warp_mma(float (&acc)[kMaxNB][4], const float *A
         a[2] = __float_as_uint(pa[4 * sak]);
         a[3] = __float_as_uint(pa[8 * sam + 4 * sak]);
 #pragma unroll
-        for (int nb = 0; nb < kMaxNB; ++nb)
+        for (int nb = 0; nb < NB; ++nb)
             if (nb < nbw) {
                 const uint32_t b0 = __float_as_uint(pb[8 * nb * sbn]);
                 const uint32_t b1 = __float_as_uint(pb[4 * sbk + 8 * nb * sbn]);
@@ -86,44 +90,49 @@ __device__ __forceinline__ void warp_mma(float (&acc)[kMaxNB][4], const float *A
     }
 }
 
-__device__ __forceinline__ void zero(float (&acc)[kMaxNB][4])
+template <int NB>
+__device__ __forceinline__ void zero(float (&acc)[NB][4])
 {
 #pragma unroll
-    for (int nb = 0; nb < kMaxNB; ++nb)
+    for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[nb][i] = 0.f;
 }
 
 // Calls f(row, col, v0, v1) for every pair of adjacent result columns this lane holds (col even).
-template <typename F>
-__device__ __forceinline__ void for_pairs(const float (&acc)[kMaxNB][4], int r0, int c0, int nbw, F f)
+template <int NB, typename F>
+__device__ __forceinline__ void for_pairs(const float (&acc)[NB][4], int r0, int c0, int nbw, F f)
 {
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
 #pragma unroll
-    for (int nb = 0; nb < kMaxNB; ++nb)
+    for (int nb = 0; nb < NB; ++nb)
         if (nb < nbw) {
             f(r0 + g, c0 + 8 * nb + 2 * t, acc[nb][0], acc[nb][1]);
             f(r0 + g + 8, c0 + 8 * nb + 2 * t, acc[nb][2], acc[nb][3]);
         }
 }
 
-// The warp tiles of an M x N result (M, N multiples of 16): 16 rows by 1/2, 1/4 or 1/8 of the columns,
-// split as far as the column count allows until every warp has a tile.
+// The warp tiles of an M x N result (M a multiple of 16, N of 8): 16 rows by a group of 8-column
+// fragments; the columns are split until every warp has a tile (the last group may be shorter).
+__host__ __device__ constexpr int tile_splits(int M, int N)
+{
+    int cs = 1;
+    while ((M >> 4) * cs < kWarps && cs < (N >> 3)) cs *= 2;
+    return cs;
+}
+__host__ __device__ constexpr int tile_frags(int M, int N) { return ((N >> 3) + tile_splits(M, N) - 1) / tile_splits(M, N); }
+// Fragments per warp tile as a compile-time bound: exact when both extents are known, else the maximum.
+__host__ __device__ constexpr int frag_bound(int M, int N) { return (M > 0 && N > 0) ? tile_frags(M, N) : kMaxNB; }
 struct Tiling {
-    int nrt, nbw, ntiles;
-    __device__ Tiling(int M, int N) : nrt(M >> 4)
-    {
-        const int nfrag = N >> 3;
-        int cs = 2;
-        while (nrt * cs < kWarps && nfrag % (2 * cs) == 0) cs *= 2;
-        nbw = nfrag / cs;
-        ntiles = nrt * cs;
-    }
-    __device__ void at(int tile, int &r0, int &c0) const
+    int nrt, nfrag, nbw, ntiles;
+    __device__ Tiling(int M, int N) : nrt(M >> 4), nfrag(N >> 3), nbw(tile_frags(M, N)), ntiles((M >> 4) * tile_splits(M, N)) {}
+    // first row, first column and fragment count (<= 0: nothing to do) of a tile
+    __device__ void at(int tile, int &r0, int &c0, int &nbt) const
     {
         const int rt = tile % nrt, ct = tile / nrt;
         r0 = 16 * rt;
         c0 = 8 * nbw * ct;
+        nbt = min(nbw, nfrag - nbw * ct);
     }
 };
 
@@ -193,7 +202,7 @@ __device__ __forceinline__ void load_gates(float *dst, int ld, const float *gate
         else *reinterpret_cast<float4 *>(dst + j * ld + c) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
-// A [dk][dv] state of the workspace -> [pad16(dk)][ld] tile (unrounded), padding zero.
+// A [dk][dv] state of the workspace (rounded to tf32 by the scan kernels) -> [pad16(dk)][ld] tile, padding zero.
 __device__ __forceinline__ void load_state(float *dst, int ld, const float *src, int dk, int dv)
 {
     const int per_row = pad16(dv) >> 2;
@@ -203,29 +212,33 @@ __device__ __forceinline__ void load_state(float *dst, int ld, const float *src,
         else *reinterpret_cast<float4 *>(dst + r * ld + c) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
-// In place: rows of a state tile times exp(row_scale[r]) (row_scale may be null), rounded to tf32.
-__device__ __forceinline__ void round_state(float *t, int ld, int dk, int dv, const float *row_scale)
-{
-    const int per_row = pad16(dv) >> 2;
-    for (int idx = threadIdx.x; idx < dk * per_row; idx += kThreads) {
-        const int r = idx / per_row, c = (idx - r * per_row) << 2;
-        const float sc = row_scale ? __expf(row_scale[r]) : 1.f;
-        float4 val = *reinterpret_cast<const float4 *>(t + r * ld + c);
-        *reinterpret_cast<float4 *>(t + r * ld + c) = make_float4(tf32r(val.x * sc), tf32r(val.y * sc), tf32r(val.z * sc), tf32r(val.w * sc));
-    }
-}
 // In place: gates -> inclusive prefix sums down the rows of the chunk; sLast receives the last row.
-__device__ __forceinline__ void prefix_gates(float *lam, int ld, int C, int dkp, float *sLast)
+// Four threads per channel take a quarter of the rows each; sSeg ([4][dkp]) carries the quarter totals.
+// Contains two barriers.
+__device__ __forceinline__ void prefix_gates(float *lam, int ld, int C, int dkp, float *sLast, float *sSeg)
 {
-    for (int c = threadIdx.x; c < dkp; c += kThreads) {
-        float run = 0.f;
+    const int rows = C >> 2;                    // C is a multiple of 16
+    const int c = threadIdx.x % dkp, seg = threadIdx.x / dkp;      // 4 * dkp <= kThreads
+    float run = 0.f;
+    if (seg < 4) {
 #pragma unroll 8
-        for (int j = 0; j < C; ++j) {
+        for (int j = seg * rows; j < (seg + 1) * rows; ++j) {
             run += lam[j * ld + c];
             lam[j * ld + c] = run;
         }
-        sLast[c] = run;
+        sSeg[seg * dkp + c] = run;
     }
+    __syncthreads();
+    if (seg < 4) {
+        float add = 0.f;
+        for (int sg = 0; sg < seg; ++sg) add += sSeg[sg * dkp + c];
+        if (seg > 0) {
+#pragma unroll 8
+            for (int j = seg * rows; j < (seg + 1) * rows; ++j) lam[j * ld + c] += add;
+        }
+        if (seg == 3) sLast[c] = run + add;
+    }
+    __syncthreads();
 }
 // In place: sQ (raw q) -> Qt = q*exp(Lam), sK (raw k) -> Kt = k*exp(-Lam), or with sLast given
 // -> Kh = k*exp(Lam_{C-1}-Lam); rounded to tf32.  Either tile may be null.
@@ -255,17 +268,19 @@ __device__ __forceinline__ void scale_qk(float *sQ, float *sK, const float *sLam
 
 // sP[t][s] = A_t . B_s for s <= t, 0 above the diagonal, rounded to tf32 (A, B: [C][ld] tiles, contraction
 // over the first K columns).  The diagonal has weight 1: the token's own k^T v enters undecayed.
+template <int NB>
 __device__ __forceinline__ void masked_scores(float *sP, int ldp, const float *A, const float *Bm, int ld, int C, int K)
 {
     const Tiling tl(C, C);
     const int warp = threadIdx.x >> 5;
     for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
-        int r0, c0;
-        tl.at(tile, r0, c0);
-        float acc[kMaxNB][4];
+        int r0, c0, nbt;
+        tl.at(tile, r0, c0, nbt);
+        if (nbt <= 0) continue;
+        float acc[NB][4];
         zero(acc);
-        if (c0 <= r0 + 15) warp_mma(acc, A, ld, 1, r0, Bm, 1, ld, c0, tl.nbw, 0, K);
-        for_pairs(acc, r0, c0, tl.nbw, [&](int t, int s, float v0, float v1) {
+        if (c0 <= r0 + 15) warp_mma(acc, A, ld, 1, r0, Bm, 1, ld, c0, nbt, 0, K);
+        for_pairs(acc, r0, c0, nbt, [&](int t, int s, float v0, float v1) {
             *reinterpret_cast<float2 *>(sP + t * ldp + s) = make_float2(s <= t ? tf32r(v0) : 0.f, s + 1 <= t ? tf32r(v1) : 0.f);
         });
     }
@@ -290,7 +305,8 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
     float *sX = sLam + C * ldk;             // k -> Kh
     float *sV = sX + C * ldk;
     float *sLast = sV + C * ldv;            // [dkp]
-    float *sQ = sLast + dkp;                // BWD: q -> Qt
+    float *sSeg = sLast + dkp;              // [4][dkp]
+    float *sQ = sSeg + 4 * dkp;             // BWD: q -> Qt
     float *sG = sQ + (BWD ? C * ldk : 0);   // BWD: dO
 
     fill_rows(sRow, g, C, b, h, chunk);
@@ -304,29 +320,30 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
     }
     cp_async_wait_all();
     __syncthreads();
-    prefix_gates(sLam, ldk, C, dkp, sLast);
-    __syncthreads();
+    prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
     const size_t chunk_id = (size_t)bh * g.N + chunk;
     for (int c = threadIdx.x; c < dk; c += kThreads) gamma[chunk_id * dk + c] = __expf(sLast[c]);
     scale_qk(BWD ? sQ : nullptr, sX, sLam, sLast, ldk, C, dk);
     __syncthreads();
-    const Tiling tl(dkp, dvp);
+    constexpr int NB = frag_bound(pad16(DM::kDK), DM::kDV);
+    const Tiling tl(dkp, dv);
     const int warp = threadIdx.x >> 5;
     float *U = states + chunk_id * dk * dv;
     float *W = BWD ? dstates + chunk_id * dk * dv : nullptr;
     for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
-        int r0, c0;
-        tl.at(tile, r0, c0);
-        float acc[kMaxNB][4];
+        int r0, c0, nbt;
+        tl.at(tile, r0, c0, nbt);
+        if (nbt <= 0) continue;
+        float acc[NB][4];
         zero(acc);
-        warp_mma(acc, sX, 1, ldk, r0, sV, ldv, 1, c0, tl.nbw, 0, C);           // sum_t Kh[t][c] V[t][e]
-        for_pairs(acc, r0, c0, tl.nbw, [&](int c, int e, float v0, float v1) {
+        warp_mma(acc, sX, 1, ldk, r0, sV, ldv, 1, c0, nbt, 0, C);           // sum_t Kh[t][c] V[t][e]
+        for_pairs(acc, r0, c0, nbt, [&](int c, int e, float v0, float v1) {
             if (c < dk && e < dv) store2(U + c * dv + e, v0, v1);
         });
         if (BWD) {
             zero(acc);
-            warp_mma(acc, sQ, 1, ldk, r0, sG, ldv, 1, c0, tl.nbw, 0, C);       // sum_t Qt[t][c] dO[t][e]
-            for_pairs(acc, r0, c0, tl.nbw, [&](int c, int e, float v0, float v1) {
+            warp_mma(acc, sQ, 1, ldk, r0, sG, ldv, 1, c0, nbt, 0, C);       // sum_t Qt[t][c] dO[t][e]
+            for_pairs(acc, r0, c0, nbt, [&](int c, int e, float v0, float v1) {
                 if (c < dk && e < dv) store2(W + c * dv + e, v0, v1);
             });
         }
@@ -353,7 +370,8 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     float *sV = sK + C * ldk;
     float *sS = sV + C * ldv;               // [dkp][ldv]
     float *sLast = sS + dkp * ldv;          // [dkp]
-    float *sP = (C <= dk) ? sLam : sLast + dkp;       // the scores reuse the gate tile when they fit
+    float *sSeg = sLast + dkp;              // [4][dkp]
+    float *sP = (C <= dk) ? sLam : sSeg + 4 * dkp;       // the scores reuse the gate tile when they fit
 
     fill_rows(sRow, g, C, b, h, chunk);
     __syncthreads();
@@ -364,23 +382,23 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     load_rows(sK, ldk, k, sRow, C, dk);
     cp_async_wait_all();
     __syncthreads();
-    prefix_gates(sLam, ldk, C, dkp, sLast);
-    __syncthreads();
+    prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
     scale_qk(sQ, sK, sLam, nullptr, ldk, C, dk);
-    round_state(sS, ldv, dk, dv, nullptr);
     __syncthreads();
-    masked_scores(sP, ldp, sQ, sK, ldk, C, dk);
+    masked_scores<frag_bound(DM::kC, DM::kC)>(sP, ldp, sQ, sK, ldk, C, dk);
     __syncthreads();
-    const Tiling tl(C, dvp);
+    constexpr int NB = frag_bound(DM::kC, DM::kDV);
+    const Tiling tl(C, dv);
     const int warp = threadIdx.x >> 5;
     for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
-        int r0, c0;
-        tl.at(tile, r0, c0);
-        float acc[kMaxNB][4];
+        int r0, c0, nbt;
+        tl.at(tile, r0, c0, nbt);
+        if (nbt <= 0) continue;
+        float acc[NB][4];
         zero(acc);
-        warp_mma(acc, sP, ldp, 1, r0, sV, ldv, 1, c0, tl.nbw, 0, r0 + 16);     // columns past the diagonal are zero
-        warp_mma(acc, sQ, ldk, 1, r0, sS, ldv, 1, c0, tl.nbw, 0, dk);
-        for_pairs(acc, r0, c0, tl.nbw, [&](int j, int e, float v0, float v1) {
+        warp_mma(acc, sP, ldp, 1, r0, sV, ldv, 1, c0, nbt, 0, r0 + 16);     // columns past the diagonal are zero
+        warp_mma(acc, sQ, ldk, 1, r0, sS, ldv, 1, c0, nbt, 0, dk);
+        for_pairs(acc, r0, c0, nbt, [&](int j, int e, float v0, float v1) {
             const int row = sRow[j];
             if (row >= 0 && e < dv) store2(out + (size_t)row * dv + e, v0, v1);
         });
@@ -413,10 +431,11 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     float *sV = sK + C * ldk;
     float *sG = sV + C * ldv;               // dO
     float *sS = sG + C * ldv;               // [dkp][ldv]
-    float *sD = sS + dkp * ldv;             // [dkp][ldv]  Dg
+    float *sD = sS + dkp * ldv;             // [dkp][ldv]  Dg, as the scan kernel stores it
     float *sP = sD + dkp * ldv;             // [C][ldp]
     float *sdP = sP + C * ldp;              // [C][ldp]
     float *sLast = sdP + C * ldp;           // [dkp]
+    float *sSeg = sLast + dkp;              // [4][dkp]
     const size_t chunk_id = (size_t)bh * g.N + chunk;
 
     fill_rows(sRow, g, C, b, h, chunk);
@@ -428,30 +447,28 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     load_rows(sG, ldv, d_out, sRow, C, dv);
     load_rows(sQ, ldk, q, sRow, C, dk);
     load_rows(sK, ldk, k, sRow, C, dk);
-    const float carry_in = threadIdx.x < dk ? carry[chunk_id * dk + threadIdx.x] : 0.f;
     cp_async_wait_all();
     __syncthreads();
-    prefix_gates(sLam, ldk, C, dkp, sLast);
-    __syncthreads();
+    prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
     scale_qk(sQ, sK, sLam, nullptr, ldk, C, dk);
-    round_state(sS, ldv, dk, dv, nullptr);
-    round_state(sD, ldv, dk, dv, sLast);                                         // Dg = diag(gamma) D
     __syncthreads();
-    masked_scores(sP, ldp, sQ, sK, ldk, C, dk);
-    masked_scores(sdP, ldp, sG, sV, ldv, C, dv);
+    masked_scores<frag_bound(DM::kC, DM::kC)>(sP, ldp, sQ, sK, ldk, C, dk);
+    masked_scores<frag_bound(DM::kC, DM::kC)>(sdP, ldp, sG, sV, ldv, C, dv);
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gi = lane >> 2, ti = lane & 3;
     {
         // dv[s][e] = sum_{t >= s} P[t][s] dO[t][e] + sum_c Kt[s][c] Dg[c][e]
-        const Tiling tl(C, dvp);
+        constexpr int NB = frag_bound(DM::kC, DM::kDV);
+        const Tiling tl(C, dv);
         for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
-            int r0, c0;
-            tl.at(tile, r0, c0);
-            float acc[kMaxNB][4];
+            int r0, c0, nbt;
+            tl.at(tile, r0, c0, nbt);
+            if (nbt <= 0) continue;
+            float acc[NB][4];
             zero(acc);
-            warp_mma(acc, sP, 1, ldp, r0, sG, ldv, 1, c0, tl.nbw, r0, C);
-            warp_mma(acc, sK, ldk, 1, r0, sD, ldv, 1, c0, tl.nbw, 0, dk);
-            for_pairs(acc, r0, c0, tl.nbw, [&](int j, int e, float v0, float v1) {
+            warp_mma(acc, sP, 1, ldp, r0, sG, ldv, 1, c0, nbt, r0, C);
+            warp_mma(acc, sK, ldk, 1, r0, sD, ldv, 1, c0, nbt, 0, dk);
+            for_pairs(acc, r0, c0, nbt, [&](int j, int e, float v0, float v1) {
                 const int row = sRow[j];
                 if (row >= 0 && e < dv) store2(dv_out + (size_t)row * dv + e, v0, v1);
             });
@@ -459,17 +476,19 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     }
     {
         // dq and dk of the same (row, channel) tile; x = q*dq - k*dk replaces Lam, element by element
-        const Tiling tl(C, dkp);
+        constexpr int NB = frag_bound(DM::kC, DM::kDK);
+        const Tiling tl(C, dk);
         for (int tile = warp; tile < tl.ntiles; tile += kWarps) {
-            int r0, c0;
-            tl.at(tile, r0, c0);
-            float acc[kMaxNB][4], xq[kMaxNB][4];
+            int r0, c0, nbt;
+            tl.at(tile, r0, c0, nbt);
+            if (nbt <= 0) continue;
+            float acc[NB][4], xq[NB][4];
             zero(acc);
-            warp_mma(acc, sdP, ldp, 1, r0, sK, ldk, 1, c0, tl.nbw, 0, r0 + 16);          // sum_{s <= t} dP[t][s] Kt[s][c]
-            warp_mma(acc, sG, ldv, 1, r0, sS, 1, ldv, c0, tl.nbw, 0, dv);                // sum_e dO[t][e] S[c][e]
+            warp_mma(acc, sdP, ldp, 1, r0, sK, ldk, 1, c0, nbt, 0, r0 + 16);          // sum_{s <= t} dP[t][s] Kt[s][c]
+            warp_mma(acc, sG, ldv, 1, r0, sS, 1, ldv, c0, nbt, 0, dv);                // sum_e dO[t][e] S[c][e]
 #pragma unroll
-            for (int nb = 0; nb < kMaxNB; ++nb)
-                if (nb < tl.nbw) {
+            for (int nb = 0; nb < NB; ++nb)
+                if (nb < nbt) {
 #pragma unroll
                     for (int i = 0; i < 4; i += 2) {
                         const float2 qt = *reinterpret_cast<const float2 *>(sQ + (r0 + gi + 4 * i) * ldk + c0 + 8 * nb + 2 * ti);
@@ -477,7 +496,7 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
                         xq[nb][i + 1] = qt.y * acc[nb][i + 1];
                     }
                 }
-            for_pairs(acc, r0, c0, tl.nbw, [&](int j, int c, float v0, float v1) {
+            for_pairs(acc, r0, c0, nbt, [&](int j, int c, float v0, float v1) {
                 const int row = sRow[j];
                 if (row >= 0 && c < dk) {
                     const float2 lam = *reinterpret_cast<const float2 *>(sLam + j * ldk + c);
@@ -485,11 +504,11 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
                 }
             });
             zero(acc);
-            warp_mma(acc, sdP, 1, ldp, r0, sQ, ldk, 1, c0, tl.nbw, r0, C);               // sum_{t >= s} dP[t][s] Qt[t][c]
-            warp_mma(acc, sV, ldv, 1, r0, sD, 1, ldv, c0, tl.nbw, 0, dv);                // sum_e V[s][e] Dg[c][e]
+            warp_mma(acc, sdP, 1, ldp, r0, sQ, ldk, 1, c0, nbt, r0, C);               // sum_{t >= s} dP[t][s] Qt[t][c]
+            warp_mma(acc, sV, ldv, 1, r0, sD, 1, ldv, c0, nbt, 0, dv);                // sum_e V[s][e] Dg[c][e]
 #pragma unroll
-            for (int nb = 0; nb < kMaxNB; ++nb)
-                if (nb < tl.nbw) {
+            for (int nb = 0; nb < NB; ++nb)
+                if (nb < nbt) {
 #pragma unroll
                     for (int i = 0; i < 4; i += 2) {
                         const float2 kt = *reinterpret_cast<const float2 *>(sK + (r0 + gi + 4 * i) * ldk + c0 + 8 * nb + 2 * ti);
@@ -497,7 +516,7 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
                         xq[nb][i + 1] -= kt.y * acc[nb][i + 1];
                     }
                 }
-            for_pairs(acc, r0, c0, tl.nbw, [&](int j, int c, float v0, float v1) {
+            for_pairs(acc, r0, c0, nbt, [&](int j, int c, float v0, float v1) {
                 const int row = sRow[j];
                 if (row >= 0 && c < dk) {
                     const float2 lam = *reinterpret_cast<const float2 *>(sLam + j * ldk + c);
@@ -505,39 +524,52 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
                 }
             });
             __syncwarp();
-            for_pairs(xq, r0, c0, tl.nbw, [&](int j, int c, float v0, float v1) {
+            for_pairs(xq, r0, c0, nbt, [&](int j, int c, float v0, float v1) {
                 *reinterpret_cast<float2 *>(sLam + j * ldk + c) = make_float2(v0, v1);
             });
         }
     }
     __syncthreads();
-    // gate gradient: suffix sums of x down the chunk plus what later chunks carry in
-    if (threadIdx.x < dk) {             // d_k <= 128 < kThreads
-        const int c = threadIdx.x;
-        float run = carry_in;
-        for (int j = C - 1; j >= 0; --j) {
-            const int row = sRow[j];
-            if (row < 0) continue;
-            run += sLam[j * ldk + c];
-            dgate[(size_t)row * dk + c] = run;
+    // gate gradient: suffix sums of x down the chunk plus what later chunks carry in; four threads per
+    // channel take a quarter of the rows each
+    {
+        const int rows = C >> 2;
+        const int c = threadIdx.x % dkp, seg = threadIdx.x / dkp;
+        float run = 0.f;
+        if (seg < 4) {
+#pragma unroll 8
+            for (int j = (seg + 1) * rows - 1; j >= seg * rows; --j) {
+                run += sLam[j * ldk + c];
+                sLam[j * ldk + c] = run;
+            }
+            sSeg[seg * dkp + c] = run;
+        }
+        __syncthreads();
+        if (seg < 4 && c < dk) {
+            float add = carry[chunk_id * dk + c];
+            for (int sg = seg + 1; sg < 4; ++sg) add += sSeg[sg * dkp + c];
+            for (int j = seg * rows; j < (seg + 1) * rows; ++j) {
+                const int row = sRow[j];
+                if (row >= 0) dgate[(size_t)row * dk + c] = sLam[j * ldk + c] + add;
+            }
         }
     }
 }
 
 size_t smem_state(const Geom &g, bool bwd)
 {
-    return sizeof(float) * ((size_t)g.C * (pitch(g.dk) * (bwd ? 3 : 2) + pitch(g.dv) * (bwd ? 2 : 1)) + pad16(g.dk));
+    return sizeof(float) * ((size_t)g.C * (pitch(g.dk) * (bwd ? 3 : 2) + pitch(g.dv) * (bwd ? 2 : 1)) + 5 * pad16(g.dk));
 }
 size_t smem_out(const Geom &g)
 {
-    size_t n = (size_t)g.C * (3 * pitch(g.dk) + pitch(g.dv)) + (size_t)pad16(g.dk) * pitch(g.dv) + pad16(g.dk);
+    size_t n = (size_t)g.C * (3 * pitch(g.dk) + pitch(g.dv)) + (size_t)pad16(g.dk) * pitch(g.dv) + 5 * pad16(g.dk);
     if (g.C > g.dk) n += (size_t)g.C * pitch(g.C);
     return sizeof(float) * n;
 }
 size_t smem_bwd(const Geom &g)
 {
     return sizeof(float) * ((size_t)g.C * (3 * pitch(g.dk) + 2 * pitch(g.dv) + 2 * pitch(g.C)) +
-                            2 * (size_t)pad16(g.dk) * pitch(g.dv) + pad16(g.dk));
+                            2 * (size_t)pad16(g.dk) * pitch(g.dv) + 5 * pad16(g.dk));
 }
 constexpr size_t kMaxSmem = 227 * 1024 - 1024;      // the row table is static shared memory
 
@@ -566,7 +598,7 @@ dig_status fwd_dims(const GlaArgs &a)
         k1<<<grid, kThreads, smem_state(g, false), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                                               nullptr, w.states, w.gamma, nullptr, g);
     }
-    if ((st = launch_state_scan_fwd(w, g, a.stream)) != DIG_OK) return st;
+    if ((st = launch_state_scan_fwd(w, g, a.stream, false, true)) != DIG_OK) return st;
     KernelTimer t(KID_MMA_OUT, a.stream);
     k3<<<grid, kThreads, smem_out(g), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate, w.states,
                                                   (TO *)a.out, g);
@@ -589,8 +621,8 @@ dig_status bwd_dims(const GlaArgs &a)
         k1<<<grid, kThreads, smem_state(g, true), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                                              (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, g);
     }
-    if ((st = launch_state_scan_fwd(w, g, a.stream)) != DIG_OK) return st;
-    if ((st = launch_state_scan_bwd(w, g, a.stream)) != DIG_OK) return st;
+    if ((st = launch_state_scan_fwd(w, g, a.stream, false, true)) != DIG_OK) return st;
+    if ((st = launch_state_scan_bwd(w, g, a.stream, true)) != DIG_OK) return st;
     KernelTimer t(KID_MMA_BWD, a.stream);
     k4<<<grid, kThreads, smem_bwd(g), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                                   (const bf16 *)a.d_out, w.states, w.dstates, w.carry, (TO *)a.dq, (TO *)a.dk,

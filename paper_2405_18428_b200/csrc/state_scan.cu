@@ -32,7 +32,8 @@ __device__ __forceinline__ float4 round4_tf32(float4 v)
 // rounded to tf32 (the running value is not).
 // The loads of a batch of kAhead chunks do not depend on the running value, so they are all in
 // flight before the short dependent chain of FMAs runs.
-template <bool TILES>
+// TF32: the stored states are rounded to tf32 although they stay row-major (warp-MMA family).
+template <bool TILES, bool TF32 = false>
 __global__ void __launch_bounds__(kScanThreads)
 state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int N, int dk, int dv)
 {
@@ -65,7 +66,7 @@ state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int 
 #pragma unroll
         for (int j = 0; j < kAhead; ++j) {
             if (i + j < N) {
-                st[(size_t)(i + j) * sstride] = TILES ? round4_tf32(run) : run;
+                st[(size_t)(i + j) * sstride] = (TILES || TF32) ? round4_tf32(run) : run;
                 run.x = fmaf(g[j].x, run.x, u[j].x);
                 run.y = fmaf(g[j].y, run.y, u[j].y);
                 run.z = fmaf(g[j].z, run.z, u[j].z);
@@ -76,9 +77,12 @@ state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int 
 }
 
 // One warp per key channel c; lanes stride over the value channels.
+// TF32: dstates receives diag(gamma_i) D_[i] rounded to tf32, the form the warp-MMA gradient kernel
+// multiplies with, instead of D_[i].
 constexpr int kRowsPerBlock = 4;
 constexpr int kMaxPerLane = 4;     // d_v <= 128
 
+template <bool TF32>
 __global__ void __launch_bounds__(32 * kRowsPerBlock)
 state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
                const float *__restrict__ gamma, float *__restrict__ carry, int N, int dk, int dv)
@@ -120,7 +124,7 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
 #pragma unroll
             for (int r = 0; r < kMaxPerLane; ++r) {
                 const int e = lane + 32 * r;
-                if (e < dv) D[(size_t)ch * sstride + e] = run[r];
+                if (e < dv) D[(size_t)ch * sstride + e] = TF32 ? round_tf32(g[j] * run[r]) : run[r];
                 dot = fmaf(sn[j][r], run[r], dot);
                 run[r] = fmaf(g[j], run[r], w[j][r]);
             }
@@ -224,24 +228,28 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
 
 }  // namespace
 
-dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tiles)
+dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tiles, bool tf32)
 {
     const dim3 grid((g.dk * g.dv / 4 + kScanThreads - 1) / kScanThreads, g.B * g.H);
     if (tiles && (g.dk != 64 || g.dv != 64)) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_SCAN_FWD, s);
     if (tiles)
         launch_pdl(state_scan_fwd<true>, grid, dim3(kScanThreads), 0, s, w.states, (const float *)w.gamma, g.N, g.dk, g.dv);
+    else if (tf32)
+        state_scan_fwd<false, true><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
     else
         state_scan_fwd<false><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
     return cuda_ok(cudaGetLastError());
 }
 
-dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s)
+dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tf32)
 {
     const dim3 grid((g.dk + kRowsPerBlock - 1) / kRowsPerBlock, g.B * g.H);
     KernelTimer t(KID_SCAN_BWD, s);
-    state_scan_bwd<<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N,
-                                                       g.dk, g.dv);
+    if (tf32)
+        state_scan_bwd<true><<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N, g.dk, g.dv);
+    else
+        state_scan_bwd<false><<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N, g.dk, g.dv);
     return cuda_ok(cudaGetLastError());
 }
 
