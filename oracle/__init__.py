@@ -48,6 +48,8 @@ def _load():
                                             ctypes.c_int, ctypes.c_int]
             lib.dig_oracle_gla_fwd.argtypes = [dp] * 5 + [ctypes.c_int] * 8
             lib.dig_oracle_gla_bwd.argtypes = [dp] * 9 + [ctypes.c_int] * 8
+            lib.dig_oracle_gla_fwd_state.argtypes = [dp] * 7 + [ctypes.c_int] * 8
+            lib.dig_oracle_gla_bwd_state.argtypes = [dp] * 12 + [ctypes.c_int] * 8
             lib.dig_oracle_dwconv.argtypes = [dp] * 4 + [ctypes.c_int] * 5
             lib.dig_oracle_dwconv_bwd.argtypes = [dp] * 6 + [ctypes.c_int] * 5
             lib.dig_oracle_outgate_fwd.argtypes = [dp] * 5 + [ctypes.c_longlong, ctypes.c_int, ctypes.c_double]
@@ -175,3 +177,44 @@ def outgate_bwd(o, r, dz, ln_w=None, ln_b=None, eps=1e-5):
     _check(_load().dig_oracle_outgate_bwd(_p(o), _p(r), wp, bp, _p(dz), _p(do), _p(dr), _p(dw), _p(db),
                                           o.size // d, d, float(eps)), "outgate_bwd")
     return do, dr, dw, db
+
+
+def gla_fwd_state(q, k, v, a, s_in, grid_h, grid_w, direction=ROW_FWD, threads=1):
+    """gla_fwd started from state s_in ([B, H, d_k, d_v] or None = zero); returns (out, s_out)."""
+    q, k, v, a = map(_f64, (q, k, v, a))
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    assert L == grid_h * grid_w and k.shape == q.shape == a.shape and v.shape == (B, L, H, dv)
+    sp = None
+    if s_in is not None:
+        s_in = _f64(s_in)
+        assert s_in.shape == (B, H, dk, dv)
+        sp = _p(s_in)
+    out, s_out = np.empty_like(v), np.empty((B, H, dk, dv))
+    _check(_load().dig_oracle_gla_fwd_state(_p(q), _p(k), _p(v), _p(a), sp, _p(out), _p(s_out), B, H, grid_h,
+                                            grid_w, dk, dv, direction, threads), "gla_fwd_state")
+    return out, s_out
+
+
+def gla_bwd_state(q, k, v, a, dout, s_in, ds_out, grid_h, grid_w, direction=ROW_FWD, threads=1):
+    """Gradients (dq, dk, dv, da, ds_in) of <dout, out> + <ds_out, s_out> for gla_fwd_state."""
+    q, k, v, a, dout = map(_f64, (q, k, v, a, dout))
+    B, L, H, dk = q.shape
+    dv_ = v.shape[-1]
+    assert L == grid_h * grid_w and dout.shape == v.shape
+    sp = dp_ = None
+    if s_in is not None:
+        s_in = _f64(s_in)
+        assert s_in.shape == (B, H, dk, dv_)
+        sp = _p(s_in)
+    if ds_out is not None:
+        ds_out = _f64(ds_out)
+        assert ds_out.shape == (B, H, dk, dv_)
+        dp_ = _p(ds_out)
+    dq, dk_, da = np.empty_like(q), np.empty_like(q), np.empty_like(q)
+    dv = np.empty_like(v)
+    ds_in = np.empty((B, H, dk, dv_))
+    _check(_load().dig_oracle_gla_bwd_state(_p(q), _p(k), _p(v), _p(a), _p(dout), sp, dp_, _p(dq), _p(dk_),
+                                            _p(dv), _p(da), _p(ds_in), B, H, grid_h, grid_w, dk, dv_, direction,
+                                            threads), "gla_bwd_state")
+    return dq, dk_, dv, da, ds_in

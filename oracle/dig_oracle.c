@@ -15,6 +15,9 @@
  *   - the 3x3 depthwise convolution of the SREM module (Algorithm 1, "DWConv2d(reshape2d(z))"),
  *     evaluated on the re-oriented token matrix by explicit gather / conv / scatter, and its
  *     reverse-mode derivative
+ *   - the recurrence started from a given state and returning the final state (the paper starts
+ *     from zero and drops it; this is what splitting a sequence into pieces needs), with the
+ *     matching terms of the derivative
  *   - the output gate z = Swish(r) (.) LN(o) that follows the recurrence (Eq. attn_gla, the line
  *     forming Y_t before the projection W_O), and its reverse-mode derivative
  *
@@ -31,7 +34,9 @@
  * dw of an identity-initialised filter on a one-pixel image; for the output gate: a library
  * layer-norm and silu on the same rows, zero-mean / unit-variance and shift-scale invariance of
  * the normalisation, Swish's values at 0 and far from 0, central finite differences of the
- * derivative, and do summing to zero over a row when the affine part is absent.
+ * derivative, and do summing to zero over a row when the affine part is absent; for the state
+ * arguments: a sequence cut in two and chained through the state equals the uncut one (values and
+ * all gradients), the final state of a constant-decay sequence in closed form, finite differences.
  * Not pinned by the paper: whether DWConv2d carries a bias (the argument is optional).
  */
 #include <math.h>
@@ -89,10 +94,12 @@ static size_t tok_off(long long b, long long t, int h, long long L, int H, int d
     return (((size_t)b * L + t) * H + h) * (size_t)d;
 }
 
-/* Forward recurrence (Eq. attn_gla), one (b,h) pair at a time, in scan order. */
-int dig_oracle_gla_fwd(const double *q, const double *k, const double *v, const double *a,
-                       double *out, int B, int H, int grid_h, int grid_w, int d_k, int d_v,
-                       int direction, int threads)
+/* Forward recurrence (Eq. attn_gla), one (b,h) pair at a time, in scan order.
+ * s_in (may be NULL = zero, the paper's case): state before the first scan position, [B][H][d_k][d_v];
+ * s_out (may be NULL): receives the state after the last scan position, same layout. */
+static int gla_fwd_impl(const double *q, const double *k, const double *v, const double *a,
+                        double *out, const double *s_in, double *s_out, int B, int H, int grid_h, int grid_w,
+                        int d_k, int d_v, int direction, int threads)
 {
     const long long L = (long long)grid_h * grid_w;
     long long *perm = (long long *)malloc(sizeof(long long) * (size_t)L);
@@ -107,6 +114,7 @@ int dig_oracle_gla_fwd(const double *q, const double *k, const double *v, const 
         const int b = bh / H, h = bh % H;
         double *S = (double *)calloc((size_t)d_k * d_v, sizeof(double));
         if (!S) { err = 2; continue; }
+        if (s_in) memcpy(S, s_in + (size_t)bh * d_k * d_v, sizeof(double) * (size_t)d_k * d_v);
         for (long long p = 0; p < L; ++p) {
             const long long t = perm[p];
             const double *qt = q + tok_off(b, t, h, L, H, d_k);
@@ -125,10 +133,27 @@ int dig_oracle_gla_fwd(const double *q, const double *k, const double *v, const 
                 ot[e] = acc;
             }
         }
+        if (s_out) memcpy(s_out + (size_t)bh * d_k * d_v, S, sizeof(double) * (size_t)d_k * d_v);
         free(S);
     }
     free(perm);
     return err;
+}
+
+int dig_oracle_gla_fwd(const double *q, const double *k, const double *v, const double *a,
+                       double *out, int B, int H, int grid_h, int grid_w, int d_k, int d_v,
+                       int direction, int threads)
+{
+    return gla_fwd_impl(q, k, v, a, out, NULL, NULL, B, H, grid_h, grid_w, d_k, d_v, direction, threads);
+}
+
+/* The same recurrence started from a given state and returning the final one: what a caller needs to
+ * split a sequence into pieces (the paper always starts from zero and drops the final state). */
+int dig_oracle_gla_fwd_state(const double *q, const double *k, const double *v, const double *a,
+                             const double *s_in, double *out, double *s_out, int B, int H, int grid_h,
+                             int grid_w, int d_k, int d_v, int direction, int threads)
+{
+    return gla_fwd_impl(q, k, v, a, out, s_in, s_out, B, H, grid_h, grid_w, d_k, d_v, direction, threads);
 }
 
 /* Reverse-mode derivative of the recurrence above.
@@ -136,11 +161,14 @@ int dig_oracle_gla_fwd(const double *q, const double *k, const double *v, const 
  *   dq_t  = S_t do_t^T,  dk_t = dS_t v_t^T,  dv_t = k_t dS_t
  *   da_t[c] = alpha_t[c] * sum_e dS_t[c,e] S_{t-1}[c,e]
  * S_{t-1} and S_t are re-created from checkpoints of the forward state taken every SEG
- * positions, so memory stays small at long L. */
-int dig_oracle_gla_bwd(const double *q, const double *k, const double *v, const double *a,
-                       const double *dout, double *dq, double *dk, double *dv, double *da,
-                       int B, int H, int grid_h, int grid_w, int d_k, int d_v,
-                       int direction, int threads)
+ * positions, so memory stays small at long L.
+ * With a start state s_in (NULL = zero) the forward sweep starts from it; ds_out (NULL = zero) is the
+ * gradient with respect to the final state and seeds dS; ds_in (may be NULL) receives the gradient
+ * with respect to s_in, which is dS after the first position has handed it on. */
+static int gla_bwd_impl(const double *q, const double *k, const double *v, const double *a,
+                        const double *dout, const double *s_in, const double *ds_out, double *dq, double *dk,
+                        double *dv, double *da, double *ds_in, int B, int H, int grid_h, int grid_w, int d_k,
+                        int d_v, int direction, int threads)
 {
     enum { SEG = 64 };
     const long long L = (long long)grid_h * grid_w;
@@ -160,9 +188,11 @@ int dig_oracle_gla_bwd(const double *q, const double *k, const double *v, const 
         double *seg = (double *)malloc(sizeof(double) * SZ * (SEG + 1));       /* seg[j] = state before local step j */
         double *dS = (double *)calloc(SZ, sizeof(double));
         if (!ckpt || !seg || !dS) { err = 2; free(ckpt); free(seg); free(dS); continue; }
+        if (ds_out) memcpy(dS, ds_out + SZ * (size_t)bh, sizeof(double) * SZ);
         /* forward sweep, storing checkpoints */
         {
             double *S = (double *)calloc(SZ, sizeof(double));
+            if (s_in) memcpy(S, s_in + SZ * (size_t)bh, sizeof(double) * SZ);
             for (long long p = 0; p < L; ++p) {
                 if (p % SEG == 0) memcpy(ckpt + SZ * (size_t)(p / SEG), S, sizeof(double) * SZ);
                 const long long t = perm[p];
@@ -227,10 +257,29 @@ int dig_oracle_gla_bwd(const double *q, const double *k, const double *v, const 
                 }
             }
         }
+        if (ds_in) memcpy(ds_in + SZ * (size_t)bh, dS, sizeof(double) * SZ);
         free(ckpt); free(seg); free(dS);
     }
     free(perm);
     return err;
+}
+
+int dig_oracle_gla_bwd(const double *q, const double *k, const double *v, const double *a,
+                       const double *dout, double *dq, double *dk, double *dv, double *da,
+                       int B, int H, int grid_h, int grid_w, int d_k, int d_v,
+                       int direction, int threads)
+{
+    return gla_bwd_impl(q, k, v, a, dout, NULL, NULL, dq, dk, dv, da, NULL, B, H, grid_h, grid_w, d_k, d_v,
+                        direction, threads);
+}
+
+int dig_oracle_gla_bwd_state(const double *q, const double *k, const double *v, const double *a,
+                             const double *dout, const double *s_in, const double *ds_out, double *dq,
+                             double *dk, double *dv, double *da, double *ds_in, int B, int H, int grid_h,
+                             int grid_w, int d_k, int d_v, int direction, int threads)
+{
+    return gla_bwd_impl(q, k, v, a, dout, s_in, ds_out, dq, dk, dv, da, ds_in, B, H, grid_h, grid_w, d_k, d_v,
+                        direction, threads);
 }
 
 /* SREM depthwise convolution (Algorithm 1: DWConv2d(reshape2d(z))).
