@@ -173,6 +173,26 @@ dig_status dig_gla_outgate_bwd(const void *o, const void *r, const float *ln_w, 
                                void *d_o, void *d_r, float *dln_w, float *dln_b, long long rows, int d_v, float eps,
                                int dtype, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* dig_gla_fwd / dig_gla_bwd with the state of the recurrence as an argument (the paper always starts
+ * from S = 0 and drops the final state; these are what a caller needs to cut a long sequence into
+ * pieces or to shard it over devices: run the pieces in scan order and chain them through the state).
+ * All state tensors are fp32 [B][H][d_k][d_v] row-major device arrays; each may be NULL.
+ *   s_in   state before the first token in scan order (NULL = 0)
+ *   s_out  receives the state after the last token (NULL = not wanted)
+ *   ds_out gradient of the loss with respect to s_out (NULL = 0)
+ *   ds_in  receives the gradient with respect to s_in (NULL = not wanted)
+ * dig_gla_bwd_state returns the gradients of  <d_out, out> + <ds_out, s_out>.  Workspace sizes are
+ * those of dig_gla_fwd / dig_gla_bwd.  The states are kept in fp32 across the whole sequence; the
+ * kernels that consume them round them to tf32 per chunk exactly as without these arguments. */
+dig_status dig_gla_fwd_state(const void *q, const void *k, const void *v, const float *gate, const float *s_in,
+                             void *out, float *s_out, int B, int H, int grid_h, int grid_w, int d_k, int d_v,
+                             int chunk, int direction, int dtype, void *workspace, size_t workspace_bytes,
+                             void *cuda_stream);
+dig_status dig_gla_bwd_state(const void *q, const void *k, const void *v, const float *gate, const void *d_out,
+                             const float *s_in, const float *ds_out, void *dq, void *dk, void *dv, float *dgate,
+                             float *ds_in, int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
+                             int direction, int dtype, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the status recorded by device code on the
  * current device: DIG_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last query,
  * DIG_ERR_CUDA if the synchronisation itself failed, DIG_OK otherwise. */

@@ -167,7 +167,8 @@ dig_status dig_gate_logsigmoid(const void *g, const float *tau_per_head, float *
     return launch_gate(g, tau_per_head, gate, B, L, H, d_k, dtype, (cudaStream_t)cuda_stream);
 }
 
-dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float *gate, void *out,
+dig_status dig_gla_fwd_state(const void *q, const void *k, const void *v, const float *gate, const float *s_in,
+                             void *out, float *s_out,
                        int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
                        int direction, int dtype, void *workspace, size_t workspace_bytes,
                        void *cuda_stream)
@@ -180,7 +181,9 @@ dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float 
     if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
     const int impl = choose_impl(d_k, d_v, chunk, dtype, false);
     if (impl < 0) return (dig_status)(-impl);
+    if ((s_in && !aligned16(s_in)) || (s_out && !aligned16(s_out))) return DIG_ERR_INVALID_ARG;
     GlaArgs a{};
+    a.sio.s_in = s_in; a.sio.s_out = s_out;
     a.q = q; a.k = k; a.v = v; a.gate = gate; a.out = out;
     a.ws = reinterpret_cast<float *>(workspace);
     a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
@@ -189,8 +192,9 @@ dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float 
     return impl == DIG_IMPL_TENSOR ? tensor_gla_fwd(a) : impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
 }
 
-dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float *gate,
-                       const void *d_out, void *dq, void *dk, void *dv, float *dgate, int B, int H,
+dig_status dig_gla_bwd_state(const void *q, const void *k, const void *v, const float *gate,
+                             const void *d_out, const float *s_in, const float *ds_out, void *dq, void *dk, void *dv,
+                             float *dgate, float *ds_in, int B, int H,
                        int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
                        void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
@@ -203,7 +207,9 @@ dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float 
     if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
     const int impl = choose_impl(d_k, d_v, chunk, dtype, true);
     if (impl < 0) return (dig_status)(-impl);
+    if ((s_in && !aligned16(s_in)) || (ds_out && !aligned16(ds_out)) || (ds_in && !aligned16(ds_in))) return DIG_ERR_INVALID_ARG;
     GlaArgs a{};
+    a.sio.s_in = s_in; a.sio.ds_out = ds_out; a.sio.ds_in = ds_in;
     a.q = q; a.k = k; a.v = v; a.gate = gate; a.d_out = d_out;
     a.dq = dq; a.dk = dk; a.dv = dv; a.dgate = dgate;
     a.ws = reinterpret_cast<float *>(workspace);
@@ -211,6 +217,23 @@ dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float 
     a.dtype = dtype;
     a.stream = (cudaStream_t)cuda_stream;
     return impl == DIG_IMPL_TENSOR ? tensor_gla_bwd(a) : impl == DIG_IMPL_MMA ? mma_gla_bwd(a) : fma_gla_bwd(a);
+}
+
+dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float *gate, void *out,
+                       int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction,
+                       int dtype, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return dig_gla_fwd_state(q, k, v, gate, nullptr, out, nullptr, B, H, grid_h, grid_w, d_k, d_v, chunk, direction,
+                             dtype, workspace, workspace_bytes, cuda_stream);
+}
+
+dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float *gate,
+                       const void *d_out, void *dq, void *dk, void *dv, float *dgate, int B, int H,
+                       int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return dig_gla_bwd_state(q, k, v, gate, d_out, nullptr, nullptr, dq, dk, dv, dgate, nullptr, B, H, grid_h, grid_w,
+                             d_k, d_v, chunk, direction, dtype, workspace, workspace_bytes, cuda_stream);
 }
 
 dig_status dig_srem_dwconv(const void *x, const void *w, const void *bias, void *y, int B,

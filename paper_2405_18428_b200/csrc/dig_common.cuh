@@ -65,7 +65,18 @@ __device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v)
 }
 
 // ---- launch plumbing shared by the .cu files --------------------------------------------
+// Optional state arguments of the recurrence (all [B][H][d_k][d_v] fp32 row-major, any may be null):
+// the state before the first scan position, the state after the last one, the gradient with
+// respect to that final state, and the gradient with respect to the start state.
+struct StateIO {
+    const float *s_in;
+    float *s_out;
+    const float *ds_out;
+    float *ds_in;
+};
+
 struct GlaArgs {
+    StateIO sio;
     const void *q, *k, *v;
     const float *gate;
     void *out;                   // forward
@@ -86,7 +97,7 @@ struct GlaArgs {
 //   dstates_m [B*H][N][dk][dv] (backward) second copy of the decayed state gradients, in the other
 //                              operand-tile order (used by the tensor-core family only)
 struct Workspace {
-    float *states, *gamma, *dstates, *carry, *dstates_m;
+    float *states, *gamma, *dstates, *carry, *dstates_m, *sfinal;
     size_t bytes;
 };
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -104,7 +115,9 @@ inline Workspace carve_workspace(float *base, const Geom &g, bool backward)
         w.dstates = reinterpret_cast<float *>(p);       p += st;
         w.carry = reinterpret_cast<float *>(p);         p += gm;
         w.dstates_m = reinterpret_cast<float *>(p);     p += st;
-        w.bytes += 2 * st + gm;
+        const size_t fin = align256(bh * g.dk * g.dv * sizeof(float));
+        w.sfinal = reinterpret_cast<float *>(p);        p += fin;
+        w.bytes += 2 * st + gm + fin;
     }
     return w;
 }
@@ -122,10 +135,11 @@ bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward);
 
 // Chunk-state scans, shared by both families (plain fp32 FMA, bandwidth-bound).
 // `tiles`: the states are stored transposed, in swizzled operand-tile order (tensor-core forward pass).
-dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tiles = false, bool tf32 = false);
-dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tf32 = false);
+dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tiles = false,
+                                 bool tf32 = false);
+dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tf32 = false);
 // Tensor-core backward pass: forward and reverse scan in one launch over states kept in tile order.
-dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s);
+dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio);
 
 // Device status word (bounded waits report here).
 int *device_status_ptr();

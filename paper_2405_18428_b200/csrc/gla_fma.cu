@@ -463,7 +463,7 @@ dig_status fwd_typed(const GlaArgs &a)
     { KernelTimer t(KID_FMA_STATE, a.stream);
     k1<<<grid, kThreads, smem_state(g, false), a.stream>>>(
         (const T *)a.q, (const T *)a.k, (const T *)a.v, a.gate, nullptr, w.states, w.gamma, nullptr, g); }
-    if ((st = launch_state_scan_fwd(w, g, a.stream)) != DIG_OK) return st;
+    if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio)) != DIG_OK) return st;
     auto k3 = fma_chunk_out<T, TO>;
     if ((st = set_smem(k3, smem_out(g))) != DIG_OK) return st;
     KernelTimer t(KID_FMA_OUT, a.stream);
@@ -487,8 +487,8 @@ dig_status bwd_typed(const GlaArgs &a)
     k1<<<grid, kThreads, smem_state(g, true), a.stream>>>(
         (const T *)a.q, (const T *)a.k, (const T *)a.v, a.gate, (const T *)a.d_out, w.states, w.gamma,
         w.dstates, g); }
-    if ((st = launch_state_scan_fwd(w, g, a.stream)) != DIG_OK) return st;
-    if ((st = launch_state_scan_bwd(w, g, a.stream)) != DIG_OK) return st;
+    if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio)) != DIG_OK) return st;
+    if ((st = launch_state_scan_bwd(w, g, a.stream, a.sio)) != DIG_OK) return st;
     KernelTimer t(KID_FMA_BWD, a.stream);
     k4<<<grid, kThreads, smem_bwd(g), a.stream>>>(
         (const T *)a.q, (const T *)a.k, (const T *)a.v, a.gate, (const T *)a.d_out, w.states, w.dstates,

@@ -598,7 +598,7 @@ dig_status fwd_dims(const GlaArgs &a)
         k1<<<grid, kThreads, smem_state(g, false), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                                               nullptr, w.states, w.gamma, nullptr, g);
     }
-    if ((st = launch_state_scan_fwd(w, g, a.stream, false, true)) != DIG_OK) return st;
+    if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, false, true)) != DIG_OK) return st;
     KernelTimer t(KID_MMA_OUT, a.stream);
     k3<<<grid, kThreads, smem_out(g), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate, w.states,
                                                   (TO *)a.out, g);
@@ -621,8 +621,8 @@ dig_status bwd_dims(const GlaArgs &a)
         k1<<<grid, kThreads, smem_state(g, true), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                                              (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, g);
     }
-    if ((st = launch_state_scan_fwd(w, g, a.stream, false, true)) != DIG_OK) return st;
-    if ((st = launch_state_scan_bwd(w, g, a.stream, true)) != DIG_OK) return st;
+    if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, false, true)) != DIG_OK) return st;
+    if ((st = launch_state_scan_bwd(w, g, a.stream, a.sio, true)) != DIG_OK) return st;
     KernelTimer t(KID_MMA_BWD, a.stream);
     k4<<<grid, kThreads, smem_bwd(g), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
                                                   (const bf16 *)a.d_out, w.states, w.dstates, w.carry, (TO *)a.dq, (TO *)a.dk,

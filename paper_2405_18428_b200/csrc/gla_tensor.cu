@@ -33,7 +33,7 @@ dig_status tensor_gla_fwd(const GlaArgs &a)
     if ((long long)g.B * g.H * g.N > (1ll << 30)) return DIG_ERR_UNSUPPORTED;      // chunk ids are 32-bit
     dig_status st;
     if ((st = launch_tc_state(a, w, false, sms, status)) != DIG_OK) return st;
-    if ((st = launch_state_scan_fwd(w, g, a.stream, true)) != DIG_OK) return st;
+    if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, true)) != DIG_OK) return st;
     return launch_tc_out(a, w, sms, status);
 }
 
@@ -47,7 +47,7 @@ dig_status tensor_gla_bwd(const GlaArgs &a)
     if ((long long)g.B * g.H * g.N > (1ll << 30)) return DIG_ERR_UNSUPPORTED;
     dig_status st;
     if ((st = launch_tc_state(a, w, true, sms, status)) != DIG_OK) return st;
-    if ((st = launch_state_scan_bwd_tiles(w, g, a.stream)) != DIG_OK) return st;
+    if ((st = launch_state_scan_bwd_tiles(w, g, a.stream, a.sio)) != DIG_OK) return st;
     return launch_tc_bwd(a, w, sms, status);
 }
 

@@ -7,6 +7,9 @@
 // leaving chunk i, and carry_i the part of the gate gradient that tokens of later chunks
 // contribute to every token of chunk i.  Plain fp32 FMAs; the work is a dependent chain over
 // the N chunks per element, so loads are issued a few chunks ahead of their use.
+// Optional state arguments ([B*H][d_k][d_v] row-major fp32, null = zero / not wanted): the forward scan
+// starts from s_in and hands out the state after the last chunk; the backward scan starts from the
+// gradient with respect to that final state and hands out the gradient with respect to s_in.
 #include "dig_common.cuh"
 
 namespace dig {
@@ -35,7 +38,8 @@ __device__ __forceinline__ float4 round4_tf32(float4 v)
 // TF32: the stored states are rounded to tf32 although they stay row-major (warp-MMA family).
 template <bool TILES, bool TF32 = false>
 __global__ void __launch_bounds__(kScanThreads)
-state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int N, int dk, int dv)
+state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, const float *__restrict__ s_in,
+               float *__restrict__ s_final, int N, int dk, int dv)
 {
     pdl_wait();
     pdl_launch_dependents();      // only once this kernel's own predecessor has completed
@@ -53,6 +57,11 @@ state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int 
     const float *gm = gamma + (size_t)blockIdx.y * N * dk + (TILES ? col : row);
     const size_t sstride = (size_t)dk * dv / 4;
     float4 run = make_float4(0.f, 0.f, 0.f, 0.f);
+    // this thread's four elements in a row-major [d_k][d_v] state: consecutive (plain layout) or a
+    // stride of d_v apart (the transposed tiles hold S[col .. col+3][row])
+    const size_t io = (size_t)blockIdx.y * dk * dv + (TILES ? (size_t)col * dv + row : (size_t)row * dv + col);
+    const size_t ios = TILES ? (size_t)dv : 1;
+    if (s_in != nullptr) run = make_float4(s_in[io], s_in[io + ios], s_in[io + 2 * ios], s_in[io + 3 * ios]);
     for (int i = 0; i < N; i += kAhead) {
         float4 u[kAhead], g[kAhead];
 #pragma unroll
@@ -74,6 +83,12 @@ state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, int 
             }
         }
     }
+    if (s_final != nullptr) {
+        s_final[io] = run.x;
+        s_final[io + ios] = run.y;
+        s_final[io + 2 * ios] = run.z;
+        s_final[io + 3 * ios] = run.w;
+    }
 }
 
 // One warp per key channel c; lanes stride over the value channels.
@@ -85,7 +100,8 @@ constexpr int kMaxPerLane = 4;     // d_v <= 128
 template <bool TF32>
 __global__ void __launch_bounds__(32 * kRowsPerBlock)
 state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
-               const float *__restrict__ gamma, float *__restrict__ carry, int N, int dk, int dv)
+               const float *__restrict__ gamma, float *__restrict__ carry, const float *__restrict__ s_final,
+               const float *__restrict__ ds_out, float *__restrict__ ds_in, int N, int dk, int dv)
 {
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * kRowsPerBlock + (threadIdx.x >> 5);
@@ -97,8 +113,12 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
     const float *gm = gamma + (size_t)blockIdx.y * N * dk + c;
     float *cr = carry + (size_t)blockIdx.y * N * dk + c;
     float run[kMaxPerLane];
+    const size_t io = ((size_t)blockIdx.y * dk + c) * dv;
 #pragma unroll
-    for (int r = 0; r < kMaxPerLane; ++r) run[r] = 0.f;
+    for (int r = 0; r < kMaxPerLane; ++r) {
+        const int e = lane + 32 * r;
+        run[r] = (ds_out != nullptr && e < dv) ? ds_out[io + e] : 0.f;
+    }
     // kLook chunks are loaded ahead of the recurrence, so the walk pays the latency of global memory
     // once per kLook chunks and not once per chunk
     constexpr int kLook = 8;
@@ -113,7 +133,11 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
             for (int r = 0; r < kMaxPerLane; ++r) {
                 const int e = lane + 32 * r;
                 w[j][r] = (ch >= 0 && e < dv) ? D[(size_t)ch * sstride + e] : 0.f;
-                sn[j][r] = (ch >= 0 && e < dv && ch + 1 < N) ? S[(size_t)(ch + 1) * sstride + e] : 0.f;
+                sn[j][r] = 0.f;          // the state leaving chunk ch: the next chunk's entry, or the final state
+                if (ch >= 0 && e < dv) {
+                    if (ch + 1 < N) sn[j][r] = S[(size_t)(ch + 1) * sstride + e];
+                    else if (ds_out != nullptr) sn[j][r] = s_final[io + e];
+                }
             }
         }
 #pragma unroll
@@ -133,6 +157,13 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
             if (lane == 0) cr[(size_t)ch * dk] = dot;
         }
     }
+    if (ds_in != nullptr) {
+#pragma unroll
+        for (int r = 0; r < kMaxPerLane; ++r) {
+            const int e = lane + 32 * r;
+            if (e < dv) ds_in[io + e] = run[r];
+        }
+    }
 }
 
 // Both scans of the tensor-core backward pass in one launch (d_k = d_v = 64).  The per-chunk
@@ -150,7 +181,8 @@ __device__ __forceinline__ float4 fma4(float g, float4 r, float4 u)
 }
 __global__ void __launch_bounds__(64)
 state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, float *__restrict__ dstates_m,
-                     const float *__restrict__ gamma, float *__restrict__ carry, int N)
+                     const float *__restrict__ gamma, float *__restrict__ carry, const float *__restrict__ s_in,
+                     const float *__restrict__ ds_out, float *__restrict__ ds_in, int N)
 {
     pdl_wait();
     pdl_launch_dependents();      // only once this kernel's own predecessor has completed
@@ -165,6 +197,12 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
     const float *gm = gamma + (size_t)blockIdx.y * N * 64 + c;
     float *cr = carry + (size_t)blockIdx.y * N * 64 + c;
     float4 r0 = make_float4(0.f, 0.f, 0.f, 0.f), r1 = r0;
+    // this thread's logical columns 4*lp .. 4*lp+3 and 32 + 4*lp .. of row c in a row-major state
+    const size_t io = ((size_t)blockIdx.y * 64 + c) * 64 + 4 * lp;
+    if (s_in != nullptr) {
+        r0 = *reinterpret_cast<const float4 *>(s_in + io);
+        r1 = *reinterpret_cast<const float4 *>(s_in + io + 32);
+    }
     for (int i = 0; i < N; i += kAhead) {
         float4 u0[kAhead], u1[kAhead];
         float g[kAhead];
@@ -185,6 +223,10 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
             }
     }
     float4 d0 = make_float4(0.f, 0.f, 0.f, 0.f), d1 = d0;
+    if (ds_out != nullptr) {
+        d0 = *reinterpret_cast<const float4 *>(ds_out + io);
+        d1 = *reinterpret_cast<const float4 *>(ds_out + io + 32);
+    }
     for (int i = N - 1; i >= 0; i -= kBack) {
         float4 w0[kBack], w1[kBack], s0[kBack], s1[kBack];
         float g[kBack];
@@ -198,8 +240,9 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
                 if (ch + 1 < N) {
                     s0[j] = S[(size_t)(ch + 1) * 1024];
                     s1[j] = S[(size_t)(ch + 1) * 1024 + 512];
-                } else {
-                    s0[j] = s1[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                } else {              // the last chunk leaves the final state, still in registers
+                    s0[j] = r0;
+                    s1[j] = r1;
                 }
             }
         }
@@ -224,41 +267,52 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
             }
         }
     }
+    if (ds_in != nullptr) {
+        *reinterpret_cast<float4 *>(ds_in + io) = d0;
+        *reinterpret_cast<float4 *>(ds_in + io + 32) = d1;
+    }
 }
 
 }  // namespace
 
-dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tiles, bool tf32)
+dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tiles, bool tf32)
 {
     const dim3 grid((g.dk * g.dv / 4 + kScanThreads - 1) / kScanThreads, g.B * g.H);
     if (tiles && (g.dk != 64 || g.dv != 64)) return DIG_ERR_UNSUPPORTED;
+    // the state after the last chunk goes to the caller if asked for, else to the workspace block the
+    // backward scan reads it from (null in a forward-only workspace)
+    float *fin = sio.s_out != nullptr ? sio.s_out : w.sfinal;
     KernelTimer t(KID_SCAN_FWD, s);
     if (tiles)
-        launch_pdl(state_scan_fwd<true>, grid, dim3(kScanThreads), 0, s, w.states, (const float *)w.gamma, g.N, g.dk, g.dv);
+        launch_pdl(state_scan_fwd<true>, grid, dim3(kScanThreads), 0, s, w.states, (const float *)w.gamma, sio.s_in, fin, g.N,
+                   g.dk, g.dv);
     else if (tf32)
-        state_scan_fwd<false, true><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
+        state_scan_fwd<false, true><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, sio.s_in, fin, g.N, g.dk, g.dv);
     else
-        state_scan_fwd<false><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, g.N, g.dk, g.dv);
+        state_scan_fwd<false><<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, sio.s_in, fin, g.N, g.dk, g.dv);
     return cuda_ok(cudaGetLastError());
 }
 
-dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, bool tf32)
+// Needs the final state in w.sfinal (left there by launch_state_scan_fwd on a backward workspace).
+dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tf32)
 {
     const dim3 grid((g.dk + kRowsPerBlock - 1) / kRowsPerBlock, g.B * g.H);
     KernelTimer t(KID_SCAN_BWD, s);
     if (tf32)
-        state_scan_bwd<true><<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N, g.dk, g.dv);
+        state_scan_bwd<true><<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, w.sfinal, sio.ds_out,
+                                                                 sio.ds_in, g.N, g.dk, g.dv);
     else
-        state_scan_bwd<false><<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, g.N, g.dk, g.dv);
+        state_scan_bwd<false><<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, w.carry, w.sfinal, sio.ds_out,
+                                                                  sio.ds_in, g.N, g.dk, g.dv);
     return cuda_ok(cudaGetLastError());
 }
 
-dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s)
+dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio)
 {
     if (g.dk != 64 || g.dv != 64) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_SCAN_BWD, s);
     launch_pdl(state_scan_bwd_tiles, dim3(8, g.B * g.H), dim3(64), 0, s, w.states, w.dstates, w.dstates_m,
-               (const float *)w.gamma, w.carry, g.N);
+               (const float *)w.gamma, w.carry, sio.s_in, sio.ds_out, sio.ds_in, g.N);
     return cuda_ok(cudaGetLastError());
 }
 

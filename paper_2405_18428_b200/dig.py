@@ -23,7 +23,7 @@ DIG_ROW_FWD, DIG_ROW_REV, DIG_COL_FWD, DIG_COL_REV = 0, 1, 2, 3
 DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR, DIG_IMPL_MMA = 0, 1, 2, 3
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
-           "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
+           "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_gla_fwd_state", "dig_gla_bwd_state", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
            "dig_srem_dwconv_bwd_workspace_bytes", "dig_gla_outgate_fwd", "dig_gla_outgate_bwd",
            "dig_gla_outgate_bwd_workspace_bytes", "dig_last_device_status",
            "dig_status_string", "dig_profile_enable", "dig_profile_kernels", "dig_profile_read")
@@ -61,6 +61,10 @@ def lib() -> ctypes.CDLL:
         L.dig_gla_fwd_static.restype = i
         L.dig_gla_bwd.argtypes = [vp] * 9 + [i] * 9 + [vp, sz, vp]
         L.dig_gla_bwd.restype = i
+        L.dig_gla_fwd_state.argtypes = [vp] * 7 + [i] * 9 + [vp, sz, vp]
+        L.dig_gla_fwd_state.restype = i
+        L.dig_gla_bwd_state.argtypes = [vp] * 12 + [i] * 9 + [vp, sz, vp]
+        L.dig_gla_bwd_state.restype = i
         L.dig_srem_dwconv.argtypes = [vp] * 4 + [i] * 6 + [vp]
         L.dig_srem_dwconv.restype = i
         L.dig_srem_dwconv_bwd_workspace_bytes.argtypes = [i] * 4
@@ -320,3 +324,54 @@ def dig_gla_outgate_bwd(o, r, dz, ln_w=None, ln_b=None, eps=1e-5, *, affine_grad
                                      None if dw is None else dw.data_ptr(), None if db is None else db.data_ptr(),
                                      rows, d, float(eps), dtype, wsp, wsn, _stream()), "dig_gla_outgate_bwd")
     return d_o, d_r, dw, db
+
+
+def _state(t, shape, name):
+    return None if t is None else _dev(t, torch.float32, shape, name)
+
+
+def dig_gla_fwd_state(q, k, v, gate, s_in, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD, *, f32_out=False,
+                      want_s_out=True, workspace=None):
+    """dig_gla_fwd started from state s_in ([B, H, d_k, d_v] fp32 or None); returns (out, s_out)."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st = _storage(dtype)
+    out = torch.empty((B, L, H, dv), dtype=_out_storage(dtype), device=q.device)
+    s_out = torch.empty((B, H, dk, dv), dtype=torch.float32, device=q.device) if want_s_out else None
+    need = dig_gla_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 0)
+    workspace = _workspace(workspace, need, q.device)
+    _check(lib().dig_gla_fwd_state(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"), _dev(v, st, (B, L, H, dv), "v"),
+                                   _dev(gate, torch.float32, q.shape, "gate"), _state(s_in, (B, H, dk, dv), "s_in"),
+                                   _dev(out, _out_storage(dtype), (B, L, H, dv), "out"),
+                                   _state(s_out, (B, H, dk, dv), "s_out"),
+                                   B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
+                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "dig_gla_fwd_state")
+    return out, s_out
+
+
+def dig_gla_bwd_state(q, k, v, gate, d_out, s_in, ds_out, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD, *,
+                      f32_out=False, workspace=None):
+    """Returns (dq, dk, dv, dgate, ds_in) for the loss <d_out, out> + <ds_out, s_out>."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st, ost = _storage(dtype), _out_storage(dtype)
+    dq = torch.empty(q.shape, dtype=ost, device=q.device)
+    dk_ = torch.empty(q.shape, dtype=ost, device=q.device)
+    dv_ = torch.empty(v.shape, dtype=ost, device=q.device)
+    dgate = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+    ds_in = torch.empty((B, H, dk, dv), dtype=torch.float32, device=q.device)
+    need = dig_gla_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 1)
+    workspace = _workspace(workspace, need, q.device)
+    _check(lib().dig_gla_bwd_state(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"), _dev(v, st, (B, L, H, dv), "v"),
+                                   _dev(gate, torch.float32, q.shape, "gate"), _dev(d_out, st, v.shape, "d_out"),
+                                   _state(s_in, (B, H, dk, dv), "s_in"), _state(ds_out, (B, H, dk, dv), "ds_out"),
+                                   _dev(dq, ost, q.shape, "dq"), _dev(dk_, ost, q.shape, "dk"),
+                                   _dev(dv_, ost, v.shape, "dv"), _dev(dgate, torch.float32, q.shape, "dgate"),
+                                   _dev(ds_in, torch.float32, (B, H, dk, dv), "ds_in"),
+                                   B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
+                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "dig_gla_bwd_state")
+    return dq, dk_, dv_, dgate, ds_in
