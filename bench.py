@@ -338,6 +338,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="C2")
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--grid", type=int, nargs=2, default=None, metavar=("H", "W"),
+                    help="patch grid to use instead of the workload's (a reduced copy of a workload, e.g. for a profiler capture)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--family", default="auto", choices=["auto", "fma", "tensor", "mma"])
     ap.add_argument("--eager", action="store_true", help="time plain stream launches instead of one CUDA graph per step")
@@ -349,6 +351,8 @@ def main():
     wl = CONFIGS[args.workload]
     if args.chunk:
         wl = wl.scaled(chunk=args.chunk)
+    if args.grid:
+        wl = wl.scaled(name=f"{wl.name}@{args.grid[0]}x{args.grid[1]}", grid_h=args.grid[0], grid_w=args.grid[1])
     if not wl.backward:
         wl = wl.scaled(backward=False)
     if args.impl == "reference":

@@ -26,6 +26,9 @@ __host__ __device__ constexpr int pad16(int d) { return (d + 15) & ~15; }
 // Row pitch (floats) of a tile whose rows hold `d` values: a multiple of 4 whose quarter is odd, so the
 // 8 rows x 4 columns a fragment load touches fall into 32 different banks.
 __host__ __device__ constexpr int pitch(int d) { return pad16(d) + 4; }
+// The same for tiles whose padding columns are never read (every kernel but the state kernel, where d_k
+// is an output extent and has to be a multiple of 16): d is a multiple of 8, so d / 4 + 1 is odd too.
+__host__ __device__ constexpr int tight(int d) { return d + 4; }
 
 // Sizes of a launch, either compile-time constants (the frequent shapes: strides fold into the
 // instructions, loops unroll, divisions become shifts) or read from the geometry (everything else).
@@ -164,10 +167,10 @@ __device__ __forceinline__ void cp_async_wait_all()
 {
     asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
-__device__ __forceinline__ void load_rows(float *dst, int ld, const __nv_bfloat16 *src, const int *sRow, int C, int d)
+__device__ __forceinline__ void load_rows(float *dst, int ld, const __nv_bfloat16 *src, const int *sRow, int C, int d, int dp)
 {
     constexpr int U = 4;
-    const int per_row = pad16(d) >> 2, n = C * per_row;
+    const int per_row = dp >> 2, n = C * per_row;      // dp: columns to fill (d, or d padded to 16)
     for (int base = threadIdx.x; base < n; base += U * kThreads) {
         uint2 raw[U];
 #pragma unroll
@@ -192,9 +195,9 @@ __device__ __forceinline__ void load_rows(float *dst, int ld, const __nv_bfloat1
         }
     }
 }
-__device__ __forceinline__ void load_gates(float *dst, int ld, const float *gate, const int *sRow, int C, int dk)
+__device__ __forceinline__ void load_gates(float *dst, int ld, const float *gate, const int *sRow, int C, int dk, int dp)
 {
-    const int per_row = pad16(dk) >> 2;
+    const int per_row = dp >> 2;
     for (int idx = threadIdx.x; idx < C * per_row; idx += kThreads) {
         const int j = idx / per_row, c = (idx - j * per_row) << 2;
         const int row = sRow[j];
@@ -202,11 +205,11 @@ __device__ __forceinline__ void load_gates(float *dst, int ld, const float *gate
         else *reinterpret_cast<float4 *>(dst + j * ld + c) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
-// A [dk][dv] state of the workspace (rounded to tf32 by the scan kernels) -> [pad16(dk)][ld] tile, padding zero.
+// A [dk][dv] state of the workspace (rounded to tf32 by the scan kernels) -> [dk][ld] tile.
 __device__ __forceinline__ void load_state(float *dst, int ld, const float *src, int dk, int dv)
 {
-    const int per_row = pad16(dv) >> 2;
-    for (int idx = threadIdx.x; idx < pad16(dk) * per_row; idx += kThreads) {
+    const int per_row = dv >> 2;
+    for (int idx = threadIdx.x; idx < dk * per_row; idx += kThreads) {
         const int r = idx / per_row, c = (idx - r * per_row) << 2;
         if (r < dk && c < dv) cp_async16(dst + r * ld + c, src + r * dv + c);
         else *reinterpret_cast<float4 *>(dst + r * ld + c) = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -242,9 +245,9 @@ __device__ __forceinline__ void prefix_gates(float *lam, int ld, int C, int dkp,
 }
 // In place: sQ (raw q) -> Qt = q*exp(Lam), sK (raw k) -> Kt = k*exp(-Lam), or with sLast given
 // -> Kh = k*exp(Lam_{C-1}-Lam); rounded to tf32.  Either tile may be null.
-__device__ __forceinline__ void scale_qk(float *sQ, float *sK, const float *sLam, const float *sLast, int ldk, int C, int dk)
+__device__ __forceinline__ void scale_qk(float *sQ, float *sK, const float *sLam, const float *sLast, int ldk, int C, int dp)
 {
-    const int per_row = pad16(dk) >> 2;
+    const int per_row = dp >> 2;
     for (int idx = threadIdx.x; idx < C * per_row; idx += kThreads) {
         const int j = idx / per_row, c = (idx - j * per_row) << 2;
         const float4 lam = *reinterpret_cast<const float4 *>(sLam + j * ldk + c);
@@ -311,19 +314,19 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
 
     fill_rows(sRow, g, C, b, h, chunk);
     __syncthreads();
-    load_gates(sLam, ldk, gate, sRow, C, dk);
-    load_rows(sX, ldk, k, sRow, C, dk);
-    load_rows(sV, ldv, v, sRow, C, dv);
+    load_gates(sLam, ldk, gate, sRow, C, dk, dkp);
+    load_rows(sX, ldk, k, sRow, C, dk, dkp);
+    load_rows(sV, ldv, v, sRow, C, dv, dvp);
     if (BWD) {
-        load_rows(sQ, ldk, q, sRow, C, dk);
-        load_rows(sG, ldv, d_out, sRow, C, dv);
+        load_rows(sQ, ldk, q, sRow, C, dk, dkp);
+        load_rows(sG, ldv, d_out, sRow, C, dv, dvp);
     }
     cp_async_wait_all();
     __syncthreads();
     prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
     const size_t chunk_id = (size_t)bh * g.N + chunk;
     for (int c = threadIdx.x; c < dk; c += kThreads) gamma[chunk_id * dk + c] = __expf(sLast[c]);
-    scale_qk(BWD ? sQ : nullptr, sX, sLam, sLast, ldk, C, dk);
+    scale_qk(BWD ? sQ : nullptr, sX, sLam, sLast, ldk, C, dkp);
     __syncthreads();
     constexpr int NB = frag_bound(pad16(DM::kDK), DM::kDV);
     const Tiling tl(dkp, dv);
@@ -363,7 +366,7 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     const DM dm(g);
     const int C = dm.C(), dk = dm.dk(), dv = dm.dv();
     const int chunk = blockIdx.x, bh = blockIdx.y, b = bh / g.H, h = bh - b * g.H;
-    const int dkp = pad16(dk), dvp = pad16(dv), ldk = pitch(dk), ldv = pitch(dv), ldp = pitch(C);
+    const int dkp = dk, ldk = tight(dk), ldv = tight(dv), ldp = tight(C);      // no padding columns here
     float *sLam = smem;
     float *sQ = sLam + C * ldk;
     float *sK = sQ + C * ldk;
@@ -375,11 +378,11 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
 
     fill_rows(sRow, g, C, b, h, chunk);
     __syncthreads();
-    load_gates(sLam, ldk, gate, sRow, C, dk);
+    load_gates(sLam, ldk, gate, sRow, C, dk, dk);
     load_state(sS, ldv, states + ((size_t)bh * g.N + chunk) * dk * dv, dk, dv);
-    load_rows(sV, ldv, v, sRow, C, dv);
-    load_rows(sQ, ldk, q, sRow, C, dk);
-    load_rows(sK, ldk, k, sRow, C, dk);
+    load_rows(sV, ldv, v, sRow, C, dv, dv);
+    load_rows(sQ, ldk, q, sRow, C, dk, dk);
+    load_rows(sK, ldk, k, sRow, C, dk, dk);
     cp_async_wait_all();
     __syncthreads();
     prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
@@ -424,7 +427,7 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     const DM dm(g);
     const int C = dm.C(), dk = dm.dk(), dv = dm.dv();
     const int chunk = blockIdx.x, bh = blockIdx.y, b = bh / g.H, h = bh - b * g.H;
-    const int dkp = pad16(dk), dvp = pad16(dv), ldk = pitch(dk), ldv = pitch(dv), ldp = pitch(C);
+    const int dkp = dk, ldk = tight(dk), ldv = tight(dv), ldp = tight(C);      // no padding columns here
     float *sLam = smem;                     // Lam, later x = q*dq - k*dk
     float *sQ = sLam + C * ldk;
     float *sK = sQ + C * ldk;
@@ -440,13 +443,13 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
 
     fill_rows(sRow, g, C, b, h, chunk);
     __syncthreads();
-    load_gates(sLam, ldk, gate, sRow, C, dk);
+    load_gates(sLam, ldk, gate, sRow, C, dk, dk);
     load_state(sS, ldv, states + chunk_id * dk * dv, dk, dv);
     load_state(sD, ldv, dstates + chunk_id * dk * dv, dk, dv);
-    load_rows(sV, ldv, v, sRow, C, dv);
-    load_rows(sG, ldv, d_out, sRow, C, dv);
-    load_rows(sQ, ldk, q, sRow, C, dk);
-    load_rows(sK, ldk, k, sRow, C, dk);
+    load_rows(sV, ldv, v, sRow, C, dv, dv);
+    load_rows(sG, ldv, d_out, sRow, C, dv, dv);
+    load_rows(sQ, ldk, q, sRow, C, dk, dk);
+    load_rows(sK, ldk, k, sRow, C, dk, dk);
     cp_async_wait_all();
     __syncthreads();
     prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
@@ -562,14 +565,14 @@ size_t smem_state(const Geom &g, bool bwd)
 }
 size_t smem_out(const Geom &g)
 {
-    size_t n = (size_t)g.C * (3 * pitch(g.dk) + pitch(g.dv)) + (size_t)pad16(g.dk) * pitch(g.dv) + 5 * pad16(g.dk);
-    if (g.C > g.dk) n += (size_t)g.C * pitch(g.C);
+    size_t n = (size_t)g.C * (3 * tight(g.dk) + tight(g.dv)) + (size_t)g.dk * tight(g.dv) + 5 * g.dk;
+    if (g.C > g.dk) n += (size_t)g.C * tight(g.C);
     return sizeof(float) * n;
 }
 size_t smem_bwd(const Geom &g)
 {
-    return sizeof(float) * ((size_t)g.C * (3 * pitch(g.dk) + 2 * pitch(g.dv) + 2 * pitch(g.C)) +
-                            2 * (size_t)pad16(g.dk) * pitch(g.dv) + 5 * pad16(g.dk));
+    return sizeof(float) * ((size_t)g.C * (3 * tight(g.dk) + 2 * tight(g.dv) + 2 * tight(g.C)) +
+                            2 * (size_t)g.dk * tight(g.dv) + 5 * g.dk);
 }
 constexpr size_t kMaxSmem = 227 * 1024 - 1024;      // the row table is static shared memory
 
