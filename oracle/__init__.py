@@ -50,6 +50,8 @@ def _load():
             lib.dig_oracle_gla_bwd.argtypes = [dp] * 9 + [ctypes.c_int] * 8
             lib.dig_oracle_gla_fwd_state.argtypes = [dp] * 7 + [ctypes.c_int] * 8
             lib.dig_oracle_gla_bwd_state.argtypes = [dp] * 12 + [ctypes.c_int] * 8
+            lib.dig_oracle_gla_fwd_beta.argtypes = [dp] * 6 + [ctypes.c_int] * 8
+            lib.dig_oracle_gla_bwd_beta.argtypes = [dp] * 11 + [ctypes.c_int] * 8
             lib.dig_oracle_dwconv.argtypes = [dp] * 4 + [ctypes.c_int] * 5
             lib.dig_oracle_dwconv_bwd.argtypes = [dp] * 6 + [ctypes.c_int] * 5
             lib.dig_oracle_outgate_fwd.argtypes = [dp] * 5 + [ctypes.c_longlong, ctypes.c_int, ctypes.c_double]
@@ -218,3 +220,30 @@ def gla_bwd_state(q, k, v, a, dout, s_in, ds_out, grid_h, grid_w, direction=ROW_
                                             _p(dv), _p(da), _p(ds_in), B, H, grid_h, grid_w, dk, dv_, direction,
                                             threads), "gla_bwd_state")
     return dq, dk_, dv, da, ds_in
+
+
+def gla_fwd_beta(q, k, v, a, bg, grid_h, grid_w, direction=ROW_FWD, threads=1) -> np.ndarray:
+    """gla_fwd with the full gate of Eq. gate_gla: S_t = diag(e^a_t) S_{t-1} diag(e^bg_t) + k_t^T v_t.
+    bg = log(beta), [B, L, H, d_v]."""
+    q, k, v, a, bg = map(_f64, (q, k, v, a, bg))
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    assert L == grid_h * grid_w and k.shape == q.shape == a.shape and v.shape == (B, L, H, dv) == bg.shape
+    out = np.empty_like(v)
+    _check(_load().dig_oracle_gla_fwd_beta(_p(q), _p(k), _p(v), _p(a), _p(bg), _p(out), B, H, grid_h, grid_w,
+                                           dk, dv, direction, threads), "gla_fwd_beta")
+    return out
+
+
+def gla_bwd_beta(q, k, v, a, bg, dout, grid_h, grid_w, direction=ROW_FWD, threads=1):
+    """Gradients (dq, dk, dv, da, dbg) of <dout, gla_fwd_beta(q, k, v, a, bg)>."""
+    q, k, v, a, bg, dout = map(_f64, (q, k, v, a, bg, dout))
+    B, L, H, dk = q.shape
+    dv_ = v.shape[-1]
+    assert L == grid_h * grid_w and dout.shape == v.shape == bg.shape
+    dq, dk_, da = np.empty_like(q), np.empty_like(q), np.empty_like(q)
+    dv, db = np.empty_like(v), np.empty_like(v)
+    _check(_load().dig_oracle_gla_bwd_beta(_p(q), _p(k), _p(v), _p(a), _p(bg), _p(dout), _p(dq), _p(dk_), _p(dv),
+                                           _p(da), _p(db), B, H, grid_h, grid_w, dk, dv_, direction, threads),
+           "gla_bwd_beta")
+    return dq, dk_, dv, da, db

@@ -18,6 +18,8 @@
  *   - the recurrence started from a given state and returning the final state (the paper starts
  *     from zero and drops it; this is what splitting a sequence into pieces needs), with the
  *     matching terms of the derivative
+ *   - the recurrence with the full gate G_t = alpha_t^T beta_t of Eq. gate_gla (value-channel decay
+ *     beta as well), and its derivative
  *   - the output gate z = Swish(r) (.) LN(o) that follows the recurrence (Eq. attn_gla, the line
  *     forming Y_t before the projection W_O), and its reverse-mode derivative
  *
@@ -36,7 +38,10 @@
  * the normalisation, Swish's values at 0 and far from 0, central finite differences of the
  * derivative, and do summing to zero over a row when the affine part is absent; for the state
  * arguments: a sequence cut in two and chained through the state equals the uncut one (values and
- * all gradients), the final state of a constant-decay sequence in closed form, finite differences.
+ * all gradients), the final state of a constant-decay sequence in closed form, finite differences;
+ * for the value-channel gate: beta == 1 gives the alpha-only recurrence back, the parallel form
+ * o_t = sum_{s<=t} (q_t e^{Lam_t} . k_s e^{-Lam_s}) v_s e^{M_t - M_s} written out in numpy, finite
+ * differences, and the suffix-sum identity d(log beta)_t = sum_{s>=t} (o_s do_s - v_s dv_s).
  * Not pinned by the paper: whether DWConv2d carries a bias (the argument is optional).
  */
 #include <math.h>
@@ -97,7 +102,7 @@ static size_t tok_off(long long b, long long t, int h, long long L, int H, int d
 /* Forward recurrence (Eq. attn_gla), one (b,h) pair at a time, in scan order.
  * s_in (may be NULL = zero, the paper's case): state before the first scan position, [B][H][d_k][d_v];
  * s_out (may be NULL): receives the state after the last scan position, same layout. */
-static int gla_fwd_impl(const double *q, const double *k, const double *v, const double *a,
+static int gla_fwd_impl(const double *q, const double *k, const double *v, const double *a, const double *bg,
                         double *out, const double *s_in, double *s_out, int B, int H, int grid_h, int grid_w,
                         int d_k, int d_v, int direction, int threads)
 {
@@ -122,10 +127,13 @@ static int gla_fwd_impl(const double *q, const double *k, const double *v, const
             const double *at = a + tok_off(b, t, h, L, H, d_k);
             const double *vt = v + tok_off(b, t, h, L, H, d_v);
             double *ot = out + tok_off(b, t, h, L, H, d_v);
+            const double *bt = bg ? bg + tok_off(b, t, h, L, H, d_v) : NULL;
             for (int c = 0; c < d_k; ++c) {
                 const double al = exp(at[c]);
-                for (int e = 0; e < d_v; ++e)           /* S'_{t-1} = G_t . S_{t-1}; S_t = S' + k^T v */
-                    S[(size_t)c * d_v + e] = al * S[(size_t)c * d_v + e] + kt[c] * vt[e];
+                for (int e = 0; e < d_v; ++e) {         /* S'_{t-1} = G_t . S_{t-1}, G_t = alpha_t^T beta_t; S_t = S' + k^T v */
+                    const double be = bt ? exp(bt[e]) : 1.0;
+                    S[(size_t)c * d_v + e] = al * be * S[(size_t)c * d_v + e] + kt[c] * vt[e];
+                }
             }
             for (int e = 0; e < d_v; ++e) {             /* o_t = q_t S_t */
                 double acc = 0.0;
@@ -144,7 +152,7 @@ int dig_oracle_gla_fwd(const double *q, const double *k, const double *v, const 
                        double *out, int B, int H, int grid_h, int grid_w, int d_k, int d_v,
                        int direction, int threads)
 {
-    return gla_fwd_impl(q, k, v, a, out, NULL, NULL, B, H, grid_h, grid_w, d_k, d_v, direction, threads);
+    return gla_fwd_impl(q, k, v, a, NULL, out, NULL, NULL, B, H, grid_h, grid_w, d_k, d_v, direction, threads);
 }
 
 /* The same recurrence started from a given state and returning the final one: what a caller needs to
@@ -153,7 +161,7 @@ int dig_oracle_gla_fwd_state(const double *q, const double *k, const double *v, 
                              const double *s_in, double *out, double *s_out, int B, int H, int grid_h,
                              int grid_w, int d_k, int d_v, int direction, int threads)
 {
-    return gla_fwd_impl(q, k, v, a, out, s_in, s_out, B, H, grid_h, grid_w, d_k, d_v, direction, threads);
+    return gla_fwd_impl(q, k, v, a, NULL, out, s_in, s_out, B, H, grid_h, grid_w, d_k, d_v, direction, threads);
 }
 
 /* Reverse-mode derivative of the recurrence above.
@@ -165,10 +173,10 @@ int dig_oracle_gla_fwd_state(const double *q, const double *k, const double *v, 
  * With a start state s_in (NULL = zero) the forward sweep starts from it; ds_out (NULL = zero) is the
  * gradient with respect to the final state and seeds dS; ds_in (may be NULL) receives the gradient
  * with respect to s_in, which is dS after the first position has handed it on. */
-static int gla_bwd_impl(const double *q, const double *k, const double *v, const double *a,
+static int gla_bwd_impl(const double *q, const double *k, const double *v, const double *a, const double *bg,
                         const double *dout, const double *s_in, const double *ds_out, double *dq, double *dk,
-                        double *dv, double *da, double *ds_in, int B, int H, int grid_h, int grid_w, int d_k,
-                        int d_v, int direction, int threads)
+                        double *dv, double *da, double *db, double *ds_in, int B, int H, int grid_h, int grid_w,
+                        int d_k, int d_v, int direction, int threads)
 {
     enum { SEG = 64 };
     const long long L = (long long)grid_h * grid_w;
@@ -199,10 +207,11 @@ static int gla_bwd_impl(const double *q, const double *k, const double *v, const
                 const double *kt = k + tok_off(b, t, h, L, H, d_k);
                 const double *at = a + tok_off(b, t, h, L, H, d_k);
                 const double *vt = v + tok_off(b, t, h, L, H, d_v);
+                const double *bt = bg ? bg + tok_off(b, t, h, L, H, d_v) : NULL;
                 for (int c = 0; c < d_k; ++c) {
                     const double al = exp(at[c]);
                     for (int e = 0; e < d_v; ++e)
-                        S[(size_t)c * d_v + e] = al * S[(size_t)c * d_v + e] + kt[c] * vt[e];
+                        S[(size_t)c * d_v + e] = al * (bt ? exp(bt[e]) : 1.0) * S[(size_t)c * d_v + e] + kt[c] * vt[e];
                 }
             }
             free(S);
@@ -218,10 +227,11 @@ static int gla_bwd_impl(const double *q, const double *k, const double *v, const
                 const double *vt = v + tok_off(b, t, h, L, H, d_v);
                 const double *Sp = seg + SZ * (size_t)j;
                 double *Sn = seg + SZ * (size_t)(j + 1);
+                const double *bt = bg ? bg + tok_off(b, t, h, L, H, d_v) : NULL;
                 for (int c = 0; c < d_k; ++c) {
                     const double al = exp(at[c]);
                     for (int e = 0; e < d_v; ++e)
-                        Sn[(size_t)c * d_v + e] = al * Sp[(size_t)c * d_v + e] + kt[c] * vt[e];
+                        Sn[(size_t)c * d_v + e] = al * (bt ? exp(bt[e]) : 1.0) * Sp[(size_t)c * d_v + e] + kt[c] * vt[e];
                 }
             }
             for (long long j = n - 1; j >= 0; --j) {
@@ -239,21 +249,27 @@ static int gla_bwd_impl(const double *q, const double *k, const double *v, const
                 const double *Scur = seg + SZ * (size_t)(j + 1);    /* S_t     */
                 for (int c = 0; c < d_k; ++c)
                     for (int e = 0; e < d_v; ++e) dS[(size_t)c * d_v + e] += qt[c] * dot[e];
+                const double *bt = bg ? bg + tok_off(b, t, h, L, H, d_v) : NULL;
+                double *dbt = db ? db + tok_off(b, t, h, L, H, d_v) : NULL;
                 for (int e = 0; e < d_v; ++e) dvt[e] = 0.0;
+                if (dbt) for (int e = 0; e < d_v; ++e) dbt[e] = 0.0;
                 for (int c = 0; c < d_k; ++c) {
                     const double al = exp(at[c]);
                     double sq = 0.0, sk = 0.0, sa = 0.0;
                     for (int e = 0; e < d_v; ++e) {
                         const double g = dS[(size_t)c * d_v + e];
+                        const double be = bt ? exp(bt[e]) : 1.0;
                         sq += Scur[(size_t)c * d_v + e] * dot[e];
                         sk += g * vt[e];
-                        sa += g * Sprev[(size_t)c * d_v + e];
+                        sa += g * be * Sprev[(size_t)c * d_v + e];            /* d/d(log alpha) of alpha*beta*S_{t-1} */
+                        if (dbt) dbt[e] += g * al * be * Sprev[(size_t)c * d_v + e];   /* d/d(log beta) of the same */
                         dvt[e] += kt[c] * g;
                     }
                     dqt[c] = sq;
                     dkt[c] = sk;
                     dat[c] = al * sa;
-                    for (int e = 0; e < d_v; ++e) dS[(size_t)c * d_v + e] *= al;   /* hand dS to step t-1 */
+                    for (int e = 0; e < d_v; ++e)                                       /* hand dS to step t-1 */
+                        dS[(size_t)c * d_v + e] *= al * (bt ? exp(bt[e]) : 1.0);
                 }
             }
         }
@@ -269,7 +285,7 @@ int dig_oracle_gla_bwd(const double *q, const double *k, const double *v, const 
                        int B, int H, int grid_h, int grid_w, int d_k, int d_v,
                        int direction, int threads)
 {
-    return gla_bwd_impl(q, k, v, a, dout, NULL, NULL, dq, dk, dv, da, NULL, B, H, grid_h, grid_w, d_k, d_v,
+    return gla_bwd_impl(q, k, v, a, NULL, dout, NULL, NULL, dq, dk, dv, da, NULL, NULL, B, H, grid_h, grid_w, d_k, d_v,
                         direction, threads);
 }
 
@@ -278,7 +294,24 @@ int dig_oracle_gla_bwd_state(const double *q, const double *k, const double *v, 
                              double *dk, double *dv, double *da, double *ds_in, int B, int H, int grid_h,
                              int grid_w, int d_k, int d_v, int direction, int threads)
 {
-    return gla_bwd_impl(q, k, v, a, dout, s_in, ds_out, dq, dk, dv, da, ds_in, B, H, grid_h, grid_w, d_k, d_v,
+    return gla_bwd_impl(q, k, v, a, NULL, dout, s_in, ds_out, dq, dk, dv, da, NULL, ds_in, B, H, grid_h, grid_w, d_k, d_v,
+                        direction, threads);
+}
+
+/* The paper's full gate G_t = alpha_t^T beta_t (Eq. gate_gla): the state decays along the key channels
+ * by alpha and along the value channels by beta.  bg = log(beta) <= 0, [B][L][H][d_v]. */
+int dig_oracle_gla_fwd_beta(const double *q, const double *k, const double *v, const double *a, const double *bg,
+                            double *out, int B, int H, int grid_h, int grid_w, int d_k, int d_v, int direction,
+                            int threads)
+{
+    return gla_fwd_impl(q, k, v, a, bg, out, NULL, NULL, B, H, grid_h, grid_w, d_k, d_v, direction, threads);
+}
+
+int dig_oracle_gla_bwd_beta(const double *q, const double *k, const double *v, const double *a, const double *bg,
+                            const double *dout, double *dq, double *dk, double *dv, double *da, double *db, int B,
+                            int H, int grid_h, int grid_w, int d_k, int d_v, int direction, int threads)
+{
+    return gla_bwd_impl(q, k, v, a, bg, dout, NULL, NULL, dq, dk, dv, da, db, NULL, B, H, grid_h, grid_w, d_k, d_v,
                         direction, threads);
 }
 
