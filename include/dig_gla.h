@@ -193,6 +193,25 @@ dig_status dig_gla_bwd_state(const void *q, const void *k, const void *v, const 
                              float *ds_in, int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
                              int direction, int dtype, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Gated linear attention with the paper's full gate G_t = alpha_t^T beta_t (Eq. gate_gla): the state
+ * also decays along the value channels,
+ *   S_t = diag(exp(gate_t)) S_{t-1} diag(exp(bgate_t)) + k_t^T v_t,   out_t = q_t S_t,
+ * bgate = log(beta) <= 0, fp32 [B][L][H][d_v]; everything else as in dig_gla_fwd / dig_gla_bwd.
+ * dig_gla_bwd_beta returns dbgate (fp32 [B][L][H][d_v]) beside the other gradients.
+ * Served by the warp-level tensor-core kernels only: bf16 storage (DIG_F32 returns DIG_ERR_UNSUPPORTED),
+ * any supported head and chunk size that fits shared memory.  The workspace is larger than that of
+ * dig_gla_fwd / dig_gla_bwd: dig_gla_beta_workspace_bytes (0 for invalid or unsupported sizes).  The same
+ * bound of 80 on the magnitude of a gate summed over one chunk applies to bgate. */
+size_t dig_gla_beta_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int dtype,
+                                    int backward);
+dig_status dig_gla_fwd_beta(const void *q, const void *k, const void *v, const float *gate, const float *bgate, void *out,
+                            int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+dig_status dig_gla_bwd_beta(const void *q, const void *k, const void *v, const float *gate, const float *bgate,
+                            const void *d_out, void *dq, void *dk, void *dv, float *dgate, float *dbgate,
+                            int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the status recorded by device code on the
  * current device: DIG_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last query,
  * DIG_ERR_CUDA if the synchronisation itself failed, DIG_OK otherwise. */

@@ -302,6 +302,59 @@ dig_status dig_gla_outgate_bwd(const void *o, const void *r, const float *ln_w, 
                               reinterpret_cast<float *>(workspace), (cudaStream_t)cuda_stream);
 }
 
+size_t dig_gla_beta_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int dtype,
+                                    int backward)
+{
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, 0, dtype)) return 0;
+    if (!mma_supports(d_k, d_v, chunk, dtype, backward != 0, true)) return 0;
+    return mma_beta_workspace_bytes(make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, 0), backward != 0);
+}
+
+dig_status dig_gla_fwd_beta(const void *q, const void *k, const void *v, const float *gate, const float *bgate, void *out,
+                            int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!q || !k || !v || !gate || !bgate || !out) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(bgate) || !aligned16(out))
+        return DIG_ERR_INVALID_ARG;
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, direction, dtype)) return DIG_ERR_INVALID_ARG;
+    if (!mma_supports(d_k, d_v, chunk, dtype, false, true)) return DIG_ERR_UNSUPPORTED;
+    const size_t need = dig_gla_beta_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, 0);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    GlaArgs a{};
+    a.bio.bgate = bgate;
+    a.q = q; a.k = k; a.v = v; a.gate = gate; a.out = out;
+    a.ws = reinterpret_cast<float *>(workspace);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, direction);
+    a.dtype = dtype;
+    a.stream = (cudaStream_t)cuda_stream;
+    return mma_gla_fwd(a);
+}
+
+dig_status dig_gla_bwd_beta(const void *q, const void *k, const void *v, const float *gate, const float *bgate,
+                            const void *d_out, void *dq, void *dk, void *dv, float *dgate, float *dbgate,
+                            int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!q || !k || !v || !gate || !bgate || !d_out || !dq || !dk || !dv || !dgate || !dbgate) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(bgate) ||
+        !aligned16(d_out) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(dgate) || !aligned16(dbgate))
+        return DIG_ERR_INVALID_ARG;
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, direction, dtype)) return DIG_ERR_INVALID_ARG;
+    if (!mma_supports(d_k, d_v, chunk, dtype, true, true)) return DIG_ERR_UNSUPPORTED;
+    const size_t need = dig_gla_beta_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, 1);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    GlaArgs a{};
+    a.bio.bgate = bgate; a.bio.dbgate = dbgate;
+    a.q = q; a.k = k; a.v = v; a.gate = gate; a.d_out = d_out;
+    a.dq = dq; a.dk = dk; a.dv = dv; a.dgate = dgate;
+    a.ws = reinterpret_cast<float *>(workspace);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, direction);
+    a.dtype = dtype;
+    a.stream = (cudaStream_t)cuda_stream;
+    return mma_gla_bwd(a);
+}
+
 dig_status dig_last_device_status(void *cuda_stream)
 {
     if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return DIG_ERR_CUDA;

@@ -75,8 +75,16 @@ struct StateIO {
     float *ds_in;
 };
 
+// Arguments of the variant with the value-channel gate (all null otherwise): log(beta) [B][L][H][d_v]
+// and the gradient with respect to it.
+struct BetaIO {
+    const float *bgate;
+    float *dbgate;
+};
+
 struct GlaArgs {
     StateIO sio;
+    BetaIO bio;
     const void *q, *k, *v;
     const float *gate;
     void *out;                   // forward
@@ -128,7 +136,8 @@ dig_status fma_gla_bwd(const GlaArgs &a);
 bool fma_supports(int dk, int dv, int chunk, int dtype, bool backward);
 dig_status mma_gla_fwd(const GlaArgs &a);
 dig_status mma_gla_bwd(const GlaArgs &a);
-bool mma_supports(int dk, int dv, int chunk, int dtype, bool backward);
+bool mma_supports(int dk, int dv, int chunk, int dtype, bool backward, bool beta = false);
+size_t mma_beta_workspace_bytes(const Geom &g, bool backward);
 dig_status tensor_gla_fwd(const GlaArgs &a);
 dig_status tensor_gla_bwd(const GlaArgs &a);
 bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward);
@@ -140,6 +149,10 @@ dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t
 dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tf32 = false);
 // Tensor-core backward pass: forward and reverse scan in one launch over states kept in tile order.
 dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio);
+// Scans with the value-channel gate (row-major states, tf32-rounded results) and the cross-chunk part of its gradient.
+dig_status launch_state_scan_fwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s);
+dig_status launch_state_scan_bwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s);
+dig_status launch_beta_carry(float *dbgate, float *xtot, const Geom &g, cudaStream_t s);
 
 // Device status word (bounded waits report here).
 int *device_status_ptr();

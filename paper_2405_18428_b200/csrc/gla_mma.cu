@@ -49,6 +49,14 @@ struct AnyDims {
     __device__ int dv() const { return dv_; }
 };
 
+// Device-side arguments of the value-channel gate (unused by the kernels instantiated without it).
+struct BetaDev {
+    const float *bgate;     // log(beta) [B][L][H][d_v]
+    float *gamma_v;         // [B*H][N][d_v]  exp of the chunk totals of bgate
+    float *dbgate;          // gradient with respect to bgate (backward pass)
+    float *xtot;            // [B*H][N][d_v]  chunk totals of o*do - v*dv (backward pass)
+};
+
 __device__ __forceinline__ float tf32r(float x)
 {
     uint32_t u;
@@ -139,6 +147,8 @@ struct Tiling {
     }
 };
 
+__device__ __forceinline__ float2 load2(const float *p) { return *reinterpret_cast<const float2 *>(p); }
+__device__ __forceinline__ float2 load2(const __nv_bfloat16 *p) { return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(p)); }
 __device__ __forceinline__ void store2(float *p, float a, float b) { *reinterpret_cast<float2 *>(p) = make_float2(a, b); }
 __device__ __forceinline__ void store2(__nv_bfloat16 *p, float a, float b)
 {
@@ -291,12 +301,14 @@ __device__ __forceinline__ void masked_scores(float *sP, int ldp, const float *A
 
 // ---- kernel 1: chunk-local state contributions ------------------------------------------------------
 // U = Kh^T V (and, for the backward pass, W = Qt^T dO); gamma = exp(Lam_{C-1}).
-template <bool BWD, typename DM>
+// BETA: with the value-channel gate the value side mirrors the key side: M = prefix sums of log(beta),
+// gamma_v = exp(M_{C-1}), U = Kh^T Vh with Vh = v*exp(M_{C-1}-M), W = Qt^T G with G = dO*exp(M).
+template <bool BWD, typename DM, bool BETA>
 __global__ void __launch_bounds__(kThreads)
 mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                 const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate,
                 const __nv_bfloat16 *__restrict__ d_out, float *__restrict__ states, float *__restrict__ gamma,
-                float *__restrict__ dstates, Geom g)
+                float *__restrict__ dstates, BetaDev bd, Geom g)
 {
     extern __shared__ __align__(16) float smem[];
     __shared__ int sRow[128];
@@ -311,9 +323,13 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
     float *sSeg = sLast + dkp;              // [4][dkp]
     float *sQ = sSeg + 4 * dkp;             // BWD: q -> Qt
     float *sG = sQ + (BWD ? C * ldk : 0);   // BWD: dO
+    float *sM = sG + (BWD ? C * ldv : 0);   // BETA: log(beta) -> M
+    float *sMlast = sM + C * ldv;           // [dvp]
+    float *sSegV = sMlast + dvp;            // [4][dvp]
 
     fill_rows(sRow, g, C, b, h, chunk);
     __syncthreads();
+    if (BETA) load_gates(sM, ldv, bd.bgate, sRow, C, dv, dvp);
     load_gates(sLam, ldk, gate, sRow, C, dk, dkp);
     load_rows(sX, ldk, k, sRow, C, dk, dkp);
     load_rows(sV, ldv, v, sRow, C, dv, dvp);
@@ -324,9 +340,14 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
     cp_async_wait_all();
     __syncthreads();
     prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
+    if (BETA) prefix_gates(sM, ldv, C, dvp, sMlast, sSegV);
     const size_t chunk_id = (size_t)bh * g.N + chunk;
     for (int c = threadIdx.x; c < dk; c += kThreads) gamma[chunk_id * dk + c] = __expf(sLast[c]);
     scale_qk(BWD ? sQ : nullptr, sX, sLam, sLast, ldk, C, dkp);
+    if (BETA) {
+        for (int e = threadIdx.x; e < dv; e += kThreads) bd.gamma_v[chunk_id * dv + e] = __expf(sMlast[e]);
+        scale_qk(BWD ? sG : nullptr, sV, sM, sMlast, ldv, C, dvp);      // G = dO*exp(M), Vh = v*exp(M_{C-1}-M)
+    }
     __syncthreads();
     constexpr int NB = frag_bound(pad16(DM::kDK), DM::kDV);
     const Tiling tl(dkp, dv);
@@ -355,11 +376,12 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
 
 // ---- kernel 3: outputs ------------------------------------------------------------------------------
 // out = tril(Qt Kt^T) V + Qt S
-template <typename TO, typename DM>
+// BETA: out = exp(M) * (tril(Qt Kt^T) Vt + Qt S) with Vt = v*exp(-M).
+template <typename TO, typename DM, bool BETA>
 __global__ void __launch_bounds__(kThreads)
 mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
               const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate, const float *__restrict__ states,
-              TO *__restrict__ out, Geom g)
+              TO *__restrict__ out, BetaDev bd, Geom g)
 {
     extern __shared__ __align__(16) float smem[];
     __shared__ int sRow[128];
@@ -375,9 +397,13 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     float *sLast = sS + dkp * ldv;          // [dkp]
     float *sSeg = sLast + dkp;              // [4][dkp]
     float *sP = (C <= dk) ? sLam : sSeg + 4 * dkp;       // the scores reuse the gate tile when they fit
+    float *sM = sSeg + 4 * dkp + (C <= dk ? 0 : C * ldp);   // BETA: log(beta) -> M
+    float *sMlast = sM + C * ldv;           // [dv]
+    float *sSegV = sMlast + dv;             // [4][dv]
 
     fill_rows(sRow, g, C, b, h, chunk);
     __syncthreads();
+    if (BETA) load_gates(sM, ldv, bd.bgate, sRow, C, dv, dv);
     load_gates(sLam, ldk, gate, sRow, C, dk, dk);
     load_state(sS, ldv, states + ((size_t)bh * g.N + chunk) * dk * dv, dk, dv);
     load_rows(sV, ldv, v, sRow, C, dv, dv);
@@ -386,7 +412,9 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     cp_async_wait_all();
     __syncthreads();
     prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
+    if (BETA) prefix_gates(sM, ldv, C, dv, sMlast, sSegV);
     scale_qk(sQ, sK, sLam, nullptr, ldk, C, dk);
+    if (BETA) scale_qk(nullptr, sV, sM, nullptr, ldv, C, dv);           // Vt = v*exp(-M)
     __syncthreads();
     masked_scores<frag_bound(DM::kC, DM::kC)>(sP, ldp, sQ, sK, ldk, C, dk);
     __syncthreads();
@@ -403,6 +431,11 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
         warp_mma(acc, sQ, ldk, 1, r0, sS, ldv, 1, c0, nbt, 0, dk);
         for_pairs(acc, r0, c0, nbt, [&](int j, int e, float v0, float v1) {
             const int row = sRow[j];
+            if (BETA) {
+                const float2 m = load2(sM + j * ldv + e);
+                v0 *= __expf(m.x);
+                v1 *= __expf(m.y);
+            }
             if (row >= 0 && e < dv) store2(out + (size_t)row * dv + e, v0, v1);
         });
     }
@@ -414,13 +447,18 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
 //   dk = (dP^T Qt + V Dg^T) * exp(-Lam)
 //   dv = P^T dO + Kt Dg
 //   dgate_j = carry + sum_{r >= j in chunk} (q*dq - k*dk)_r,   q*dq = Qt*(dq accumulator), k*dk alike
-template <typename TO, typename DM>
+// BETA: the same formulas with Vt = v*exp(-M) for V and G = dO*exp(M) for dO (Dg then carries both
+// decays); dv = (P^T G + Kt Dg) * exp(-M), and the gradient of log(beta) is, mirroring dgate,
+//   dbgate_j = sum_{r >= j} (o*dO - v*dv)_r  with  o*dO = (P Vt + Qt S)*G  and  v*dv = Vt*(dv accumulator)
+// (the unscaled output P Vt + Qt S is recomputed here, two more products, rather than read back in
+// storage precision), summed here inside the chunk; the chunk total goes to xtot for the cross-chunk part.
+template <typename TO, typename DM, bool BETA>
 __global__ void __launch_bounds__(kThreads)
 mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
               const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate,
               const __nv_bfloat16 *__restrict__ d_out, const float *__restrict__ states,
               const float *__restrict__ dstates, const float *__restrict__ carry, TO *__restrict__ dq,
-              TO *__restrict__ dk_out, TO *__restrict__ dv_out, float *__restrict__ dgate, Geom g)
+              TO *__restrict__ dk_out, TO *__restrict__ dv_out, float *__restrict__ dgate, BetaDev bd, Geom g)
 {
     extern __shared__ __align__(16) float smem[];
     __shared__ int sRow[128];
@@ -439,10 +477,14 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     float *sdP = sP + C * ldp;              // [C][ldp]
     float *sLast = sdP + C * ldp;           // [dkp]
     float *sSeg = sLast + dkp;              // [4][dkp]
+    float *sM = sSeg + 4 * dkp;             // BETA: log(beta) -> M, later x = o*dO - v*dv
+    float *sMlast = sM + C * ldv;           // [dv]
+    float *sSegV = sMlast + dv;             // [4][dv]
     const size_t chunk_id = (size_t)bh * g.N + chunk;
 
     fill_rows(sRow, g, C, b, h, chunk);
     __syncthreads();
+    if (BETA) load_gates(sM, ldv, bd.bgate, sRow, C, dv, dv);
     load_gates(sLam, ldk, gate, sRow, C, dk, dk);
     load_state(sS, ldv, states + chunk_id * dk * dv, dk, dv);
     load_state(sD, ldv, dstates + chunk_id * dk * dv, dk, dv);
@@ -453,7 +495,9 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     cp_async_wait_all();
     __syncthreads();
     prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
+    if (BETA) prefix_gates(sM, ldv, C, dv, sMlast, sSegV);
     scale_qk(sQ, sK, sLam, nullptr, ldk, C, dk);
+    if (BETA) scale_qk(sG, sV, sM, nullptr, ldv, C, dv);                // G = dO*exp(M), Vt = v*exp(-M)
     __syncthreads();
     masked_scores<frag_bound(DM::kC, DM::kC)>(sP, ldp, sQ, sK, ldk, C, dk);
     masked_scores<frag_bound(DM::kC, DM::kC)>(sdP, ldp, sG, sV, ldv, C, dv);
@@ -471,10 +515,39 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
             zero(acc);
             warp_mma(acc, sP, 1, ldp, r0, sG, ldv, 1, c0, nbt, r0, C);
             warp_mma(acc, sK, ldk, 1, r0, sD, ldv, 1, c0, nbt, 0, dk);
-            for_pairs(acc, r0, c0, nbt, [&](int j, int e, float v0, float v1) {
-                const int row = sRow[j];
-                if (row >= 0 && e < dv) store2(dv_out + (size_t)row * dv + e, v0, v1);
-            });
+            if (BETA) {
+                // unscaled output of the same tile, then x = o*dO - v*dv = (P Vt + Qt S)*G - Vt*(dv accumulator)
+                float oh[NB][4];
+                zero(oh);
+                warp_mma(oh, sP, ldp, 1, r0, sV, ldv, 1, c0, nbt, 0, r0 + 16);
+                warp_mma(oh, sQ, ldk, 1, r0, sS, ldv, 1, c0, nbt, 0, dk);
+#pragma unroll
+                for (int nb = 0; nb < NB; ++nb)
+                    if (nb < nbt) {
+#pragma unroll
+                        for (int i = 0; i < 4; i += 2) {
+                            const int off = (r0 + gi + 4 * i) * ldv + c0 + 8 * nb + 2 * ti;
+                            const float2 vt = load2(sV + off), gg = load2(sG + off);
+                            oh[nb][i] = oh[nb][i] * gg.x - vt.x * acc[nb][i];
+                            oh[nb][i + 1] = oh[nb][i + 1] * gg.y - vt.y * acc[nb][i + 1];
+                        }
+                    }
+                // this thread alone touches its elements of M: scale dv by exp(-M), then leave x there
+                for_pairs(acc, r0, c0, nbt, [&](int j, int e, float v0, float v1) {
+                    const int row = sRow[j];
+                    const float2 m = load2(sM + j * ldv + e);
+                    if (row >= 0 && e < dv) store2(dv_out + (size_t)row * dv + e, v0 * __expf(-m.x), v1 * __expf(-m.y));
+                });
+                __syncwarp();
+                for_pairs(oh, r0, c0, nbt, [&](int j, int e, float v0, float v1) {
+                    *reinterpret_cast<float2 *>(sM + j * ldv + e) = make_float2(v0, v1);
+                });
+            } else {
+                for_pairs(acc, r0, c0, nbt, [&](int j, int e, float v0, float v1) {
+                    const int row = sRow[j];
+                    if (row >= 0 && e < dv) store2(dv_out + (size_t)row * dv + e, v0, v1);
+                });
+            }
         }
     }
     {
@@ -547,6 +620,17 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
             }
             sSeg[seg * dkp + c] = run;
         }
+        // the value-channel gate: the same inside the chunk, without the carry (added by a later pass)
+        const int cv = threadIdx.x % dv, segv = threadIdx.x / dv;
+        if (BETA && segv < 4) {
+            float runv = 0.f;
+#pragma unroll 8
+            for (int j = (segv + 1) * rows - 1; j >= segv * rows; --j) {
+                runv += sM[j * ldv + cv];
+                sM[j * ldv + cv] = runv;
+            }
+            sSegV[segv * dv + cv] = runv;
+        }
         __syncthreads();
         if (seg < 4 && c < dk) {
             float add = carry[chunk_id * dk + c];
@@ -556,23 +640,36 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
                 if (row >= 0) dgate[(size_t)row * dk + c] = sLam[j * ldk + c] + add;
             }
         }
+        if (BETA && segv < 4) {
+            float add = 0.f;
+            for (int sg = segv + 1; sg < 4; ++sg) add += sSegV[sg * dv + cv];
+            for (int j = segv * rows; j < (segv + 1) * rows; ++j) {
+                const int row = sRow[j];
+                if (row >= 0) bd.dbgate[(size_t)row * dv + cv] = sM[j * ldv + cv] + add;
+            }
+            if (segv == 0) bd.xtot[chunk_id * dv + cv] = sSegV[cv] + add;
+        }
     }
 }
 
-size_t smem_state(const Geom &g, bool bwd)
+size_t smem_state(const Geom &g, bool bwd, bool beta)
 {
-    return sizeof(float) * ((size_t)g.C * (pitch(g.dk) * (bwd ? 3 : 2) + pitch(g.dv) * (bwd ? 2 : 1)) + 5 * pad16(g.dk));
+    size_t n = (size_t)g.C * (pitch(g.dk) * (bwd ? 3 : 2) + pitch(g.dv) * (bwd ? 2 : 1)) + 5 * pad16(g.dk);
+    if (beta) n += (size_t)g.C * pitch(g.dv) + 5 * pad16(g.dv);
+    return sizeof(float) * n;
 }
-size_t smem_out(const Geom &g)
+size_t smem_out(const Geom &g, bool beta)
 {
     size_t n = (size_t)g.C * (3 * tight(g.dk) + tight(g.dv)) + (size_t)g.dk * tight(g.dv) + 5 * g.dk;
     if (g.C > g.dk) n += (size_t)g.C * tight(g.C);
+    if (beta) n += (size_t)g.C * tight(g.dv) + 5 * g.dv;
     return sizeof(float) * n;
 }
-size_t smem_bwd(const Geom &g)
+size_t smem_bwd(const Geom &g, bool beta)
 {
-    return sizeof(float) * ((size_t)g.C * (3 * tight(g.dk) + 2 * tight(g.dv) + 2 * tight(g.C)) +
-                            2 * (size_t)g.dk * tight(g.dv) + 5 * g.dk);
+    size_t n = (size_t)g.C * (3 * tight(g.dk) + 2 * tight(g.dv) + 2 * tight(g.C)) + 2 * (size_t)g.dk * tight(g.dv) + 5 * g.dk;
+    if (beta) n += (size_t)g.C * tight(g.dv) + 5 * g.dv;
+    return sizeof(float) * n;
 }
 constexpr size_t kMaxSmem = 227 * 1024 - 1024;      // the row table is static shared memory
 
@@ -585,95 +682,135 @@ dig_status set_smem(K kernel, size_t bytes)
 
 using bf16 = __nv_bfloat16;
 
-template <typename TO, typename DM>
+// The value-channel gate keeps two more blocks behind the common workspace: gamma_v and, for the
+// backward pass, the chunk totals of o*do - v*dv, both [B*H][N][d_v].
+size_t beta_block(const Geom &g) { return align256((size_t)g.B * g.H * g.N * g.dv * sizeof(float)); }
+BetaDev beta_dev(const GlaArgs &a, const Workspace &w, bool backward)
+{
+    BetaDev bd{};
+    if (a.bio.bgate == nullptr) return bd;
+    char *p = reinterpret_cast<char *>(a.ws) + w.bytes;
+    bd.bgate = a.bio.bgate;
+    bd.gamma_v = reinterpret_cast<float *>(p);
+    if (backward) {
+        bd.dbgate = a.bio.dbgate;
+        bd.xtot = reinterpret_cast<float *>(p + beta_block(a.g));
+    }
+    return bd;
+}
+
+template <typename TO, typename DM, bool BETA>
 dig_status fwd_dims(const GlaArgs &a)
 {
     const Geom &g = a.g;
     const Workspace w = carve_workspace(a.ws, g, false);
+    const BetaDev bd = beta_dev(a, w, false);
     const dim3 grid(g.N, g.B * g.H);
     dig_status st;
-    auto k1 = mma_chunk_state<false, DM>;
-    if ((st = set_smem(k1, smem_state(g, false))) != DIG_OK) return st;
-    auto k3 = mma_chunk_out<TO, DM>;
-    if ((st = set_smem(k3, smem_out(g))) != DIG_OK) return st;
+    auto k1 = mma_chunk_state<false, DM, BETA>;
+    if ((st = set_smem(k1, smem_state(g, false, BETA))) != DIG_OK) return st;
+    auto k3 = mma_chunk_out<TO, DM, BETA>;
+    if ((st = set_smem(k3, smem_out(g, BETA))) != DIG_OK) return st;
     {
         KernelTimer t(KID_MMA_STATE, a.stream);
-        k1<<<grid, kThreads, smem_state(g, false), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
-                                                              nullptr, w.states, w.gamma, nullptr, g);
+        k1<<<grid, kThreads, smem_state(g, false, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
+                                                                    a.gate, nullptr, w.states, w.gamma, nullptr, bd, g);
     }
-    if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, false, true)) != DIG_OK) return st;
+    if (BETA) st = launch_state_scan_fwd_beta(w, bd.gamma_v, g, a.stream);
+    else st = launch_state_scan_fwd(w, g, a.stream, a.sio, false, true);
+    if (st != DIG_OK) return st;
     KernelTimer t(KID_MMA_OUT, a.stream);
-    k3<<<grid, kThreads, smem_out(g), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate, w.states,
-                                                  (TO *)a.out, g);
+    k3<<<grid, kThreads, smem_out(g, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
+                                                        w.states, (TO *)a.out, bd, g);
     return cuda_ok(cudaGetLastError());
 }
 
-template <typename TO, typename DM>
+template <typename TO, typename DM, bool BETA>
 dig_status bwd_dims(const GlaArgs &a)
 {
     const Geom &g = a.g;
     const Workspace w = carve_workspace(a.ws, g, true);
+    const BetaDev bd = beta_dev(a, w, true);
     const dim3 grid(g.N, g.B * g.H);
     dig_status st;
-    auto k1 = mma_chunk_state<true, DM>;
-    if ((st = set_smem(k1, smem_state(g, true))) != DIG_OK) return st;
-    auto k4 = mma_chunk_bwd<TO, DM>;
-    if ((st = set_smem(k4, smem_bwd(g))) != DIG_OK) return st;
+    auto k1 = mma_chunk_state<true, DM, BETA>;
+    if ((st = set_smem(k1, smem_state(g, true, BETA))) != DIG_OK) return st;
+    auto k4 = mma_chunk_bwd<TO, DM, BETA>;
+    if ((st = set_smem(k4, smem_bwd(g, BETA))) != DIG_OK) return st;
     {
         KernelTimer t(KID_MMA_STATE, a.stream);
-        k1<<<grid, kThreads, smem_state(g, true), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
-                                                             (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, g);
+        k1<<<grid, kThreads, smem_state(g, true, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
+                                                                   a.gate, (const bf16 *)a.d_out, w.states, w.gamma, w.dstates,
+                                                                   bd, g);
     }
-    if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, false, true)) != DIG_OK) return st;
-    if ((st = launch_state_scan_bwd(w, g, a.stream, a.sio, true)) != DIG_OK) return st;
-    KernelTimer t(KID_MMA_BWD, a.stream);
-    k4<<<grid, kThreads, smem_bwd(g), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
-                                                  (const bf16 *)a.d_out, w.states, w.dstates, w.carry, (TO *)a.dq, (TO *)a.dk,
-                                                  (TO *)a.dv, a.dgate, g);
-    return cuda_ok(cudaGetLastError());
+    if (BETA) {
+        if ((st = launch_state_scan_fwd_beta(w, bd.gamma_v, g, a.stream)) != DIG_OK) return st;
+        if ((st = launch_state_scan_bwd_beta(w, bd.gamma_v, g, a.stream)) != DIG_OK) return st;
+    } else {
+        if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, false, true)) != DIG_OK) return st;
+        if ((st = launch_state_scan_bwd(w, g, a.stream, a.sio, true)) != DIG_OK) return st;
+    }
+    {
+        KernelTimer t(KID_MMA_BWD, a.stream);
+        k4<<<grid, kThreads, smem_bwd(g, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
+                                                            (const bf16 *)a.d_out, w.states, w.dstates, w.carry, (TO *)a.dq,
+                                                            (TO *)a.dk, (TO *)a.dv, a.dgate, bd, g);
+    }
+    if (cudaGetLastError() != cudaSuccess) return DIG_ERR_CUDA;
+    if (BETA) return launch_beta_carry(bd.dbgate, bd.xtot, g, a.stream);
+    return DIG_OK;
 }
 
 // The shapes of the paper's models that the tcgen05 family leaves to this one get kernels with
 // compile-time sizes: 72-wide heads with 64-token chunks, 64-wide heads with 32-token chunks.
-template <typename TO>
+template <typename TO, bool BETA>
 dig_status fwd_typed(const GlaArgs &a)
 {
     const Geom &g = a.g;
-    if (g.C == 64 && g.dk == 72 && g.dv == 72) return fwd_dims<TO, FixedDims<64, 72, 72>>(a);
-    if (g.C == 32 && g.dk == 64 && g.dv == 64) return fwd_dims<TO, FixedDims<32, 64, 64>>(a);
-    return fwd_dims<TO, AnyDims>(a);
+    if (g.C == 64 && g.dk == 72 && g.dv == 72) return fwd_dims<TO, FixedDims<64, 72, 72>, BETA>(a);
+    if (!BETA && g.C == 32 && g.dk == 64 && g.dv == 64) return fwd_dims<TO, FixedDims<32, 64, 64>, false>(a);
+    if (BETA && g.C == 64 && g.dk == 64 && g.dv == 64) return fwd_dims<TO, FixedDims<64, 64, 64>, true>(a);
+    return fwd_dims<TO, AnyDims, BETA>(a);
 }
-template <typename TO>
+template <typename TO, bool BETA>
 dig_status bwd_typed(const GlaArgs &a)
 {
     const Geom &g = a.g;
-    if (g.C == 64 && g.dk == 72 && g.dv == 72) return bwd_dims<TO, FixedDims<64, 72, 72>>(a);
-    if (g.C == 32 && g.dk == 64 && g.dv == 64) return bwd_dims<TO, FixedDims<32, 64, 64>>(a);
-    return bwd_dims<TO, AnyDims>(a);
+    if (g.C == 64 && g.dk == 72 && g.dv == 72) return bwd_dims<TO, FixedDims<64, 72, 72>, BETA>(a);
+    if (!BETA && g.C == 32 && g.dk == 64 && g.dv == 64) return bwd_dims<TO, FixedDims<32, 64, 64>, false>(a);
+    if (BETA && g.C == 64 && g.dk == 64 && g.dv == 64) return bwd_dims<TO, FixedDims<64, 64, 64>, true>(a);
+    return bwd_dims<TO, AnyDims, BETA>(a);
 }
 
 }  // namespace
 
-bool mma_supports(int dk, int dv, int chunk, int dtype, bool backward)
+bool mma_supports(int dk, int dv, int chunk, int dtype, bool backward, bool beta)
 {
     if (dtype == DIG_F32) return false;      // one tf32 pass is not fp32-accurate
     Geom g{};
     g.dk = dk; g.dv = dv; g.C = chunk;
-    if (backward) return smem_bwd(g) <= kMaxSmem && smem_state(g, true) <= kMaxSmem;
-    return smem_out(g) <= kMaxSmem && smem_state(g, false) <= kMaxSmem;
+    if (backward) return smem_bwd(g, beta) <= kMaxSmem && smem_state(g, true, beta) <= kMaxSmem;
+    return smem_out(g, beta) <= kMaxSmem && smem_state(g, false, beta) <= kMaxSmem;
+}
+
+size_t mma_beta_workspace_bytes(const Geom &g, bool backward)
+{
+    return carve_workspace(nullptr, g, backward).bytes + beta_block(g) * (backward ? 2 : 1);
 }
 
 dig_status mma_gla_fwd(const GlaArgs &a)
 {
-    if (a.dtype == DIG_BF16) return fwd_typed<__nv_bfloat16>(a);
-    if (a.dtype == DIG_BF16_F32OUT) return fwd_typed<float>(a);
+    const bool beta = a.bio.bgate != nullptr;
+    if (a.dtype == DIG_BF16) return beta ? fwd_typed<__nv_bfloat16, true>(a) : fwd_typed<__nv_bfloat16, false>(a);
+    if (a.dtype == DIG_BF16_F32OUT) return beta ? fwd_typed<float, true>(a) : fwd_typed<float, false>(a);
     return DIG_ERR_UNSUPPORTED;
 }
 
 dig_status mma_gla_bwd(const GlaArgs &a)
 {
-    if (a.dtype == DIG_BF16) return bwd_typed<__nv_bfloat16>(a);
-    if (a.dtype == DIG_BF16_F32OUT) return bwd_typed<float>(a);
+    const bool beta = a.bio.bgate != nullptr;
+    if (a.dtype == DIG_BF16) return beta ? bwd_typed<__nv_bfloat16, true>(a) : bwd_typed<__nv_bfloat16, false>(a);
+    if (a.dtype == DIG_BF16_F32OUT) return beta ? bwd_typed<float, true>(a) : bwd_typed<float, false>(a);
     return DIG_ERR_UNSUPPORTED;
 }
 

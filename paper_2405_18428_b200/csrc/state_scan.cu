@@ -273,6 +273,137 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
     }
 }
 
+// ---- the same scans with the value-channel gate (full gate G = alpha^T beta of Eq. gate_gla) ---------
+// The state decays along its rows by gamma (key channels) and along its columns by gamma_v (value
+// channels): S_[i+1] = diag(gamma_i) S_[i] diag(gamma_v_i) + U_i, and the mirror image for D.  Row-major
+// states only (warp-MMA family); stored states and diag(gamma) D diag(gamma_v) are rounded to tf32.
+__global__ void __launch_bounds__(kScanThreads)
+state_scan_fwd_beta(float *__restrict__ states, const float *__restrict__ gamma, const float *__restrict__ gamma_v,
+                    float *__restrict__ s_final, int N, int dk, int dv)
+{
+    const int e4 = blockIdx.x * kScanThreads + threadIdx.x;
+    if (e4 * 4 >= dk * dv) return;
+    const int row = (e4 * 4) / dv, col = (e4 * 4) - row * dv;
+    float4 *st = reinterpret_cast<float4 *>(states + (size_t)blockIdx.y * N * dk * dv) + e4;
+    const float *gm = gamma + (size_t)blockIdx.y * N * dk + row;
+    const float *gv = gamma_v + (size_t)blockIdx.y * N * dv + col;
+    const size_t sstride = (size_t)dk * dv / 4;
+    float4 run = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < N; i += kAhead) {
+        float4 u[kAhead], g[kAhead];
+#pragma unroll
+        for (int j = 0; j < kAhead; ++j) {
+            if (i + j < N) {
+                u[j] = st[(size_t)(i + j) * sstride];
+                const float gr = gm[(size_t)(i + j) * dk];
+                const float4 gc = *reinterpret_cast<const float4 *>(gv + (size_t)(i + j) * dv);
+                g[j] = make_float4(gr * gc.x, gr * gc.y, gr * gc.z, gr * gc.w);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kAhead; ++j) {
+            if (i + j < N) {
+                st[(size_t)(i + j) * sstride] = round4_tf32(run);
+                run.x = fmaf(g[j].x, run.x, u[j].x);
+                run.y = fmaf(g[j].y, run.y, u[j].y);
+                run.z = fmaf(g[j].z, run.z, u[j].z);
+                run.w = fmaf(g[j].w, run.w, u[j].w);
+            }
+        }
+    }
+    if (s_final != nullptr) *reinterpret_cast<float4 *>(s_final + (size_t)blockIdx.y * dk * dv + (size_t)e4 * 4) = run;
+}
+
+__global__ void __launch_bounds__(32 * kRowsPerBlock)
+state_scan_bwd_beta(const float *__restrict__ states, float *__restrict__ dstates, const float *__restrict__ gamma,
+                    const float *__restrict__ gamma_v, float *__restrict__ carry, int N, int dk, int dv)
+{
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * kRowsPerBlock + (threadIdx.x >> 5);
+    if (c >= dk) return;
+    const size_t sstride = (size_t)dk * dv;
+    const size_t base = (size_t)blockIdx.y * N * sstride + (size_t)c * dv;
+    const float *S = states + base;
+    float *D = dstates + base;
+    const float *gm = gamma + (size_t)blockIdx.y * N * dk + c;
+    const float *gv = gamma_v + (size_t)blockIdx.y * N * dv;
+    float *cr = carry + (size_t)blockIdx.y * N * dk + c;
+    float run[kMaxPerLane];
+#pragma unroll
+    for (int r = 0; r < kMaxPerLane; ++r) run[r] = 0.f;
+    constexpr int kLook = 4;
+    for (int i = N - 1; i >= 0; i -= kLook) {
+        float w[kLook][kMaxPerLane], sn[kLook][kMaxPerLane], g[kLook][kMaxPerLane];
+#pragma unroll
+        for (int j = 0; j < kLook; ++j) {
+            const int ch = i - j;
+            const float gr = ch >= 0 ? gm[(size_t)ch * dk] : 0.f;
+#pragma unroll
+            for (int r = 0; r < kMaxPerLane; ++r) {
+                const int e = lane + 32 * r;
+                const bool on = ch >= 0 && e < dv;
+                w[j][r] = on ? D[(size_t)ch * sstride + e] : 0.f;
+                g[j][r] = on ? gr * gv[(size_t)ch * dv + e] : 0.f;
+                sn[j][r] = (on && ch + 1 < N) ? S[(size_t)(ch + 1) * sstride + e] : 0.f;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kLook; ++j) {
+            const int ch = i - j;
+            if (ch < 0) break;          // uniform over the warp
+            float dot = 0.f;
+#pragma unroll
+            for (int r = 0; r < kMaxPerLane; ++r) {
+                const int e = lane + 32 * r;
+                if (e < dv) D[(size_t)ch * sstride + e] = round_tf32(g[j][r] * run[r]);
+                dot = fmaf(sn[j][r], run[r], dot);
+                run[r] = fmaf(g[j][r], run[r], w[j][r]);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+            if (lane == 0) cr[(size_t)ch * dk] = dot;
+        }
+    }
+}
+
+// Gate gradient of the value-channel gate across chunks.  xtot[i][e] holds chunk i's total of
+// (o*do - v*dv); it is turned in place into the sum over the later chunks (what every token of chunk
+// i still has to receive), one thread per (sequence, value channel).
+__global__ void __launch_bounds__(128)
+beta_suffix_totals(float *__restrict__ xtot, int N, int dv, int total)
+{
+    const int idx = blockIdx.x * 128 + threadIdx.x;
+    if (idx >= total) return;
+    const int bh = idx / dv, e = idx - bh * dv;
+    float *x = xtot + (size_t)bh * N * dv + e;
+    float run = 0.f;
+    for (int i = N - 1; i >= 0; --i) {
+        const float t = x[(size_t)i * dv];
+        x[(size_t)i * dv] = run;
+        run += t;
+    }
+}
+
+// dbgate[token][e] += what later chunks contribute; one thread per 4 value channels of a scan position.
+__global__ void __launch_bounds__(256)
+beta_add_carry(float *__restrict__ dbgate, const float *__restrict__ xtot, Geom g)
+{
+    const int per_row = g.dv >> 2;
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long total = (long long)g.B * g.H * g.L * per_row;
+    if (idx >= total) return;
+    const int e = (int)(idx % per_row) << 2;
+    const long long r = idx / per_row;
+    const int p = (int)(r % g.L);
+    const int bh = (int)(r / g.L), b = bh / g.H, h = bh - b * g.H;
+    const int chunk = p / g.C;
+    const float4 add = *reinterpret_cast<const float4 *>(xtot + ((size_t)bh * g.N + chunk) * g.dv + e);
+    float4 *dst = reinterpret_cast<float4 *>(dbgate + tok_offset(g, b, scan_token(p, g.dir, g.gh, g.gw, g.L), h, g.dv) + e);
+    float4 v = *dst;
+    v.x += add.x; v.y += add.y; v.z += add.z; v.w += add.w;
+    *dst = v;
+}
+
 }  // namespace
 
 dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tiles, bool tf32)
@@ -313,6 +444,33 @@ dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaSt
     KernelTimer t(KID_SCAN_BWD, s);
     launch_pdl(state_scan_bwd_tiles, dim3(8, g.B * g.H), dim3(64), 0, s, w.states, w.dstates, w.dstates_m,
                (const float *)w.gamma, w.carry, sio.s_in, sio.ds_out, sio.ds_in, g.N);
+    return cuda_ok(cudaGetLastError());
+}
+
+dig_status launch_state_scan_fwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s)
+{
+    const dim3 grid((g.dk * g.dv / 4 + kScanThreads - 1) / kScanThreads, g.B * g.H);
+    KernelTimer t(KID_SCAN_FWD, s);
+    state_scan_fwd_beta<<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, gamma_v, w.sfinal, g.N, g.dk, g.dv);
+    return cuda_ok(cudaGetLastError());
+}
+
+dig_status launch_state_scan_bwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s)
+{
+    const dim3 grid((g.dk + kRowsPerBlock - 1) / kRowsPerBlock, g.B * g.H);
+    KernelTimer t(KID_SCAN_BWD, s);
+    state_scan_bwd_beta<<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, gamma_v, w.carry, g.N, g.dk, g.dv);
+    return cuda_ok(cudaGetLastError());
+}
+
+dig_status launch_beta_carry(float *dbgate, float *xtot, const Geom &g, cudaStream_t s)
+{
+    KernelTimer t(KID_SCAN_BWD, s);
+    const int total = g.B * g.H * g.dv;
+    beta_suffix_totals<<<(total + 127) / 128, 128, 0, s>>>(xtot, g.N, g.dv, total);
+    if (cudaGetLastError() != cudaSuccess) return DIG_ERR_CUDA;
+    const long long n = (long long)g.B * g.H * g.L * (g.dv >> 2);
+    beta_add_carry<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(dbgate, xtot, g);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -23,7 +23,8 @@ DIG_ROW_FWD, DIG_ROW_REV, DIG_COL_FWD, DIG_COL_REV = 0, 1, 2, 3
 DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR, DIG_IMPL_MMA = 0, 1, 2, 3
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
-           "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_gla_fwd_state", "dig_gla_bwd_state", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
+           "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_gla_fwd_state", "dig_gla_bwd_state",
+           "dig_gla_fwd_beta", "dig_gla_bwd_beta", "dig_gla_beta_workspace_bytes", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
            "dig_srem_dwconv_bwd_workspace_bytes", "dig_gla_outgate_fwd", "dig_gla_outgate_bwd",
            "dig_gla_outgate_bwd_workspace_bytes", "dig_last_device_status",
            "dig_status_string", "dig_profile_enable", "dig_profile_kernels", "dig_profile_read")
@@ -61,6 +62,12 @@ def lib() -> ctypes.CDLL:
         L.dig_gla_fwd_static.restype = i
         L.dig_gla_bwd.argtypes = [vp] * 9 + [i] * 9 + [vp, sz, vp]
         L.dig_gla_bwd.restype = i
+        L.dig_gla_beta_workspace_bytes.argtypes = [i] * 9
+        L.dig_gla_beta_workspace_bytes.restype = sz
+        L.dig_gla_fwd_beta.argtypes = [vp] * 6 + [i] * 9 + [vp, sz, vp]
+        L.dig_gla_fwd_beta.restype = i
+        L.dig_gla_bwd_beta.argtypes = [vp] * 11 + [i] * 9 + [vp, sz, vp]
+        L.dig_gla_bwd_beta.restype = i
         L.dig_gla_fwd_state.argtypes = [vp] * 7 + [i] * 9 + [vp, sz, vp]
         L.dig_gla_fwd_state.restype = i
         L.dig_gla_bwd_state.argtypes = [vp] * 12 + [i] * 9 + [vp, sz, vp]
@@ -375,3 +382,51 @@ def dig_gla_bwd_state(q, k, v, gate, d_out, s_in, ds_out, grid_h, grid_w, chunk=
                                    workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
            "dig_gla_bwd_state")
     return dq, dk_, dv_, dgate, ds_in
+
+
+def dig_gla_fwd_beta(q, k, v, gate, bgate, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD, *, f32_out=False,
+                     workspace=None) -> torch.Tensor:
+    """dig_gla_fwd with the value-channel gate: bgate = log(beta), fp32 [B, L, H, d_v]."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st = _storage(dtype)
+    need = lib().dig_gla_beta_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 0)
+    if need == 0:
+        raise DigError(DIG_ERR_UNSUPPORTED, "dig_gla_beta_workspace_bytes")
+    workspace = _workspace(workspace, need, q.device)
+    out = torch.empty((B, L, H, dv), dtype=_out_storage(dtype), device=q.device)
+    _check(lib().dig_gla_fwd_beta(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"), _dev(v, st, (B, L, H, dv), "v"),
+                                  _dev(gate, torch.float32, q.shape, "gate"), _dev(bgate, torch.float32, v.shape, "bgate"),
+                                  _dev(out, _out_storage(dtype), name="out"),
+                                  B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
+                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "dig_gla_fwd_beta")
+    return out
+
+
+def dig_gla_bwd_beta(q, k, v, gate, bgate, d_out, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD, *,
+                     f32_out=False, workspace=None):
+    """Returns (dq, dk, dv, dgate, dbgate)."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st, ost = _storage(dtype), _out_storage(dtype)
+    need = lib().dig_gla_beta_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 1)
+    if need == 0:
+        raise DigError(DIG_ERR_UNSUPPORTED, "dig_gla_beta_workspace_bytes")
+    workspace = _workspace(workspace, need, q.device)
+    dq = torch.empty(q.shape, dtype=ost, device=q.device)
+    dk_ = torch.empty(q.shape, dtype=ost, device=q.device)
+    dv_ = torch.empty(v.shape, dtype=ost, device=q.device)
+    dgate = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+    dbgate = torch.empty(v.shape, dtype=torch.float32, device=q.device)
+    _check(lib().dig_gla_bwd_beta(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"), _dev(v, st, (B, L, H, dv), "v"),
+                                  _dev(gate, torch.float32, q.shape, "gate"), _dev(bgate, torch.float32, v.shape, "bgate"),
+                                  _dev(d_out, st, v.shape, "d_out"),
+                                  _dev(dq, ost, name="dq"), _dev(dk_, ost, name="dk"), _dev(dv_, ost, name="dv"),
+                                  _dev(dgate, torch.float32, name="dgate"), _dev(dbgate, torch.float32, name="dbgate"),
+                                  B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
+                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "dig_gla_bwd_beta")
+    return dq, dk_, dv_, dgate, dbgate

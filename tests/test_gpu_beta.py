@@ -1,0 +1,83 @@
+"""GPU parity of gated linear attention with the full gate alpha^T beta of Eq. gate_gla
+(dig_gla_fwd_beta, dig_gla_bwd_beta) against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2405_18428_b200.inputs import CONFIGS, Workload, make_inputs, round_to_bf16
+from parity import TOL_BF16, oracle_threads, rel_err, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(wl, direction, seed, tau_v=8.0):
+    from paper_2405_18428_b200 import dig
+    x = make_inputs(wl, conv=False)
+    rng = np.random.default_rng(seed)
+    gb = round_to_bf16(rng.standard_normal((wl.B, wl.grid_h * wl.grid_w, wl.H, wl.d_v)).astype(np.float32))
+    a = oracle.gate(x["g"], x["tau"])
+    bg = oracle.gate(gb, np.full(wl.H, tau_v, dtype=np.float32))          # log(beta) = logsigmoid / tau
+    thr = oracle_threads()
+    ro = oracle.gla_fwd_beta(x["q"], x["k"], x["v"], a, bg, wl.grid_h, wl.grid_w, direction, threads=thr)
+    rg = oracle.gla_bwd_beta(x["q"], x["k"], x["v"], a, bg, x["dO"], wl.grid_h, wl.grid_w, direction, threads=thr)
+    q, k, v, g, dO = (to_dev(x[n], wl) for n in ("q", "k", "v", "g", "dO"))
+    gate = dig.dig_gate_logsigmoid(g, x["tau"])
+    bgate = dig.dig_gate_logsigmoid(to_dev(gb, wl), np.full(wl.H, tau_v, dtype=np.float32))
+    res = {}
+    for f32_out in (True, False):
+        out = dig.dig_gla_fwd_beta(q, k, v, gate, bgate, wl.grid_h, wl.grid_w, wl.chunk, direction, f32_out=f32_out)
+        grads = dig.dig_gla_bwd_beta(q, k, v, gate, bgate, dO, wl.grid_h, wl.grid_w, wl.chunk, direction, f32_out=f32_out)
+        torch.cuda.synchronize()
+        assert dig.dig_last_device_status() == dig.DIG_OK
+        res[f32_out] = dict(zip(("out", "dq", "dk", "dv", "dgate", "dbgate"), (out, *grads)))
+    errs = {n: rel_err(t.cpu().numpy(), r) for (n, t), r in zip(res[True].items(), (ro, *rg))}
+    assert all(np.isfinite(e) and e <= TOL_BF16 for e in errs.values()), errs
+    # bf16-stored results are exactly the fp32 results rounded to nearest-even bf16; the gate gradients are fp32 in both
+    for n in ("out", "dq", "dk", "dv"):
+        assert torch.equal(res[False][n], res[True][n].to(torch.bfloat16)), n
+    for n in ("dgate", "dbgate"):
+        assert torch.equal(res[False][n], res[True][n]), n
+    return errs
+
+
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+def test_small_ragged_all_directions(direction):
+    wl = Workload("beta", B=2, H=3, grid_h=7, grid_w=9, d_k=24, d_v=40, chunk=16, dtype="bf16", backward=True,
+                  tau=(16.0, 2.0, 1.0), seed=31)
+    print(_run(wl, direction, direction))
+
+
+@pytest.mark.parametrize("d,chunk", [(64, 64), (72, 64), (64, 32), (8, 16)])
+def test_head_and_chunk_sizes(d, chunk):
+    wl = Workload("beta", B=1, H=2, grid_h=12, grid_w=11, d_k=d, d_v=d, chunk=chunk, dtype="bf16", backward=True,
+                  tau=(16.0, 4.0), seed=32)
+    print(_run(wl, 2, 5))
+
+
+def test_long_sequence_many_chunks():
+    wl = CONFIGS["C5"].scaled(B=1, H=2, grid_h=40, grid_w=40, backward=True)       # 1600 tokens, 25 chunks, d = 72
+    print(_run(wl, 3, 6))
+
+
+def test_beta_one_equals_the_alpha_only_entry_point():
+    from paper_2405_18428_b200 import dig
+    wl = Workload("beta1", B=1, H=2, grid_h=8, grid_w=16, d_k=72, d_v=72, chunk=64, dtype="bf16", backward=True, seed=33)
+    x = make_inputs(wl, conv=False)
+    q, k, v, g, dO = (to_dev(x[n], wl) for n in ("q", "k", "v", "g", "dO"))
+    gate = dig.dig_gate_logsigmoid(g, x["tau"])
+    zero = torch.zeros(v.shape, dtype=torch.float32, device="cuda")
+    a = dig.dig_gla_fwd(q, k, v, gate, 8, 16, 64, 1, f32_out=True)
+    b = dig.dig_gla_fwd_beta(q, k, v, gate, zero, 8, 16, 64, 1, f32_out=True)
+    assert torch.equal(a, b)
+    ga = dig.dig_gla_bwd(q, k, v, gate, dO, 8, 16, 64, 1, f32_out=True)
+    gb = dig.dig_gla_bwd_beta(q, k, v, gate, zero, dO, 8, 16, 64, 1, f32_out=True)
+    for x1, x2 in zip(ga, gb[:4]):
+        assert torch.equal(x1, x2)
+
+
+def test_fp32_storage_is_refused():
+    from paper_2405_18428_b200 import dig
+    q = torch.zeros(1, 16, 1, 8, device="cuda")
+    with pytest.raises(dig.DigError):
+        dig.dig_gla_fwd_beta(q, q, q, q, q, 4, 4, 16, 0)
