@@ -91,6 +91,58 @@ state_scan_fwd(float *__restrict__ states, const float *__restrict__ gamma, cons
     }
 }
 
+// The same scan with one element per thread and 16 chunks of loads in flight: four times the threads
+// of the kernel above, for calls with so few (batch, head) sequences that float4 threads would leave
+// most SMs idle and too few loads in flight (long sequences of a small batch).
+constexpr int kScan1Threads = 256, kAhead1 = 16;
+template <bool TILES, bool TF32>
+__global__ void __launch_bounds__(kScan1Threads)
+state_scan_fwd1(float *__restrict__ states, const float *__restrict__ gamma, const float *__restrict__ s_in,
+                float *__restrict__ s_final, int N, int dk, int dv)
+{
+    pdl_wait();
+    pdl_launch_dependents();      // only once this kernel's own predecessor has completed
+    const int e = blockIdx.x * kScan1Threads + threadIdx.x;          // element index inside one stored state
+    if (e >= dk * dv) return;
+    int row, col;
+    if (TILES) {
+        row = (e & 2047) >> 5;
+        col = (e >> 11) * 32 + ((((e & 31) >> 2) ^ (row & 7)) << 2) + (e & 3);
+    } else {
+        row = e / dv;
+        col = e - row * dv;
+    }
+    float *st = states + (size_t)blockIdx.y * N * dk * dv + e;
+    const float *gm = gamma + (size_t)blockIdx.y * N * dk + (TILES ? col : row);
+    const size_t sstride = (size_t)dk * dv;
+    const size_t io = (size_t)blockIdx.y * dk * dv + (TILES ? (size_t)col * dv + row : (size_t)row * dv + col);
+    float run = s_in != nullptr ? s_in[io] : 0.f;
+    for (int i = 0; i < N; i += kAhead1) {
+        float u[kAhead1], g[kAhead1];
+        const float *pu = st;
+        const float *pg = gm;
+#pragma unroll
+        for (int j = 0; j < kAhead1; ++j) {
+            if (i + j < N) {
+                u[j] = *pu;
+                g[j] = *pg;
+            }
+            pu += sstride;
+            pg += dk;
+        }
+#pragma unroll
+        for (int j = 0; j < kAhead1; ++j) {
+            if (i + j < N) {
+                *st = (TILES || TF32) ? round_tf32(run) : run;
+                run = fmaf(g[j], run, u[j]);
+            }
+            st += sstride;
+        }
+        gm += (size_t)kAhead1 * dk;
+    }
+    if (s_final != nullptr) s_final[io] = run;
+}
+
 // One warp per key channel c; lanes stride over the value channels.
 // TF32: dstates receives diag(gamma_i) D_[i] rounded to tf32, the form the warp-MMA gradient kernel
 // multiplies with, instead of D_[i].
@@ -414,6 +466,17 @@ dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t
     // backward scan reads it from (null in a forward-only workspace)
     float *fin = sio.s_out != nullptr ? sio.s_out : w.sfinal;
     KernelTimer t(KID_SCAN_FWD, s);
+    if ((long long)grid.x * grid.y * kScanThreads < 16384) {       // few sequences: one element per thread
+        const dim3 grid1((g.dk * g.dv + kScan1Threads - 1) / kScan1Threads, g.B * g.H);
+        if (tiles)
+            launch_pdl(state_scan_fwd1<true, true>, grid1, dim3(kScan1Threads), 0, s, w.states, (const float *)w.gamma, sio.s_in,
+                       fin, g.N, g.dk, g.dv);
+        else if (tf32)
+            state_scan_fwd1<false, true><<<grid1, kScan1Threads, 0, s>>>(w.states, w.gamma, sio.s_in, fin, g.N, g.dk, g.dv);
+        else
+            state_scan_fwd1<false, false><<<grid1, kScan1Threads, 0, s>>>(w.states, w.gamma, sio.s_in, fin, g.N, g.dk, g.dv);
+        return cuda_ok(cudaGetLastError());
+    }
     if (tiles)
         launch_pdl(state_scan_fwd<true>, grid, dim3(kScanThreads), 0, s, w.states, (const float *)w.gamma, sio.s_in, fin, g.N,
                    g.dk, g.dv);
