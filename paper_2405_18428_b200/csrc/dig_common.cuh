@@ -35,15 +35,6 @@ __host__ __device__ __forceinline__ size_t tok_offset(const Geom &g, int b, int 
 }
 
 // ---- storage conversion ---------------------------------------------------------------
-__device__ __forceinline__ float to_f32(float x) { return x; }
-__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
-template <typename T> __device__ __forceinline__ T from_f32(float x);
-template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
-template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x)
-{
-    return __float2bfloat16_rn(x);
-}
-
 // Load 4 consecutive elements (16-byte aligned for float, 8-byte for bf16) as floats.
 __device__ __forceinline__ float4 load4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
 __device__ __forceinline__ float4 load4(const __nv_bfloat16 *p)

@@ -66,17 +66,6 @@ __device__ __forceinline__ size_t row_offset(const Geom &g, const Item &it, int 
 __device__ __forceinline__ uint4 ldg16(const bf16 *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }
 __device__ __forceinline__ float4 ldg16(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
 
-// 8 consecutive bf16 / 4 consecutive floats of a token row.  The load is unconditional so that it
-// can stay in flight across a loop iteration: for tok < 0 (a row past the end of the sequence)
-// token 0 is read instead and the consumer zeroes the values.
-__device__ __forceinline__ uint4 ld_row8(const bf16 *base, const Geom &g, int b, int tok, int h, int d, int col)
-{
-    return __ldg(reinterpret_cast<const uint4 *>(base + tok_offset(g, b, tok < 0 ? 0 : tok, h, d) + col));
-}
-__device__ __forceinline__ float4 ld_row4(const float *base, const Geom &g, int b, int tok, int h, int d, int col)
-{
-    return __ldg(reinterpret_cast<const float4 *>(base + tok_offset(g, b, tok < 0 ? 0 : tok, h, d) + col));
-}
 // `keep` = false turns the row into zeros.
 // `flip`: the lanes that hold columns 32-63 of a row keep the two 4-column halves of their 8 columns
 // exchanged in registers (f[0..3] = columns col8+4..col8+7) and store the upper half first.  The 8
@@ -179,30 +168,6 @@ __device__ __forceinline__ void gate_prefix(float *sLam, float *sLast, float *sT
     for (int j = 0; j < R; ++j) sLam[(R * seg + j) * kLamPitch + c] = a[j] + add;
     if (seg - first == SEG_PER_CH - 1) sLast[(seg / SEG_PER_CH) * 64 + c] = a[R - 1] + add;
     if (GROUP) sync_group(NT); else __syncthreads();
-}
-
-// Fetches 32 gate rows (rows 32*part .. 32*part+31 of the stacked table; `it` is the item those
-// rows belong to) into sLam: one bulk copy of 256 bytes per token row, rows past the end of the
-// sequence are zero-filled.  Called by one full warp per part; `bar` (initialised with one arrival
-// per part) receives this warp's arrival plus its bytes in flight.  The caller guarantees that
-// nobody reads or writes sLam until the barrier completes (zero-filled rows: until the next
-// __syncthreads).
-__device__ __forceinline__ void fetch_gate_rows(float *sLam, const float *gate, const Geom &g, const Item &it, int part,
-                                                uint64_t *bar, int lane)
-{
-    fence_async_smem();          // earlier generic-proxy reads of sLam come before the asynchronous writes
-    const int row = 32 * part + lane;
-    const int tok = item_token(g, it, row % T);
-    const uint32_t rows = __popc(__ballot_sync(0xffffffffu, tok >= 0));
-    if (lane == 0) mbar_arrive_expect_tx(bar, rows * DK * 4);
-    __syncwarp();
-    float *dst = sLam + row * kLamPitch;
-    if (tok >= 0) {
-        bulk_g2s(dst, gate + tok_offset(g, it.b, tok, it.h, DK), DK * 4, bar);
-    } else {
-#pragma unroll
-        for (int j = 0; j < DK / 4; ++j) *reinterpret_cast<float4 *>(dst + 4 * j) = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
 }
 
 __device__ __forceinline__ void read_lam8(const float *sLam, int row, int col8, float (&lam)[8], bool flip = false)
