@@ -325,6 +325,107 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
     }
 }
 
+// The same two scans for calls with few sequences: one warp per row, lane l holds logical columns l
+// and 32 + l (the same offset in the two column blocks, so a warp touches one 128-byte line per
+// block), 32 chunks of loads in flight.  Four times the threads and twice the look-ahead of the kernel
+// above; slower than it when there are enough sequences to fill the GPU.
+constexpr int kTileRows = 4, kLook1 = 32;
+__global__ void __launch_bounds__(32 * kTileRows)
+state_scan_bwd_tiles1(float *__restrict__ states, float *__restrict__ dstates, float *__restrict__ dstates_m,
+                      const float *__restrict__ gamma, float *__restrict__ carry, const float *__restrict__ s_in,
+                      const float *__restrict__ ds_out, float *__restrict__ ds_in, int N)
+{
+    pdl_wait();
+    pdl_launch_dependents();      // only once this kernel's own predecessor has completed
+    const int lane = threadIdx.x & 31, c = kTileRows * blockIdx.x + (threadIdx.x >> 5);
+    const size_t base = (size_t)blockIdx.y * N * 4096;
+    const int offk = c * 32 + ((((lane >> 2) ^ (c & 7)) << 2) | (lane & 3));
+    const int offm = c * 32 + ((((lane >> 3) ^ (c & 3)) << 3) | (lane & 7));
+    float *S = states + base + offk;
+    float *D = dstates + base + offk;
+    float *DM = dstates_m + base + offm;
+    const float *gm = gamma + (size_t)blockIdx.y * N * 64 + c;
+    float *cr = carry + (size_t)blockIdx.y * N * 64 + c;
+    const size_t io = ((size_t)blockIdx.y * 64 + c) * 64 + lane;       // row-major state: columns lane, lane + 32
+    float r0 = 0.f, r1 = 0.f;
+    if (s_in != nullptr) {
+        r0 = s_in[io];
+        r1 = s_in[io + 32];
+    }
+    for (int i = 0; i < N; i += kLook1) {
+        float u0[kLook1], u1[kLook1], g[kLook1];
+        const float *ps = S + (size_t)i * 4096;
+        const float *pg = gm + (size_t)i * 64;
+#pragma unroll
+        for (int j = 0; j < kLook1; ++j) {
+            if (i + j < N) {
+                u0[j] = ps[0];
+                u1[j] = ps[2048];
+                g[j] = *pg;
+            }
+            ps += 4096;
+            pg += 64;
+        }
+        float *pw = S + (size_t)i * 4096;
+#pragma unroll
+        for (int j = 0; j < kLook1; ++j) {
+            if (i + j < N) {
+                pw[0] = round_tf32(r0);
+                pw[2048] = round_tf32(r1);
+                r0 = fmaf(g[j], r0, u0[j]);
+                r1 = fmaf(g[j], r1, u1[j]);
+            }
+            pw += 4096;
+        }
+    }
+    float d0 = 0.f, d1 = 0.f;
+    if (ds_out != nullptr) {
+        d0 = ds_out[io];
+        d1 = ds_out[io + 32];
+    }
+    constexpr int kB = kLook1 / 2;
+    for (int i = N - 1; i >= 0; i -= kB) {
+        float w0[kB], w1[kB], s0[kB], s1[kB], g[kB];
+#pragma unroll
+        for (int j = 0; j < kB; ++j) {
+            const int ch = i - j;
+            if (ch >= 0) {
+                w0[j] = D[(size_t)ch * 4096];
+                w1[j] = D[(size_t)ch * 4096 + 2048];
+                g[j] = gm[(size_t)ch * 64];
+                if (ch + 1 < N) {
+                    s0[j] = S[(size_t)(ch + 1) * 4096];
+                    s1[j] = S[(size_t)(ch + 1) * 4096 + 2048];
+                } else {              // the last chunk leaves the final state, still in registers
+                    s0[j] = r0;
+                    s1[j] = r1;
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kB; ++j) {
+            const int ch = i - j;
+            if (ch >= 0) {            // uniform over the block
+                float dot = fmaf(s0[j], d0, s1[j] * d1);
+                const float e0 = round_tf32(g[j] * d0), e1 = round_tf32(g[j] * d1);
+                D[(size_t)ch * 4096] = e0;
+                D[(size_t)ch * 4096 + 2048] = e1;
+                DM[(size_t)ch * 4096] = e0;
+                DM[(size_t)ch * 4096 + 2048] = e1;
+                d0 = fmaf(g[j], d0, w0[j]);
+                d1 = fmaf(g[j], d1, w1[j]);
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+                if (lane == 0) cr[(size_t)ch * 64] = dot;
+            }
+        }
+    }
+    if (ds_in != nullptr) {
+        ds_in[io] = d0;
+        ds_in[io + 32] = d1;
+    }
+}
+
 // ---- the same scans with the value-channel gate (full gate G = alpha^T beta of Eq. gate_gla) ---------
 // The state decays along its rows by gamma (key channels) and along its columns by gamma_v (value
 // channels): S_[i+1] = diag(gamma_i) S_[i] diag(gamma_v_i) + U_i, and the mirror image for D.  Row-major
@@ -505,8 +606,12 @@ dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaSt
 {
     if (g.dk != 64 || g.dv != 64) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_SCAN_BWD, s);
-    launch_pdl(state_scan_bwd_tiles, dim3(8, g.B * g.H), dim3(64), 0, s, w.states, w.dstates, w.dstates_m,
-               (const float *)w.gamma, w.carry, sio.s_in, sio.ds_out, sio.ds_in, g.N);
+    if (g.B * g.H < 16)      // few sequences: the finer kernel with the deeper look-ahead
+        launch_pdl(state_scan_bwd_tiles1, dim3(64 / kTileRows, g.B * g.H), dim3(32 * kTileRows), 0, s, w.states, w.dstates,
+                   w.dstates_m, (const float *)w.gamma, w.carry, sio.s_in, sio.ds_out, sio.ds_in, g.N);
+    else
+        launch_pdl(state_scan_bwd_tiles, dim3(8, g.B * g.H), dim3(64), 0, s, w.states, w.dstates, w.dstates_m,
+                   (const float *)w.gamma, w.carry, sio.s_in, sio.ds_out, sio.ds_in, g.N);
     return cuda_ok(cudaGetLastError());
 }
 
