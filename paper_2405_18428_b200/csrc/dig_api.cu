@@ -12,6 +12,8 @@ dig_status launch_gate(const void *g, const float *tau_host, float *gate, int B,
 dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y, int B, int gh,
                          int gw, int D, int dir, int dtype, cudaStream_t stream);
 size_t outgate_bwd_workspace_bytes(long long rows, int dv);
+dig_status launch_outgate_fwd_mixed(const void *o, const void *r, const float *ln_w, const float *ln_b, void *z,
+                                    long long rows, int dv, float eps, int dtype, cudaStream_t stream);
 dig_status launch_outgate_fwd(const void *o, const void *r, const float *ln_w, const float *ln_b, void *z,
                               long long rows, int dv, float eps, int dtype, cudaStream_t stream);
 dig_status launch_outgate_bwd(const void *o, const void *r, const void *dz, const float *ln_w, const float *ln_b,
@@ -300,6 +302,39 @@ dig_status dig_gla_outgate_bwd(const void *o, const void *r, const float *ln_w, 
     }
     return launch_outgate_bwd(o, r, dz, ln_w, ln_b, d_o, d_r, dln_w, dln_b, rows, d_v, eps, dtype,
                               reinterpret_cast<float *>(workspace), (cudaStream_t)cuda_stream);
+}
+
+dig_status dig_gla_fwd_outgate(const void *q, const void *k, const void *v, const float *gate, const void *r,
+                               const float *ln_w, const float *ln_b, float eps, void *out, void *z, int B, int H,
+                               int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!q || !k || !v || !gate || !r || !z) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(r) || !aligned16(z) ||
+        (out && !aligned16(out)) || (ln_w && !aligned16(ln_w)) || (ln_b && !aligned16(ln_b)) || !(eps >= 0.f))
+        return DIG_ERR_INVALID_ARG;
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, direction, dtype)) return DIG_ERR_INVALID_ARG;
+    const size_t need = dig_gla_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, 0);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    const int impl = choose_impl(d_k, d_v, chunk, dtype, false);
+    if (impl < 0) return (dig_status)(-impl);
+    GlaArgs a{};
+    a.q = q; a.k = k; a.v = v; a.gate = gate;
+    a.ws = reinterpret_cast<float *>(workspace);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
+    a.dtype = dtype;
+    a.stream = (cudaStream_t)cuda_stream;
+    if (impl == DIG_IMPL_TENSOR) {          // the readout kernel applies the gate while it stores
+        a.out = out;
+        a.og.r = r; a.og.ln_w = ln_w; a.og.ln_b = ln_b; a.og.eps = eps; a.og.z = z;
+        return tensor_gla_fwd(a);
+    }
+    // other families: the plain forward pass (into z when the caller does not want `out`), then the
+    // gate kernel, which may work in place
+    a.out = out ? out : z;
+    const dig_status st = impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
+    if (st != DIG_OK) return st;
+    return launch_outgate_fwd_mixed(a.out, r, ln_w, ln_b, z, (long long)B * grid_h * grid_w * H, d_v, eps, dtype, a.stream);
 }
 
 size_t dig_gla_beta_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int dtype,

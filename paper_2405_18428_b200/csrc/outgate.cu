@@ -73,10 +73,13 @@ template <int LPR> __device__ __forceinline__ float normalise(const float (&o)[8
 
 __device__ __forceinline__ float sigmoidf(float r) { return 1.f / (1.f + __expf(-r)); }
 
-template <typename TI, typename TO, int LPR>
+// TA: type of o (the GLA output: input storage type when it comes from memory written by a caller, output
+// storage type when it comes straight from the forward pass), TR: type of r, TZ: type of z.  o and z may
+// be the same buffer: a lane reads its values of a row before it writes them.
+template <typename TA, typename TR, typename TZ, int LPR>
 __global__ void __launch_bounds__(kThreads)
-outgate_fwd(const TI *__restrict__ o, const TI *__restrict__ r, const float *__restrict__ ln_w,
-            const float *__restrict__ ln_b, TO *__restrict__ z, long long rows, int dv, float eps)
+outgate_fwd(const TA *o, const TR *__restrict__ r, const float *__restrict__ ln_w,
+            const float *__restrict__ ln_b, TZ *z, long long rows, int dv, float eps)
 {
     constexpr int kRows = kThreads / LPR;
     const int lane = threadIdx.x % LPR, slot = threadIdx.x / LPR, col = lane * 8;
@@ -199,16 +202,22 @@ int grid_for(long long rows, int lpr)
     return (int)(need < kMaxCtas ? need : kMaxCtas);
 }
 
+template <typename TA, typename TR, typename TZ>
+void fwd_dispatch3(const void *o, const void *r, const float *w, const float *b, void *z, long long rows, int dv,
+                   float eps, cudaStream_t stream)
+{
+    if (dv <= 64)
+        launch_pdl(outgate_fwd<TA, TR, TZ, 8>, dim3(grid_for(rows, 8)), dim3(kThreads), 0, stream, (const TA *)o,
+                   (const TR *)r, w, b, (TZ *)z, rows, dv, eps);
+    else
+        launch_pdl(outgate_fwd<TA, TR, TZ, 16>, dim3(grid_for(rows, 16)), dim3(kThreads), 0, stream, (const TA *)o,
+                   (const TR *)r, w, b, (TZ *)z, rows, dv, eps);
+}
 template <typename TI, typename TO>
 void fwd_dispatch(const void *o, const void *r, const float *w, const float *b, void *z, long long rows, int dv,
                   float eps, cudaStream_t stream)
 {
-    if (dv <= 64)
-        launch_pdl(outgate_fwd<TI, TO, 8>, dim3(grid_for(rows, 8)), dim3(kThreads), 0, stream, (const TI *)o,
-                   (const TI *)r, w, b, (TO *)z, rows, dv, eps);
-    else
-        launch_pdl(outgate_fwd<TI, TO, 16>, dim3(grid_for(rows, 16)), dim3(kThreads), 0, stream, (const TI *)o,
-                   (const TI *)r, w, b, (TO *)z, rows, dv, eps);
+    fwd_dispatch3<TI, TI, TO>(o, r, w, b, z, rows, dv, eps, stream);
 }
 
 template <typename TI, typename TO>
@@ -237,6 +246,17 @@ dig_status launch_outgate_fwd(const void *o, const void *r, const float *ln_w, c
     if (dtype == DIG_F32) fwd_dispatch<float, float>(o, r, ln_w, ln_b, z, rows, dv, eps, stream);
     else if (dtype == DIG_BF16) fwd_dispatch<__nv_bfloat16, __nv_bfloat16>(o, r, ln_w, ln_b, z, rows, dv, eps, stream);
     else fwd_dispatch<__nv_bfloat16, float>(o, r, ln_w, ln_b, z, rows, dv, eps, stream);
+    return cuda_ok(cudaGetLastError());
+}
+
+// o in the output storage type of `dtype` (as the forward pass writes it), r in the input storage type.
+dig_status launch_outgate_fwd_mixed(const void *o, const void *r, const float *ln_w, const float *ln_b, void *z,
+                                    long long rows, int dv, float eps, int dtype, cudaStream_t stream)
+{
+    KernelTimer t(KID_OUTGATE, stream);
+    if (dtype == DIG_F32) fwd_dispatch3<float, float, float>(o, r, ln_w, ln_b, z, rows, dv, eps, stream);
+    else if (dtype == DIG_BF16) fwd_dispatch3<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16>(o, r, ln_w, ln_b, z, rows, dv, eps, stream);
+    else fwd_dispatch3<float, __nv_bfloat16, float>(o, r, ln_w, ln_b, z, rows, dv, eps, stream);
     return cuda_ok(cudaGetLastError());
 }
 

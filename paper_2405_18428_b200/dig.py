@@ -24,7 +24,7 @@ DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR, DIG_IMPL_MMA = 0, 1, 2, 3
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
            "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_gla_fwd_state", "dig_gla_bwd_state",
-           "dig_gla_fwd_beta", "dig_gla_bwd_beta", "dig_gla_beta_workspace_bytes", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
+           "dig_gla_fwd_beta", "dig_gla_bwd_beta", "dig_gla_beta_workspace_bytes", "dig_gla_fwd_outgate", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
            "dig_srem_dwconv_bwd_workspace_bytes", "dig_gla_outgate_fwd", "dig_gla_outgate_bwd",
            "dig_gla_outgate_bwd_workspace_bytes", "dig_last_device_status",
            "dig_status_string", "dig_profile_enable", "dig_profile_kernels", "dig_profile_read")
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.dig_gla_fwd_static.restype = i
         L.dig_gla_bwd.argtypes = [vp] * 9 + [i] * 9 + [vp, sz, vp]
         L.dig_gla_bwd.restype = i
+        L.dig_gla_fwd_outgate.argtypes = [vp] * 7 + [ctypes.c_float, vp, vp] + [i] * 9 + [vp, sz, vp]
+        L.dig_gla_fwd_outgate.restype = i
         L.dig_gla_beta_workspace_bytes.argtypes = [i] * 9
         L.dig_gla_beta_workspace_bytes.restype = sz
         L.dig_gla_fwd_beta.argtypes = [vp] * 6 + [i] * 9 + [vp, sz, vp]
@@ -430,3 +432,24 @@ def dig_gla_bwd_beta(q, k, v, gate, bgate, d_out, grid_h, grid_w, chunk=64, dire
                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
            "dig_gla_bwd_beta")
     return dq, dk_, dv_, dgate, dbgate
+
+
+def dig_gla_fwd_outgate(q, k, v, gate, r, grid_h, grid_w, chunk=64, direction=DIG_ROW_FWD, *, ln_w=None, ln_b=None,
+                        eps=1e-5, f32_out=False, want_out=True, workspace=None):
+    """dig_gla_fwd and the output gate z = Swish(r) * LN(out) in one call; returns (out or None, z)."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st, ost = _storage(dtype), _out_storage(dtype)
+    out = torch.empty((B, L, H, dv), dtype=ost, device=q.device) if want_out else None
+    z = torch.empty((B, L, H, dv), dtype=ost, device=q.device)
+    need = dig_gla_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 0)
+    workspace = _workspace(workspace, need, q.device)
+    _check(lib().dig_gla_fwd_outgate(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"), _dev(v, st, (B, L, H, dv), "v"),
+                                     _dev(gate, torch.float32, q.shape, "gate"), _dev(r, st, v.shape, "r"),
+                                     _affine(ln_w, dv, "ln_w"), _affine(ln_b, dv, "ln_b"), float(eps),
+                                     None if out is None else out.data_ptr(), z.data_ptr(),
+                                     B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
+                                     workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "dig_gla_fwd_outgate")
+    return out, z
