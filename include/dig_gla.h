@@ -196,9 +196,8 @@ dig_status dig_gla_bwd_state(const void *q, const void *k, const void *v, const 
 /* dig_gla_fwd followed by the output gate of the layer, z = Swish(r) * LN(out) (dig_gla_outgate_fwd),
  * in one call.  r: gate pre-activation [B][L][H][d_v] in the input storage type of `dtype`; ln_w, ln_b:
  * fp32 [d_v] or NULL; z: [B][L][H][d_v] in the output storage type; `out` may be NULL when only z is
- * wanted.  LN sees `out` as it is stored (rounded to bf16 for DIG_BF16).  With the tcgen05 kernels the
- * gate is applied while the readout kernel stores its rows, so `out` is not read back; the other
- * families run the two steps one after the other.  Workspace as for dig_gla_fwd. */
+ * wanted (z then serves as the intermediate buffer).  LN sees `out` as it is stored (rounded to bf16 for
+ * DIG_BF16).  The two steps run one after the other on the stream.  Workspace as for dig_gla_fwd. */
 dig_status dig_gla_fwd_outgate(const void *q, const void *k, const void *v, const float *gate, const void *r,
                                const float *ln_w, const float *ln_b, float eps, void *out, void *z, int B, int H,
                                int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,

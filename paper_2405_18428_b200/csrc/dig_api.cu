@@ -324,15 +324,10 @@ dig_status dig_gla_fwd_outgate(const void *q, const void *k, const void *v, cons
     a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
     a.dtype = dtype;
     a.stream = (cudaStream_t)cuda_stream;
-    if (impl == DIG_IMPL_TENSOR) {          // the readout kernel applies the gate while it stores
-        a.out = out;
-        a.og.r = r; a.og.ln_w = ln_w; a.og.ln_b = ln_b; a.og.eps = eps; a.og.z = z;
-        return tensor_gla_fwd(a);
-    }
-    // other families: the plain forward pass (into z when the caller does not want `out`), then the
-    // gate kernel, which may work in place
+    // the plain forward pass (into z when the caller does not want `out`), then the gate kernel, which may
+    // work in place
     a.out = out ? out : z;
-    const dig_status st = impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
+    const dig_status st = impl == DIG_IMPL_TENSOR ? tensor_gla_fwd(a) : impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
     if (st != DIG_OK) return st;
     return launch_outgate_fwd_mixed(a.out, r, ln_w, ln_b, z, (long long)B * grid_h * grid_w * H, d_v, eps, dtype, a.stream);
 }

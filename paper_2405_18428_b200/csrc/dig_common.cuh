@@ -73,20 +73,9 @@ struct BetaIO {
     float *dbgate;
 };
 
-// Arguments of the forward pass with the output gate applied on the way out (all null otherwise):
-// gate pre-activation r [B][L][H][d_v] in the input storage type, LayerNorm weight / bias (fp32 [d_v] or
-// null), eps, and z = Swish(r) * LN(out) in the output storage type.  `out` itself may then be null.
-struct OutGateIO {
-    const void *r;
-    const float *ln_w, *ln_b;
-    float eps;
-    void *z;
-};
-
 struct GlaArgs {
     StateIO sio;
     BetaIO bio;
-    OutGateIO og;
     const void *q, *k, *v;
     const float *gate;
     void *out;                   // forward

@@ -62,40 +62,11 @@ __device__ __forceinline__ void fetch_states(char *tS, const float *states, int 
     }
 }
 
-// 16 staged bytes as floats (8 bf16 or 4 fp32), the matching loads of the gate pre-activation (always
-// bf16 in memory) and the stores of the gated result.
-__device__ __forceinline__ void unpack_staged(const uint4 &u, float (&x)[8]) { unpack8(u, x); }
-__device__ __forceinline__ void unpack_staged(const uint4 &u, float (&x)[4])
-{
-    x[0] = __uint_as_float(u.x); x[1] = __uint_as_float(u.y); x[2] = __uint_as_float(u.z); x[3] = __uint_as_float(u.w);
-}
-__device__ __forceinline__ void load_gate_pre(const bf16 *p, float (&x)[8]) { unpack8(ldg16(p), x); }
-__device__ __forceinline__ void load_gate_pre(const bf16 *p, float (&x)[4])
-{
-    const uint2 u = __ldg(reinterpret_cast<const uint2 *>(p));
-    x[0] = __uint_as_float(u.x << 16); x[1] = __uint_as_float(u.x & 0xffff0000u);
-    x[2] = __uint_as_float(u.y << 16); x[3] = __uint_as_float(u.y & 0xffff0000u);
-}
-__device__ __forceinline__ void store_z(bf16 *p, const float (&z)[8])
-{
-    uint4 u;
-    __nv_bfloat162 t;
-    t = __floats2bfloat162_rn(z[0], z[1]); u.x = *reinterpret_cast<uint32_t *>(&t);
-    t = __floats2bfloat162_rn(z[2], z[3]); u.y = *reinterpret_cast<uint32_t *>(&t);
-    t = __floats2bfloat162_rn(z[4], z[5]); u.z = *reinterpret_cast<uint32_t *>(&t);
-    t = __floats2bfloat162_rn(z[6], z[7]); u.w = *reinterpret_cast<uint32_t *>(&t);
-    *reinterpret_cast<uint4 *>(p) = u;
-}
-__device__ __forceinline__ void store_z(float *p, const float (&z)[4]) { *reinterpret_cast<float4 *>(p) = make_float4(z[0], z[1], z[2], z[3]); }
-
-// GATE: the staged rows pass through the output gate of the layer on their way out,
-// z = Swish(r) * LN(row) (Eq. attn_gla), computed by the 8 or 16 lanes that store one row; `out` is
-// written too unless it is null.
-template <typename TO, bool GATE>
+template <typename TO>
 __global__ void __launch_bounds__(NTA)
 tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *__restrict__ v,
             const float *__restrict__ gate, const float *__restrict__ states, TO *__restrict__ out,
-            OutGateIO og, int *status, Geom g)
+            int *status, Geom g)
 {
     extern __shared__ char smem_raw[];
     char *base = align1024(smem_raw);
@@ -227,45 +198,9 @@ tc_out_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *
                     const int u = threadIdx.x + NT * i, rr = u / PER_ROW, piece = u % PER_ROW;
                     const Item it = pick(cur[0], cur[1], rr >> 6);
                     const int tr = item_token(g, it, rr & 63);
-                    const uint4 staged = *reinterpret_cast<const uint4 *>(stage + rr * kOutPitch + piece * 16);
-                    const size_t tok = tok_offset(g, it.b, tr < 0 ? 0 : tr, it.h, DV);
-                    if (!GATE || out != nullptr) {
-                        if (tr >= 0) *reinterpret_cast<uint4 *>(reinterpret_cast<char *>(out) + tok * sizeof(TO) + piece * 16) = staged;
-                    }
-                    if (GATE) {
-                        // the PER_ROW consecutive lanes of a row hold it completely: statistics by shuffles
-                        // (every lane takes part, rows past the end of the sequence compute on zeros)
-                        constexpr int NV = 16 / (int)sizeof(TO);
-                        float x[NV];
-                        unpack_staged(staged, x);
-                        float sum = 0.f;
-#pragma unroll
-                        for (int e = 0; e < NV; ++e) sum += x[e];
-#pragma unroll
-                        for (int m = PER_ROW / 2; m >= 1; m >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, m);
-                        const float mean = sum * (1.f / 64.f);
-                        float var = 0.f;
-#pragma unroll
-                        for (int e = 0; e < NV; ++e) {
-                            x[e] -= mean;
-                            var = fmaf(x[e], x[e], var);
-                        }
-#pragma unroll
-                        for (int m = PER_ROW / 2; m >= 1; m >>= 1) var += __shfl_xor_sync(0xffffffffu, var, m);
-                        const float rstd = rsqrtf(var * (1.f / 64.f) + og.eps);
-                        if (tr >= 0) {
-                            const int c = piece * NV;
-                            float rv[NV], zz[NV];
-                            load_gate_pre(reinterpret_cast<const bf16 *>(og.r) + tok + c, rv);
-#pragma unroll
-                            for (int e = 0; e < NV; ++e) {
-                                const float wv = og.ln_w != nullptr ? og.ln_w[c + e] : 1.f;
-                                const float bv = og.ln_b != nullptr ? og.ln_b[c + e] : 0.f;
-                                zz[e] = rv[e] / (1.f + __expf(-rv[e])) * fmaf(x[e] * rstd, wv, bv);
-                            }
-                            store_z(reinterpret_cast<TO *>(og.z) + tok + c, zz);
-                        }
-                    }
+                    if (tr >= 0)
+                        *reinterpret_cast<uint4 *>(reinterpret_cast<char *>(out) + tok_offset(g, it.b, tr, it.h, DV) * sizeof(TO) + piece * 16) =
+                            *reinterpret_cast<const uint4 *>(stage + rr * kOutPitch + piece * 16);
                 }
             }
         }
@@ -282,18 +217,18 @@ constexpr size_t out_smem()
     return 1024 + 4 * (size_t)kTileK + kTileM + sizeof(float) * (2 * T * kLamPitch + 128 + NT) + sizeof(Control);
 }
 
-template <typename TO, bool GATE>
+template <typename TO>
 dig_status launch_typed(const GlaArgs &a, const Workspace &w, int sm_count, int *status)
 {
     const Geom &g = a.g;
     const int total = g.B * g.H * g.N, npairs = (total + 1) / 2;
-    auto kern = tc_out_pair<TO, GATE>;
+    auto kern = tc_out_pair<TO>;
     constexpr size_t smem = out_smem();
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
     const int grid = npairs < sm_count ? npairs : sm_count;
     KernelTimer t(KID_TC_OUT, a.stream);
     launch_pdl(kern, dim3(grid), dim3(NTA), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
-               a.gate, (const float *)w.states, (TO *)a.out, a.og, status, g);
+               a.gate, (const float *)w.states, (TO *)a.out, status, g);
     return cuda_ok(cudaGetLastError());
 }
 
@@ -301,9 +236,7 @@ dig_status launch_typed(const GlaArgs &a, const Workspace &w, int sm_count, int 
 
 dig_status launch_tc_out(const GlaArgs &a, const Workspace &w, int sm_count, int *status)
 {
-    if (a.og.z != nullptr)
-        return a.dtype == DIG_BF16 ? launch_typed<bf16, true>(a, w, sm_count, status) : launch_typed<float, true>(a, w, sm_count, status);
-    return a.dtype == DIG_BF16 ? launch_typed<bf16, false>(a, w, sm_count, status) : launch_typed<float, false>(a, w, sm_count, status);
+    return a.dtype == DIG_BF16 ? launch_typed<bf16>(a, w, sm_count, status) : launch_typed<float>(a, w, sm_count, status);
 }
 
 }  // namespace dig

@@ -88,9 +88,8 @@ def test_outgate_argument_checks():
 @pytest.mark.parametrize("d,chunk,direction", [(64, 64, 0), (64, 64, 3), (72, 64, 2), (64, 32, 1)])
 @pytest.mark.parametrize("f32_out", [True, False])
 def test_fwd_outgate_one_call(d, chunk, direction, f32_out):
-    """tcgen05 family: the readout kernel applies the gate while storing; other families: two steps inside
-    the call.  Against the oracle (recurrence, then gate, on the stored form of the outputs) and against
-    the two public calls made one after the other."""
+    """Against the oracle (recurrence, then gate, on the stored form of the outputs) and against the two
+    public calls made one after the other, on every kernel family."""
     from paper_2405_18428_b200 import dig
     from paper_2405_18428_b200.inputs import Workload, make_inputs
     from parity import TOL_BF16, to_dev
