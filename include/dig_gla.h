@@ -51,10 +51,9 @@ typedef enum { DIG_ROW_FWD = 0, DIG_ROW_REV = 1, DIG_COL_FWD = 2, DIG_COL_REV = 
  * cover the request (bf16 storage, d_k = d_v = 64, chunks of 64 or 128), else the warp-level
  * tensor-core kernels (MMA: bf16 storage, any supported head and chunk size that fits shared
  * memory), else the fp32-FMA kernels (fp32 storage, whose products must be fp32-accurate).  Forcing
- * a family that does not cover the request returns DIG_ERR_UNSUPPORTED.  TENSOR_TF32 forces TENSOR and
- * switches off its fp16 operand path (the gradient kernel then always multiplies in tf32); any other
- * value switches it back on.  Process-wide; meant for tests and benchmarks. */
-typedef enum { DIG_IMPL_AUTO = 0, DIG_IMPL_FMA = 1, DIG_IMPL_TENSOR = 2, DIG_IMPL_MMA = 3, DIG_IMPL_TENSOR_TF32 = 4 } dig_impl;
+ * a family that does not cover the request returns DIG_ERR_UNSUPPORTED.  Process-wide; meant for
+ * tests and benchmarks. */
+typedef enum { DIG_IMPL_AUTO = 0, DIG_IMPL_FMA = 1, DIG_IMPL_TENSOR = 2, DIG_IMPL_MMA = 3 } dig_impl;
 dig_status dig_set_impl(int impl);
 /* The family the next call with these parameters would use (DIG_IMPL_FMA, _TENSOR or _MMA),
  * or a negative dig_status if no family covers it. */

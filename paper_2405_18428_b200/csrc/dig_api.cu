@@ -81,7 +81,7 @@ const char *const kKernelNames[KID_COUNT] = {
     "gate_logsigmoid", "srem_dwconv3x3", "srem_dwconv_wgrad", "gla_outgate", "state_scan_fwd", "state_scan_bwd",
     "fma_chunk_state", "fma_chunk_out", "fma_chunk_bwd",
     "mma_chunk_state", "mma_chunk_out", "mma_chunk_bwd",
-    "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd", "tc_chunk_bwd_fp16"};
+    "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd"};
 struct Profile {
     bool on = false;
     std::vector<cudaEvent_t> ev;      // 2 per timed launch, created lazily and reused
@@ -139,10 +139,8 @@ extern "C" {
 
 dig_status dig_set_impl(int impl)
 {
-    if (impl < DIG_IMPL_AUTO || impl > DIG_IMPL_TENSOR_TF32) return DIG_ERR_INVALID_ARG;
-    // TENSOR_TF32 is the tcgen05 family with its fp16 operand path switched off
-    tensor_set_half_path(impl != DIG_IMPL_TENSOR_TF32);
-    g_impl.store(impl == DIG_IMPL_TENSOR_TF32 ? DIG_IMPL_TENSOR : impl);
+    if (impl < DIG_IMPL_AUTO || impl > DIG_IMPL_MMA) return DIG_ERR_INVALID_ARG;
+    g_impl.store(impl);
     return DIG_OK;
 }
 

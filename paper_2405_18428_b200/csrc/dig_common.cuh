@@ -97,8 +97,6 @@ struct GlaArgs {
 //                              operand-tile order (used by the tensor-core family only)
 struct Workspace {
     float *states, *gamma, *dstates, *carry, *dstates_m, *sfinal;
-    void *states_h, *dstates_h;      // fp16 copies of the scaled states for the fp16 operand path (64-wide heads)
-    int *flags;                      // range flags that select the fp16 or the tf32 gradient kernel
     size_t bytes;
 };
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -119,12 +117,6 @@ inline Workspace carve_workspace(float *base, const Geom &g, bool backward)
         const size_t fin = align256(bh * g.dk * g.dv * sizeof(float));
         w.sfinal = reinterpret_cast<float *>(p);        p += fin;
         w.bytes += 2 * st + gm + fin;
-        if (g.dk == 64 && g.dv == 64) {
-            w.states_h = p;                             p += st / 2;
-            w.dstates_h = p;                            p += st / 2;
-            w.flags = reinterpret_cast<int *>(p);       p += 256;
-            w.bytes += st + 256;
-        }
     }
     return w;
 }
@@ -140,8 +132,6 @@ size_t mma_beta_workspace_bytes(const Geom &g, bool backward);
 dig_status tensor_gla_fwd(const GlaArgs &a);
 dig_status tensor_gla_bwd(const GlaArgs &a);
 bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward);
-void tensor_set_half_path(bool on);
-void tensor_set_half_path(bool on);
 
 // Chunk-state scans, shared by both families (plain fp32 FMA, bandwidth-bound).
 // `tiles`: the states are stored transposed, in swizzled operand-tile order (tensor-core forward pass).
@@ -171,7 +161,7 @@ enum KernelId {
     KID_GATE = 0, KID_DWCONV, KID_DWCONV_WGRAD, KID_OUTGATE, KID_SCAN_FWD, KID_SCAN_BWD,
     KID_FMA_STATE, KID_FMA_OUT, KID_FMA_BWD,
     KID_MMA_STATE, KID_MMA_OUT, KID_MMA_BWD,
-    KID_TC_STATE, KID_TC_OUT, KID_TC_BWD, KID_TC_BWD_H,
+    KID_TC_STATE, KID_TC_OUT, KID_TC_BWD,
     KID_COUNT
 };
 struct KernelTimer {

@@ -16,15 +16,6 @@
 // gate rows of the next chunk are prefetched into registers.  A seventeenth warp issues the MMAs
 // and the bulk copies, so the tensor pipe runs while the other warps build operands.  Results are
 // staged in shared memory and leave with coalesced 16-byte stores.
-//
-// HALF = true is the same kernel with fp16 operands (kind::f16; 11 significant bits like tf32): one
-// 8 KB tile per operand serves both orientations, tile builds and MMA steps halve.  To stay inside
-// fp16's range the decay is referred to the middle of the chunk: with c = Lam_C / 2 per channel the
-// tiles hold q*exp(Lam-c), k*exp(c-Lam), sqrt(gamma)*S and sqrt(gamma)*D (the scan kernel writes the
-// last two as fp16 tiles), the accumulators are rescaled by exp(Lam-c) / exp(c-Lam), and nothing else
-// changes.  It runs when the range flags left by the earlier kernels allow it; otherwise it returns at
-// once and the tf32 instance, launched right after it, does the work (and returns at once when the
-// flags are good).
 #include "tc_tiles.cuh"
 
 namespace dig {
@@ -70,42 +61,28 @@ __device__ __forceinline__ void fetch_states(char *tSk, char *tDk, char *tDm, co
     bulk_g2s(tDm, dstates_m + (size_t)id * (DK * DV), kTile, bar);
 }
 
-__device__ __forceinline__ void fetch_states_h(char *tS, char *tD, const __half *states_h, const __half *dstates_h, int id,
-                                               uint64_t *bar)
-{
-    fence_async_smem();
-    mbar_arrive_expect_tx(bar, 2u * kTileH);
-    bulk_g2s(tS, states_h + (size_t)id * (DK * DV), kTileH, bar);
-    bulk_g2s(tD, dstates_h + (size_t)id * (DK * DV), kTileH, bar);
-}
-
-template <typename TO, bool HALF>
-__global__ void __launch_bounds__(NTA, HALF ? 2 : 1)
+template <typename TO>
+__global__ void __launch_bounds__(NTA)
 tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *__restrict__ v,
              const float *__restrict__ gate, const bf16 *__restrict__ d_out, const float *__restrict__ states,
              const float *__restrict__ dstates, const float *__restrict__ dstates_m, const float *__restrict__ carry,
-             const __half *__restrict__ states_h, const __half *__restrict__ dstates_h, const int *__restrict__ flags,
              TO *__restrict__ dq,
              TO *__restrict__ dk, TO *__restrict__ dv, float *__restrict__ dgate, int *status, Geom g)
 {
     extern __shared__ char smem_raw[];
     char *base = align1024(smem_raw);
-    constexpr int kOutPitch = 64 * (int)sizeof(TO) + 16, kOutStage = T * kOutPitch;
-    // tf32: K-format tiles Q K V G S D, then M-format tiles Q K G D.  fp16: one tile each of Q K V G S D.
-    constexpr int kT = HALF ? kTileH : kTile;
-    // (fp16: the six tiles are all live or being refilled while results are staged, so staging gets its own space)
-    constexpr int kTilesBytes = HALF ? 6 * kTileH + ((3 * kOutStage + 1023) / 1024) * 1024 : 10 * kTile;
-    char *tQk = base + 0 * kT, *tKk = base + 1 * kT, *tVk = base + 2 * kT, *tGk = base + 3 * kT;
-    char *tSk = base + 4 * kT, *tDk = base + 5 * kT;
-    char *tQm = HALF ? tQk : base + 6 * kTile, *tKm = HALF ? tKk : base + 7 * kTile, *tGm = HALF ? tGk : base + 8 * kTile;
-    char *tDm = HALF ? tDk : base + 9 * kTile;
+    // K-format tiles
+    char *tQk = base + 0 * kTile, *tKk = base + 1 * kTile, *tVk = base + 2 * kTile, *tGk = base + 3 * kTile;
+    char *tSk = base + 4 * kTile, *tDk = base + 5 * kTile;
+    // M-format tiles
+    char *tQm = base + 6 * kTile, *tKm = base + 7 * kTile, *tGm = base + 8 * kTile, *tDm = base + 9 * kTile;
     // written after the first group of products has completed, over tiles that group has finished with
-    // (fp16: the scores go over S, which only the first group reads; Q is still needed)
-    char *tPm = HALF ? tSk : tQk, *tdPk = tVk, *tdPm = HALF ? tVk : tSk;
-    // tf32: results are staged over tiles 0-3 once every product has completed
-    static_assert(HALF || 3 * kOutStage <= 4 * kTile, "output staging must fit in the four tiles it reuses");
-    char *stage = HALF ? base + 6 * kTileH : base;
-    float *sLamBuf = reinterpret_cast<float *>(base + kTilesBytes);         // gate table, later q*dq - k*dk and the gate gradient
+    char *tPm = tQk, *tdPk = tVk, *tdPm = tSk;
+    // results are staged over tiles 0-3 once every product has completed
+    constexpr int kOutPitch = 64 * (int)sizeof(TO) + 16, kOutStage = T * kOutPitch;
+    static_assert(3 * kOutStage <= 4 * kTile, "output staging must fit in the four tiles it reuses");
+    char *stage = base;
+    float *sLamBuf = reinterpret_cast<float *>(base + 10 * kTile);          // gate table, later q*dq - k*dk and the gate gradient
     float *sLast = sLamBuf + T * kLamPitch, *sTot = sLast + 64;
     Control *ctl = reinterpret_cast<Control *>(sTot + NT);
     uint64_t *barA = &ctl->bar[0], *barB = &ctl->bar[1], *barS = &ctl->bar[2];
@@ -127,13 +104,7 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
     if (id < total && !issuer) load_raw(raw, q, k, v, d_out, gate, g, it);
     pdl_wait();
     pdl_launch_dependents();          // only once this kernel's own predecessor has completed
-    // one of the two instances does the work: the fp16 one inside fp16's range, the tf32 one otherwise
-    const bool mine = flags == nullptr || half_range_ok(flags) == HALF;
-    if (!mine) id = total;
-    if (id < total && issuer && lane == 0) {
-        if constexpr (HALF) fetch_states_h(tSk, tDk, states_h, dstates_h, id, barS);
-        else fetch_states(tSk, tDk, tDm, states, dstates, dstates_m, id, barS);
-    }
+    if (id < total && issuer && lane == 0) fetch_states(tSk, tDk, tDm, states, dstates, dstates_m, id, barS);
     uint32_t parity = 0;
     bool ok = true;
     for (; id < total; id += gridDim.x) {
@@ -148,18 +119,11 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
             carry_in = __ldg(carry + (size_t)id * DK + (threadIdx.x & 63));
             sync_group(NT);              // the previous chunk's results have left the staging area
             float x[8];
-            if constexpr (HALF) {
-                unpack8(raw.v, x, keep);
-                st_h8(tVk, row, col, x);
-                unpack8(raw.d, x, keep);
-                st_h8(tGk, row, col, x);
-            } else {
-                unpack8(raw.v, x, keep, flip);
-                st_k8<T, false>(tVk, row, col, x, flip);
-                unpack8(raw.d, x, keep, flip);
-                st_k8<T, false>(tGk, row, col, x, flip);
-                st_m8<T, false>(tGm, row, col, x, flip);
-            }
+            unpack8(raw.v, x, keep, flip);
+            st_k8<T, false>(tVk, row, col, x, flip);
+            unpack8(raw.d, x, keep, flip);
+            st_k8<T, false>(tGk, row, col, x, flip);
+            st_m8<T, false>(tGm, row, col, x, flip);
             fence_async_smem();
         }
         tc_fence_before_sync();
@@ -169,15 +133,9 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
                 // products of operands that need no gate: they run while the other warps build Qt and Kt
                 ok = mbar_wait(barS, parity, status);      // S, Dg (both tile orders) have landed
                 tc_fence_after_sync();
-                if constexpr (HALF) {
-                    issue_h<false, false>(tmem + aQK, kdesc_h(tGk), kdesc_h(tSk), false);                       // dO S^T
-                    issue_h<false, false>(tmem + aQK + kUpper, kdesc_h(tVk), kdesc_h(tDk), false);              // V Dg^T
-                    issue_h<false, false>(tmem + aP + kUpper, kdesc_h(tGk), kdesc_h(tVk), false);               // dO V^T
-                } else {
-                    issue<64, 64, false, false, T, T>(tmem + aQK, kdesc<T>(tGk), kdesc<T>(tSk), false);             // dO S^T
-                    issue<64, 64, false, false, T, T>(tmem + aQK + kUpper, kdesc<T>(tVk), kdesc<T>(tDk), false);    // V Dg^T
-                    issue<64, 64, false, false, T, T>(tmem + aP + kUpper, kdesc<T>(tGk), kdesc<T>(tVk), false);     // dO V^T
-                }
+                issue<64, 64, false, false, T, T>(tmem + aQK, kdesc<T>(tGk), kdesc<T>(tSk), false);             // dO S^T
+                issue<64, 64, false, false, T, T>(tmem + aQK + kUpper, kdesc<T>(tVk), kdesc<T>(tDk), false);    // V Dg^T
+                issue<64, 64, false, false, T, T>(tmem + aP + kUpper, kdesc<T>(tGk), kdesc<T>(tVk), false);     // dO V^T
             }
         } else {
             {
@@ -190,35 +148,17 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
             sync_group(NT);
             gate_prefix<NT, 1, true>(sLam, sLast, sTot);
             float lam[8], x[8];
-            if constexpr (HALF) {
-                // decay referred to the middle of the chunk: lam - Lam_C / 2 lies in [Lam_C / 2, -Lam_C / 2]
-                float half_tot[8];
-                read_lam8(sLam, row, col, lam);
-                read_lam8(sLast, 0, col, half_tot);
-                unpack8(raw.q, x, keep);
+            read_lam8(sLam, row, col, lam, flip);
+            unpack8(raw.q, x, keep, flip);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    lam[e] -= 0.5f * half_tot[e];
-                    x[e] *= ex2(lam[e]);
-                }
-                st_h8(tQk, row, col, x);
-                unpack8(raw.k, x, keep);
+            for (int e = 0; e < 8; ++e) x[e] = to_tf32(x[e] * ex2(lam[e]));
+            st_k8<T, false>(tQk, row, col, x, flip);
+            st_m8<T, false>(tQm, row, col, x, flip);
+            unpack8(raw.k, x, keep, flip);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) x[e] *= ex2(-lam[e]);
-                st_h8(tKk, row, col, x);
-            } else {
-                read_lam8(sLam, row, col, lam, flip);
-                unpack8(raw.q, x, keep, flip);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) x[e] = to_tf32(x[e] * ex2(lam[e]));
-                st_k8<T, false>(tQk, row, col, x, flip);
-                st_m8<T, false>(tQm, row, col, x, flip);
-                unpack8(raw.k, x, keep, flip);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) x[e] = to_tf32(x[e] * ex2(-lam[e]));
-                st_k8<T, false>(tKk, row, col, x, flip);
-                st_m8<T, false>(tKm, row, col, x, flip);
-            }
+            for (int e = 0; e < 8; ++e) x[e] = to_tf32(x[e] * ex2(-lam[e]));
+            st_k8<T, false>(tKk, row, col, x, flip);
+            st_m8<T, false>(tKm, row, col, x, flip);
             fence_async_smem();
         }
         tc_fence_before_sync();
@@ -226,15 +166,9 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
         if (issuer) {
             if (lane == 0) {
                 tc_fence_after_sync();
-                if constexpr (HALF) {
-                    issue_h<false, false>(tmem + aP, kdesc_h(tQk), kdesc_h(tKk), false);                        // Qt Kt^T
-                    mma_commit(barA);
-                    issue_h<false, true>(tmem + aV, kdesc_h(tKk), mdesc_h(tDk), false);                         // Kt Dg
-                } else {
-                    issue<64, 64, false, false, T, T>(tmem + aP, kdesc<T>(tQk), kdesc<T>(tKk), false);              // Qt Kt^T
-                    mma_commit(barA);
-                    issue<64, 64, false, true, T, T>(tmem + aV, kdesc<T>(tKk), mdesc<T>(tDm), false);               // Kt Dg
-                }
+                issue<64, 64, false, false, T, T>(tmem + aP, kdesc<T>(tQk), kdesc<T>(tKk), false);              // Qt Kt^T
+                mma_commit(barA);
+                issue<64, 64, false, true, T, T>(tmem + aV, kdesc<T>(tKk), mdesc<T>(tDm), false);               // Kt Dg
             }
         } else {
             ok = mbar_wait(barA, parity, status);
@@ -244,17 +178,8 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
                 tmem_ld(tmem + lane_base + aP + (uint32_t)c0, p);       // lanes 0-15: scores, lanes 16-31: dO V^T
 #pragma unroll
                 for (int jj = 0; jj < W; ++jj)
-                    p[jj] = c0 + jj > arow ? 0.f : (HALF ? p[jj] : to_tf32(p[jj]));      // keep s <= t; the diagonal has weight 1
-                if constexpr (HALF) {
-                    char *dst = hf == 0 ? tPm : tdPk;                    // scores | dO V^T, one tile each
-                    float h8[8];
-#pragma unroll
-                    for (int jj = 0; jj < W / 8; ++jj) {
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) h8[e] = p[8 * jj + e];
-                        st_h8(dst, arow, c0 + 8 * jj, h8);
-                    }
-                } else if (hf == 0) {
+                    p[jj] = c0 + jj > arow ? 0.f : to_tf32(p[jj]);       // keep s <= t; the diagonal has weight 1
+                if (hf == 0) {
 #pragma unroll
                     for (int jj = 0; jj < W / 4; ++jj)
                         st_m4<T, false>(tPm, arow, c0 + 4 * jj, make_float4(p[4 * jj], p[4 * jj + 1], p[4 * jj + 2], p[4 * jj + 3]));
@@ -274,21 +199,12 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
         if (issuer) {
             if (lane == 0) {
                 tc_fence_after_sync();
-                if constexpr (HALF) {
-                    issue_h<false, true>(tmem + aQK, kdesc_h(tdPk), mdesc_h(tKm), true);                        // + dP Kt
-                    issue_h<true, true>(tmem + aQK + kUpper, mdesc_h(tdPm), mdesc_h(tQm), true);                // + dP^T Qt
-                    issue_h<true, true>(tmem + aV, mdesc_h(tPm), mdesc_h(tGm), true);                           // + P^T dO
-                } else {
-                    issue<64, 64, false, true, T, T>(tmem + aQK, kdesc<T>(tdPk), mdesc<T>(tKm), true);              // + dP Kt
-                    issue<64, 64, true, true, T, T>(tmem + aQK + kUpper, mdesc<T>(tdPm), mdesc<T>(tQm), true);      // + dP^T Qt
-                    issue<64, 64, true, true, T, T>(tmem + aV, mdesc<T>(tPm), mdesc<T>(tGm), true);                 // + P^T dO
-                }
+                issue<64, 64, false, true, T, T>(tmem + aQK, kdesc<T>(tdPk), mdesc<T>(tKm), true);              // + dP Kt
+                issue<64, 64, true, true, T, T>(tmem + aQK + kUpper, mdesc<T>(tdPm), mdesc<T>(tQm), true);      // + dP^T Qt
+                issue<64, 64, true, true, T, T>(tmem + aV, mdesc<T>(tPm), mdesc<T>(tGm), true);                 // + P^T dO
                 mma_commit(barB);
                 // once everything has completed the state tiles are free for the next chunk
-                if (mbar_wait(barB, parity, status) && next < total) {
-                    if constexpr (HALF) fetch_states_h(tSk, tDk, states_h, dstates_h, next, barS);
-                    else fetch_states(tSk, tDk, tDm, states, dstates, dstates_m, next, barS);
-                }
+                if (mbar_wait(barB, parity, status) && next < total) fetch_states(tSk, tDk, tDm, states, dstates, dstates_m, next, barS);
             }
         } else {
             // the tensor pipe is busy for a while: a good moment to start the next chunk's loads
@@ -301,21 +217,15 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
                 for (int jj = 0; jj < W / 4; ++jj) {
                     const float4 l4 = *reinterpret_cast<const float4 *>(sLam + arow * kLamPitch + c0 + 4 * jj);
                     lam[4 * jj] = l4.x; lam[4 * jj + 1] = l4.y; lam[4 * jj + 2] = l4.z; lam[4 * jj + 3] = l4.w;
-                    if constexpr (HALF) {            // the same reference point as in the operand tiles
-                        const float4 t4 = *reinterpret_cast<const float4 *>(sLast + c0 + 4 * jj);
-                        lam[4 * jj] -= 0.5f * t4.x; lam[4 * jj + 1] -= 0.5f * t4.y; lam[4 * jj + 2] -= 0.5f * t4.z; lam[4 * jj + 3] -= 0.5f * t4.w;
-                    }
                 }
                 tmem_ld(tmem + lane_base + aQK + (uint32_t)c0, a);      // lanes 0-15: dq part, lanes 16-31: dk part
                 {
                     // q*dq = Qt*(dq accumulator), k*dk = Kt*(dk accumulator): the decay factors cancel
                     float t8[8];
-                    if constexpr (HALF) ld_h8(hf == 0 ? tQm : tKm, arow, c0, t8);
-                    else ld_m8<T>(hf == 0 ? tQm : tKm, arow, c0, t8);
+                    ld_m8<T>(hf == 0 ? tQm : tKm, arow, c0, t8);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) x[e] = t8[e] * a[e];
-                    if constexpr (HALF) ld_h8(hf == 0 ? tQm : tKm, arow, c0 + 8, t8);
-                    else ld_m8<T>(hf == 0 ? tQm : tKm, arow, c0 + 8, t8);
+                    ld_m8<T>(hf == 0 ? tQm : tKm, arow, c0 + 8, t8);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) x[8 + e] = t8[e] * a[8 + e];
                 }
@@ -392,40 +302,25 @@ tc_chunk_bwd(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
     teardown(ctl, kCols);
 }
 
-template <typename TO, bool HALF>
 constexpr size_t bwd_smem()
 {
-    constexpr size_t stage = 3 * (size_t)T * (64 * sizeof(TO) + 16);
-    constexpr size_t tiles = HALF ? 6 * (size_t)kTileH + ((stage + 1023) / 1024) * 1024 : 10 * (size_t)kTile;
-    return 1024 + tiles + kLamBytes + sizeof(float) * (64 + NT) + sizeof(Control);
+    return 1024 + 10 * (size_t)kTile + kLamBytes + sizeof(float) * (64 + NT) + sizeof(Control);
 }
 
-template <typename TO, bool HALF>
-dig_status launch_one(const GlaArgs &a, const Workspace &w, int sm_count, int *status, const int *flags)
-{
-    const Geom &g = a.g;
-    const int total = g.B * g.H * g.N;
-    auto kern = tc_chunk_bwd<TO, HALF>;
-    constexpr size_t smem = bwd_smem<TO, HALF>();
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
-    const int ctas = (HALF ? 2 : 1) * sm_count;
-    const int grid = total < ctas ? total : ctas;
-    KernelTimer t(HALF ? KID_TC_BWD_H : KID_TC_BWD, a.stream);
-    launch_pdl(kern, dim3(grid), dim3(NTA), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
-               (const bf16 *)a.d_out, (const float *)w.states, (const float *)w.dstates, (const float *)w.dstates_m,
-               (const float *)w.carry, (const __half *)w.states_h, (const __half *)w.dstates_h, flags, (TO *)a.dq, (TO *)a.dk,
-               (TO *)a.dv, a.dgate, status, g);
-    return cuda_ok(cudaGetLastError());
-}
-
-// With range flags: the fp16 instance first, then the tf32 one; exactly one of them does the work.
 template <typename TO>
 dig_status launch_typed(const GlaArgs &a, const Workspace &w, int sm_count, int *status)
 {
-    if (w.flags == nullptr) return launch_one<TO, false>(a, w, sm_count, status, nullptr);
-    const dig_status st = launch_one<TO, true>(a, w, sm_count, status, w.flags);
-    if (st != DIG_OK) return st;
-    return launch_one<TO, false>(a, w, sm_count, status, w.flags);
+    const Geom &g = a.g;
+    const int total = g.B * g.H * g.N;
+    auto kern = tc_chunk_bwd<TO>;
+    constexpr size_t smem = bwd_smem();
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DIG_ERR_CUDA;
+    const int grid = total < sm_count ? total : sm_count;
+    KernelTimer t(KID_TC_BWD, a.stream);
+    launch_pdl(kern, dim3(grid), dim3(NTA), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
+               (const bf16 *)a.d_out, (const float *)w.states, (const float *)w.dstates, (const float *)w.dstates_m,
+               (const float *)w.carry, (TO *)a.dq, (TO *)a.dk, (TO *)a.dv, a.dgate, status, g);
+    return cuda_ok(cudaGetLastError());
 }
 
 }  // namespace

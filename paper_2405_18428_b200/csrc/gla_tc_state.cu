@@ -62,7 +62,7 @@ template <int NT, bool BWD>
 __global__ void __launch_bounds__(NT, BWD ? 1 : 2)
 tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 *__restrict__ v,
               const float *__restrict__ gate, const bf16 *__restrict__ d_out, float *__restrict__ states,
-              float *__restrict__ gamma, float *__restrict__ dstates, int *__restrict__ flags, int *status, Geom g)
+              float *__restrict__ gamma, float *__restrict__ dstates, int *status, Geom g)
 {
     constexpr int W = 64 / (NT / 128);        // accumulator columns per thread
     constexpr int NROW = StateRaw<NT, BWD>::NROW;
@@ -112,14 +112,6 @@ tc_state_pair(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16
         if (threadIdx.x < 128) {
             const int id = 2 * pair + (threadIdx.x >> 6);
             if (id < total) gamma[(size_t)id * DK + (threadIdx.x & 63)] = ex2(sLast[threadIdx.x]);
-            if (BWD && flags != nullptr) {
-                // range flag of the fp16 gradient kernel: the largest chunk total of the gates (log2 units)
-                float m = id < total ? fabsf(sLast[threadIdx.x]) : 0.f;
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-                if (!(m <= 3.0e38f)) m = 3.0e38f;
-                if ((threadIdx.x & 31) == 0) atomicMax(flags, __float_as_int(m));
-            }
         }
         // operands
 #pragma unroll
@@ -218,7 +210,7 @@ dig_status launch_tc_state(const GlaArgs &a, const Workspace &w, bool backward, 
         const int grid = npairs < sm_count ? npairs : sm_count;
         KernelTimer t(KID_TC_STATE, a.stream);
         launch_pdl(kern, dim3(grid), dim3(NT), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
-                   a.gate, (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, w.flags, status, g);
+                   a.gate, (const bf16 *)a.d_out, w.states, w.gamma, w.dstates, status, g);
     } else {
         constexpr int NT = 256;           // 100 KB of shared memory: two CTAs per SM overlap each other's phases
         auto kern = tc_state_pair<NT, false>;
@@ -227,7 +219,7 @@ dig_status launch_tc_state(const GlaArgs &a, const Workspace &w, bool backward, 
         const int grid = npairs < 2 * sm_count ? npairs : 2 * sm_count;
         KernelTimer t(KID_TC_STATE, a.stream);
         launch_pdl(kern, dim3(grid), dim3(NT), smem, a.stream, (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
-                   a.gate, (const bf16 *)nullptr, w.states, w.gamma, (float *)nullptr, (int *)nullptr, status, g);
+                   a.gate, (const bf16 *)nullptr, w.states, w.gamma, (float *)nullptr, status, g);
     }
     return cuda_ok(cudaGetLastError());
 }

@@ -37,25 +37,15 @@ dig_status tensor_gla_fwd(const GlaArgs &a)
     return launch_tc_out(a, w, sms, status);
 }
 
-// The fp16 operand path of the gradient kernel can be switched off (kernel-family switch of the API).
-static bool g_half_path = true;
-void tensor_set_half_path(bool on) { g_half_path = on; }
-
 dig_status tensor_gla_bwd(const GlaArgs &a)
 {
     const Geom &g = a.g;
-    Workspace w = carve_workspace(a.ws, g, true);
-    if (!g_half_path) {
-        w.flags = nullptr;
-        w.states_h = w.dstates_h = nullptr;
-    }
+    const Workspace w = carve_workspace(a.ws, g, true);
     int *status = device_status_ptr();
     const int sms = device_sm_count();
     if (!status || sms <= 0) return DIG_ERR_CUDA;
     if ((long long)g.B * g.H * g.N > (1ll << 30)) return DIG_ERR_UNSUPPORTED;
     dig_status st;
-    // the range flags start at zero; the state and scan kernels raise them
-    if (w.flags != nullptr && cudaMemsetAsync(w.flags, 0, 2 * sizeof(int), a.stream) != cudaSuccess) return DIG_ERR_CUDA;
     if ((st = launch_tc_state(a, w, true, sms, status)) != DIG_OK) return st;
     if ((st = launch_state_scan_bwd_tiles(w, g, a.stream, a.sio)) != DIG_OK) return st;
     return launch_tc_bwd(a, w, sms, status);

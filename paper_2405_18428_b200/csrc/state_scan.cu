@@ -10,8 +10,6 @@
 // Optional state arguments ([B*H][d_k][d_v] row-major fp32, null = zero / not wanted): the forward scan
 // starts from s_in and hands out the state after the last chunk; the backward scan starts from the
 // gradient with respect to that final state and hands out the gradient with respect to s_in.
-#include <cuda_fp16.h>
-
 #include "dig_common.cuh"
 
 namespace dig {
@@ -236,29 +234,11 @@ __device__ __forceinline__ float4 fma4(float g, float4 r, float4 u)
 __global__ void __launch_bounds__(64)
 state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, float *__restrict__ dstates_m,
                      const float *__restrict__ gamma, float *__restrict__ carry, const float *__restrict__ s_in,
-                     const float *__restrict__ ds_out, float *__restrict__ ds_in, __half *__restrict__ states_h,
-                     __half *__restrict__ dstates_h, int *__restrict__ flags, int N)
+                     const float *__restrict__ ds_out, float *__restrict__ ds_in, int N)
 {
     pdl_wait();
     pdl_launch_dependents();      // only once this kernel's own predecessor has completed
     const int t = threadIdx.x, c = 8 * blockIdx.x + (t >> 3);
-    // fp16 copies for the fp16 operand path (states_h != null): sqrt(gamma_i) S_[i] and sqrt(gamma_i) D_[i] as
-    // 64 x 64 fp16 tiles (128 bytes per row, 16-byte pieces XOR-ed with row & 7); this thread's logical columns
-    // 4*lp .. 4*lp+3 and 32 + 4*lp .. are 8 bytes each.  flags[1] collects the largest magnitude written.
-    const int lp_h = (t & 7) ^ (c & 7);
-    const size_t hoff0 = (size_t)c * 64 + ((((lp_h >> 1)) ^ (c & 7)) << 3) + ((lp_h & 1) << 2);
-    const size_t hoff1 = (size_t)c * 64 + (((4 + (lp_h >> 1)) ^ (c & 7)) << 3) + ((lp_h & 1) << 2);
-    __half *SH = states_h != nullptr ? states_h + (size_t)blockIdx.y * N * 4096 : nullptr;
-    __half *DH = states_h != nullptr ? dstates_h + (size_t)blockIdx.y * N * 4096 : nullptr;
-    float hmax = 0.f;
-    auto put_h = [&](__half *tile, float4 a, float4 b, float sc) {
-        const __half2 a0 = __floats2half2_rn(a.x * sc, a.y * sc), a1 = __floats2half2_rn(a.z * sc, a.w * sc);
-        const __half2 b0 = __floats2half2_rn(b.x * sc, b.y * sc), b1 = __floats2half2_rn(b.z * sc, b.w * sc);
-        *reinterpret_cast<uint2 *>(tile + hoff0) = make_uint2(*reinterpret_cast<const uint32_t *>(&a0), *reinterpret_cast<const uint32_t *>(&a1));
-        *reinterpret_cast<uint2 *>(tile + hoff1) = make_uint2(*reinterpret_cast<const uint32_t *>(&b0), *reinterpret_cast<const uint32_t *>(&b1));
-        hmax = fmaxf(hmax, sc * fmaxf(fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))),
-                                      fmaxf(fmaxf(fabsf(b.x), fabsf(b.y)), fmaxf(fabsf(b.z), fabsf(b.w)))));
-    };
     const size_t base = (size_t)blockIdx.y * N * 4096;
     float4 *S = reinterpret_cast<float4 *>(states + base) + c * 8 + (t & 7);
     float4 *D = reinterpret_cast<float4 *>(dstates + base) + c * 8 + (t & 7);
@@ -290,7 +270,6 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
             if (i + j < N) {
                 S[(size_t)(i + j) * 1024] = round4_tf32(r0);
                 S[(size_t)(i + j) * 1024 + 512] = round4_tf32(r1);
-                if (SH != nullptr) put_h(SH + (size_t)(i + j) * 4096, r0, r1, sqrtf(g[j]));
                 r0 = fma4(g[j], r0, u0[j]);
                 r1 = fma4(g[j], r1, u1[j]);
             }
@@ -331,7 +310,6 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
                 D[(size_t)ch * 1024 + 512] = e1;
                 DM[(size_t)ch * 1024] = e0;
                 DM[(size_t)ch * 1024 + 512] = e1;
-                if (DH != nullptr) put_h(DH + (size_t)ch * 4096, d0, d1, sqrtf(g[j]));
                 d0 = fma4(g[j], d0, w0[j]);
                 d1 = fma4(g[j], d1, w1[j]);
                 dot += __shfl_xor_sync(0xffffffffu, dot, 1);
@@ -344,13 +322,6 @@ state_scan_bwd_tiles(float *__restrict__ states, float *__restrict__ dstates, fl
     if (ds_in != nullptr) {
         *reinterpret_cast<float4 *>(ds_in + io) = d0;
         *reinterpret_cast<float4 *>(ds_in + io + 32) = d1;
-    }
-    if (flags != nullptr) {
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) hmax = fmaxf(hmax, __shfl_xor_sync(0xffffffffu, hmax, off));
-        // non-finite magnitudes must read as out of range: NaN would lose every comparison
-        if (!(hmax <= 3.0e38f)) hmax = 3.0e38f;
-        if ((t & 31) == 0) atomicMax(flags + 1, __float_as_int(hmax));
     }
 }
 
@@ -635,13 +606,12 @@ dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaSt
 {
     if (g.dk != 64 || g.dv != 64) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_SCAN_BWD, s);
-    if (g.B * g.H < 16 && w.flags == nullptr)      // few sequences (tf32 path only): the finer kernel with the deeper look-ahead
+    if (g.B * g.H < 16)      // few sequences: the finer kernel with the deeper look-ahead
         launch_pdl(state_scan_bwd_tiles1, dim3(64 / kTileRows, g.B * g.H), dim3(32 * kTileRows), 0, s, w.states, w.dstates,
                    w.dstates_m, (const float *)w.gamma, w.carry, sio.s_in, sio.ds_out, sio.ds_in, g.N);
     else
         launch_pdl(state_scan_bwd_tiles, dim3(8, g.B * g.H), dim3(64), 0, s, w.states, w.dstates, w.dstates_m,
-                   (const float *)w.gamma, w.carry, sio.s_in, sio.ds_out, sio.ds_in, (__half *)w.states_h, (__half *)w.dstates_h,
-                   w.flags, g.N);
+                   (const float *)w.gamma, w.carry, sio.s_in, sio.ds_out, sio.ds_in, g.N);
     return cuda_ok(cudaGetLastError());
 }
 

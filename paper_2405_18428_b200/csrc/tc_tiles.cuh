@@ -3,8 +3,6 @@
 // the in-chunk cumulative gate table, and lean tcgen05.mma issue loops.
 #pragma once
 
-#include <cuda_fp16.h>
-
 #include "dig_common.cuh"
 #include "umma.cuh"
 
@@ -214,51 +212,6 @@ __device__ __forceinline__ void issue(uint32_t d_tmem, uint64_t a0, uint64_t b0,
         const uint64_t db = b0 + (B_MN ? mstep(kk) : kstep<BROWS>(kk));
         mma_tf32(d_tmem, da, db, idesc, accumulate || kk > 0);
     }
-}
-
-// ---- fp16 operand tiles ------------------------------------------------------------------------
-// 64 rows x 64 halfs, 128 bytes per row, 16-byte pieces of a row XOR-ed with row & 7.  With 16-bit
-// operands one tile serves both orientations: read K-major (contraction along the row, 32 bytes per
-// 16-wide step) or MN-major (contraction down the rows, 16 rows = 2048 bytes per step).
-constexpr int kTileH = T * 128;
-__device__ __forceinline__ uint32_t pack_h2(float a, float b)
-{
-    const __half2 h = __floats2half2_rn(a, b);
-    return *reinterpret_cast<const uint32_t *>(&h);
-}
-__device__ __forceinline__ void st_h8(char *tile, int row, int col8, const float (&f)[8])
-{
-    *reinterpret_cast<uint4 *>(tile + row * 128 + (((col8 >> 3) ^ (row & 7)) << 4)) =
-        make_uint4(pack_h2(f[0], f[1]), pack_h2(f[2], f[3]), pack_h2(f[4], f[5]), pack_h2(f[6], f[7]));
-}
-__device__ __forceinline__ void ld_h8(const char *tile, int row, int col8, float (&f)[8])
-{
-    const uint4 u = *reinterpret_cast<const uint4 *>(tile + row * 128 + (((col8 >> 3) ^ (row & 7)) << 4));
-    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float2 v = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
-        f[2 * i] = v.x;
-        f[2 * i + 1] = v.y;
-    }
-}
-__device__ __forceinline__ uint64_t kdesc_h(const void *tile) { return make_desc(smem_u32(tile), 16, 1024, 2); }
-__device__ __forceinline__ uint64_t mdesc_h(const void *tile) { return make_desc(smem_u32(tile), 8192, 1024, 2); }
-// D[tmem] (+)= A * B for 64 x 64 x 64 fp16 tiles: four steps of 16 along the contraction.
-template <bool A_MN, bool B_MN>
-__device__ __forceinline__ void issue_h(uint32_t d_tmem, uint64_t a0, uint64_t b0, bool accumulate)
-{
-    constexpr uint32_t idesc = idesc_f16(64, 64, A_MN, B_MN);
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk)
-        mma_f16(d_tmem, a0 + (uint64_t)(kk * (A_MN ? 128 : 2)), b0 + (uint64_t)(kk * (B_MN ? 128 : 2)), idesc, accumulate || kk > 0);
-}
-// The fp16 operand path is taken when the decay inside a chunk and the states stay inside fp16's range:
-// flags[0] = bits of max |chunk total of the gate| (log2 units), flags[1] = bits of the largest scaled
-// state entry; both are non-negative floats, so their bit patterns order like the values.
-__device__ __forceinline__ bool half_range_ok(const int *flags)
-{
-    return __int_as_float(flags[0]) <= 23.0f && __int_as_float(flags[1]) <= 30000.0f;
 }
 
 __device__ __forceinline__ char *align1024(char *p)

@@ -20,7 +20,7 @@ DIG_ERR_SCRATCH_LIMIT = 6
 DIG_GLA_STATIC_SCRATCH_BYTES = 16 << 20
 DIG_F32, DIG_BF16, DIG_BF16_F32OUT = 0, 1, 2
 DIG_ROW_FWD, DIG_ROW_REV, DIG_COL_FWD, DIG_COL_REV = 0, 1, 2, 3
-DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR, DIG_IMPL_MMA, DIG_IMPL_TENSOR_TF32 = 0, 1, 2, 3, 4
+DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR, DIG_IMPL_MMA = 0, 1, 2, 3
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
            "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_gla_fwd_state", "dig_gla_bwd_state",

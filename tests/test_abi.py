@@ -40,11 +40,9 @@ def test_workspace_bytes(L):
     # forward: states [B*H][N][dk][dv] + gamma [B*H][N][dk], fp32, each block 256-byte aligned
     n = L.dig_gla_workspace_bytes(1, 6, 16, 16, 64, 64, 64, 0, 0)
     assert n == 6 * 4 * 64 * 64 * 4 + 6 * 4 * 64 * 4
-    # backward: + dstates, carry, a second copy of dstates in the other operand-tile order, the state
-    # after the last chunk [B*H][dk][dv] and, for 64-wide heads, fp16 copies of both state arrays plus a
-    # 256-byte block of range flags
-    st = 6 * 4 * 64 * 64 * 4
-    assert L.dig_gla_workspace_bytes(1, 6, 16, 16, 64, 64, 64, 0, 1) == 2 * n + st + 6 * 64 * 64 * 4 + st + 256
+    # backward: + dstates, carry, a second copy of dstates in the other operand-tile order and the
+    # state after the last chunk [B*H][dk][dv]
+    assert L.dig_gla_workspace_bytes(1, 6, 16, 16, 64, 64, 64, 0, 1) == 2 * n + 6 * 4 * 64 * 64 * 4 + 6 * 64 * 64 * 4
     # ragged tail: 10x10 = 100 tokens in chunks of 64 -> 2 chunks
     assert L.dig_gla_workspace_bytes(1, 1, 10, 10, 8, 8, 64, 1, 0) == 2 * 8 * 8 * 4 + 256
     for bad in [(0, 6, 16, 16, 64, 64, 64, 0, 0), (1, 6, 16, 16, 60, 64, 64, 0, 0),
