@@ -118,8 +118,8 @@ dig_status dig_gla_fwd_static(const void *q, const void *k, const void *v, const
  * (reverse-mode derivative of Eq. attn_gla; the paper trains through the operator but does not
  * print it).  Nothing is saved by the forward call: chunk states are recomputed here.
  *   d_out: [B][L][H][d_v]; dq, dk: [B][L][H][d_k]; dv: [B][L][H][d_v]; dgate: fp32 [B][L][H][d_k].
- * The fp32-FMA family covers chunk <= 64 here; chunk = 128 is served by the tensor-core family only
- * (bf16 storage, d_k = d_v = 64). */
+ * The fp32-FMA and warp-level families cover chunk <= 64 here (shared memory); chunk = 128 is served by
+ * the tcgen05 family only (bf16 storage, d_k = d_v = 64, 64-token tiles). */
 dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float *gate,
                        const void *d_out, void *dq, void *dk, void *dv, float *dgate,
                        int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
