@@ -123,22 +123,29 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
 // ---- reverse mode: filter and bias gradients ------------------------------------------------------
 // dw'[u][v][c] = sum over pixels of dy[i][j][c] * x[i+u-1][j+v-1][c] (zero outside the grid), computed
 // in canonical taps and written to the stored tap the scan order maps (u, v) to; dbias = sum of dy.
-// A CTA takes 128 consecutive pixels and one block of channels: its threads (8 channels each, 8
-// pixels in flight) read dy and the nine neighbours straight from global memory (they hit L1 / L2),
-// reduce over their pixel groups in shared memory and write one partial sum per CTA; a second kernel
-// adds the partial sums in a fixed order, so the result does not depend on scheduling.
-constexpr int kWgPixels = 128, kWgGroups = 8;
+// Same tiling as the forward kernel: a CTA stages the halo tile of x and the tile of dy of TY x TX pixels
+// and one block of channels in shared memory; a thread owns 8 channels of one tile column and adds the
+// nine products of its TY pixels to 72 + 8 accumulators.  CTA y of a channel block takes the tiles
+// y, y + gridDim.y, ... in that order, then the CTA's column threads are summed in shared memory and
+// one partial sum per CTA is written; a second kernel adds the partial sums in a fixed order, so the
+// result does not depend on scheduling.
+constexpr int kWgPixels = 128;       // pixels per partial sum (sizes the workspace)
 
 template <typename T>
-__global__ void __launch_bounds__(Cfg<T>::kLanes * kWgGroups)
+__global__ void __launch_bounds__(Cfg<T>::kThreads)
 srem_dwconv_wgrad(const T *__restrict__ x, const T *__restrict__ dy, float *__restrict__ partial,
-                  int npix, int gh, int gw, int D, int dir)
+                  int B, int gh, int gw, int D, int dir)
 {
-    constexpr int CH = Cfg<T>::CH, kLanes = Cfg<T>::kLanes;
-    __shared__ float red[kWgGroups][10][CH];
-    const int lane = threadIdx.x % kLanes, grp = threadIdx.x / kLanes;
-    const int ch = blockIdx.x * CH + lane * VEC;
-    const bool ch_ok = ch < D;
+    constexpr int CH = Cfg<T>::CH, kLanes = Cfg<T>::kLanes, kConvThreads = Cfg<T>::kThreads;
+    // halo tile of x and tile of dy; the same memory later holds the per-warp sums [warps][10][CH]
+    constexpr int kHalo = (TY + 2) * (TX + 2) * kLanes, kInner = TY * TX * kLanes, kWarps = kConvThreads / 32;
+    constexpr size_t kBytes = sizeof(Vec8<T>) * (kHalo + kInner) > sizeof(float) * kWarps * 10 * CH
+                                  ? sizeof(Vec8<T>) * (kHalo + kInner) : sizeof(float) * kWarps * 10 * CH;
+    __shared__ __align__(16) char sm[kBytes];
+    Vec8<T> (*tile)[TX + 2][kLanes] = reinterpret_cast<Vec8<T> (*)[TX + 2][kLanes]>(sm);
+    Vec8<T> (*gtile)[TX][kLanes] = reinterpret_cast<Vec8<T> (*)[TX][kLanes]>(sm + sizeof(Vec8<T>) * kHalo);
+    const int lane = threadIdx.x % kLanes, col = threadIdx.x / kLanes;
+    const int tiles_x = (gw + TX - 1) / TX, tiles_y = (gh + TY - 1) / TY, ntiles = B * tiles_x * tiles_y;
     pdl_wait();
     pdl_launch_dependents();
     float acc[10][8];
@@ -146,43 +153,71 @@ srem_dwconv_wgrad(const T *__restrict__ x, const T *__restrict__ dy, float *__re
     for (int k = 0; k < 10; ++k)
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[k][i] = 0.f;
-    const int p0 = blockIdx.y * kWgPixels, p1 = min(p0 + kWgPixels, npix);
-    if (ch_ok) {
-        for (int p = p0 + grp; p < p1; p += kWgGroups) {
-            const int b = p / (gh * gw), ij = p - b * (gh * gw), i = ij / gw, j = ij - i * gw;
+    for (int t = blockIdx.y; t < ntiles; t += gridDim.y) {
+        const int b = t / (tiles_x * tiles_y), r = t - b * (tiles_x * tiles_y);
+        const int y0 = (r / tiles_x) * TY, x0 = (r % tiles_x) * TX;
+        const size_t img = (size_t)b * gh * gw;
+        __syncthreads();                 // the previous tile has been consumed
+        for (int idx = threadIdx.x; idx < (TY + 2) * (TX + 2) * kLanes; idx += kConvThreads) {
+            const int l = idx % kLanes, pix = idx / kLanes;
+            const int tx = pix % (TX + 2), ty = pix / (TX + 2);
+            const int gy = y0 + ty - 1, gx = x0 + tx - 1, c = blockIdx.x * CH + l * VEC;
+            Vec8<T> v = Vec8<T>::zero();
+            if (gy >= 0 && gy < gh && gx >= 0 && gx < gw && c < D) v = Vec8<T>::load(x + (img + (size_t)gy * gw + gx) * D + c);
+            tile[ty][tx][l] = v;
+        }
+        for (int idx = threadIdx.x; idx < TY * TX * kLanes; idx += kConvThreads) {
+            const int l = idx % kLanes, pix = idx / kLanes;
+            const int tx = pix % TX, ty = pix / TX;
+            const int gy = y0 + ty, gx = x0 + tx, c = blockIdx.x * CH + l * VEC;
+            Vec8<T> v = Vec8<T>::zero();         // pixels outside the grid contribute nothing
+            if (gy < gh && gx < gw && c < D) v = Vec8<T>::load(dy + (img + (size_t)gy * gw + gx) * D + c);
+            gtile[ty][tx][l] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int ty = 0; ty < TY; ++ty) {
             float g[8];
-            Vec8<T>::load(dy + (size_t)p * D + ch).unpack(g);
+            gtile[ty][col][lane].unpack(g);
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[9][e] += g[e];
 #pragma unroll
             for (int u = 0; u < 3; ++u)
 #pragma unroll
                 for (int v = 0; v < 3; ++v) {
-                    const int ii = i + u - 1, jj = j + v - 1;
-                    if (ii < 0 || ii >= gh || jj < 0 || jj >= gw) continue;
                     float xv[8];
-                    Vec8<T>::load(x + ((size_t)b * gh * gw + (size_t)ii * gw + jj) * D + ch).unpack(xv);
+                    tile[ty + u][col + v][lane].unpack(xv);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) acc[u * 3 + v][e] = fmaf(g[e], xv[e], acc[u * 3 + v][e]);
                 }
         }
     }
+    __syncthreads();
+    // sum over the tile columns: the columns a warp holds by shuffles (a warp is 32 / kLanes columns of all
+    // lanes), the warps through shared memory
+    float *red = reinterpret_cast<float *>(sm);
+    const int warp = threadIdx.x >> 5;
 #pragma unroll
     for (int k = 0; k < 10; ++k)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) red[grp][k][lane * VEC + e] = acc[k][e];
+        for (int e = 0; e < 8; ++e) {
+            float v = acc[k][e];
+#pragma unroll
+            for (int m = kLanes; m < 32; m <<= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+            if ((threadIdx.x & 31) < kLanes) red[(warp * 10 + k) * CH + lane * VEC + e] = v;
+        }
     __syncthreads();
-    // partial[slab][k][D]: k = stored tap index 0..8, 9 = bias
-    for (int idx = threadIdx.x; idx < 10 * CH; idx += kLanes * kWgGroups) {
+    // partial[part][k][D]: k = stored tap index 0..8, 9 = bias
+    for (int idx = threadIdx.x; idx < 10 * CH; idx += kConvThreads) {
         const int k = idx / CH, c = idx - k * CH;
         if (blockIdx.x * CH + c >= D) continue;
         float sum = 0.f;
 #pragma unroll
-        for (int gidx = 0; gidx < kWgGroups; ++gidx) sum += red[gidx][k][c];
+        for (int j = 0; j < kWarps; ++j) sum += red[(j * 10 + k) * CH + c];
         int ks = k;
         if (k < 9) {
             int su = k / 3, sv = k - 3 * su;
-            if (dir & 2) { const int t = su; su = sv; sv = t; }
+            if (dir & 2) { const int tt = su; su = sv; sv = tt; }
             if (dir & 1) { su = 2 - su; sv = 2 - sv; }
             ks = su * 3 + sv;
         }
@@ -247,18 +282,21 @@ dig_status launch_dwconv_bwd(const void *x, const void *w, const void *dy, void 
 {
     dig_status st = launch_dwconv(dy, w, nullptr, dx, B, gh, gw, D, dir ^ 1, dtype, stream);
     if (st != DIG_OK) return st;
-    const int npix = B * gh * gw, nslab = (npix + kWgPixels - 1) / kWgPixels;
+    // one partial sum per CTA row; never more rows than tiles, never more than the workspace holds
+    const int npix = B * gh * gw, ntiles = B * ((gh + TY - 1) / TY) * ((gw + TX - 1) / TX);
+    int nslab = (npix + kWgPixels - 1) / kWgPixels;
+    if (nslab > ntiles) nslab = ntiles;
     if (nslab > 65535) return DIG_ERR_UNSUPPORTED;
     {
         KernelTimer t(KID_DWCONV_WGRAD, stream);
         if (dtype == DIG_F32) {
             const dim3 grid((D + Cfg<float>::CH - 1) / Cfg<float>::CH, nslab);
-            launch_pdl(srem_dwconv_wgrad<float>, grid, dim3(Cfg<float>::kLanes * kWgGroups), 0, stream,
-                       (const float *)x, (const float *)dy, partial, npix, gh, gw, D, dir);
+            launch_pdl(srem_dwconv_wgrad<float>, grid, dim3(Cfg<float>::kThreads), 0, stream,
+                       (const float *)x, (const float *)dy, partial, B, gh, gw, D, dir);
         } else {
             const dim3 grid((D + Cfg<__nv_bfloat16>::CH - 1) / Cfg<__nv_bfloat16>::CH, nslab);
-            launch_pdl(srem_dwconv_wgrad<__nv_bfloat16>, grid, dim3(Cfg<__nv_bfloat16>::kLanes * kWgGroups), 0, stream,
-                       (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)dy, partial, npix, gh, gw, D, dir);
+            launch_pdl(srem_dwconv_wgrad<__nv_bfloat16>, grid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
+                       (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)dy, partial, B, gh, gw, D, dir);
         }
     }
     if (cudaGetLastError() != cudaSuccess) return DIG_ERR_CUDA;
