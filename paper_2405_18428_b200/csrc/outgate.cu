@@ -11,7 +11,10 @@ namespace dig {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kMaxCtas = 148 * 8;
+// Grid caps (measured): the reverse kernel does best with as many CTAs as stay resident together, three
+// per SM at its register count, so that the grid-stride loops end together and not in a ragged last
+// wave; the forward kernel does best with eight per SM.
+constexpr int kSMs = 148, kFwdPerSM = 8, kBwdPerSM = 3;
 
 __device__ __forceinline__ void load8(const float *p, float (&f)[8])
 {
@@ -196,8 +199,9 @@ outgate_affine_sum(const float *__restrict__ partial, float *__restrict__ dln_w,
     }
 }
 
-int grid_for(long long rows, int lpr)
+int grid_for(long long rows, int lpr, int per_sm = kBwdPerSM)
 {
+    const int kMaxCtas = kSMs * per_sm;
     const long long per = kThreads / lpr, need = (rows + per - 1) / per;
     return (int)(need < kMaxCtas ? need : kMaxCtas);
 }
@@ -207,10 +211,10 @@ void fwd_dispatch3(const void *o, const void *r, const float *w, const float *b,
                    float eps, cudaStream_t stream)
 {
     if (dv <= 64)
-        launch_pdl(outgate_fwd<TA, TR, TZ, 8>, dim3(grid_for(rows, 8)), dim3(kThreads), 0, stream, (const TA *)o,
+        launch_pdl(outgate_fwd<TA, TR, TZ, 8>, dim3(grid_for(rows, 8, kFwdPerSM)), dim3(kThreads), 0, stream, (const TA *)o,
                    (const TR *)r, w, b, (TZ *)z, rows, dv, eps);
     else
-        launch_pdl(outgate_fwd<TA, TR, TZ, 16>, dim3(grid_for(rows, 16)), dim3(kThreads), 0, stream, (const TA *)o,
+        launch_pdl(outgate_fwd<TA, TR, TZ, 16>, dim3(grid_for(rows, 16, kFwdPerSM)), dim3(kThreads), 0, stream, (const TA *)o,
                    (const TR *)r, w, b, (TZ *)z, rows, dv, eps);
 }
 template <typename TI, typename TO>
