@@ -286,6 +286,14 @@ dig_status launch_dwconv_bwd(const void *x, const void *w, const void *dy, void 
     const int npix = B * gh * gw, ntiles = B * ((gh + TY - 1) / TY) * ((gw + TX - 1) / TX);
     int nslab = (npix + kWgPixels - 1) / kWgPixels;
     if (nslab > ntiles) nslab = ntiles;
+    {
+        // no more CTAs than stay resident together (three per SM at this kernel's register count), so that
+        // their tile loops end together
+        const int CHb = dtype == DIG_F32 ? Cfg<float>::CH : Cfg<__nv_bfloat16>::CH;
+        const int nchb = (D + CHb - 1) / CHb, resident = 148 * 3;
+        const int cap = resident / nchb > 0 ? resident / nchb : 1;
+        if (nslab > cap) nslab = cap;
+    }
     if (nslab > 65535) return DIG_ERR_UNSUPPORTED;
     {
         KernelTimer t(KID_DWCONV_WGRAD, stream);
