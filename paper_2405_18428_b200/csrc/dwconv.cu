@@ -120,6 +120,100 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
     }
 }
 
+// The same convolution for grids with several tiles per resident CTA: a persistent CTA walks over tiles
+// (x fastest, then y, batch, channel block) and fills the halo tile of its next tile with cp.async into a
+// second buffer while it computes the current one, so the load latency is paid once per CTA, not once
+// per tile.  Out-of-grid pixels and channels are zero-filled by the copy itself (source size 0).
+template <typename T, typename TO>
+__global__ void __launch_bounds__(Cfg<T>::kThreads)
+srem_dwconv3x3_stream(const T *__restrict__ x, const T *__restrict__ w, const T *__restrict__ bias,
+                      TO *__restrict__ y, int B, int gh, int gw, int D, int dir, int tiles_x, int tiles_y, int ntiles)
+{
+    constexpr int CH = Cfg<T>::CH, kLanes = Cfg<T>::kLanes, kConvThreads = Cfg<T>::kThreads;
+    constexpr int kPieces = (int)sizeof(Vec8<T>) / 16;
+    __shared__ Vec8<T> tile[2][TY + 2][TX + 2][kLanes];
+    const int lane = threadIdx.x % kLanes, col = threadIdx.x / kLanes;
+    pdl_wait();
+    pdl_launch_dependents();
+    auto decode = [&](int t, int &b, int &chb, int &y0, int &x0) {
+        const int per_img = tiles_x * tiles_y, z = t / per_img, r = t - z * per_img;
+        chb = z / B;
+        b = z - chb * B;
+        y0 = (r / tiles_x) * TY;
+        x0 = (r % tiles_x) * TX;
+    };
+    auto fill = [&](int t, int buf) {
+        int b, chb, y0, x0;
+        decode(t, b, chb, y0, x0);
+        const T *xb = x + (size_t)b * gh * gw * D;
+        for (int idx = threadIdx.x; idx < (TY + 2) * (TX + 2) * kLanes; idx += kConvThreads) {
+            const int l = idx % kLanes, pix = idx / kLanes;
+            const int tx = pix % (TX + 2), ty = pix / (TX + 2);
+            const int gy = y0 + ty - 1, gx = x0 + tx - 1, c = chb * CH + l * VEC;
+            const bool in = gy >= 0 && gy < gh && gx >= 0 && gx < gw && c < D;
+            const char *src = reinterpret_cast<const char *>(in ? xb + ((size_t)gy * gw + gx) * D + c : x);
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&tile[buf][ty][tx][l]);
+#pragma unroll
+            for (int p = 0; p < kPieces; ++p)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 16 * p), "l"(src + (in ? 16 * p : 0)),
+                             "r"(in ? 16 : 0) : "memory");
+        }
+    };
+    int t = blockIdx.x, cur_chb = -1;
+    if (t < ntiles) fill(t, 0);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    Vec8<T> wt[3][3];
+    float bs[8];
+    for (int buf = 0; t < ntiles; t += gridDim.x, buf ^= 1) {
+        if (t + (int)gridDim.x < ntiles) fill(t + gridDim.x, buf ^ 1);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        int b, chb, y0, x0;
+        decode(t, b, chb, y0, x0);
+        const int ch = chb * CH + lane * VEC;
+        const bool ch_ok = ch < D;
+        if (chb != cur_chb) {            // uniform over the CTA: the taps of this channel block, re-oriented
+            cur_chb = chb;
+#pragma unroll
+            for (int u = 0; u < 3; ++u)
+#pragma unroll
+                for (int v = 0; v < 3; ++v) {
+                    int su = u, sv = v;
+                    if (dir & 2) { su = v; sv = u; }
+                    if (dir & 1) { su = 2 - su; sv = 2 - sv; }
+                    wt[u][v] = ch_ok ? Vec8<T>::load(w + (size_t)(su * 3 + sv) * D + ch) : Vec8<T>::zero();
+                }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) bs[i] = 0.f;
+            if (bias != nullptr && ch_ok) Vec8<T>::load(bias + ch).unpack(bs);
+        }
+        asm volatile("cp.async.wait_group 1;" ::: "memory");      // everything but the newest group: this tile has landed
+        __syncthreads();
+        if (ch_ok && x0 + col < gw) {
+#pragma unroll
+            for (int ty = 0; ty < TY; ++ty) {
+                if (y0 + ty < gh) {
+                    float acc[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[i] = bs[i];
+#pragma unroll
+                    for (int u = 0; u < 3; ++u)
+#pragma unroll
+                        for (int v = 0; v < 3; ++v) {
+                            float xv[8], wv[8];
+                            tile[buf][ty + u][col + v][lane].unpack(xv);
+                            wt[u][v].unpack(wv);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) acc[i] = fmaf(wv[i], xv[i], acc[i]);
+                        }
+                    store8(y + (((size_t)b * gh + y0 + ty) * gw + x0 + col) * D + ch, acc);
+                }
+            }
+        }
+        __syncthreads();                 // this buffer is refilled during the next iteration
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
 // ---- reverse mode: filter and bias gradients ------------------------------------------------------
 // dw'[u][v][c] = sum over pixels of dy[i][j][c] * x[i+u-1][j+v-1][c] (zero outside the grid), computed
 // in canonical taps and written to the stored tap the scan order maps (u, v) to; dbias = sum of dy.
@@ -249,6 +343,30 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
     const dim3 grid((gw + TX - 1) / TX, (gh + TY - 1) / TY, B * nchb);
     if (grid.y > 65535 || (size_t)B * nchb > 65535) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_DWCONV, stream);
+    // two or more tiles per CTA that can be resident: the persistent, double-buffered kernel
+    const long long ntiles = (long long)grid.x * grid.y * grid.z;
+    const int resident = 148 * 4;       // four CTAs of the persistent kernel fit an SM at its register count
+    if (ntiles >= 2 * resident && ntiles < (1ll << 31)) {
+        const dim3 pgrid(resident);
+        switch (dtype) {
+            case DIG_F32:
+                launch_pdl(srem_dwconv3x3_stream<float, float>, pgrid, dim3(Cfg<float>::kThreads), 0, stream, (const float *)x,
+                           (const float *)w, (const float *)bias, (float *)y, B, gh, gw, D, dir, (int)grid.x, (int)grid.y, (int)ntiles);
+                break;
+            case DIG_BF16:
+                launch_pdl(srem_dwconv3x3_stream<__nv_bfloat16, __nv_bfloat16>, pgrid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
+                           (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias, (__nv_bfloat16 *)y, B, gh,
+                           gw, D, dir, (int)grid.x, (int)grid.y, (int)ntiles);
+                break;
+            case DIG_BF16_F32OUT:
+                launch_pdl(srem_dwconv3x3_stream<__nv_bfloat16, float>, pgrid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
+                           (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias, (float *)y, B, gh, gw, D,
+                           dir, (int)grid.x, (int)grid.y, (int)ntiles);
+                break;
+            default: return DIG_ERR_INVALID_ARG;
+        }
+        return cuda_ok(cudaGetLastError());
+    }
     switch (dtype) {
         case DIG_F32:
             launch_pdl(srem_dwconv3x3<float, float>, grid, dim3(Cfg<float>::kThreads), 0, stream,

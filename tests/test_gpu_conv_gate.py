@@ -145,3 +145,11 @@ def test_conv_bwd_rejects_short_workspace():
     ws = torch.empty(16, dtype=torch.uint8, device="cuda")
     with pytest.raises(RuntimeError):
         dig.dig_srem_dwconv_bwd(x, w, x, 4, 4, 0, workspace=ws)
+
+
+@pytest.mark.parametrize("dtype,direction,bias", [("f32", 1, True), ("bf16", 2, True), ("bf16", 3, False)])
+def test_conv_many_tiles_per_cta(dtype, direction, bias):
+    """3 x 96 x 96 pixels x 136 channels: 1728 tiles, which selects the persistent double-buffered kernel
+    (ragged last channel block, every scan order's tap permutation, bf16 and fp32 storage and output)."""
+    _conv_case(3, 96, 96, 136, dtype, direction, bias=bias, seed=9)
+    _conv_bwd_case(3, 96, 96, 136, dtype, direction, with_bias=bias, seed=9)      # dx runs through the same kernel
