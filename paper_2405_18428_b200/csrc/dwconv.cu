@@ -125,7 +125,7 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
 // second buffer while it computes the current one, so the load latency is paid once per CTA, not once
 // per tile.  Out-of-grid pixels and channels are zero-filled by the copy itself (source size 0).
 template <typename T, typename TO>
-__global__ void __launch_bounds__(Cfg<T>::kThreads)
+__global__ void __launch_bounds__(Cfg<T>::kThreads, 3)
 srem_dwconv3x3_stream(const T *__restrict__ x, const T *__restrict__ w, const T *__restrict__ bias,
                       TO *__restrict__ y, int B, int gh, int gw, int D, int dir, int tiles_x, int tiles_y, int ntiles)
 {
@@ -162,8 +162,9 @@ srem_dwconv3x3_stream(const T *__restrict__ x, const T *__restrict__ w, const T 
     int t = blockIdx.x, cur_chb = -1;
     if (t < ntiles) fill(t, 0);
     asm volatile("cp.async.commit_group;" ::: "memory");
-    Vec8<T> wt[3][3];
-    float bs[8];
+    // with the loads off the critical path the kernel is bound by instruction issue: the taps are kept as
+    // fp32 in registers and every input row is read and widened once for the three output rows it feeds
+    float wf[3][3][8], bs[8];
     for (int buf = 0; t < ntiles; t += gridDim.x, buf ^= 1) {
         if (t + (int)gridDim.x < ntiles) fill(t + gridDim.x, buf ^ 1);
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -180,7 +181,7 @@ srem_dwconv3x3_stream(const T *__restrict__ x, const T *__restrict__ w, const T 
                     int su = u, sv = v;
                     if (dir & 2) { su = v; sv = u; }
                     if (dir & 1) { su = 2 - su; sv = 2 - sv; }
-                    wt[u][v] = ch_ok ? Vec8<T>::load(w + (size_t)(su * 3 + sv) * D + ch) : Vec8<T>::zero();
+                    (ch_ok ? Vec8<T>::load(w + (size_t)(su * 3 + sv) * D + ch) : Vec8<T>::zero()).unpack(wf[u][v]);
                 }
 #pragma unroll
             for (int i = 0; i < 8; ++i) bs[i] = 0.f;
@@ -189,24 +190,30 @@ srem_dwconv3x3_stream(const T *__restrict__ x, const T *__restrict__ w, const T 
         asm volatile("cp.async.wait_group 1;" ::: "memory");      // everything but the newest group: this tile has landed
         __syncthreads();
         if (ch_ok && x0 + col < gw) {
+            // acc[r % 3] belongs to output row r; tile row rr (0 = the halo row above) feeds output rows rr - u,
+            // u = 0..2, and completes output row rr - 2
+            float acc[3][8];
 #pragma unroll
-            for (int ty = 0; ty < TY; ++ty) {
-                if (y0 + ty < gh) {
-                    float acc[8];
+            for (int rr = 0; rr < TY + 2; ++rr) {
+                if (rr < TY) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[i] = bs[i];
-#pragma unroll
-                    for (int u = 0; u < 3; ++u)
-#pragma unroll
-                        for (int v = 0; v < 3; ++v) {
-                            float xv[8], wv[8];
-                            tile[buf][ty + u][col + v][lane].unpack(xv);
-                            wt[u][v].unpack(wv);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) acc[i] = fmaf(wv[i], xv[i], acc[i]);
-                        }
-                    store8(y + (((size_t)b * gh + y0 + ty) * gw + x0 + col) * D + ch, acc);
+                    for (int i = 0; i < 8; ++i) acc[rr % 3][i] = bs[i];
                 }
+                float xv[3][8];
+#pragma unroll
+                for (int v = 0; v < 3; ++v) tile[buf][rr][col + v][lane].unpack(xv[v]);
+#pragma unroll
+                for (int u = 0; u < 3; ++u) {
+                    const int ty = rr - u;
+                    if (ty >= 0 && ty < TY) {
+#pragma unroll
+                        for (int v = 0; v < 3; ++v)
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) acc[ty % 3][i] = fmaf(wf[u][v][i], xv[v][i], acc[ty % 3][i]);
+                    }
+                }
+                const int done = rr - 2;
+                if (done >= 0 && y0 + done < gh) store8(y + (((size_t)b * gh + y0 + done) * gw + x0 + col) * D + ch, acc[done % 3]);
             }
         }
         __syncthreads();                 // this buffer is refilled during the next iteration
@@ -345,7 +352,7 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
     KernelTimer t(KID_DWCONV, stream);
     // two or more tiles per CTA that can be resident: the persistent, double-buffered kernel
     const long long ntiles = (long long)grid.x * grid.y * grid.z;
-    const int resident = 148 * 4;       // four CTAs of the persistent kernel fit an SM at its register count
+    const int resident = 148 * 3;       // three CTAs of the persistent kernel fit an SM at its register count
     if (ntiles >= 2 * resident && ntiles < (1ll << 31)) {
         const dim3 pgrid(resident);
         switch (dtype) {
