@@ -350,11 +350,11 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
     const dim3 grid((gw + TX - 1) / TX, (gh + TY - 1) / TY, B * nchb);
     if (grid.y > 65535 || (size_t)B * nchb > 65535) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_DWCONV, stream);
-    // two or more tiles per CTA that can be resident: the persistent, double-buffered kernel
+    // at least as many tiles as CTAs can be resident: the persistent, double-buffered kernel, two or more tiles per CTA
     const long long ntiles = (long long)grid.x * grid.y * grid.z;
     const int resident = 148 * 3;       // three CTAs of the persistent kernel fit an SM at its register count
-    if (ntiles >= 2 * resident && ntiles < (1ll << 31)) {
-        const dim3 pgrid(resident);
+    if (ntiles >= resident && ntiles < (1ll << 31)) {
+        const dim3 pgrid((unsigned)(ntiles >= 2 * resident ? resident : (ntiles + 1) / 2));
         switch (dtype) {
             case DIG_F32:
                 launch_pdl(srem_dwconv3x3_stream<float, float>, pgrid, dim3(Cfg<float>::kThreads), 0, stream, (const float *)x,
