@@ -31,7 +31,8 @@ typedef enum {
     DIG_ERR_WORKSPACE = 3,     /* workspace missing or smaller than dig_gla_workspace_bytes */
     DIG_ERR_CUDA = 4,          /* a CUDA runtime call failed (launch, attribute, ...) */
     DIG_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (see dig_last_device_status) */
-    DIG_ERR_SCRATCH_LIMIT = 6  /* dig_gla_fwd_static: the problem needs more than its built-in scratch */
+    DIG_ERR_SCRATCH_LIMIT = 6, /* dig_gla_fwd_static: the problem needs more than its built-in scratch */
+    DIG_ERR_RANGE = 7          /* gates decay faster than the kernels can represent (see dig_gla_fwd, dig_last_device_status) */
 } dig_status;
 
 /* Storage type of q, k, v, out, d_out, dq, dk, dv, x, y, w, bias.  Gates are always fp32.

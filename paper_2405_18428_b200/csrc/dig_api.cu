@@ -4,6 +4,7 @@
 #include <vector>
 
 #include "dig_common.cuh"
+#include "sweep.cuh"
 
 namespace dig {
 
@@ -53,14 +54,14 @@ Geom make_geom(int B, int H, int gh, int gw, int dk, int dv, int chunk, int dir)
 }
 
 // DIG_IMPL_FMA / DIG_IMPL_TENSOR / DIG_IMPL_MMA, or a negative status.
-// The tensor-core kernels hold 64 tokens per tile; a request for chunks of 128 is evaluated by them
-// with 64-token tiles (the result does not depend on the chunk size beyond rounding).
-int tile_chunk(int impl, int chunk) { return (impl == DIG_IMPL_TENSOR && chunk == 128) ? 64 : chunk; }
+// The tcgen05 kernels take the requested chunk size as it is (they work in 64-token tiles and treat
+// shorter chunks as sub-chunks of a tile, longer ones as 64).
+int tile_chunk(int impl, int chunk) { (void)impl; return chunk; }
 
 int choose_impl(int dk, int dv, int chunk, int dtype, bool backward)
 {
     const int want = g_impl.load();
-    const bool t_ok = tensor_supports(dk, dv, chunk, dtype, backward);
+    const bool t_ok = sweep_supports(dk, dv, chunk, dtype);
     const bool f_ok = fma_supports(dk, dv, chunk, dtype, backward);
     const bool m_ok = mma_supports(dk, dv, chunk, dtype, backward);
     if (want == DIG_IMPL_TENSOR) return t_ok ? DIG_IMPL_TENSOR : -(int)DIG_ERR_UNSUPPORTED;
@@ -81,7 +82,8 @@ const char *const kKernelNames[KID_COUNT] = {
     "gate_logsigmoid", "srem_dwconv3x3", "srem_dwconv_wgrad", "gla_outgate", "state_scan_fwd", "state_scan_bwd",
     "fma_chunk_state", "fma_chunk_out", "fma_chunk_bwd",
     "mma_chunk_state", "mma_chunk_out", "mma_chunk_bwd",
-    "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd"};
+    "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd",
+    "sweep_local", "seg_scan", "sweep_fwd", "sweep_bwd"};
 struct Profile {
     bool on = false;
     std::vector<cudaEvent_t> ev;      // 2 per timed launch, created lazily and reused
@@ -155,10 +157,15 @@ size_t dig_gla_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, in
                                int dtype, int backward)
 {
     if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, 0, dtype)) return 0;
-    // sized for whichever family may serve the call (the tensor family uses 64-token tiles for chunk 128)
-    const bool tensor_ok = tensor_supports(d_k, d_v, chunk, dtype, backward != 0);
-    const Geom g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(tensor_ok ? DIG_IMPL_TENSOR : DIG_IMPL_FMA, chunk), 0);
-    return carve_workspace(nullptr, g, backward != 0).bytes;
+    // sized for whichever family may serve the call
+    const Geom g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, 0);
+    size_t need = 0;
+    if (sweep_supports(d_k, d_v, chunk, dtype)) need = sweep_workspace_bytes(g, backward != 0);
+    if (fma_supports(d_k, d_v, chunk, dtype, backward != 0) || mma_supports(d_k, d_v, chunk, dtype, backward != 0)) {
+        const size_t other = carve_workspace(nullptr, g, backward != 0).bytes;
+        need = other > need ? other : need;
+    }
+    return need;
 }
 
 dig_status dig_gate_logsigmoid(const void *g, const float *tau_per_head, float *gate, int B, int L,
@@ -191,7 +198,7 @@ dig_status dig_gla_fwd_state(const void *q, const void *k, const void *v, const 
     a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
     a.dtype = dtype;
     a.stream = (cudaStream_t)cuda_stream;
-    return impl == DIG_IMPL_TENSOR ? tensor_gla_fwd(a) : impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
+    return impl == DIG_IMPL_TENSOR ? sweep_gla_fwd(a) : impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
 }
 
 dig_status dig_gla_bwd_state(const void *q, const void *k, const void *v, const float *gate,
@@ -218,7 +225,7 @@ dig_status dig_gla_bwd_state(const void *q, const void *k, const void *v, const 
     a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, tile_chunk(impl, chunk), direction);
     a.dtype = dtype;
     a.stream = (cudaStream_t)cuda_stream;
-    return impl == DIG_IMPL_TENSOR ? tensor_gla_bwd(a) : impl == DIG_IMPL_MMA ? mma_gla_bwd(a) : fma_gla_bwd(a);
+    return impl == DIG_IMPL_TENSOR ? sweep_gla_bwd(a) : impl == DIG_IMPL_MMA ? mma_gla_bwd(a) : fma_gla_bwd(a);
 }
 
 dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float *gate, void *out,
@@ -327,7 +334,7 @@ dig_status dig_gla_fwd_outgate(const void *q, const void *k, const void *v, cons
     // the plain forward pass (into z when the caller does not want `out`), then the gate kernel, which may
     // work in place
     a.out = out ? out : z;
-    const dig_status st = impl == DIG_IMPL_TENSOR ? tensor_gla_fwd(a) : impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
+    const dig_status st = impl == DIG_IMPL_TENSOR ? sweep_gla_fwd(a) : impl == DIG_IMPL_MMA ? mma_gla_fwd(a) : fma_gla_fwd(a);
     if (st != DIG_OK) return st;
     return launch_outgate_fwd_mixed(a.out, r, ln_w, ln_b, z, (long long)B * grid_h * grid_w * H, d_v, eps, dtype, a.stream);
 }
@@ -393,7 +400,7 @@ dig_status dig_last_device_status(void *cuda_stream)
     if (host != 0) {
         const int zero = 0;
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return DIG_ERR_CUDA;
-        return DIG_ERR_TIMEOUT;
+        return (host & 1) ? DIG_ERR_TIMEOUT : DIG_ERR_RANGE;          // bit 0: a wait expired; bit 1: gates out of range
     }
     return DIG_OK;
 }
@@ -439,6 +446,7 @@ const char *dig_status_string(int status)
         case DIG_ERR_CUDA: return "CUDA runtime error";
         case DIG_ERR_TIMEOUT: return "device-side wait timed out";
         case DIG_ERR_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of dig_gla_fwd_static";
+        case DIG_ERR_RANGE: return "gate decay inside a chunk exceeds the documented range";
     }
     return "unknown status";
 }

@@ -162,6 +162,7 @@ enum KernelId {
     KID_FMA_STATE, KID_FMA_OUT, KID_FMA_BWD,
     KID_MMA_STATE, KID_MMA_OUT, KID_MMA_BWD,
     KID_TC_STATE, KID_TC_OUT, KID_TC_BWD,
+    KID_SW_LOCAL, KID_SW_SCAN, KID_SW_FWD, KID_SW_BWD,
     KID_COUNT
 };
 struct KernelTimer {

@@ -1,0 +1,938 @@
+// tcgen05 "sweep" kernels of chunkwise gated linear attention (Eq. attn_gla, Section 3.5): the
+// recurrence S_t = diag(exp(a_t)) S_{t-1} + k_t^T v_t, o_t = q_t S_t worked in 64-token tiles, with
+// the d_k x d_v state held on chip while a CTA walks over a segment of consecutive tiles.
+//
+// A sequence of N tiles is cut into segments of G tiles; one CTA sweeps one segment.
+//   forward : sweep_local  per segment, from a zero state: the state it leaves and its total decay
+//             seg_scan     per sequence, over the few segment ends: the state entering each segment
+//             sweep_fwd    per segment, from its true entry state: out = tril(Qc Kc^T) V + Qc Sc per tile
+//   backward: sweep_local  (backward flavour) also stores, per (sub-)chunk, the zero-start state in
+//                          fp16 and the decay since the segment start, and accumulates the segment's
+//                          contribution to the state gradient
+//             seg_scan     forward over the states, backward over the state gradients, gate-gradient carry
+//             sweep_bwd    per segment in reverse: dq, dk, dv, dgate with the state gradient on chip
+// Per (sub-)chunk, with Lam the cumulative gate inside it, c = Lam_end / 2 per channel,
+//   Qc = q exp(Lam - c), Kc = k exp(c - Lam), Sc = diag(exp(c)) S_in, Dc = diag(exp(c)) D_out:
+//   P   = tril(Qc Kc^T)                         dP = tril(dO V^T)
+//   out = P V + Qc Sc                           S_out = exp(2c) S_in + exp(c) (Kc^T V)
+//   dq  = (dP Kc + dO Sc^T) exp(Lam - c)        dk = (dP^T Qc + V Dc^T) exp(c - Lam)
+//   dv  = P^T dO + Kc Dc                        D_in = exp(2c) D_out + exp(c) (Qc^T dO)
+//   dgate_j = sum_{r >= j} (q dq - k dk)_r  (running over the whole sequence in reverse scan order)
+// In the backward sweep S_in = S_local + diag(G) S_segment, G the decay since the segment start, so
+// dO Sc^T = dO Sc_local^T + (dO S_segment^T) diag(exp(c) G): two products and one fused multiply-add.
+//
+// Every product is a tcgen05.mma (kind::f16, fp16 operands, fp32 accumulators in tensor memory)
+// issued by one extra warp; the other warps build operand tiles, mask the scores and post-process
+// accumulators.  Token rows of the next tile are prefetched into registers; with 256 worker
+// threads two CTAs share an SM, so one builds while the other's products are in the tensor pipe.
+#include "sweep.cuh"
+
+namespace dig {
+namespace {
+
+using namespace sw;
+
+struct SweepArgs {
+    const bf16 *q, *k, *v, *d_out;
+    const float *gate;
+    void *out, *dq, *dk, *dv;
+    float *dgate;
+    float *seg_state, *seg_gamma, *seg_dstate, *seg_carry;
+    __half *seg_state16, *slot_s;
+    float *slot_g;
+    int *status;
+    Geom g;
+    Plan plan;
+};
+
+// ---- shared phases ------------------------------------------------------------------------------
+__device__ __forceinline__ void cta_setup(Ctl *ctl, int nbar, uint32_t tmem_cols, char *tiles, int tile_bytes)
+{
+    const int tid = threadIdx.x;
+    if (tid < 32) tmem_alloc(&ctl->tmem_base, tmem_cols);
+    if (tid == 32) {
+        for (int i = 0; i < nbar; ++i) mbar_init(&ctl->bar[i], 1);
+        fence_barrier_init();
+    }
+    zero_smem(tiles, tile_bytes);
+    fence_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+}
+__device__ __forceinline__ void cta_teardown(Ctl *ctl, uint32_t tmem_cols)
+{
+    tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x < 32) tmem_dealloc(ctl->tmem_base, tmem_cols);
+}
+
+// Operand tiles of rows [lo, hi) of the prefetched tile (the other rows are zero):
+//   tK <- k 2^(off - Lam), tV <- v, and where present tQ <- q 2^(Lam - off), tG <- dO.
+template <int D, int NT, bool HQ, bool HD>
+__device__ __forceinline__ void build_tiles(const Raw<Lay<D, NT>::NIT, HQ, HD> &r, char *tQ, char *tK, char *tV, char *tG,
+                                            const float *table, const float *off, const int *row_tok, int lo, int hi)
+{
+    using C = Cfg<D>;
+#pragma unroll
+    for (int i = 0; i < Lay<D, NT>::NIT; ++i) {
+        const int it = (int)threadIdx.x + NT * i;
+        if (it < T * C::NCH) {
+            const int row = it / C::NCH, j = it - row * C::NCH;
+            const int o = j * C::CHT + row * 16;
+            if (row >= lo && row < hi && row_tok[row] >= 0) {
+                float lam[8], of[8], x[8], y[8];
+                ld8(table + row * C::LAMP + 8 * j, lam);
+                ld8(off + 8 * j, of);
+                unpack_b8(r.k[i], x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) y[e] = x[e] * ex2(of[e] - lam[e]);
+                *reinterpret_cast<uint4 *>(tK + o) = pack_h8(y);
+                unpack_b8(r.v[i], x);
+                *reinterpret_cast<uint4 *>(tV + o) = pack_h8(x);
+                if (HQ) {
+                    unpack_b8(r.q[i], x);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) y[e] = x[e] * ex2(lam[e] - of[e]);
+                    *reinterpret_cast<uint4 *>(tQ + o) = pack_h8(y);
+                }
+                if (HD) {
+                    unpack_b8(r.d[i], x);
+                    *reinterpret_cast<uint4 *>(tG + o) = pack_h8(x);
+                }
+            } else {
+                const uint4 z = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4 *>(tK + o) = z;
+                *reinterpret_cast<uint4 *>(tV + o) = z;
+                if (HQ) *reinterpret_cast<uint4 *>(tQ + o) = z;
+                if (HD) *reinterpret_cast<uint4 *>(tG + o) = z;
+            }
+        }
+    }
+}
+
+// State product with channels along M: acc <- A^T B, A and B token tiles read down their rows
+// (contraction over the 64 tokens).  Small heads: two value-column halves into the two lane halves.
+template <int D>
+__device__ __forceinline__ void issue_state_product(uint32_t tmem_acc, const char *tA, const char *tB)
+{
+    using C = Cfg<D>;
+    const uint32_t a = smem_u32(tA), b = smem_u32(tB);
+    if constexpr (C::BIGM) {
+        issue<128, C::NACC, true, true>(tmem_acc, a, C::CHT, b, C::CHT, T / 16, false);
+    } else {
+        constexpr int HCH = C::NCH / 2;
+        issue<64, D / 2, true, true>(tmem_acc, a, C::CHT, b, C::CHT, T / 16, false);
+        issue<64, D / 2, true, true>(tmem_acc + (16u << 16), a, C::CHT, b + HCH * C::CHT, C::CHT, T / 16, false);
+    }
+}
+
+// Bounded wait whose verdict is uniform over the warp (tcgen05.ld must never run under a
+// lane-divergent condition).
+__device__ __forceinline__ bool wait_all(uint64_t *bar, uint32_t parity, int *status)
+{
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, status)) != 0;
+}
+
+#define SYNC_OR_DIE()                               \
+    do {                                            \
+        if (!__syncthreads_and(ok)) goto die;       \
+    } while (0)
+
+// =================================================================================================
+// sweep_local: a segment from a zero state.
+// =================================================================================================
+template <int D, int NT, bool BWD>
+struct LocalSmem {
+    using C = Cfg<D>;
+    using L = Lay<D, NT>;
+    static constexpr int kTiles = (BWD ? 4 : 2) * C::TILE_T;
+    // an M = 128 operand read down the rows of tQ / tK covers 16 chunks (more than the tile has): the
+    // bytes behind it belong to the next tile, which is mapped and holds finite fp16 values
+    static constexpr int kTilesPad = kTiles;
+    static_assert(!C::BIGM || 16 * C::CHT <= 2 * C::TILE_T, "an M = 128 operand must stay inside the tile area");
+    static constexpr int kFloats = T * C::LAMP + L::NSEG * D + 8 * D;
+    static constexpr size_t bytes = kTilesPad + kFloats * 4 + 3 * T * 4 + sizeof(Ctl);
+    static constexpr uint32_t tmem_cols = C::BIGM ? (BWD ? 256 : 128) : (BWD ? 64 : 32);
+};
+
+template <int D, int NT, bool BWD>
+__global__ void __launch_bounds__(NT, NT == 256 ? 2 : 1)
+sweep_local(const SweepArgs a)
+{
+    using C = Cfg<D>;
+    using L = Lay<D, NT>;
+    using SM = LocalSmem<D, NT, BWD>;
+    extern __shared__ __align__(128) char smem[];
+    char *tQ = smem, *tK = BWD ? tQ + C::TILE_T : smem, *tV = tK + C::TILE_T, *tG = tV + C::TILE_T;
+    float *table = reinterpret_cast<float *>(smem + SM::kTilesPad);
+    float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D;
+    int *rowTok = reinterpret_cast<int *>(vecb + 8 * D);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowTok + 3 * T);
+    constexpr uint32_t aU = 0, aW = C::BIGM ? C::NACC : D / 2;
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    cta_setup(ctl, 1, SM::tmem_cols, smem, SM::kTilesPad);
+    const uint32_t tmem = ctl->tmem_base, lane_base = (uint32_t)(32 * ((tid >> 5) & 3)) << 16;
+    const Geom &g = a.g;
+    const Plan &pl = a.plan;
+    const StateMap<D, NT> sm;
+    float S[L::NPS][8], Wl[L::NPS][8];
+    Raw<L::NIT, BWD, BWD> raw;
+    float gcum = 0.f;
+    uint32_t par = 0;
+    bool ok = true;
+    int cur = 0, iter = 0;
+    const int total = g.B * g.H * pl.nseg;
+
+    pdl_wait();
+    pdl_launch_dependents();
+    for (int sid = blockIdx.x; sid < total; sid += gridDim.x) {
+        const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg, b = bh / g.H, h = bh - b * g.H;
+        const int t0 = sg * pl.G, t1 = min(t0 + pl.G, pl.ntile);
+        load_state<D, NT>(nullptr, sm, S);
+        if (BWD) load_state<D, NT>(nullptr, sm, Wl);
+        gcum = 0.f;
+        if (tid < T) rowTok[cur * T + tid] = tile_token(g, t0, tid);
+        __syncthreads();
+        load_raw<D, NT, BWD, BWD>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, b, h, rowTok + cur * T);
+        for (int tile = t0; tile < t1; ++tile) {
+            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
+            if (tid < T) rowTok[nxt * T + tid] = tile + 1 < t1 ? tile_token(g, tile + 1, tid) : -1;
+            write_gates<D, NT, BWD, BWD>(raw, table, rowTok + cur * T);
+            __syncthreads();
+            float tot_unused;
+            const bool need = gate_prefix<D, NT>(table, sTot, tot_unused);
+            int s = pl.sub_max;
+            if (need || s < T) {
+                bool bad;
+                s = choose_sub<D>(table, need ? min(s, T / 2) : s, &bad);
+                if (bad && tid == 0) atomicOr(a.status, kStatusRange);
+            }
+            const int nsub = (nrow + s - 1) / s;
+            for (int u = 0; u < nsub; ++u, ++iter) {
+                const int lo = u * s, hi = min(lo + s, T);
+                const Vec vc = vec_of<D>(vecb, iter & 1);
+                if (tid < D) {
+                    const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
+                    const float t = table[(hi - 1) * C::LAMP + tid] - base, cv = 0.5f * t;
+                    vc.off[tid] = base + cv;
+                    vc.ec[tid] = ex2(cv);
+                    vc.e2c[tid] = ex2(t);
+                    if (BWD) {
+                        vc.aux[tid] = ex2(gcum + cv);           // decay from the segment start to the sub-chunk's centre
+                        const size_t slot = ((size_t)(nsub - 1 - u) * g.B * g.H + bh) * pl.ntile + tile;
+                        a.slot_g[slot * D + tid] = gcum;
+                    }
+                    gcum += t;
+                }
+                __syncthreads();
+                {
+                    build_tiles<D, NT, BWD, BWD>(raw, tQ, tK, tV, tG, table, vc.off, rowTok + cur * T, lo, min(hi, nrow));
+                    if (BWD) {
+                        const size_t slot = ((size_t)(nsub - 1 - u) * g.B * g.H + bh) * pl.ntile + tile;
+                        write_state_slot<D, NT>(a.slot_s + slot * (D * D), sm, S, vc.ec);
+                    }
+                    fence_async_smem();
+                }
+                tc_fence_before_sync();
+                SYNC_OR_DIE();
+                if (tid == 0) {
+                    tc_fence_after_sync();
+                    issue_state_product<D>(tmem + aU, tK, tV);                   // Kc^T V
+                    if (BWD) issue_state_product<D>(tmem + aW, tQ, tG);         // Qc^T dO
+                    mma_commit(&ctl->bar[0]);
+                }
+                {
+                    if (u == nsub - 1 && tile + 1 < t1)
+                        load_raw<D, NT, BWD, BWD>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, b, h, rowTok + nxt * T);
+                    ok = wait_all(&ctl->bar[0], par, a.status);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        update_state<D, NT>(lane_base, tmem + aU, sm, S, vc.e2c, vc.ec);
+                        if (BWD) {
+                            // W_segment += (decay since the segment start) * exp(c) * (Qc^T dO)
+                            const float fs = sm.valid ? vc.aux[sm.c] : 0.f;
+#pragma unroll
+                            for (int i = 0; i < L::NPS; ++i)
+                                if (sm.has(i)) {
+                                    float w[8];
+                                    tmem_ld8(lane_base + tmem + aW + sm.tcol(i), w);
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) Wl[i][e] += fs * w[e];
+                                }
+                        }
+                    }
+                    tc_fence_before_sync();
+                }
+                par ^= 1;
+            }
+            cur = nxt;
+        }
+        {
+            store_state<D, NT>(a.seg_state + (size_t)sid * D * D, sm, S);
+            if (BWD) store_state<D, NT>(a.seg_dstate + (size_t)sid * D * D, sm, Wl);
+            if (tid < D) a.seg_gamma[(size_t)sid * D + tid] = gcum;
+        }
+    }
+die:
+    cta_teardown(ctl, SM::tmem_cols);
+}
+
+// =================================================================================================
+// seg_scan: the recurrence over segment ends, one sequence per blockIdx.y, 8 state rows per block,
+// 8 lanes per row.  Forward: seg_state[s] (state a segment leaves from a zero start) becomes the
+// state entering segment s.  Backward flavour: seg_dstate[s] (the segment's own contribution)
+// becomes the gradient with respect to the state leaving segment s, seg_carry the gate-gradient
+// carried into the segment from later ones, seg_state16 an fp16 copy of the entry states in the
+// dense chunk-major order the backward sweep bulk-copies.
+// =================================================================================================
+template <int D, bool BWD>
+__global__ void __launch_bounds__(64)
+seg_scan(float *seg_state, const float *seg_gamma, float *seg_dstate, float *seg_carry, __half *seg_state16,
+         const float *s_in, float *s_out, const float *ds_out, float *ds_in, int nseg)
+{
+    constexpr int NV = (D / 4 + 7) / 8;               // float4 pieces per lane
+    const int bh = blockIdx.y, c = blockIdx.x * 8 + (threadIdx.x >> 3), l8 = threadIdx.x & 7;
+    pdl_wait();
+    pdl_launch_dependents();
+    float4 s[NV];
+    const size_t row = (size_t)c * D;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const int e = 4 * (l8 + 8 * i);
+        s[i] = (s_in && e < D) ? *reinterpret_cast<const float4 *>(s_in + (size_t)bh * D * D + row + e) : make_float4(0, 0, 0, 0);
+    }
+    for (int sg = 0; sg < nseg; ++sg) {
+        float *st = seg_state + ((size_t)bh * nseg + sg) * D * D + row;
+        const float gam = exp2f(seg_gamma[((size_t)bh * nseg + sg) * D + c]);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int e = 4 * (l8 + 8 * i);
+            if (e < D) {
+                const float4 t = *reinterpret_cast<const float4 *>(st + e);
+                *reinterpret_cast<float4 *>(st + e) = s[i];
+                if (BWD) {
+                    __half2 lo = __floats2half2_rn(s[i].x, s[i].y), hi = __floats2half2_rn(s[i].z, s[i].w);
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<uint32_t *>(&lo);
+                    pk.y = *reinterpret_cast<uint32_t *>(&hi);
+                    char *dst = reinterpret_cast<char *>(seg_state16 + ((size_t)bh * nseg + sg) * D * D);
+                    *reinterpret_cast<uint2 *>(dst + ((e >> 3) * D + c) * 16 + (e & 7) * 2) = pk;
+                }
+                s[i] = make_float4(gam * s[i].x + t.x, gam * s[i].y + t.y, gam * s[i].z + t.z, gam * s[i].w + t.w);
+            }
+        }
+    }
+    if (s_out) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int e = 4 * (l8 + 8 * i);
+            if (e < D) *reinterpret_cast<float4 *>(s_out + (size_t)bh * D * D + row + e) = s[i];
+        }
+    }
+    if (BWD) {
+        float4 d[NV];
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int e = 4 * (l8 + 8 * i);
+            d[i] = (ds_out && e < D) ? *reinterpret_cast<const float4 *>(ds_out + (size_t)bh * D * D + row + e) : make_float4(0, 0, 0, 0);
+        }
+        // s holds the state leaving the last segment; walking back, it is replaced by the entry
+        // state of the following segment, which is the state leaving this one
+        for (int sg = nseg - 1; sg >= 0; --sg) {
+            float *dt = seg_dstate + ((size_t)bh * nseg + sg) * D * D + row;
+            const float gam = exp2f(seg_gamma[((size_t)bh * nseg + sg) * D + c]);
+            float dot = 0.f;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int e = 4 * (l8 + 8 * i);
+                if (e < D) {
+                    const float4 t = *reinterpret_cast<const float4 *>(dt + e);
+                    *reinterpret_cast<float4 *>(dt + e) = d[i];
+                    dot += s[i].x * d[i].x + s[i].y * d[i].y + s[i].z * d[i].z + s[i].w * d[i].w;
+                    d[i] = make_float4(gam * d[i].x + t.x, gam * d[i].y + t.y, gam * d[i].z + t.z, gam * d[i].w + t.w);
+                    s[i] = *reinterpret_cast<const float4 *>(seg_state + ((size_t)bh * nseg + sg) * D * D + row + e);
+                }
+            }
+            dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+            dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+            dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+            if (l8 == 0) seg_carry[((size_t)bh * nseg + sg) * D + c] = dot;
+        }
+        if (ds_in) {
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int e = 4 * (l8 + 8 * i);
+                if (e < D) *reinterpret_cast<float4 *>(ds_in + (size_t)bh * D * D + row + e) = d[i];
+            }
+        }
+    }
+}
+
+// =================================================================================================
+// sweep_fwd: a segment from its entry state; writes out.
+// =================================================================================================
+template <int D, int NT>
+struct FwdSmem {
+    using C = Cfg<D>;
+    using L = Lay<D, NT>;
+    static constexpr int kTiles = 3 * C::TILE_T + C::TILE_S + C::TILE_P;      // tQ tK tV tS tP
+    static constexpr int kFloats = T * C::LAMP + L::NSEG * D + 8 * D;
+    static constexpr size_t bytes = kTiles + kFloats * 4 + 3 * T * 4 + sizeof(Ctl);
+    static constexpr uint32_t tmem_cols = 256;
+};
+
+template <int D, int NT, typename TO>
+__global__ void __launch_bounds__(NT, NT == 256 ? 2 : 1)
+sweep_fwd(const SweepArgs a)
+{
+    using C = Cfg<D>;
+    using L = Lay<D, NT>;
+    using SM = FwdSmem<D, NT>;
+    extern __shared__ __align__(128) char smem[];
+    char *tQ = smem, *tK = tQ + C::TILE_T, *tV = tK + C::TILE_T, *tS = tV + C::TILE_T, *tP = tS + C::TILE_S;
+    float *table = reinterpret_cast<float *>(smem + SM::kTiles);
+    float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D;
+    int *rowTok = reinterpret_cast<int *>(vecb + 8 * D);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowTok + 3 * T);
+    constexpr uint32_t aP = 0, aO = 64, aU = 64 + C::NACC;
+
+    const int tid = threadIdx.x, lane = tid & 31, q4 = (tid >> 5) & 3, cg = tid >> 7, hf = lane >> 4;
+    const int r16 = 16 * q4 + (lane & 15);
+    cta_setup(ctl, 2, SM::tmem_cols, smem, SM::kTiles);
+    const uint32_t tmem = ctl->tmem_base, lane_base = (uint32_t)(32 * q4) << 16;
+    const Geom &g = a.g;
+    const Plan &pl = a.plan;
+    const StateMap<D, NT> sm;
+    float S[L::NPS][8];
+    Raw<L::NIT, true, false> raw;
+    uint32_t par = 0;
+    bool ok = true;
+    int cur = 0, iter = 0;
+    const int total = g.B * g.H * pl.nseg;
+    TO *out = reinterpret_cast<TO *>(a.out);
+
+    // the first tile's rows are inputs of the call: their loads need not wait for the scan kernel
+    {
+        const int sid = blockIdx.x;
+        if (sid < total) {
+            const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg;
+            if (tid < T) rowTok[cur * T + tid] = tile_token(g, sg * pl.G, tid);
+            __syncthreads();
+            load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, g, bh / g.H, bh % g.H, rowTok + cur * T);
+        }
+    }
+    pdl_wait();
+    pdl_launch_dependents();
+    for (int sid = blockIdx.x; sid < total; sid += gridDim.x) {
+        const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg, b = bh / g.H, h = bh - b * g.H;
+        const int t0 = sg * pl.G, t1 = min(t0 + pl.G, pl.ntile);
+        load_state<D, NT>(a.seg_state + (size_t)sid * D * D, sm, S);
+        if (sid != (int)blockIdx.x) {
+            if (tid < T) rowTok[cur * T + tid] = tile_token(g, t0, tid);
+            __syncthreads();
+            load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, g, b, h, rowTok + cur * T);
+        }
+        for (int tile = t0; tile < t1; ++tile) {
+            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
+            if (tid < T) rowTok[nxt * T + tid] = tile + 1 < t1 ? tile_token(g, tile + 1, tid) : -1;
+            write_gates<D, NT, true, false>(raw, table, rowTok + cur * T);
+            __syncthreads();
+            const int my_tok = rowTok[cur * T + r16];
+            float tot_unused;
+            const bool need = gate_prefix<D, NT>(table, sTot, tot_unused);
+            int s = pl.sub_max;
+            if (need || s < T) {
+                bool bad;
+                s = choose_sub<D>(table, need ? min(s, T / 2) : s, &bad);
+                if (bad && tid == 0) atomicOr(a.status, kStatusRange);
+            }
+            const int nsub = (nrow + s - 1) / s;
+            for (int u = 0; u < nsub; ++u, ++iter) {
+                const int lo = u * s, hi = min(lo + s, T);
+                const Vec vc = vec_of<D>(vecb, iter & 1);
+                if (tid < D) {
+                    const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
+                    const float t = table[(hi - 1) * C::LAMP + tid] - base, cv = 0.5f * t;
+                    vc.off[tid] = base + cv;
+                    vc.ec[tid] = ex2(cv);
+                    vc.e2c[tid] = ex2(t);
+                }
+                __syncthreads();
+                {
+                    build_tiles<D, NT, true, false>(raw, tQ, tK, tV, nullptr, table, vc.off, rowTok + cur * T, lo, min(hi, nrow));
+                    write_state_tile<D, NT>(tS, sm, S, vc.ec);                       // Sc = diag(2^c) S
+                    fence_async_smem();
+                }
+                tc_fence_before_sync();
+                SYNC_OR_DIE();
+                if (tid == 0) {
+                    tc_fence_after_sync();
+                    issue<64, 64, false, false>(tmem + aP, smem_u32(tQ), C::CHT, smem_u32(tK), C::CHT, C::KS, false);   // Qc Kc^T
+                    mma_commit(&ctl->bar[0]);
+                    issue<64, D, false, true>(tmem + aO, smem_u32(tQ), C::CHT, smem_u32(tS), C::CHS, C::KS, false);     // Qc Sc
+                    issue_state_product<D>(tmem + aU, tK, tV);                                                         // Kc^T V
+                    mma_commit(&ctl->bar[1]);
+                }
+                {
+                    if (u == nsub - 1 && tile + 1 < t1)
+                        load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, g, b, h, rowTok + nxt * T);
+                    ok = wait_all(&ctl->bar[0], 0, a.status);          // completes twice per iteration: parities 0, 1
+                    if (ok) {
+                        tc_fence_after_sync();
+                        // scores of row r16 (lanes 0-15 hold accumulator rows): keep s <= t, the diagonal has weight 1
+#pragma unroll
+                        for (int i = 0; i < L::NPT; ++i) {
+                            const int sc = cg + L::NCG * i;
+                            float p[8];
+                            tmem_ld8(lane_base + tmem + aP + 8 * sc, p);
+                            if (hf == 0) {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) p[e] = (8 * sc + e <= r16) ? p[e] : 0.f;
+                                *reinterpret_cast<uint4 *>(tP + sc * C::CHT + r16 * 16) = pack_h8(p);
+                            }
+                        }
+                    }
+                    fence_async_smem();
+                }
+                tc_fence_before_sync();
+                SYNC_OR_DIE();
+                if (tid == 0) {
+                    tc_fence_after_sync();
+                    issue<64, D, false, true>(tmem + aO, smem_u32(tP), C::CHT, smem_u32(tV), C::CHT, T / 16, true);     // + P V
+                    mma_commit(&ctl->bar[0]);
+                }
+                {
+                    // Kc^T V has completed with the first group: advance the state while P V is in the pipe
+                    ok = wait_all(&ctl->bar[1], par, a.status);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        update_state<D, NT>(lane_base, tmem + aU, sm, S, vc.e2c, vc.ec);
+                    }
+                    if (ok) ok = wait_all(&ctl->bar[0], 1, a.status);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        const bool inrow = hf == 0 && r16 >= lo && r16 < hi && my_tok >= 0;
+                        const size_t ro = tok_offset(g, b, my_tok < 0 ? 0 : my_tok, h, D);
+#pragma unroll
+                        for (int i = 0; i < L::NPC; ++i) {
+                            const int jc = cg + L::NCG * i;
+                            if (jc < C::NCH) {
+                                float o[8];
+                                tmem_ld8(lane_base + tmem + aO + 8 * jc, o);
+                                if (inrow) store_out8(out + ro + 8 * jc, o);
+                            }
+                        }
+                    }
+                    tc_fence_before_sync();
+                }
+                par ^= 1;          // parity of bar[1], which completes once per iteration
+            }
+            cur = nxt;
+        }
+    }
+die:
+    cta_teardown(ctl, SM::tmem_cols);
+}
+
+// =================================================================================================
+// sweep_bwd: a segment in reverse scan order with the state gradient on chip.
+// =================================================================================================
+template <int D, int NT>
+struct BwdSmem {
+    using C = Cfg<D>;
+    using L = Lay<D, NT>;
+    static constexpr int kTiles = 4 * C::TILE_T + 3 * C::TILE_S + 2 * C::TILE_P;      // tQ tK tV tG | tS tI tD | tP tdP
+    static constexpr int kFloats = T * C::LAMP + L::NSEG * D + 8 * D + 2 * D;
+    static constexpr size_t bytes = kTiles + kFloats * 4 + 3 * T * 4 + sizeof(Ctl);
+    static constexpr uint32_t tmem_cols = 256;
+};
+
+template <int D, int NT, typename TO>
+__global__ void __launch_bounds__(NT, NT == 256 ? 2 : 1)
+sweep_bwd(const SweepArgs a)
+{
+    using C = Cfg<D>;
+    using L = Lay<D, NT>;
+    using SM = BwdSmem<D, NT>;
+    extern __shared__ __align__(128) char smem[];
+    char *tQ = smem, *tK = tQ + C::TILE_T, *tV = tK + C::TILE_T, *tG = tV + C::TILE_T;
+    char *tS = tG + C::TILE_T, *tI = tS + C::TILE_S, *tD = tI + C::TILE_S;
+    char *tP = tD + C::TILE_S, *tdP = tP + C::TILE_P;
+    float *table = reinterpret_cast<float *>(smem + SM::kTiles);
+    float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D, *sCarry = vecb + 8 * D;
+    int *rowTok = reinterpret_cast<int *>(sCarry + 2 * D);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowTok + 3 * T);
+    constexpr uint32_t W0 = C::BIGM ? C::NACC : 64;
+    constexpr uint32_t aP = 0, aQK = W0, aV = W0 + C::NACC, kHi = 16u << 16;
+    static_assert(aV + C::NACC <= SM::tmem_cols, "tensor memory");
+
+    const int tid = threadIdx.x, lane = tid & 31, q4 = (tid >> 5) & 3, cg = tid >> 7, hf = lane >> 4;
+    const int r16 = 16 * q4 + (lane & 15);
+    cta_setup(ctl, 2, SM::tmem_cols, smem, SM::kTiles);
+    const uint32_t tmem = ctl->tmem_base, lane_base = (uint32_t)(32 * q4) << 16;
+    uint64_t *barG1 = &ctl->bar[0], *barS = &ctl->bar[1];
+    const Geom &g = a.g;
+    const Plan &pl = a.plan;
+    const StateMap<D, NT> sm;
+    float Dst[L::NPS][8];
+    Raw<L::NIT, true, true> raw;
+    uint32_t par = 0;
+    bool ok = true;
+    int cur = 0, iter = 0, cpar = 0;
+    const int total = g.B * g.H * pl.nseg;
+    TO *dq = reinterpret_cast<TO *>(a.dq), *dk = reinterpret_cast<TO *>(a.dk), *dv = reinterpret_cast<TO *>(a.dv);
+
+    {
+        const int sid = blockIdx.x;
+        if (sid < total) {
+            const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg;
+            const int t1 = min(sg * pl.G + pl.G, pl.ntile);
+            if (tid < T) rowTok[cur * T + tid] = tile_token(g, t1 - 1, tid);
+            __syncthreads();
+            load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, bh / g.H, bh % g.H, rowTok + cur * T);
+        }
+    }
+    pdl_wait();
+    pdl_launch_dependents();
+    for (int sid = blockIdx.x; sid < total; sid += gridDim.x) {
+        const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg, b = bh / g.H, h = bh - b * g.H;
+        const int t0 = sg * pl.G, t1 = min(t0 + pl.G, pl.ntile);
+        load_state<D, NT>(a.seg_dstate + (size_t)sid * D * D, sm, Dst);
+        if (tid < D) sCarry[cpar * D + tid] = a.seg_carry[(size_t)sid * D + tid];
+        if (sid != (int)blockIdx.x) {
+            if (tid < T) rowTok[cur * T + tid] = tile_token(g, t1 - 1, tid);
+            __syncthreads();
+            load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, b, h, rowTok + cur * T);
+        }
+        const char *seg16 = reinterpret_cast<const char *>(a.seg_state16 + (size_t)sid * D * D);
+        for (int tile = t1 - 1; tile >= t0; --tile) {
+            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
+            if (tid < T) rowTok[nxt * T + tid] = tile > t0 ? tile_token(g, tile - 1, tid) : -1;
+            write_gates<D, NT, true, true>(raw, table, rowTok + cur * T);
+            __syncthreads();
+            const int my_tok = rowTok[cur * T + r16];
+            // decay since the segment start of the sub-chunk worked first (always slot 0): fetched ahead of its use
+            const float g_first = tid < D ? a.slot_g[((size_t)bh * pl.ntile + tile) * D + tid] : 0.f;
+            float tot_unused;
+            const bool need = gate_prefix<D, NT>(table, sTot, tot_unused);
+            int s = pl.sub_max;
+            if (need || s < T) {
+                bool bad;
+                s = choose_sub<D>(table, need ? min(s, T / 2) : s, &bad);
+                if (bad && tid == 0) atomicOr(a.status, kStatusRange);
+            }
+            const int nsub = (nrow + s - 1) / s;
+            for (int u = nsub - 1; u >= 0; --u, ++iter) {
+                const int lo = u * s, hi = min(lo + s, T), hiv = min(hi, nrow);
+                const size_t slot = ((size_t)(nsub - 1 - u) * g.B * g.H + bh) * pl.ntile + tile;
+                const Vec vc = vec_of<D>(vecb, iter & 1);
+                if (tid < D) {
+                    const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
+                    const float t = table[(hi - 1) * C::LAMP + tid] - base, cv = 0.5f * t;
+                    vc.off[tid] = base + cv;
+                    vc.ec[tid] = ex2(cv);
+                    vc.e2c[tid] = ex2(t);
+                    vc.aux[tid] = ex2(cv + (u == nsub - 1 ? g_first : a.slot_g[slot * D + tid]));   // exp(c) * decay since the segment start
+                }
+                // every thread has passed its wait for the previous products: the two state tiles are free again
+                __syncthreads();
+                if (tid == 0) {
+                    const char *src = reinterpret_cast<const char *>(a.slot_s + slot * (D * D));
+                    fence_async_smem();
+                    mbar_arrive_expect_tx(barS, 2u * C::NCH * D * 16u);
+                    for (int j = 0; j < C::NCH; ++j) {
+                        bulk_g2s(tS + j * C::CHS, src + j * D * 16, D * 16, barS);
+                        bulk_g2s(tI + j * C::CHS, seg16 + j * D * 16, D * 16, barS);
+                    }
+                }
+                {
+                    build_tiles<D, NT, true, true>(raw, tQ, tK, tV, tG, table, vc.off, rowTok + cur * T, lo, hiv);
+                    write_state_tile<D, NT>(tD, sm, Dst, vc.ec);                    // Dc = diag(2^c) D
+                    fence_async_smem();
+                }
+                tc_fence_before_sync();
+                SYNC_OR_DIE();
+                if (tid == 0) {
+                    ok = mbar_wait(barS, par, a.status);          // both state tiles have landed
+                    tc_fence_after_sync();
+                    const uint32_t sQ = smem_u32(tQ), sK = smem_u32(tK), sV = smem_u32(tV), sG = smem_u32(tG);
+                    const uint32_t sS = smem_u32(tS), sI = smem_u32(tI), sD = smem_u32(tD);
+                    issue<64, 64, false, false>(tmem + aP, sQ, C::CHT, sK, C::CHT, C::KS, false);             // Qc Kc^T
+                    issue<64, 64, false, false>(tmem + aP + kHi, sG, C::CHT, sV, C::CHT, C::KS, false);       // dO V^T
+                    mma_commit(barG1);
+                    issue<64, D, false, false>(tmem + aQK, sG, C::CHT, sS, C::CHS, C::KS, false);             // dO Sc_local^T
+                    issue<64, D, false, false>(tmem + aV, sG, C::CHT, sI, C::CHS, C::KS, false);              // dO S_segment^T
+                    issue<64, D, false, false>(tmem + aQK + kHi, sV, C::CHT, sD, C::CHS, C::KS, false);       // V Dc^T
+                    issue<64, D, false, true>(tmem + aV + kHi, sK, C::CHT, sD, C::CHS, C::KS, false);         // Kc Dc
+                }
+                {
+                    if (u == 0 && tile > t0)
+                        load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, b, h, rowTok + nxt * T);
+                    ok = wait_all(barG1, 0, a.status);                 // completes twice per iteration: parities 0, 1
+                    if (ok) {
+                        tc_fence_after_sync();
+                        // lanes 0-15: scores, lanes 16-31: dO V^T; keep s <= t, the diagonal has weight 1
+#pragma unroll
+                        for (int i = 0; i < L::NPT; ++i) {
+                            const int sc = cg + L::NCG * i;
+                            float p[8];
+                            tmem_ld8(lane_base + tmem + aP + 8 * sc, p);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) p[e] = (8 * sc + e <= r16) ? p[e] : 0.f;
+                            *reinterpret_cast<uint4 *>((hf ? tdP : tP) + sc * C::CHT + r16 * 16) = pack_h8(p);
+                        }
+                    }
+                    fence_async_smem();
+                }
+                tc_fence_before_sync();
+                SYNC_OR_DIE();
+                if (tid == 0) {
+                    tc_fence_after_sync();
+                    const uint32_t sQ = smem_u32(tQ), sK = smem_u32(tK), sG = smem_u32(tG);
+                    const uint32_t sP = smem_u32(tP), sdP = smem_u32(tdP);
+                    issue<64, D, false, true>(tmem + aQK, sdP, C::CHT, sK, C::CHT, T / 16, true);             // + dP Kc
+                    issue<64, D, true, true>(tmem + aQK + kHi, sdP, C::CHT, sQ, C::CHT, T / 16, true);        // + dP^T Qc
+                    issue<64, D, true, true>(tmem + aV + kHi, sP, C::CHT, sG, C::CHT, T / 16, true);          // + P^T dO
+                    issue_state_product<D>(tmem + aP, tQ, tG);                                                // Qc^T dO
+                    mma_commit(barG1);
+                }
+                {
+                    ok = wait_all(barG1, 1, a.status);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        const bool inrow = r16 >= lo && r16 < hiv;
+                        const size_t ro = tok_offset(g, b, my_tok < 0 ? 0 : my_tok, h, D);
+#pragma unroll
+                        for (int i = 0; i < L::NPC; ++i) {
+                            const int jc = cg + L::NCG * i;
+                            if (jc < C::NCH) {          // uniform over the warp
+                                float a1[8], a2[8], lam[8], of[8], t8[8], x[8];
+                                // lanes 0-15: dq accumulator and dO S_segment^T; lanes 16-31: dk and dv accumulators
+                                tmem_ld8_pair(lane_base + tmem + aQK + 8 * jc, lane_base + tmem + aV + 8 * jc, a1, a2);
+                                ld8(table + r16 * C::LAMP + 8 * jc, lam);
+                                ld8(vc.off + 8 * jc, of);
+                                unpack_h8(*reinterpret_cast<const uint4 *>((hf ? tK : tQ) + jc * C::CHT + r16 * 16), t8);
+                                if (hf == 0) {
+                                    float hh[8];
+                                    ld8(vc.aux + 8 * jc, hh);
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) a1[e] = fmaf(hh[e], a2[e], a1[e]);
+                                }
+                                // q*dq = Qc * (dq accumulator), k*dk = Kc * (dk accumulator): the decay factors cancel
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    x[e] = t8[e] * a1[e];
+                                    a1[e] *= ex2(hf ? of[e] - lam[e] : lam[e] - of[e]);
+                                }
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) x[e] -= __shfl_xor_sync(0xffffffffu, x[e], 16);
+                                __syncwarp();           // both halves have read their gates before the table is overwritten
+                                if (inrow) {
+                                    if (hf == 0) {
+                                        st8(table + r16 * C::LAMP + 8 * jc, x);                 // q*dq - k*dk
+                                        store_out8(dq + ro + 8 * jc, a1);
+                                    } else {
+                                        store_out8(dk + ro + 8 * jc, a1);
+                                        store_out8(dv + ro + 8 * jc, a2);
+                                    }
+                                }
+                            }
+                        }
+                        // D <- 2^(2c) D + 2^c (Qc^T dO)
+                        update_state<D, NT>(lane_base, tmem + aP, sm, Dst, vc.e2c, vc.ec);
+                    }
+                    tc_fence_before_sync();
+                }
+                par ^= 1;
+            }
+            // gate gradient of the tile: suffix sums of q*dq - k*dk down the rows plus what later tiles carry in
+            SYNC_OR_DIE();
+            {
+                const bool active = tid < L::NSEG * D;
+                const int seg = tid / D, c = tid - seg * D, r0 = seg * L::RPS;
+                float sfx[L::RPS];
+                if (active) {
+                    float run = 0.f;
+#pragma unroll
+                    for (int j = L::RPS - 1; j >= 0; --j) {
+                        if (r0 + j < nrow) run += table[(r0 + j) * C::LAMP + c];
+                        sfx[j] = run;
+                    }
+                    sTot[seg * D + c] = run;
+                }
+                __syncthreads();
+                if (active) {
+                    float add = sCarry[cpar * D + c], all = 0.f;
+#pragma unroll
+                    for (int sgm = 0; sgm < L::NSEG; ++sgm) {
+                        const float t = sTot[sgm * D + c];
+                        if (sgm > seg) add += t;
+                        all += t;
+                    }
+                    if (seg == 0) sCarry[(cpar ^ 1) * D + c] = sCarry[cpar * D + c] + all;
+#pragma unroll
+                    for (int j = 0; j < L::RPS; ++j) {
+                        const int tok = r0 + j < nrow ? rowTok[cur * T + r0 + j] : -1;
+                        if (tok >= 0) a.dgate[tok_offset(g, b, tok, h, D) + c] = sfx[j] + add;
+                    }
+                }
+                cpar ^= 1;
+            }
+            cur = nxt;
+        }
+    }
+die:
+    if (!ok && tid == 0) mbar_wait(barS, par, a.status);      // let bulk copies in flight land
+    cta_teardown(ctl, SM::tmem_cols);
+}
+
+#undef SYNC_OR_DIE
+
+// ---- host side ----------------------------------------------------------------------------------
+template <int D>
+constexpr int ctas_per_sm() { return 2; }
+template <>
+constexpr int ctas_per_sm<72>() { return 1; }
+template <int D>
+constexpr int worker_threads() { return ctas_per_sm<D>() == 2 ? 256 : 512; }
+
+Plan make_plan(const Geom &g, int sms, int per_sm)
+{
+    Plan p;
+    p.ntile = (g.L + T - 1) / T;
+    p.sub_max = g.C < T ? g.C : T;
+    const long long slots = (long long)sms * per_sm, bh = (long long)g.B * g.H;
+    long long best = -1;
+    p.G = p.ntile;
+    for (int G = p.ntile; G >= 1; --G) {
+        const int nseg = (p.ntile + G - 1) / G;
+        const long long rounds = (bh * nseg + slots - 1) / slots;
+        const long long cost = rounds * (G + 1);          // a segment costs about one tile of fill and drain
+        if (best < 0 || cost < best) {
+            best = cost;
+            p.G = G;
+        }
+    }
+    p.nseg = (p.ntile + p.G - 1) / p.G;
+    return p;
+}
+
+struct SweepWs {
+    float *seg_state, *seg_gamma, *seg_dstate, *seg_carry, *slot_g;
+    __half *seg_state16, *slot_s;
+    size_t bytes;
+};
+SweepWs carve(char *base, const Geom &g, const Plan &pl, bool backward)
+{
+    SweepWs w{};
+    const size_t segs = (size_t)g.B * g.H * pl.nseg, dd = (size_t)g.dk * g.dv;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { char *p = base + o; o += align256(bytes); return p; };
+    w.seg_state = reinterpret_cast<float *>(take(segs * dd * 4));
+    w.seg_gamma = reinterpret_cast<float *>(take(segs * g.dk * 4));
+    if (backward) {
+        const size_t slots = (size_t)kSlots * g.B * g.H * pl.ntile;
+        w.seg_dstate = reinterpret_cast<float *>(take(segs * dd * 4));
+        w.seg_carry = reinterpret_cast<float *>(take(segs * g.dk * 4));
+        w.seg_state16 = reinterpret_cast<__half *>(take(segs * dd * 2));
+        w.slot_s = reinterpret_cast<__half *>(take(slots * dd * 2));
+        w.slot_g = reinterpret_cast<float *>(take(slots * g.dk * 4));
+    }
+    w.bytes = o;
+    return w;
+}
+
+int sweep_per_sm(int d) { return d == 64 ? ctas_per_sm<64>() : ctas_per_sm<72>(); }
+
+template <typename K>
+dig_status set_smem(K kern, size_t bytes)
+{
+    return cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+}
+
+template <int D, bool BWD>
+dig_status run(const GlaArgs &ga)
+{
+    constexpr int NT = worker_threads<D>();
+    const Geom &g = ga.g;
+    const int sms = device_sm_count();
+    int *status = device_status_ptr();
+    if (!status || sms <= 0) return DIG_ERR_CUDA;
+    const Plan pl = make_plan(g, sms, ctas_per_sm<D>());
+    const SweepWs w = carve(reinterpret_cast<char *>(ga.ws), g, pl, BWD);
+    const long long total = (long long)g.B * g.H * pl.nseg;
+    if (total > (1ll << 30)) return DIG_ERR_UNSUPPORTED;
+    SweepArgs a{};
+    a.q = (const bf16 *)ga.q; a.k = (const bf16 *)ga.k; a.v = (const bf16 *)ga.v; a.d_out = (const bf16 *)ga.d_out;
+    a.gate = ga.gate;
+    a.out = ga.out; a.dq = ga.dq; a.dk = ga.dk; a.dv = ga.dv; a.dgate = ga.dgate;
+    a.seg_state = w.seg_state; a.seg_gamma = w.seg_gamma; a.seg_dstate = w.seg_dstate; a.seg_carry = w.seg_carry;
+    a.seg_state16 = w.seg_state16; a.slot_s = w.slot_s; a.slot_g = w.slot_g;
+    a.status = status;
+    a.g = g;
+    a.plan = pl;
+    const int grid = (int)(total < (long long)sms * ctas_per_sm<D>() ? total : (long long)sms * ctas_per_sm<D>());
+    dig_status st;
+    {
+        auto kern = sweep_local<D, NT, BWD>;
+        constexpr size_t smem = LocalSmem<D, NT, BWD>::bytes;
+        if ((st = set_smem(kern, smem)) != DIG_OK) return st;
+        KernelTimer t(KID_SW_LOCAL, ga.stream);
+        launch_pdl(kern, dim3(grid), dim3(NT), smem, ga.stream, a);
+        if ((st = cuda_ok(cudaGetLastError())) != DIG_OK) return st;
+    }
+    {
+        auto kern = seg_scan<D, BWD>;
+        KernelTimer t(KID_SW_SCAN, ga.stream);
+        launch_pdl(kern, dim3(D / 8, g.B * g.H), dim3(64), 0, ga.stream, w.seg_state, (const float *)w.seg_gamma, w.seg_dstate,
+                   w.seg_carry, w.seg_state16, ga.sio.s_in, ga.sio.s_out, ga.sio.ds_out, ga.sio.ds_in, pl.nseg);
+        if ((st = cuda_ok(cudaGetLastError())) != DIG_OK) return st;
+    }
+    const bool f32 = ga.dtype == DIG_BF16_F32OUT;
+    if (!BWD) {
+        constexpr size_t smem = FwdSmem<D, NT>::bytes;
+        auto k16 = sweep_fwd<D, NT, bf16>;
+        auto k32 = sweep_fwd<D, NT, float>;
+        if ((st = set_smem(k16, smem)) != DIG_OK || (st = set_smem(k32, smem)) != DIG_OK) return st;
+        KernelTimer t(KID_SW_FWD, ga.stream);
+        launch_pdl(f32 ? k32 : k16, dim3(grid), dim3(NT), smem, ga.stream, a);
+    } else {
+        constexpr size_t smem = BwdSmem<D, NT>::bytes;
+        auto k16 = sweep_bwd<D, NT, bf16>;
+        auto k32 = sweep_bwd<D, NT, float>;
+        if ((st = set_smem(k16, smem)) != DIG_OK || (st = set_smem(k32, smem)) != DIG_OK) return st;
+        KernelTimer t(KID_SW_BWD, ga.stream);
+        launch_pdl(f32 ? k32 : k16, dim3(grid), dim3(NT), smem, ga.stream, a);
+    }
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace
+
+bool sweep_supports(int dk, int dv, int chunk, int dtype)
+{
+    if (dtype != DIG_BF16 && dtype != DIG_BF16_F32OUT) return false;
+    (void)chunk;                     // every chunk size is worked in 64-token tiles, shorter ones as sub-chunks
+    return dk == dv && (dk == 64 || dk == 72);
+}
+
+size_t sweep_workspace_bytes(const Geom &g, bool backward)
+{
+    int sms = device_sm_count();
+    if (sms <= 0) sms = 148;
+    const Plan pl = make_plan(g, sms, sweep_per_sm(g.dk));
+    return carve(nullptr, g, pl, backward).bytes;
+}
+
+dig_status sweep_gla_fwd(const GlaArgs &a)
+{
+    return a.g.dk == 64 ? run<64, false>(a) : run<72, false>(a);
+}
+dig_status sweep_gla_bwd(const GlaArgs &a)
+{
+    return a.g.dk == 64 ? run<64, true>(a) : run<72, true>(a);
+}
+
+}  // namespace dig

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libdig_gla.so")
 DIG_OK = 0
 DIG_ERR_INVALID_ARG, DIG_ERR_UNSUPPORTED, DIG_ERR_WORKSPACE, DIG_ERR_CUDA, DIG_ERR_TIMEOUT = 1, 2, 3, 4, 5
 DIG_ERR_SCRATCH_LIMIT = 6
+DIG_ERR_RANGE = 7
 DIG_GLA_STATIC_SCRATCH_BYTES = 16 << 20
 DIG_F32, DIG_BF16, DIG_BF16_F32OUT = 0, 1, 2
 DIG_ROW_FWD, DIG_ROW_REV, DIG_COL_FWD, DIG_COL_REV = 0, 1, 2, 3

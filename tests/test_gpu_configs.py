@@ -29,7 +29,7 @@ def test_c5_other_directions_four_heads(direction):
 @pytest.mark.parametrize("chunk", [32, 64, 128])
 def test_c4_chunk_sweep(chunk):
     """112 x 112 grid: 64 does not divide the column length, so column orders straddle columns.
-    Chunk 32 runs on the fp32-FMA kernels, 64 and 128 on the tensor-core kernels (128 in 64-token tiles)."""
+    Every chunk size must be served by some kernel family, forward and backward."""
     from paper_2405_18428_b200 import dig
     from parity import check_workload
     wl = CONFIGS["C4"]

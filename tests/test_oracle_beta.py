@@ -84,3 +84,18 @@ def test_suffix_sum_identities_of_both_gate_gradients():
     xb = (o * dO - v * dv)[:, p]
     np.testing.assert_allclose(da[:, p], np.cumsum(xa[:, ::-1], axis=1)[:, ::-1], rtol=1e-11, atol=1e-12)
     np.testing.assert_allclose(db[:, p], np.cumsum(xb[:, ::-1], axis=1)[:, ::-1], rtol=1e-11, atol=1e-12)
+
+
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+def test_suffix_sum_identities_across_checkpoint_segments(direction):
+    """Both identities on 200 scan positions, more than one stored-state segment of the backward sweep."""
+    q, k, v, a, bg, dO = _inputs(5 + direction, B=1, L=200)
+    a, bg = a * 0.4, bg * 0.4
+    gh, gw = 10, 20
+    o = oracle.gla_fwd_beta(q, k, v, a, bg, gh, gw, direction)
+    dq, dk, dv, da, db = oracle.gla_bwd_beta(q, k, v, a, bg, dO, gh, gw, direction)
+    p = oracle.perm(direction, gh, gw)
+    xa = (q * dq - k * dk)[:, p]
+    xb = (o * dO - v * dv)[:, p]
+    np.testing.assert_allclose(da[:, p], np.cumsum(xa[:, ::-1], axis=1)[:, ::-1], rtol=1e-9, atol=1e-10)
+    np.testing.assert_allclose(db[:, p], np.cumsum(xb[:, ::-1], axis=1)[:, ::-1], rtol=1e-9, atol=1e-10)

@@ -189,6 +189,23 @@ def test_gate_gradient_suffix_sum_identity(direction):
     np.testing.assert_allclose(np.sum(v * dv), np.sum(dO * o), rtol=1e-11)
 
 
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+def test_gate_gradient_suffix_sum_identity_across_checkpoint_segments(direction):
+    """The same identity on 200 scan positions (10 x 20 grid): the oracle's backward sweep restarts
+    from a stored state several times on the way, so a slip in how the gate gradient uses the
+    recomputed states would break the running sum here while leaving short sequences intact."""
+    rng = np.random.default_rng(20 + direction)
+    gh, gw = 10, 20
+    q, k, v, a = _rand(rng, 1, gh * gw, 2, 4, 3, decay_scale=0.25)
+    dO = rng.standard_normal(v.shape)
+    dq, dk, dv, da = oracle.gla_bwd(q, k, v, a, dO, gh, gw, direction)
+    p = _scan_orders(gh, gw)[direction]
+    x = (q * dq - k * dk)[:, p]
+    suffix = np.cumsum(x[:, ::-1], axis=1)[:, ::-1]
+    np.testing.assert_allclose(da[:, p], suffix, rtol=1e-9, atol=1e-10)
+    np.testing.assert_allclose(da[:, p[0]], 0.0, atol=1e-10)
+
+
 def test_threads_do_not_change_results():
     rng = np.random.default_rng(11)
     q, k, v, a = _rand(rng, 2, 64, 3, 8, 8)

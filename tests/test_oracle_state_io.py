@@ -93,3 +93,33 @@ def test_state_gradients_by_finite_differences(direction):
             pa[which], ma[which] = ap, am
             fd = (loss(*pa) - loss(*ma)) / (2 * h)
             assert abs(fd - grad[idx]) <= 2e-7 * max(1.0, abs(fd)), (which, idx, fd, grad[idx])
+
+
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+def test_two_pieces_chained_equal_the_whole_across_checkpoint_segments(direction):
+    """A 300-position sequence cut at 170: both pieces are longer than one stored-state segment of
+    the backward sweep, so ds_in, da and the other gradients are pinned where states are recomputed.
+    The cut is made in scan order (pieces are 1 x n rows holding the tokens in the order visited)."""
+    B, H, dk, dv, gh, gw, cut = 1, 2, 3, 4, 15, 20, 170
+    L = gh * gw
+    q, k, v, a, dO = _inputs(40 + direction, B=B, H=H, L=L, dk=dk, dv=dv)
+    a = a * 0.3
+    rng = np.random.default_rng(41)
+    s_in, ds_out = rng.standard_normal((B, H, dk, dv)), rng.standard_normal((B, H, dk, dv))
+    o, s_out = oracle.gla_fwd_state(q, k, v, a, s_in, gh, gw, direction)
+    dq, dk_, dv_, da, ds_in = oracle.gla_bwd_state(q, k, v, a, dO, s_in, ds_out, gh, gw, direction)
+    idx = np.arange(L)
+    col = idx.reshape(gh, gw).T.ravel()
+    p = {0: idx, 1: idx[::-1], 2: col, 3: col[::-1]}[direction]          # scan position -> token
+    sq, sk, sv, sa, sdO = (x[:, p] for x in (q, k, v, a, dO))
+    A = tuple(x[:, :cut] for x in (sq, sk, sv, sa, sdO))
+    Bp = tuple(x[:, cut:] for x in (sq, sk, sv, sa, sdO))
+    oA, sA = oracle.gla_fwd_state(*A[:4], s_in, 1, cut, 0)
+    oB, sB = oracle.gla_fwd_state(*Bp[:4], sA, 1, L - cut, 0)
+    np.testing.assert_allclose(np.concatenate([oA, oB], axis=1), o[:, p], rtol=1e-11, atol=1e-11)
+    np.testing.assert_allclose(sB, s_out, rtol=1e-11, atol=1e-11)
+    gB = oracle.gla_bwd_state(*Bp, sA, ds_out, 1, L - cut, 0)
+    gA = oracle.gla_bwd_state(*A, s_in, gB[4], 1, cut, 0)
+    for whole, pa, pb in zip((dq, dk_, dv_, da), gA[:4], gB[:4]):
+        np.testing.assert_allclose(np.concatenate([pa, pb], axis=1), whole[:, p], rtol=1e-9, atol=1e-10)
+    np.testing.assert_allclose(gA[4], ds_in, rtol=1e-9, atol=1e-10)

@@ -31,6 +31,7 @@ def _inputs(wl):
 
 def test_static_scratch_forward_matches_workspace_forward_twice():
     import torch
+    import oracle
     from parity import TOL_BF16, rel_err
     from paper_2405_18428_b200 import dig
 
@@ -41,16 +42,30 @@ def test_static_scratch_forward_matches_workspace_forward_twice():
     second = Workload("static-b", B=1, H=2, grid_h=9, grid_w=31, d_k=64, d_v=64, chunk=64, dtype="bf16",
                       tau=(4.0,), seed=12)
     for wl, direction in ((first, 0), (second, 3)):
+        x = make_inputs(wl, conv=False)
         q, k, v, gate = _inputs(wl)
         want = dig.dig_gla_fwd(q, k, v, gate, wl.grid_h, wl.grid_w, wl.chunk, direction, f32_out=True)
         out = torch.full(want.shape, float("nan"), dtype=torch.float32, device="cuda")   # caller-owned output
+        dig.dig_gla_fwd_static(q, k, v, gate, out, wl.grid_h, wl.grid_w, wl.chunk, direction)   # first call on the device: set-up
+        torch.cuda.synchronize()
+        # a second call must leave both torch's allocator and the device's free memory untouched
+        out.fill_(float("nan"))
+        torch.cuda.synchronize()
+        held, (free0, _) = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()
         dig.dig_gla_fwd_static(q, k, v, gate, out, wl.grid_h, wl.grid_w, wl.chunk, direction)
         torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == held
+        assert torch.cuda.mem_get_info()[0] == free0
         assert dig.dig_last_device_status() == dig.DIG_OK
-        got, ref = out.cpu().numpy(), want.cpu().numpy().astype(np.float64)
+        got = out.cpu().numpy()
         assert np.isfinite(got).all()
+        # the header promises the same kernels on other scratch memory: the same bits
+        np.testing.assert_array_equal(got, want.cpu().numpy())
+        # and, like every other entry point, it is held against the fp64 oracle
+        a = oracle.gate(x["g"], x["tau"])
+        ref = oracle.gla_fwd(x["q"], x["k"], x["v"], a, wl.grid_h, wl.grid_w, direction)
         err = rel_err(got, ref)
-        assert err <= TOL_BF16, f"{wl.name}: static-scratch forward differs from dig_gla_fwd by {err:.3e}"
+        assert err <= TOL_BF16, f"{wl.name}: static-scratch forward differs from the oracle by {err:.3e}"
 
 
 def test_static_scratch_rejects_problems_beyond_its_limit():
