@@ -69,43 +69,41 @@ __device__ __forceinline__ void cta_teardown(Ctl *ctl, uint32_t tmem_cols)
 
 // Operand tiles of rows [lo, hi) of the prefetched tile (the other rows are zero):
 //   tK <- k 2^(off - Lam), tV <- v, and where present tQ <- q 2^(Lam - off), tG <- dO.
+__device__ __forceinline__ uint4 keep4(const uint4 &u, uint32_t m) { return make_uint4(u.x & m, u.y & m, u.z & m, u.w & m); }
 template <int D, int NT, bool HQ, bool HD>
 __device__ __forceinline__ void build_tiles(const Raw<Lay<D, NT>::NIT, HQ, HD> &r, char *tQ, char *tK, char *tV, char *tG,
-                                            const float *table, const float *off, const int *row_tok, int lo, int hi)
+                                            const float *table, const float *off, const int *row_off, int lo, int hi)
 {
     using C = Cfg<D>;
 #pragma unroll
     for (int i = 0; i < Lay<D, NT>::NIT; ++i) {
         const int it = (int)threadIdx.x + NT * i;
-        if (it < T * C::NCH) {
+        if (item_exists<D, NT>(it)) {
             const int row = it / C::NCH, j = it - row * C::NCH;
             const int o = j * C::CHT + row * 16;
-            if (row >= lo && row < hi && row_tok[row] >= 0) {
-                float lam[8], of[8], x[8], y[8];
-                ld8(table + row * C::LAMP + 8 * j, lam);
-                ld8(off + 8 * j, of);
-                unpack_b8(r.k[i], x);
+            // rows outside the sub-chunk or past the end of the sequence become zeros: no branch, a mask on the
+            // packed result (which also discards whatever an out-of-range exponent produced there)
+            const uint32_t m = (row >= lo && row < hi && row_off[row] >= 0) ? 0xffffffffu : 0u;
+            float lam[8], of[8], x[8], y[8];
+            ld8(table + row * C::LAMP + 8 * j, lam);
+            ld8(off + 8 * j, of);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) y[e] = x[e] * ex2(of[e] - lam[e]);
-                *reinterpret_cast<uint4 *>(tK + o) = pack_h8(y);
-                unpack_b8(r.v[i], x);
-                *reinterpret_cast<uint4 *>(tV + o) = pack_h8(x);
-                if (HQ) {
-                    unpack_b8(r.q[i], x);
+            for (int e = 0; e < 8; ++e) lam[e] -= of[e];
+            unpack_b8(r.k[i], x);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) y[e] = x[e] * ex2(lam[e] - of[e]);
-                    *reinterpret_cast<uint4 *>(tQ + o) = pack_h8(y);
-                }
-                if (HD) {
-                    unpack_b8(r.d[i], x);
-                    *reinterpret_cast<uint4 *>(tG + o) = pack_h8(x);
-                }
-            } else {
-                const uint4 z = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4 *>(tK + o) = z;
-                *reinterpret_cast<uint4 *>(tV + o) = z;
-                if (HQ) *reinterpret_cast<uint4 *>(tQ + o) = z;
-                if (HD) *reinterpret_cast<uint4 *>(tG + o) = z;
+            for (int e = 0; e < 8; ++e) y[e] = x[e] * ex2(-lam[e]);
+            *reinterpret_cast<uint4 *>(tK + o) = keep4(pack_h8(y), m);
+            unpack_b8(r.v[i], x);
+            *reinterpret_cast<uint4 *>(tV + o) = keep4(pack_h8(x), m);
+            if (HQ) {
+                unpack_b8(r.q[i], x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) y[e] = x[e] * ex2(lam[e]);
+                *reinterpret_cast<uint4 *>(tQ + o) = keep4(pack_h8(y), m);
+            }
+            if (HD) {
+                unpack_b8(r.d[i], x);
+                *reinterpret_cast<uint4 *>(tG + o) = keep4(pack_h8(x), m);
             }
         }
     }
@@ -167,8 +165,8 @@ sweep_local(const SweepArgs a)
     char *tQ = smem, *tK = BWD ? tQ + C::TILE_T : smem, *tV = tK + C::TILE_T, *tG = tV + C::TILE_T;
     float *table = reinterpret_cast<float *>(smem + SM::kTilesPad);
     float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D;
-    int *rowTok = reinterpret_cast<int *>(vecb + 8 * D);
-    Ctl *ctl = reinterpret_cast<Ctl *>(rowTok + 3 * T);
+    int *rowOff = reinterpret_cast<int *>(vecb + 8 * D);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 3 * T);
     constexpr uint32_t aU = 0, aW = C::BIGM ? C::NACC : D / 2;
 
     const int tid = threadIdx.x, lane = tid & 31;
@@ -193,13 +191,13 @@ sweep_local(const SweepArgs a)
         load_state<D, NT>(nullptr, sm, S);
         if (BWD) load_state<D, NT>(nullptr, sm, Wl);
         gcum = 0.f;
-        if (tid < T) rowTok[cur * T + tid] = tile_token(g, t0, tid);
+        if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, t0, tid);
         __syncthreads();
-        load_raw<D, NT, BWD, BWD>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, b, h, rowTok + cur * T);
+        load_raw<D, NT, BWD, BWD>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
         for (int tile = t0; tile < t1; ++tile) {
             const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
-            if (tid < T) rowTok[nxt * T + tid] = tile + 1 < t1 ? tile_token(g, tile + 1, tid) : -1;
-            write_gates<D, NT, BWD, BWD>(raw, table, rowTok + cur * T);
+            if (tid < T) rowOff[nxt * T + tid] = tile + 1 < t1 ? tile_row_offset(g, b, h, D, tile + 1, tid) : -1;
+            write_gates<D, NT, BWD, BWD>(raw, table, rowOff + cur * T);
             __syncthreads();
             float tot_unused;
             const bool need = gate_prefix<D, NT>(table, sTot, tot_unused);
@@ -228,7 +226,7 @@ sweep_local(const SweepArgs a)
                 }
                 __syncthreads();
                 {
-                    build_tiles<D, NT, BWD, BWD>(raw, tQ, tK, tV, tG, table, vc.off, rowTok + cur * T, lo, min(hi, nrow));
+                    build_tiles<D, NT, BWD, BWD>(raw, tQ, tK, tV, tG, table, vc.off, rowOff + cur * T, lo, min(hi, nrow));
                     if (BWD) {
                         const size_t slot = ((size_t)(nsub - 1 - u) * g.B * g.H + bh) * pl.ntile + tile;
                         write_state_slot<D, NT>(a.slot_s + slot * (D * D), sm, S, vc.ec);
@@ -245,7 +243,7 @@ sweep_local(const SweepArgs a)
                 }
                 {
                     if (u == nsub - 1 && tile + 1 < t1)
-                        load_raw<D, NT, BWD, BWD>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, b, h, rowTok + nxt * T);
+                        load_raw<D, NT, BWD, BWD>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + nxt * T);
                     ok = wait_all(&ctl->bar[0], par, a.status);
                     if (ok) {
                         tc_fence_after_sync();
@@ -293,34 +291,53 @@ seg_scan(float *seg_state, const float *seg_gamma, float *seg_dstate, float *seg
          const float *s_in, float *s_out, const float *ds_out, float *ds_in, int nseg)
 {
     constexpr int NV = (D / 4 + 7) / 8;               // float4 pieces per lane
+    constexpr int NB = 4;                             // segments whose loads are in flight together
     const int bh = blockIdx.y, c = blockIdx.x * 8 + (threadIdx.x >> 3), l8 = threadIdx.x & 7;
     pdl_wait();
     pdl_launch_dependents();
     float4 s[NV];
     const size_t row = (size_t)c * D;
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
         const int e = 4 * (l8 + 8 * i);
-        s[i] = (s_in && e < D) ? *reinterpret_cast<const float4 *>(s_in + (size_t)bh * D * D + row + e) : make_float4(0, 0, 0, 0);
+        s[i] = (s_in && e < D) ? *reinterpret_cast<const float4 *>(s_in + (size_t)bh * D * D + row + e) : zero4;
     }
-    for (int sg = 0; sg < nseg; ++sg) {
-        float *st = seg_state + ((size_t)bh * nseg + sg) * D * D + row;
-        const float gam = exp2f(seg_gamma[((size_t)bh * nseg + sg) * D + c]);
+    for (int sg0 = 0; sg0 < nseg; sg0 += NB) {
+        float4 t[NB][NV];
+        float gam[NB];
 #pragma unroll
-        for (int i = 0; i < NV; ++i) {
-            const int e = 4 * (l8 + 8 * i);
-            if (e < D) {
-                const float4 t = *reinterpret_cast<const float4 *>(st + e);
-                *reinterpret_cast<float4 *>(st + e) = s[i];
-                if (BWD) {
-                    __half2 lo = __floats2half2_rn(s[i].x, s[i].y), hi = __floats2half2_rn(s[i].z, s[i].w);
-                    uint2 pk;
-                    pk.x = *reinterpret_cast<uint32_t *>(&lo);
-                    pk.y = *reinterpret_cast<uint32_t *>(&hi);
-                    char *dst = reinterpret_cast<char *>(seg_state16 + ((size_t)bh * nseg + sg) * D * D);
-                    *reinterpret_cast<uint2 *>(dst + ((e >> 3) * D + c) * 16 + (e & 7) * 2) = pk;
+        for (int j = 0; j < NB; ++j) {
+            const int sg = min(sg0 + j, nseg - 1);
+            gam[j] = seg_gamma[((size_t)bh * nseg + sg) * D + c];
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int e = 4 * (l8 + 8 * i);
+                t[j][i] = e < D ? *reinterpret_cast<const float4 *>(seg_state + ((size_t)bh * nseg + sg) * D * D + row + e) : zero4;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            const int sg = sg0 + j;
+            if (sg < nseg) {
+                const float gm = exp2f(gam[j]);
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int e = 4 * (l8 + 8 * i);
+                    if (e < D) {
+                        *reinterpret_cast<float4 *>(seg_state + ((size_t)bh * nseg + sg) * D * D + row + e) = s[i];
+                        if (BWD) {
+                            __half2 lo = __floats2half2_rn(s[i].x, s[i].y), hi = __floats2half2_rn(s[i].z, s[i].w);
+                            uint2 pk;
+                            pk.x = *reinterpret_cast<uint32_t *>(&lo);
+                            pk.y = *reinterpret_cast<uint32_t *>(&hi);
+                            char *dst = reinterpret_cast<char *>(seg_state16 + ((size_t)bh * nseg + sg) * D * D);
+                            *reinterpret_cast<uint2 *>(dst + ((e >> 3) * D + c) * 16 + (e & 7) * 2) = pk;
+                        }
+                        s[i] = make_float4(gm * s[i].x + t[j][i].x, gm * s[i].y + t[j][i].y, gm * s[i].z + t[j][i].z,
+                                           gm * s[i].w + t[j][i].w);
+                    }
                 }
-                s[i] = make_float4(gam * s[i].x + t.x, gam * s[i].y + t.y, gam * s[i].z + t.z, gam * s[i].w + t.w);
             }
         }
     }
@@ -336,29 +353,47 @@ seg_scan(float *seg_state, const float *seg_gamma, float *seg_dstate, float *seg
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
             const int e = 4 * (l8 + 8 * i);
-            d[i] = (ds_out && e < D) ? *reinterpret_cast<const float4 *>(ds_out + (size_t)bh * D * D + row + e) : make_float4(0, 0, 0, 0);
+            d[i] = (ds_out && e < D) ? *reinterpret_cast<const float4 *>(ds_out + (size_t)bh * D * D + row + e) : zero4;
         }
-        // s holds the state leaving the last segment; walking back, it is replaced by the entry
-        // state of the following segment, which is the state leaving this one
-        for (int sg = nseg - 1; sg >= 0; --sg) {
-            float *dt = seg_dstate + ((size_t)bh * nseg + sg) * D * D + row;
-            const float gam = exp2f(seg_gamma[((size_t)bh * nseg + sg) * D + c]);
-            float dot = 0.f;
+        // s holds the state leaving the last segment; walking back, it is replaced by the entry state of
+        // the segment just handled, which is the state leaving the one before it
+        for (int sg0 = nseg - 1; sg0 >= 0; sg0 -= NB) {
+            float4 t[NB][NV], sp[NB][NV];
+            float gam[NB];
 #pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                const int e = 4 * (l8 + 8 * i);
-                if (e < D) {
-                    const float4 t = *reinterpret_cast<const float4 *>(dt + e);
-                    *reinterpret_cast<float4 *>(dt + e) = d[i];
-                    dot += s[i].x * d[i].x + s[i].y * d[i].y + s[i].z * d[i].z + s[i].w * d[i].w;
-                    d[i] = make_float4(gam * d[i].x + t.x, gam * d[i].y + t.y, gam * d[i].z + t.z, gam * d[i].w + t.w);
-                    s[i] = *reinterpret_cast<const float4 *>(seg_state + ((size_t)bh * nseg + sg) * D * D + row + e);
+            for (int j = 0; j < NB; ++j) {
+                const int sg = max(sg0 - j, 0);
+                gam[j] = seg_gamma[((size_t)bh * nseg + sg) * D + c];
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int e = 4 * (l8 + 8 * i);
+                    t[j][i] = e < D ? *reinterpret_cast<const float4 *>(seg_dstate + ((size_t)bh * nseg + sg) * D * D + row + e) : zero4;
+                    sp[j][i] = e < D ? *reinterpret_cast<const float4 *>(seg_state + ((size_t)bh * nseg + sg) * D * D + row + e) : zero4;
                 }
             }
-            dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-            dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-            dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-            if (l8 == 0) seg_carry[((size_t)bh * nseg + sg) * D + c] = dot;
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                const int sg = sg0 - j;
+                if (sg >= 0) {
+                    const float gm = exp2f(gam[j]);
+                    float dot = 0.f;
+#pragma unroll
+                    for (int i = 0; i < NV; ++i) {
+                        const int e = 4 * (l8 + 8 * i);
+                        if (e < D) {
+                            *reinterpret_cast<float4 *>(seg_dstate + ((size_t)bh * nseg + sg) * D * D + row + e) = d[i];
+                            dot += s[i].x * d[i].x + s[i].y * d[i].y + s[i].z * d[i].z + s[i].w * d[i].w;
+                            d[i] = make_float4(gm * d[i].x + t[j][i].x, gm * d[i].y + t[j][i].y, gm * d[i].z + t[j][i].z,
+                                               gm * d[i].w + t[j][i].w);
+                            s[i] = sp[j][i];
+                        }
+                    }
+                    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                    if (l8 == 0) seg_carry[((size_t)bh * nseg + sg) * D + c] = dot;
+                }
+            }
         }
         if (ds_in) {
 #pragma unroll
@@ -394,8 +429,8 @@ sweep_fwd(const SweepArgs a)
     char *tQ = smem, *tK = tQ + C::TILE_T, *tV = tK + C::TILE_T, *tS = tV + C::TILE_T, *tP = tS + C::TILE_S;
     float *table = reinterpret_cast<float *>(smem + SM::kTiles);
     float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D;
-    int *rowTok = reinterpret_cast<int *>(vecb + 8 * D);
-    Ctl *ctl = reinterpret_cast<Ctl *>(rowTok + 3 * T);
+    int *rowOff = reinterpret_cast<int *>(vecb + 8 * D);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 3 * T);
     constexpr uint32_t aP = 0, aO = 64, aU = 64 + C::NACC;
 
     const int tid = threadIdx.x, lane = tid & 31, q4 = (tid >> 5) & 3, cg = tid >> 7, hf = lane >> 4;
@@ -417,10 +452,10 @@ sweep_fwd(const SweepArgs a)
     {
         const int sid = blockIdx.x;
         if (sid < total) {
-            const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg;
-            if (tid < T) rowTok[cur * T + tid] = tile_token(g, sg * pl.G, tid);
+            const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg, b = bh / g.H, h = bh - b * g.H;
+            if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, sg * pl.G, tid);
             __syncthreads();
-            load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, g, bh / g.H, bh % g.H, rowTok + cur * T);
+            load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, rowOff + cur * T);
         }
     }
     pdl_wait();
@@ -430,16 +465,16 @@ sweep_fwd(const SweepArgs a)
         const int t0 = sg * pl.G, t1 = min(t0 + pl.G, pl.ntile);
         load_state<D, NT>(a.seg_state + (size_t)sid * D * D, sm, S);
         if (sid != (int)blockIdx.x) {
-            if (tid < T) rowTok[cur * T + tid] = tile_token(g, t0, tid);
+            if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, t0, tid);
             __syncthreads();
-            load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, g, b, h, rowTok + cur * T);
+            load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, rowOff + cur * T);
         }
         for (int tile = t0; tile < t1; ++tile) {
             const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
-            if (tid < T) rowTok[nxt * T + tid] = tile + 1 < t1 ? tile_token(g, tile + 1, tid) : -1;
-            write_gates<D, NT, true, false>(raw, table, rowTok + cur * T);
+            if (tid < T) rowOff[nxt * T + tid] = tile + 1 < t1 ? tile_row_offset(g, b, h, D, tile + 1, tid) : -1;
+            write_gates<D, NT, true, false>(raw, table, rowOff + cur * T);
             __syncthreads();
-            const int my_tok = rowTok[cur * T + r16];
+            const int my_off = rowOff[cur * T + r16];
             float tot_unused;
             const bool need = gate_prefix<D, NT>(table, sTot, tot_unused);
             int s = pl.sub_max;
@@ -461,7 +496,7 @@ sweep_fwd(const SweepArgs a)
                 }
                 __syncthreads();
                 {
-                    build_tiles<D, NT, true, false>(raw, tQ, tK, tV, nullptr, table, vc.off, rowTok + cur * T, lo, min(hi, nrow));
+                    build_tiles<D, NT, true, false>(raw, tQ, tK, tV, nullptr, table, vc.off, rowOff + cur * T, lo, min(hi, nrow));
                     write_state_tile<D, NT>(tS, sm, S, vc.ec);                       // Sc = diag(2^c) S
                     fence_async_smem();
                 }
@@ -477,20 +512,24 @@ sweep_fwd(const SweepArgs a)
                 }
                 {
                     if (u == nsub - 1 && tile + 1 < t1)
-                        load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, g, b, h, rowTok + nxt * T);
+                        load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, rowOff + nxt * T);
                     ok = wait_all(&ctl->bar[0], 0, a.status);          // completes twice per iteration: parities 0, 1
                     if (ok) {
                         tc_fence_after_sync();
-                        // scores of row r16 (lanes 0-15 hold accumulator rows): keep s <= t, the diagonal has weight 1
+                        // scores of row r16 (lanes 0-15 hold accumulator rows): keep s <= t, the diagonal has weight 1.
+                        // Column chunks entirely above the diagonal for all 16 rows of the warp are never written (the
+                        // tile starts out zero), chunks entirely below it need no selects.
 #pragma unroll
                         for (int i = 0; i < L::NPT; ++i) {
                             const int sc = cg + L::NCG * i;
-                            float p[8];
-                            tmem_ld8(lane_base + tmem + aP + 8 * sc, p);
-                            if (hf == 0) {
+                            if (8 * sc <= 16 * q4 + 15) {           // uniform over the warp
+                                float p[8];
+                                tmem_ld8(lane_base + tmem + aP + 8 * sc, p);
+                                if (8 * sc + 7 > 16 * q4) {
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) p[e] = (8 * sc + e <= r16) ? p[e] : 0.f;
-                                *reinterpret_cast<uint4 *>(tP + sc * C::CHT + r16 * 16) = pack_h8(p);
+                                    for (int e = 0; e < 8; ++e) p[e] = (8 * sc + e <= r16) ? p[e] : 0.f;
+                                }
+                                if (hf == 0) *reinterpret_cast<uint4 *>(tP + sc * C::CHT + r16 * 16) = pack_h8(p);
                             }
                         }
                     }
@@ -513,8 +552,8 @@ sweep_fwd(const SweepArgs a)
                     if (ok) ok = wait_all(&ctl->bar[0], 1, a.status);
                     if (ok) {
                         tc_fence_after_sync();
-                        const bool inrow = hf == 0 && r16 >= lo && r16 < hi && my_tok >= 0;
-                        const size_t ro = tok_offset(g, b, my_tok < 0 ? 0 : my_tok, h, D);
+                        const bool inrow = hf == 0 && r16 >= lo && r16 < hi && my_off >= 0;
+                        const size_t ro = (size_t)(my_off < 0 ? 0 : my_off);
 #pragma unroll
                         for (int i = 0; i < L::NPC; ++i) {
                             const int jc = cg + L::NCG * i;
@@ -562,8 +601,8 @@ sweep_bwd(const SweepArgs a)
     char *tP = tD + C::TILE_S, *tdP = tP + C::TILE_P;
     float *table = reinterpret_cast<float *>(smem + SM::kTiles);
     float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D, *sCarry = vecb + 8 * D;
-    int *rowTok = reinterpret_cast<int *>(sCarry + 2 * D);
-    Ctl *ctl = reinterpret_cast<Ctl *>(rowTok + 3 * T);
+    int *rowOff = reinterpret_cast<int *>(sCarry + 2 * D);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 3 * T);
     constexpr uint32_t W0 = C::BIGM ? C::NACC : 64;
     constexpr uint32_t aP = 0, aQK = W0, aV = W0 + C::NACC, kHi = 16u << 16;
     static_assert(aV + C::NACC <= SM::tmem_cols, "tensor memory");
@@ -587,11 +626,11 @@ sweep_bwd(const SweepArgs a)
     {
         const int sid = blockIdx.x;
         if (sid < total) {
-            const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg;
+            const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg, b = bh / g.H, h = bh - b * g.H;
             const int t1 = min(sg * pl.G + pl.G, pl.ntile);
-            if (tid < T) rowTok[cur * T + tid] = tile_token(g, t1 - 1, tid);
+            if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, t1 - 1, tid);
             __syncthreads();
-            load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, bh / g.H, bh % g.H, rowTok + cur * T);
+            load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
         }
     }
     pdl_wait();
@@ -602,17 +641,28 @@ sweep_bwd(const SweepArgs a)
         load_state<D, NT>(a.seg_dstate + (size_t)sid * D * D, sm, Dst);
         if (tid < D) sCarry[cpar * D + tid] = a.seg_carry[(size_t)sid * D + tid];
         if (sid != (int)blockIdx.x) {
-            if (tid < T) rowTok[cur * T + tid] = tile_token(g, t1 - 1, tid);
+            if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, t1 - 1, tid);
             __syncthreads();
-            load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, b, h, rowTok + cur * T);
+            load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
         }
-        const char *seg16 = reinterpret_cast<const char *>(a.seg_state16 + (size_t)sid * D * D);
+        if (tid == 0) {
+            // the zero-start state of the sub-chunk worked first (always slot 0 of its tile) and, once per
+            // segment, the state entering the segment; later sub-chunks' states are fetched as soon as the
+            // products of the one before are done
+            const char *src = reinterpret_cast<const char *>(a.slot_s + ((size_t)bh * pl.ntile + (t1 - 1)) * (D * D));
+            const char *seg16 = reinterpret_cast<const char *>(a.seg_state16 + (size_t)sid * D * D);
+            mbar_arrive_expect_tx(barS, 2u * C::NCH * D * 16u);
+            for (int j = 0; j < C::NCH; ++j) {
+                bulk_g2s(tS + j * C::CHS, src + j * D * 16, D * 16, barS);
+                bulk_g2s(tI + j * C::CHS, seg16 + j * D * 16, D * 16, barS);
+            }
+        }
         for (int tile = t1 - 1; tile >= t0; --tile) {
             const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
-            if (tid < T) rowTok[nxt * T + tid] = tile > t0 ? tile_token(g, tile - 1, tid) : -1;
-            write_gates<D, NT, true, true>(raw, table, rowTok + cur * T);
+            if (tid < T) rowOff[nxt * T + tid] = tile > t0 ? tile_row_offset(g, b, h, D, tile - 1, tid) : -1;
+            write_gates<D, NT, true, true>(raw, table, rowOff + cur * T);
             __syncthreads();
-            const int my_tok = rowTok[cur * T + r16];
+            const int my_off = rowOff[cur * T + r16];
             // decay since the segment start of the sub-chunk worked first (always slot 0): fetched ahead of its use
             const float g_first = tid < D ? a.slot_g[((size_t)bh * pl.ntile + tile) * D + tid] : 0.f;
             float tot_unused;
@@ -636,19 +686,9 @@ sweep_bwd(const SweepArgs a)
                     vc.e2c[tid] = ex2(t);
                     vc.aux[tid] = ex2(cv + (u == nsub - 1 ? g_first : a.slot_g[slot * D + tid]));   // exp(c) * decay since the segment start
                 }
-                // every thread has passed its wait for the previous products: the two state tiles are free again
                 __syncthreads();
-                if (tid == 0) {
-                    const char *src = reinterpret_cast<const char *>(a.slot_s + slot * (D * D));
-                    fence_async_smem();
-                    mbar_arrive_expect_tx(barS, 2u * C::NCH * D * 16u);
-                    for (int j = 0; j < C::NCH; ++j) {
-                        bulk_g2s(tS + j * C::CHS, src + j * D * 16, D * 16, barS);
-                        bulk_g2s(tI + j * C::CHS, seg16 + j * D * 16, D * 16, barS);
-                    }
-                }
                 {
-                    build_tiles<D, NT, true, true>(raw, tQ, tK, tV, tG, table, vc.off, rowTok + cur * T, lo, hiv);
+                    build_tiles<D, NT, true, true>(raw, tQ, tK, tV, tG, table, vc.off, rowOff + cur * T, lo, hiv);
                     write_state_tile<D, NT>(tD, sm, Dst, vc.ec);                    // Dc = diag(2^c) D
                     fence_async_smem();
                 }
@@ -668,20 +708,28 @@ sweep_bwd(const SweepArgs a)
                     issue<64, D, false, true>(tmem + aV + kHi, sK, C::CHT, sD, C::CHS, C::KS, false);         // Kc Dc
                 }
                 {
+                    // the raw rows are spent: the next tile's gates (needed first) start now, its q, k, v, dO rows
+                    // after the epilogue, which needs the registers
                     if (u == 0 && tile > t0)
-                        load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, g, b, h, rowTok + nxt * T);
+                        load_raw<D, NT, true, true, true, false>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + nxt * T);
                     ok = wait_all(barG1, 0, a.status);                 // completes twice per iteration: parities 0, 1
                     if (ok) {
                         tc_fence_after_sync();
-                        // lanes 0-15: scores, lanes 16-31: dO V^T; keep s <= t, the diagonal has weight 1
+                        // lanes 0-15: scores, lanes 16-31: dO V^T; keep s <= t, the diagonal has weight 1.  Column
+                        // chunks entirely above the diagonal for all rows of the warp are never written (the tiles
+                        // start out zero), chunks entirely below it need no selects.
 #pragma unroll
                         for (int i = 0; i < L::NPT; ++i) {
                             const int sc = cg + L::NCG * i;
-                            float p[8];
-                            tmem_ld8(lane_base + tmem + aP + 8 * sc, p);
+                            if (8 * sc <= 16 * q4 + 15) {           // uniform over the warp
+                                float p[8];
+                                tmem_ld8(lane_base + tmem + aP + 8 * sc, p);
+                                if (8 * sc + 7 > 16 * q4) {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) p[e] = (8 * sc + e <= r16) ? p[e] : 0.f;
-                            *reinterpret_cast<uint4 *>((hf ? tdP : tP) + sc * C::CHT + r16 * 16) = pack_h8(p);
+                                    for (int e = 0; e < 8; ++e) p[e] = (8 * sc + e <= r16) ? p[e] : 0.f;
+                                }
+                                *reinterpret_cast<uint4 *>((hf ? tdP : tP) + sc * C::CHT + r16 * 16) = pack_h8(p);
+                            }
                         }
                     }
                     fence_async_smem();
@@ -702,46 +750,57 @@ sweep_bwd(const SweepArgs a)
                     ok = wait_all(barG1, 1, a.status);
                     if (ok) {
                         tc_fence_after_sync();
+                        if (tid == 0 && (u > 0 || tile > t0)) {
+                            // every product has completed: fetch the next sub-chunk's zero-start state
+                            const size_t nslot = u > 0 ? slot + (size_t)g.B * g.H * pl.ntile : (size_t)bh * pl.ntile + (tile - 1);
+                            const char *src = reinterpret_cast<const char *>(a.slot_s + nslot * (D * D));
+                            mbar_arrive_expect_tx(barS, (uint32_t)C::NCH * D * 16u);
+                            for (int j = 0; j < C::NCH; ++j) bulk_g2s(tS + j * C::CHS, src + j * D * 16, D * 16, barS);
+                        }
                         const bool inrow = r16 >= lo && r16 < hiv;
-                        const size_t ro = tok_offset(g, b, my_tok < 0 ? 0 : my_tok, h, D);
+                        const size_t ro = (size_t)(my_off < 0 ? 0 : my_off);
 #pragma unroll
                         for (int i = 0; i < L::NPC; ++i) {
                             const int jc = cg + L::NCG * i;
                             if (jc < C::NCH) {          // uniform over the warp
-                                float a1[8], a2[8], lam[8], of[8], t8[8], x[8];
+                                float a1[8], a2[8], x[8];
                                 // lanes 0-15: dq accumulator and dO S_segment^T; lanes 16-31: dk and dv accumulators
                                 tmem_ld8_pair(lane_base + tmem + aQK + 8 * jc, lane_base + tmem + aV + 8 * jc, a1, a2);
-                                ld8(table + r16 * C::LAMP + 8 * jc, lam);
-                                ld8(vc.off + 8 * jc, of);
-                                unpack_h8(*reinterpret_cast<const uint4 *>((hf ? tK : tQ) + jc * C::CHT + r16 * 16), t8);
                                 if (hf == 0) {
                                     float hh[8];
                                     ld8(vc.aux + 8 * jc, hh);
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) a1[e] = fmaf(hh[e], a2[e], a1[e]);
+                                } else if (inrow) {
+                                    store_out8(dv + ro + 8 * jc, a2);
                                 }
-                                // q*dq = Qc * (dq accumulator), k*dk = Kc * (dk accumulator): the decay factors cancel
+                                {
+                                    // q*dq = Qc * (dq accumulator), k*dk = Kc * (dk accumulator): the decay factors cancel
+                                    float t8[8];
+                                    unpack_h8(*reinterpret_cast<const uint4 *>((hf ? tK : tQ) + jc * C::CHT + r16 * 16), t8);
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    x[e] = t8[e] * a1[e];
-                                    a1[e] *= ex2(hf ? of[e] - lam[e] : lam[e] - of[e]);
+                                    for (int e = 0; e < 8; ++e) x[e] = t8[e] * a1[e];
                                 }
 #pragma unroll
                                 for (int e = 0; e < 8; ++e) x[e] -= __shfl_xor_sync(0xffffffffu, x[e], 16);
+                                {
+                                    float lam[8], of[8];
+                                    ld8(table + r16 * C::LAMP + 8 * jc, lam);
+                                    ld8(vc.off + 8 * jc, of);
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) a1[e] *= ex2(hf ? of[e] - lam[e] : lam[e] - of[e]);
+                                }
                                 __syncwarp();           // both halves have read their gates before the table is overwritten
                                 if (inrow) {
-                                    if (hf == 0) {
-                                        st8(table + r16 * C::LAMP + 8 * jc, x);                 // q*dq - k*dk
-                                        store_out8(dq + ro + 8 * jc, a1);
-                                    } else {
-                                        store_out8(dk + ro + 8 * jc, a1);
-                                        store_out8(dv + ro + 8 * jc, a2);
-                                    }
+                                    if (hf == 0) st8(table + r16 * C::LAMP + 8 * jc, x);        // q*dq - k*dk
+                                    store_out8((hf ? dk : dq) + ro + 8 * jc, a1);
                                 }
                             }
                         }
                         // D <- 2^(2c) D + 2^c (Qc^T dO)
                         update_state<D, NT>(lane_base, tmem + aP, sm, Dst, vc.e2c, vc.ec);
+                        if (u == 0 && tile > t0)
+                            load_raw<D, NT, true, true, false, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + nxt * T);
                     }
                     tc_fence_before_sync();
                 }
@@ -774,8 +833,8 @@ sweep_bwd(const SweepArgs a)
                     if (seg == 0) sCarry[(cpar ^ 1) * D + c] = sCarry[cpar * D + c] + all;
 #pragma unroll
                     for (int j = 0; j < L::RPS; ++j) {
-                        const int tok = r0 + j < nrow ? rowTok[cur * T + r0 + j] : -1;
-                        if (tok >= 0) a.dgate[tok_offset(g, b, tok, h, D) + c] = sfx[j] + add;
+                        const int ro = r0 + j < nrow ? rowOff[cur * T + r0 + j] : -1;
+                        if (ro >= 0) a.dgate[(size_t)ro + c] = sfx[j] + add;
                     }
                 }
                 cpar ^= 1;
@@ -863,7 +922,7 @@ dig_status run(const GlaArgs &ga)
     const Plan pl = make_plan(g, sms, ctas_per_sm<D>());
     const SweepWs w = carve(reinterpret_cast<char *>(ga.ws), g, pl, BWD);
     const long long total = (long long)g.B * g.H * pl.nseg;
-    if (total > (1ll << 30)) return DIG_ERR_UNSUPPORTED;
+    if (total > (1ll << 30) || (long long)g.B * g.L * g.H * D >= (1ll << 31)) return DIG_ERR_UNSUPPORTED;     // 31-bit row offsets
     SweepArgs a{};
     a.q = (const bf16 *)ga.q; a.k = (const bf16 *)ga.k; a.v = (const bf16 *)ga.v; a.d_out = (const bf16 *)ga.d_out;
     a.gate = ga.gate;

@@ -170,11 +170,12 @@ struct Ctl {
     uint32_t pad;
 };
 
-// Canonical token of scan position 64*tile + row, or -1 past the end of the sequence.
-__device__ __forceinline__ int tile_token(const Geom &g, int tile, int row)
+// Element offset of the (batch b, head h) row of the token at scan position 64*tile + row in a
+// [B][L][H][D] tensor, or -1 past the end of the sequence (the host checks that offsets fit 31 bits).
+__device__ __forceinline__ int tile_row_offset(const Geom &g, int b, int h, int d, int tile, int row)
 {
     const int p = tile * T + row;
-    return p < g.L ? scan_token(p, g.dir, g.gh, g.gw, g.L) : -1;
+    return p < g.L ? (int)tok_offset(g, b, scan_token(p, g.dir, g.gh, g.gw, g.L), h, d) : -1;
 }
 
 // ---- rows of q, k, v, dO and the gates of one tile, prefetched into registers ------------------
@@ -187,41 +188,50 @@ __device__ __forceinline__ uint4 ldg16(const bf16 *p) { return __ldg(reinterpret
 __device__ __forceinline__ float4 ldg16(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
 
 // Item i of a thread is (row, chunk) = divmod(tid + NT*i, NCH): consecutive threads read consecutive
-// 16-byte pieces of a token row.  Rows past the end of the sequence read token 0 (masked later).
-template <int D, int NT, bool HQ, bool HD>
+// 16-byte pieces of a token row.  Rows past the end of the sequence read the tensor's first row (masked later).
+// GATES / ROWS: which part to load (the gates are needed first, the bf16 rows can follow later).
+template <int D, int NT>
+__device__ __forceinline__ bool item_exists(int it)
+{
+    return (T * Cfg<D>::NCH) % NT == 0 || it < T * Cfg<D>::NCH;     // every thread has all its items when NT divides the count
+}
+template <int D, int NT, bool HQ, bool HD, bool GATES = true, bool ROWS = true>
 __device__ __forceinline__ void load_raw(Raw<Lay<D, NT>::NIT, HQ, HD> &r, const bf16 *q, const bf16 *k, const bf16 *v,
-                                         const bf16 *d_out, const float *gate, const Geom &g, int b, int h,
-                                         const int *row_tok)
+                                         const bf16 *d_out, const float *gate, const int *row_off)
 {
     constexpr int NCH = Cfg<D>::NCH;
 #pragma unroll
     for (int i = 0; i < Lay<D, NT>::NIT; ++i) {
         const int it = (int)threadIdx.x + NT * i;
-        if (it < T * NCH) {
+        if (item_exists<D, NT>(it)) {
             const int row = it / NCH, j = it - row * NCH;
-            const int tok = row_tok[row];
-            const size_t off = tok_offset(g, b, tok < 0 ? 0 : tok, h, D) + 8 * j;
-            r.k[i] = ldg16(k + off);
-            r.v[i] = ldg16(v + off);
-            if (HQ) r.q[i] = ldg16(q + off);
-            if (HD) r.d[i] = ldg16(d_out + off);
-            r.g0[i] = ldg16(gate + off);
-            r.g1[i] = ldg16(gate + off + 4);
+            const int ro = row_off[row];
+            const uint32_t off = (uint32_t)(ro < 0 ? 0 : ro) + 8u * j;
+            if (ROWS) {
+                r.k[i] = ldg16(k + off);
+                r.v[i] = ldg16(v + off);
+                if (HQ) r.q[i] = ldg16(q + off);
+                if (HD) r.d[i] = ldg16(d_out + off);
+            }
+            if (GATES) {
+                r.g0[i] = ldg16(gate + off);
+                r.g1[i] = ldg16(gate + off + 4);
+            }
         }
     }
 }
 
 // Gates of the prefetched tile into the table, in log2 units, zero for rows past the end.
 template <int D, int NT, bool HQ, bool HD>
-__device__ __forceinline__ void write_gates(const Raw<Lay<D, NT>::NIT, HQ, HD> &r, float *table, const int *row_tok)
+__device__ __forceinline__ void write_gates(const Raw<Lay<D, NT>::NIT, HQ, HD> &r, float *table, const int *row_off)
 {
     constexpr int NCH = Cfg<D>::NCH, LAMP = Cfg<D>::LAMP;
 #pragma unroll
     for (int i = 0; i < Lay<D, NT>::NIT; ++i) {
         const int it = (int)threadIdx.x + NT * i;
-        if (it < T * NCH) {
+        if (item_exists<D, NT>(it)) {
             const int row = it / NCH, j = it - row * NCH;
-            const float sc = row_tok[row] >= 0 ? kLog2e : 0.f;
+            const float sc = row_off[row] >= 0 ? kLog2e : 0.f;
             float *dst = table + row * LAMP + 8 * j;
             *reinterpret_cast<float4 *>(dst) = make_float4(r.g0[i].x * sc, r.g0[i].y * sc, r.g0[i].z * sc, r.g0[i].w * sc);
             *reinterpret_cast<float4 *>(dst + 4) = make_float4(r.g1[i].x * sc, r.g1[i].y * sc, r.g1[i].z * sc, r.g1[i].w * sc);

@@ -150,11 +150,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *s
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+            : "=r"(ok) : "r"(addr), "r"(parity), "r"(20000u) : "memory");      // may sleep up to 20 us per try
         if (ok) return true;
-        if ((it & 63) == 63) {
+        if ((it & 7) == 7) {
             const uint64_t now = global_ns();
             if (t0 == 0) t0 = now;
             else if (now - t0 > 250000000ull) {

@@ -20,9 +20,10 @@ def _force_mma():
 def test_auto_picks_this_family_where_tcgen05_does_not_apply():
     from paper_2405_18428_b200 import dig
     dig.dig_set_impl(dig.DIG_IMPL_AUTO)
-    assert dig.dig_gla_query_impl(72, 72, 64, dig.DIG_BF16, 1) == dig.DIG_IMPL_MMA
-    assert dig.dig_gla_query_impl(64, 64, 32, dig.DIG_BF16, 1) == dig.DIG_IMPL_MMA
+    assert dig.dig_gla_query_impl(72, 72, 64, dig.DIG_BF16, 1) == dig.DIG_IMPL_TENSOR     # the paper's XL head size
+    assert dig.dig_gla_query_impl(64, 64, 32, dig.DIG_BF16, 1) == dig.DIG_IMPL_TENSOR
     assert dig.dig_gla_query_impl(64, 64, 64, dig.DIG_BF16, 1) == dig.DIG_IMPL_TENSOR
+    assert dig.dig_gla_query_impl(24, 40, 16, dig.DIG_BF16, 1) == dig.DIG_IMPL_MMA        # d_k != d_v, other head sizes
     assert dig.dig_gla_query_impl(72, 72, 64, dig.DIG_F32, 1) == dig.DIG_IMPL_FMA
     dig.dig_set_impl(dig.DIG_IMPL_MMA)
     assert dig.dig_gla_query_impl(72, 72, 64, dig.DIG_F32, 1) < 0          # fp32 storage is not served
