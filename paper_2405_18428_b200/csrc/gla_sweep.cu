@@ -154,8 +154,8 @@ struct LocalSmem {
     static constexpr uint32_t tmem_cols = C::BIGM ? (BWD ? 256 : 128) : (BWD ? 64 : 32);
 };
 
-template <int D, int NT, bool BWD>
-__global__ void __launch_bounds__(NT, NT == 256 ? 2 : 1)
+template <int D, int NT, bool BWD, int OCC>
+__global__ void __launch_bounds__(NT, OCC)
 sweep_local(const SweepArgs a)
 {
     using C = Cfg<D>;
@@ -415,11 +415,11 @@ struct FwdSmem {
     static constexpr int kTiles = 3 * C::TILE_T + C::TILE_S + C::TILE_P;      // tQ tK tV tS tP
     static constexpr int kFloats = T * C::LAMP + L::NSEG * D + 8 * D;
     static constexpr size_t bytes = kTiles + kFloats * 4 + 3 * T * 4 + sizeof(Ctl);
-    static constexpr uint32_t tmem_cols = 256;
+    static constexpr uint32_t tmem_cols = C::BIGM ? 256 : 128;
 };
 
-template <int D, int NT, typename TO>
-__global__ void __launch_bounds__(NT, NT == 256 ? 2 : 1)
+template <int D, int NT, typename TO, int OCC>
+__global__ void __launch_bounds__(NT, OCC)
 sweep_fwd(const SweepArgs a)
 {
     using C = Cfg<D>;
@@ -431,11 +431,13 @@ sweep_fwd(const SweepArgs a)
     float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D;
     int *rowOff = reinterpret_cast<int *>(vecb + 8 * D);
     Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 3 * T);
-    constexpr uint32_t aP = 0, aO = 64, aU = 64 + C::NACC;
+    // the state product is issued after the scores have been read and reuses their columns
+    constexpr uint32_t aP = 0, aO = C::BIGM ? C::NACC : 64, aU = aP;
+    static_assert(aO + C::NACC <= SM::tmem_cols, "tensor memory");
 
     const int tid = threadIdx.x, lane = tid & 31, q4 = (tid >> 5) & 3, cg = tid >> 7, hf = lane >> 4;
     const int r16 = 16 * q4 + (lane & 15);
-    cta_setup(ctl, 2, SM::tmem_cols, smem, SM::kTiles);
+    cta_setup(ctl, 1, SM::tmem_cols, smem, SM::kTiles);
     const uint32_t tmem = ctl->tmem_base, lane_base = (uint32_t)(32 * q4) << 16;
     const Geom &g = a.g;
     const Plan &pl = a.plan;
@@ -507,8 +509,6 @@ sweep_fwd(const SweepArgs a)
                     issue<64, 64, false, false>(tmem + aP, smem_u32(tQ), C::CHT, smem_u32(tK), C::CHT, C::KS, false);   // Qc Kc^T
                     mma_commit(&ctl->bar[0]);
                     issue<64, D, false, true>(tmem + aO, smem_u32(tQ), C::CHT, smem_u32(tS), C::CHS, C::KS, false);     // Qc Sc
-                    issue_state_product<D>(tmem + aU, tK, tV);                                                         // Kc^T V
-                    mma_commit(&ctl->bar[1]);
                 }
                 {
                     if (u == nsub - 1 && tile + 1 < t1)
@@ -522,7 +522,7 @@ sweep_fwd(const SweepArgs a)
 #pragma unroll
                         for (int i = 0; i < L::NPT; ++i) {
                             const int sc = cg + L::NCG * i;
-                            if (8 * sc <= 16 * q4 + 15) {           // uniform over the warp
+                            if (sc < T / 8 && 8 * sc <= 16 * q4 + 15) {           // uniform over the warp
                                 float p[8];
                                 tmem_ld8(lane_base + tmem + aP + 8 * sc, p);
                                 if (8 * sc + 7 > 16 * q4) {
@@ -540,18 +540,14 @@ sweep_fwd(const SweepArgs a)
                 if (tid == 0) {
                     tc_fence_after_sync();
                     issue<64, D, false, true>(tmem + aO, smem_u32(tP), C::CHT, smem_u32(tV), C::CHT, T / 16, true);     // + P V
+                    issue_state_product<D>(tmem + aU, tK, tV);                                                         // Kc^T V
                     mma_commit(&ctl->bar[0]);
                 }
                 {
-                    // Kc^T V has completed with the first group: advance the state while P V is in the pipe
-                    ok = wait_all(&ctl->bar[1], par, a.status);
+                    ok = wait_all(&ctl->bar[0], 1, a.status);
                     if (ok) {
                         tc_fence_after_sync();
                         update_state<D, NT>(lane_base, tmem + aU, sm, S, vc.e2c, vc.ec);
-                    }
-                    if (ok) ok = wait_all(&ctl->bar[0], 1, a.status);
-                    if (ok) {
-                        tc_fence_after_sync();
                         const bool inrow = hf == 0 && r16 >= lo && r16 < hi && my_off >= 0;
                         const size_t ro = (size_t)(my_off < 0 ? 0 : my_off);
 #pragma unroll
@@ -566,7 +562,7 @@ sweep_fwd(const SweepArgs a)
                     }
                     tc_fence_before_sync();
                 }
-                par ^= 1;          // parity of bar[1], which completes once per iteration
+                par ^= 1;
             }
             cur = nxt;
         }
@@ -588,8 +584,8 @@ struct BwdSmem {
     static constexpr uint32_t tmem_cols = 256;
 };
 
-template <int D, int NT, typename TO>
-__global__ void __launch_bounds__(NT, NT == 256 ? 2 : 1)
+template <int D, int NT, typename TO, int OCC>
+__global__ void __launch_bounds__(NT, OCC)
 sweep_bwd(const SweepArgs a)
 {
     using C = Cfg<D>;
@@ -721,7 +717,7 @@ sweep_bwd(const SweepArgs a)
 #pragma unroll
                         for (int i = 0; i < L::NPT; ++i) {
                             const int sc = cg + L::NCG * i;
-                            if (8 * sc <= 16 * q4 + 15) {           // uniform over the warp
+                            if (sc < T / 8 && 8 * sc <= 16 * q4 + 15) {           // uniform over the warp
                                 float p[8];
                                 tmem_ld8(lane_base + tmem + aP + 8 * sc, p);
                                 if (8 * sc + 7 > 16 * q4) {
@@ -850,12 +846,16 @@ die:
 #undef SYNC_OR_DIE
 
 // ---- host side ----------------------------------------------------------------------------------
+// Launch shapes per head size: worker threads per CTA and CTAs per SM of each kernel (the light
+// kernels run more CTAs per SM on fewer registers, which hides the latency of their short tiles).
 template <int D>
-constexpr int ctas_per_sm() { return 2; }
+struct Shape {          // d = 64: two CTAs of 256 threads per SM
+    static constexpr int NT_LOCAL_F = 256, NT_LOCAL_B = 256, NT_FWD = 256, NT_BWD = 256, OCC = 2;
+};
 template <>
-constexpr int ctas_per_sm<72>() { return 1; }
-template <int D>
-constexpr int worker_threads() { return ctas_per_sm<D>() == 2 ? 256 : 512; }
+struct Shape<72> {
+    static constexpr int NT_LOCAL_F = 640, NT_LOCAL_B = 640, NT_FWD = 640, NT_BWD = 640, OCC = 1;
+};
 
 Plan make_plan(const Geom &g, int sms, int per_sm)
 {
@@ -903,7 +903,12 @@ SweepWs carve(char *base, const Geom &g, const Plan &pl, bool backward)
     return w;
 }
 
-int sweep_per_sm(int d) { return d == 64 ? ctas_per_sm<64>() : ctas_per_sm<72>(); }
+// CTAs per SM of the heaviest kernel of a pass: segments are sized for that many slots
+int sweep_per_sm(int d, bool backward)
+{
+    (void)backward;
+    return d == 64 ? Shape<64>::OCC : Shape<72>::OCC;
+}
 
 template <typename K>
 dig_status set_smem(K kern, size_t bytes)
@@ -914,12 +919,14 @@ dig_status set_smem(K kern, size_t bytes)
 template <int D, bool BWD>
 dig_status run(const GlaArgs &ga)
 {
-    constexpr int NT = worker_threads<D>();
+    using SH = Shape<D>;
+    constexpr int NT_L = BWD ? SH::NT_LOCAL_B : SH::NT_LOCAL_F, NT_M = BWD ? SH::NT_BWD : SH::NT_FWD;
+    constexpr int OCC_L = SH::OCC, OCC_M = SH::OCC;
     const Geom &g = ga.g;
     const int sms = device_sm_count();
     int *status = device_status_ptr();
     if (!status || sms <= 0) return DIG_ERR_CUDA;
-    const Plan pl = make_plan(g, sms, ctas_per_sm<D>());
+    const Plan pl = make_plan(g, sms, OCC_M);
     const SweepWs w = carve(reinterpret_cast<char *>(ga.ws), g, pl, BWD);
     const long long total = (long long)g.B * g.H * pl.nseg;
     if (total > (1ll << 30) || (long long)g.B * g.L * g.H * D >= (1ll << 31)) return DIG_ERR_UNSUPPORTED;     // 31-bit row offsets
@@ -932,14 +939,15 @@ dig_status run(const GlaArgs &ga)
     a.status = status;
     a.g = g;
     a.plan = pl;
-    const int grid = (int)(total < (long long)sms * ctas_per_sm<D>() ? total : (long long)sms * ctas_per_sm<D>());
+    const int grid_l = (int)(total < (long long)sms * OCC_L ? total : (long long)sms * OCC_L);
+    const int grid_m = (int)(total < (long long)sms * OCC_M ? total : (long long)sms * OCC_M);
     dig_status st;
     {
-        auto kern = sweep_local<D, NT, BWD>;
-        constexpr size_t smem = LocalSmem<D, NT, BWD>::bytes;
+        auto kern = sweep_local<D, NT_L, BWD, OCC_L>;
+        constexpr size_t smem = LocalSmem<D, NT_L, BWD>::bytes;
         if ((st = set_smem(kern, smem)) != DIG_OK) return st;
         KernelTimer t(KID_SW_LOCAL, ga.stream);
-        launch_pdl(kern, dim3(grid), dim3(NT), smem, ga.stream, a);
+        launch_pdl(kern, dim3(grid_l), dim3(NT_L), smem, ga.stream, a);
         if ((st = cuda_ok(cudaGetLastError())) != DIG_OK) return st;
     }
     {
@@ -950,20 +958,20 @@ dig_status run(const GlaArgs &ga)
         if ((st = cuda_ok(cudaGetLastError())) != DIG_OK) return st;
     }
     const bool f32 = ga.dtype == DIG_BF16_F32OUT;
-    if (!BWD) {
-        constexpr size_t smem = FwdSmem<D, NT>::bytes;
-        auto k16 = sweep_fwd<D, NT, bf16>;
-        auto k32 = sweep_fwd<D, NT, float>;
+    if constexpr (!BWD) {
+        constexpr size_t smem = FwdSmem<D, NT_M>::bytes;
+        auto k16 = sweep_fwd<D, NT_M, bf16, OCC_M>;
+        auto k32 = sweep_fwd<D, NT_M, float, OCC_M>;
         if ((st = set_smem(k16, smem)) != DIG_OK || (st = set_smem(k32, smem)) != DIG_OK) return st;
         KernelTimer t(KID_SW_FWD, ga.stream);
-        launch_pdl(f32 ? k32 : k16, dim3(grid), dim3(NT), smem, ga.stream, a);
+        launch_pdl(f32 ? k32 : k16, dim3(grid_m), dim3(NT_M), smem, ga.stream, a);
     } else {
-        constexpr size_t smem = BwdSmem<D, NT>::bytes;
-        auto k16 = sweep_bwd<D, NT, bf16>;
-        auto k32 = sweep_bwd<D, NT, float>;
+        constexpr size_t smem = BwdSmem<D, NT_M>::bytes;
+        auto k16 = sweep_bwd<D, NT_M, bf16, OCC_M>;
+        auto k32 = sweep_bwd<D, NT_M, float, OCC_M>;
         if ((st = set_smem(k16, smem)) != DIG_OK || (st = set_smem(k32, smem)) != DIG_OK) return st;
         KernelTimer t(KID_SW_BWD, ga.stream);
-        launch_pdl(f32 ? k32 : k16, dim3(grid), dim3(NT), smem, ga.stream, a);
+        launch_pdl(f32 ? k32 : k16, dim3(grid_m), dim3(NT_M), smem, ga.stream, a);
     }
     return cuda_ok(cudaGetLastError());
 }
@@ -981,7 +989,7 @@ size_t sweep_workspace_bytes(const Geom &g, bool backward)
 {
     int sms = device_sm_count();
     if (sms <= 0) sms = 148;
-    const Plan pl = make_plan(g, sms, sweep_per_sm(g.dk));
+    const Plan pl = make_plan(g, sms, sweep_per_sm(g.dk, backward));
     return carve(nullptr, g, pl, backward).bytes;
 }
 

@@ -64,10 +64,10 @@ struct Lay {
     static constexpr int RPS = (T + NSEG - 1) / NSEG;             // rows per segment
     static constexpr int NIT = (T * C::NCH + NT - 1) / NT;        // (row, chunk) items per thread of one tensor
     static constexpr int NPC = (C::NCH + NCG - 1) / NCG;          // channel chunks per thread in row-wise epilogues
-    static constexpr int NPT = (T / 8) / NCG;                     // token-column chunks per thread of a score tile
+    static constexpr int NPT = (T / 8 + NCG - 1) / NCG;           // token-column chunks per thread of a score tile
     static constexpr int HCH = C::NCH / 2;                        // chunks per half (state products of small heads)
     static constexpr int NPS = C::BIGM ? NPC : (HCH + NCG - 1) / NCG;   // state chunks per thread
-    static_assert(NSEG >= 1 && (T / 8) % NCG == 0, "thread count");
+    static_assert(NSEG >= 1, "thread count");
 };
 
 struct Plan {
