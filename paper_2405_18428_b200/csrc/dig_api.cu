@@ -82,7 +82,6 @@ const char *const kKernelNames[KID_COUNT] = {
     "gate_logsigmoid", "srem_dwconv3x3", "srem_dwconv_wgrad", "gla_outgate", "state_scan_fwd", "state_scan_bwd",
     "fma_chunk_state", "fma_chunk_out", "fma_chunk_bwd",
     "mma_chunk_state", "mma_chunk_out", "mma_chunk_bwd",
-    "tc_chunk_state", "tc_chunk_out", "tc_chunk_bwd",
     "sweep_local", "seg_scan", "sweep_fwd", "sweep_bwd"};
 struct Profile {
     bool on = false;

@@ -93,10 +93,8 @@ struct GlaArgs {
 //   gamma   [B*H][N][dk]       exp(sum of the chunk's gates)
 //   dstates [B*H][N][dk][dv]   (backward) chunk-local Q^T dO, turned in place into dL/d(state leaving the chunk)
 //   carry   [B*H][N][dk]       (backward) gate-gradient carried in from later chunks
-//   dstates_m [B*H][N][dk][dv] (backward) second copy of the decayed state gradients, in the other
-//                              operand-tile order (used by the tensor-core family only)
 struct Workspace {
-    float *states, *gamma, *dstates, *carry, *dstates_m, *sfinal;
+    float *states, *gamma, *dstates, *carry, *sfinal;
     size_t bytes;
 };
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -113,10 +111,9 @@ inline Workspace carve_workspace(float *base, const Geom &g, bool backward)
     if (backward) {
         w.dstates = reinterpret_cast<float *>(p);       p += st;
         w.carry = reinterpret_cast<float *>(p);         p += gm;
-        w.dstates_m = reinterpret_cast<float *>(p);     p += st;
         const size_t fin = align256(bh * g.dk * g.dv * sizeof(float));
         w.sfinal = reinterpret_cast<float *>(p);        p += fin;
-        w.bytes += 2 * st + gm + fin;
+        w.bytes += st + gm + fin;
     }
     return w;
 }
@@ -129,17 +126,10 @@ dig_status mma_gla_fwd(const GlaArgs &a);
 dig_status mma_gla_bwd(const GlaArgs &a);
 bool mma_supports(int dk, int dv, int chunk, int dtype, bool backward, bool beta = false);
 size_t mma_beta_workspace_bytes(const Geom &g, bool backward);
-dig_status tensor_gla_fwd(const GlaArgs &a);
-dig_status tensor_gla_bwd(const GlaArgs &a);
-bool tensor_supports(int dk, int dv, int chunk, int dtype, bool backward);
 
 // Chunk-state scans, shared by both families (plain fp32 FMA, bandwidth-bound).
-// `tiles`: the states are stored transposed, in swizzled operand-tile order (tensor-core forward pass).
-dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tiles = false,
-                                 bool tf32 = false);
+dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tf32 = false);
 dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tf32 = false);
-// Tensor-core backward pass: forward and reverse scan in one launch over states kept in tile order.
-dig_status launch_state_scan_bwd_tiles(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio);
 // Scans with the value-channel gate (row-major states, tf32-rounded results) and the cross-chunk part of its gradient.
 dig_status launch_state_scan_fwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s);
 dig_status launch_state_scan_bwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s);
@@ -150,18 +140,12 @@ int *device_status_ptr();
 // Streaming multiprocessors of the current device (cached per device), 0 on error.
 int device_sm_count();
 
-// Tensor-core kernels (one .cu file each).
-dig_status launch_tc_state(const GlaArgs &a, const Workspace &w, bool backward, int sm_count, int *status);
-dig_status launch_tc_out(const GlaArgs &a, const Workspace &w, int sm_count, int *status);
-dig_status launch_tc_bwd(const GlaArgs &a, const Workspace &w, int sm_count, int *status);
-
 // Optional per-kernel timing (dig_profile_*): when enabled, every launch site brackets its
 // kernel with two CUDA events on the launching stream.
 enum KernelId {
     KID_GATE = 0, KID_DWCONV, KID_DWCONV_WGRAD, KID_OUTGATE, KID_SCAN_FWD, KID_SCAN_BWD,
     KID_FMA_STATE, KID_FMA_OUT, KID_FMA_BWD,
     KID_MMA_STATE, KID_MMA_OUT, KID_MMA_BWD,
-    KID_TC_STATE, KID_TC_OUT, KID_TC_BWD,
     KID_SW_LOCAL, KID_SW_SCAN, KID_SW_FWD, KID_SW_BWD,
     KID_COUNT
 };

@@ -717,7 +717,7 @@ dig_status fwd_dims(const GlaArgs &a)
                                                                     a.gate, nullptr, w.states, w.gamma, nullptr, bd, g);
     }
     if (BETA) st = launch_state_scan_fwd_beta(w, bd.gamma_v, g, a.stream);
-    else st = launch_state_scan_fwd(w, g, a.stream, a.sio, false, true);
+    else st = launch_state_scan_fwd(w, g, a.stream, a.sio, true);
     if (st != DIG_OK) return st;
     KernelTimer t(KID_MMA_OUT, a.stream);
     k3<<<grid, kThreads, smem_out(g, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
@@ -747,7 +747,7 @@ dig_status bwd_dims(const GlaArgs &a)
         if ((st = launch_state_scan_fwd_beta(w, bd.gamma_v, g, a.stream)) != DIG_OK) return st;
         if ((st = launch_state_scan_bwd_beta(w, bd.gamma_v, g, a.stream)) != DIG_OK) return st;
     } else {
-        if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, false, true)) != DIG_OK) return st;
+        if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, true)) != DIG_OK) return st;
         if ((st = launch_state_scan_bwd(w, g, a.stream, a.sio, true)) != DIG_OK) return st;
     }
     {
