@@ -4,9 +4,17 @@
 A step is one pass of the whole hot path over one batch of synthetic, seeded input: for every
 scan direction of the workload (one DiG block each) the gate transform, GLA forward, GLA backward
 and, where the workload has one, the SREM depthwise conv.  Every block owns its own input and
-output buffers, so a step streams far more than the 126 MB L2 and no flush is needed.
+output buffers.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C5] [--impl ours|reference]
+
+Headline (`value`): the largest single-GPU workload (C5: 128 x 128 grid, 16 heads of 72 channels,
+four scan directions + conv).  K steps are captured as CUDA-graph replays and timed with CUDA
+events; the K-step region is repeated until at least a second of device time has been measured and
+the median repetition is reported, with the spread and the SM clock sampled meanwhile.  The other
+workloads (C1 - C4 and the chunk sweep of C4) follow as `sweep` entries: a whole step each, median
+of 20 repetitions with the L2 flushed before every one ("cold") and without ("warm"), forward and
+backward also on their own, each with its roofline fractions and clock record.
 
 Prints one JSON line (rank 0).  N > 1 (torchrun) shards nothing across ranks: every rank runs the
 same workload on its own GPU (weak scaling over independent batches, no collective in the path).
@@ -14,7 +22,9 @@ same workload on its own GPU (weak scaling over independent batches, no collecti
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
 import sys
 import threading
@@ -26,12 +36,10 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu capture summarised
-# in profiles/; only valid for the kernel as it stood when the capture was taken (reset to None on change).
-NCU_TRAFFIC = {("C2", "tc_chunk_bwd"): 80.6e6}
-
 METRIC = "gla_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
+TILE = 64                      # tokens per tile of the tcgen05 kernels, whatever chunk size was asked for
+FAMILY = {1: "fma", 2: "tensor", 3: "mma"}
 
 
 def load_peaks():
@@ -43,27 +51,98 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-def flops_per_token_head(wl, chunk):
+def executed_tile(family, chunk):
+    """Tokens per tile the kernels actually work on: the tcgen05 family always uses 64-token tiles
+    (shorter chunks are sub-chunks of a tile whose other rows are zero), the others the chunk itself."""
+    return TILE if family == 2 else chunk
+
+
+def flops_per_token_head(wl, tile):
     """(algorithmic, executed) flops per (token, head) for fwd+bwd: causal-useful work without the
-    backward's recomputation, and full chunk x chunk blocks with it."""
-    dk, dv, C = wl.d_k, wl.d_v, chunk
+    backward's recomputation, and full tile x tile blocks with it."""
+    dk, dv, C = wl.d_k, wl.d_v, tile
     alg = 3 * (C + 1) * (dk + dv) + 12 * dk * dv
     exe = 2 * C * (dk + dv) + 4 * dk * dv + 2 * C * (3 * dk + 2 * dv) + 10 * dk * dv
+    if not wl.backward:
+        alg = (C + 1) * (dk + dv) + 4 * dk * dv
+        exe = 2 * C * (dk + dv) + 4 * dk * dv
     return alg, exe
 
 
 def bytes_per_token_head(wl):
-    """Algorithmic HBM bytes per (token, head): every operand touched once per pass; bf16 tensors,
-    fp32 gate and gate gradient."""
+    """Algorithmic HBM bytes per (token, head): every operand touched once per pass; bf16 (or fp32)
+    tensors, fp32 gate and gate gradient."""
     e = 2 if wl.dtype == "bf16" else 4
     dk, dv = wl.d_k, wl.d_v
     fwd = e * (2 * dk + dv) + 4 * dk + e * dv
     bwd = e * (2 * dk + 2 * dv) + 4 * dk + e * (2 * dk + dv) + 4 * dk
-    return fwd, bwd
+    return fwd, (bwd if wl.backward else 0)
+
+
+def step_work(wl, family):
+    """Algorithmic bytes and executed flops of one step (all blocks) of a workload."""
+    fwd_b, bwd_b = bytes_per_token_head(wl)
+    th = wl.B * wl.L * wl.H
+    e = 2 if wl.dtype == "bf16" else 4
+    nb = len(wl.directions)
+    conv_b = 2 * e * wl.B * wl.L * wl.H * wl.d_v if wl.conv else 0
+    alg_f, exe_f = flops_per_token_head(wl, executed_tile(family, wl.chunk))
+    return {"bytes": nb * (th * (fwd_b + bwd_b) + conv_b), "flops_alg": nb * th * alg_f, "flops_exec": nb * th * exe_f}
+
+
+def roofline_fracs(work, seconds, peaks):
+    t_hbm = work["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_tc = work["flops_exec"] / (peaks["bf16_tflops_sustained"] * 1e12)
+    return {"hbm_frac": t_hbm / seconds, "tensor_frac_exec": t_tc / seconds, "frac": max(t_hbm, t_tc) / seconds,
+            "bound": "hbm" if t_hbm >= t_tc else "tensor",
+            "tflops_alg": work["flops_alg"] / seconds / 1e12, "tflops_exec": work["flops_exec"] / seconds / 1e12,
+            "gbs_alg": work["bytes"] / seconds / 1e9}
+
+
+def kernel_alg_bytes(wl):
+    """Algorithmic bytes per launch of the kernels that have a plain bandwidth model."""
+    fwd_b, bwd_b = bytes_per_token_head(wl)
+    th = wl.B * wl.L * wl.H
+    e = 2 if wl.dtype == "bf16" else 4
+    out = {}
+    for name in ("sweep_fwd", "mma_chunk_out", "fma_chunk_out"):
+        out[name] = fwd_b * th
+    for name in ("sweep_bwd", "mma_chunk_bwd", "fma_chunk_bwd"):
+        out[name] = bwd_b * th
+    out["gate_logsigmoid"] = (e + 4) * th * wl.d_k
+    out["srem_dwconv3x3"] = 2 * e * wl.B * wl.L * wl.H * wl.d_v
+    return out
+
+
+def source_hash():
+    h = hashlib.sha256()
+    src = os.path.join(ROOT, "paper_2405_18428_b200", "csrc")
+    for f in sorted(os.listdir(src)):
+        if f.endswith((".cu", ".cuh")):
+            h.update(open(os.path.join(src, f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(kernel, workload):
+    """DRAM bytes per launch of a kernel from the ncu capture recorded beside the profile summaries;
+    None when no capture exists for this kernel and workload or the kernel sources changed since."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    try:
+        rec = json.load(open(path))
+    except ValueError:
+        return None
+    if rec.get("source_hash") != source_hash():
+        return None
+    for r in rec.get("kernels", []):
+        if r["kernel"] == kernel and r["workload"] == workload:
+            return r["dram_bytes_per_launch"]
+    return None
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons through NVML while the timed region runs (read only)."""
+    """Samples SM clock and throttle reasons through NVML while a timed region runs (read only)."""
 
     def __init__(self, index):
         self.samples, self.reasons, self.stop_flag, self.thread, self.max_mhz = [], set(), False, None, None
@@ -95,6 +174,7 @@ class ClockSampler:
         if self.nv is not None:
             self.thread = threading.Thread(target=self._loop, daemon=True)
             self.thread.start()
+        return self
 
     def stop(self):
         self.stop_flag = True
@@ -119,22 +199,24 @@ class Block:
         self.grads = (torch.empty(self.q.shape, dtype=ost, device="cuda"), torch.empty(self.q.shape, dtype=ost, device="cuda"),
                       torch.empty(self.v.shape, dtype=ost, device="cuda"), torch.empty(self.q.shape, dtype=torch.float32, device="cuda"))
         dt = dig.DIG_BF16 if wl.dtype == "bf16" else dig.DIG_F32
-        need = dig.dig_gla_workspace_bytes(wl.B, wl.H, wl.grid_h, wl.grid_w, wl.d_k, wl.d_v, wl.chunk, dt, 1)
-        self.ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        need = dig.dig_gla_workspace_bytes(wl.B, wl.H, wl.grid_h, wl.grid_w, wl.d_k, wl.d_v, wl.chunk, dt, int(wl.backward))
+        self.ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
         self.tau = x["tau"]
         if wl.conv:
             self.cx, self.cw = dev(x["conv_x"]), dev(x["conv_w"])
             self.cy = torch.empty_like(self.cx)
 
-    def run(self, dig):
+    def run(self, dig, part="all"):
+        """part: "all" (the step), "fwd" (gate transform + forward), "bwd" (backward alone)."""
         wl = self.wl
-        dig.dig_gate_logsigmoid(self.g, self.tau, self.gate)
-        dig.dig_gla_fwd(self.q, self.k, self.v, self.gate, wl.grid_h, wl.grid_w, wl.chunk, self.direction,
-                        out=self.out, workspace=self.ws)
-        if wl.backward:
+        if part in ("all", "fwd"):
+            dig.dig_gate_logsigmoid(self.g, self.tau, self.gate)
+            dig.dig_gla_fwd(self.q, self.k, self.v, self.gate, wl.grid_h, wl.grid_w, wl.chunk, self.direction,
+                            out=self.out, workspace=self.ws)
+        if wl.backward and part in ("all", "bwd"):
             dig.dig_gla_bwd(self.q, self.k, self.v, self.gate, self.dO, wl.grid_h, wl.grid_w, wl.chunk,
                             self.direction, grads=self.grads, workspace=self.ws)
-        if wl.conv:
+        if wl.conv and part == "all":
             dig.dig_srem_dwconv(self.cx, self.cw, None, wl.grid_h, wl.grid_w, self.direction, y=self.cy)
 
     def host_io(self, torch):
@@ -213,10 +295,11 @@ def job_tokens_per_s(tokens_per_step_per_rank, steps, world, ms):
     return tokens_per_step_per_rank * steps * world / (ms * 1e-3)
 
 
-def time_steps(blocks, dig, torch, steps, warmup, dist, e2e=False, before_timed=None):
+def time_steps(blocks, dig, torch, steps, warmup, dist, e2e=False, before_timed=None, part="all"):
+    """K steps of plain stream launches between two CUDA events (barrier + synchronize on both sides)."""
     for _ in range(warmup):
         for b in blocks:
-            b.run_e2e(dig, torch) if e2e else b.run(dig)
+            b.run_e2e(dig, torch) if e2e else b.run(dig, part)
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
@@ -227,7 +310,7 @@ def time_steps(blocks, dig, torch, steps, warmup, dist, e2e=False, before_timed=
     t0.record()
     for _ in range(steps):
         for b in blocks:
-            b.run_e2e(dig, torch) if e2e else b.run(dig)
+            b.run_e2e(dig, torch) if e2e else b.run(dig, part)
     if e2e:
         Block.join_copies(torch)
     t1.record()
@@ -237,25 +320,27 @@ def time_steps(blocks, dig, torch, steps, warmup, dist, e2e=False, before_timed=
     return max_over_ranks(t0.elapsed_time(t1), dist)
 
 
-def time_graph_steps(blocks, dig, torch, steps, warmup, dist):
-    """The same K steps as time_steps, with one step captured in a CUDA graph and replayed (the
-    kernels and their order are unchanged; only the host-side launch cost goes away).  Returns None
-    if the capture fails."""
+def capture_step(blocks, dig, torch, part="all"):
+    """One step (or its forward / backward part) as a CUDA graph: the kernels and their order are
+    those of the plain launches, only the host-side launch cost goes away.  None if capture fails."""
     try:
         side = torch.cuda.Stream()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.stream(side):
             for b in blocks:
-                b.run(dig)          # first calls outside the capture (per-kernel attribute set-up)
+                b.run(dig, part)          # first calls outside the capture (per-kernel attribute set-up)
             torch.cuda.synchronize()
             with torch.cuda.graph(graph, stream=side):
                 for b in blocks:
-                    b.run(dig)
+                    b.run(dig, part)
         torch.cuda.synchronize()
+        return graph
     except Exception:
         return None
-    for _ in range(warmup):
-        graph.replay()
+
+
+def time_replays(graph, torch, steps, dist):
+    """`steps` replays of a captured step between two CUDA events."""
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
@@ -271,20 +356,97 @@ def time_graph_steps(blocks, dig, torch, steps, warmup, dist):
     return max_over_ranks(t0.elapsed_time(t1), dist)
 
 
-def cpu_baseline(wl, budget_s=20.0):
+def median_single(run_once, torch, reps, flush=None):
+    """Median (and min, max) over `reps` single timed runs, optionally with the L2 flushed before each."""
+    ts = []
+    for _ in range(reps):
+        if flush is not None:
+            flush.zero_()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        run_once()
+        t1.record()
+        torch.cuda.synchronize()
+        ts.append(t0.elapsed_time(t1))
+    ts.sort()
+    return {"median_ms": float(np.median(ts)), "min_ms": ts[0], "max_ms": ts[-1], "reps": reps}
+
+
+def profile_kernels(blocks, dig, torch, steps):
+    """Per-kernel device time of `steps` steps, every launch bracketed by two CUDA events."""
+    for b in blocks:
+        b.run(dig)
+    torch.cuda.synchronize()
+    dig.dig_profile_enable(True)
+    for _ in range(steps):
+        for b in blocks:
+            b.run(dig)
+    torch.cuda.synchronize()
+    prof = dig.dig_profile_read()
+    dig.dig_profile_enable(False)
+    total = sum(t for n, t in prof.values() if n) or 1.0
+    return {k: {"launches": n, "ms_per_launch": t / n, "share": t / total} for k, (n, t) in prof.items() if n}
+
+
+def kernel_rooflines(shares, wl, peaks):
+    """Achieved algorithmic GB/s of every kernel with a bandwidth model, against the measured copy bandwidth."""
+    alg = kernel_alg_bytes(wl)
+    out = {}
+    for k, s in shares.items():
+        if k in alg and alg[k] > 0:
+            a = alg[k] / (s["ms_per_launch"] * 1e-3) / 1e9
+            out[k] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
+                      "algorithmic_bytes_per_launch": alg[k], "us_per_launch": s["ms_per_launch"] * 1e3,
+                      "traffic": recorded_traffic(k, wl.name), "peak_source": peaks["source"]}
+    return out
+
+
+def sweep_entry(name, wl, torch, dig, peaks, local, flush, reps=20):
+    dt = dig.DIG_BF16 if wl.dtype == "bf16" else dig.DIG_F32
+    fam = dig.dig_gla_query_impl(wl.d_k, wl.d_v, wl.chunk, dt, int(wl.backward))
+    blocks = make_blocks(wl, torch, dig)
+    sampler = ClockSampler(local).start()
+    res = {"L": wl.L, "B": wl.B, "H": wl.H, "d": wl.d_k, "chunk_requested": wl.chunk,
+           "tile_executed": executed_tile(fam, wl.chunk), "storage": wl.dtype, "kernel_family": FAMILY.get(fam, str(fam)),
+           "directions": list(wl.directions), "conv": wl.conv, "backward": wl.backward}
+    graphs = {p: capture_step(blocks, dig, torch, p) for p in (("all", "fwd", "bwd") if wl.backward else ("all",))}
+    run = {p: (g.replay if g is not None else (lambda p=p: [b.run(dig, p) for b in blocks])) for p, g in graphs.items()}
+    for p in run:
+        for _ in range(3):
+            run[p]()
+    torch.cuda.synchronize()
+    res["step_cold"] = median_single(run["all"], torch, reps, flush)
+    res["step_warm"] = median_single(run["all"], torch, reps, None)
+    if wl.backward:
+        res["fwd_cold"] = median_single(run["fwd"], torch, reps, flush)
+        res["bwd_cold"] = median_single(run["bwd"], torch, reps, flush)
+    sec = res["step_cold"]["median_ms"] * 1e-3
+    res["tokens_per_s"] = wl.B * wl.L * len(wl.directions) / sec
+    res["roofline"] = roofline_fracs(step_work(wl, fam), sec, peaks)
+    shares = profile_kernels(blocks, dig, torch, 3)
+    rl = kernel_rooflines(shares, wl, peaks)
+    dom = max(shares, key=lambda k: shares[k]["share"])
+    res["dominant_kernel"] = {"name": dom, "share": shares[dom]["share"], **(rl.get(dom) or {})}
+    res["clocks"] = sampler.stop()
+    res["launch"] = "cuda_graph" if graphs["all"] is not None else "eager"
+    del blocks, graphs, run
+    torch.cuda.empty_cache()
+    return res
+
+
+def cpu_baseline(wl, budget_s=16.0, threads=None):
     """The fp64 oracle, as it stands, on a bounded sample of the workload: whole (batch, head)
-    pairs of the first scan direction, all host cores, gate + fwd + bwd (+ conv on those batches)."""
+    pairs, every scan direction of the workload, gate + fwd + bwd (+ conv on those batches)."""
     import oracle
     from paper_2405_18428_b200.inputs import make_inputs
-    cores = max(1, len(os.sched_getaffinity(0)))
-    # one (b, h) pair costs about L*dk*dv*(2 + 8) fp64 multiply-adds at ~1e9/s per core
-    per_pair = wl.L * wl.d_k * wl.d_v * 10 / 1.0e9
-    pairs_budget = max(1, int(budget_s * cores / max(per_pair, 1e-9)))
-    nb = max(1, min(wl.B, pairs_budget // wl.H))
-    sub = wl.scaled(B=nb)
+    cores = max(1, len(os.sched_getaffinity(0))) if threads is None else threads
+    # one (b, h) pair costs about L*dk*dv*(2 + 8) fp64 multiply-adds at ~1e9/s per core, per direction
+    per_pair = wl.L * wl.d_k * wl.d_v * 10 / 1.0e9 * len(wl.directions)
+    pairs_budget = max(1, int(0.5 * budget_s * cores / max(per_pair, 1e-9)))
+    nh = max(1, min(wl.H, pairs_budget))
+    nb = max(1, min(wl.B, pairs_budget // wl.H)) if nh == wl.H else 1
+    sub = wl.scaled(B=nb, H=nh)
     x = make_inputs(sub)
-    # whole steps of the sample (every scan direction of the workload), repeated until about half the
-    # budget is spent, so that the timing is not dominated by start-up effects
     t0 = time.perf_counter()
     passes = 0
     while True:
@@ -299,10 +461,11 @@ def cpu_baseline(wl, budget_s=20.0):
         if time.perf_counter() - t0 >= 0.5 * budget_s:
             break
     dt = time.perf_counter() - t0
-    tokens = nb * wl.L * len(wl.directions) * passes
+    # tokens of a full-width batch this much head-work corresponds to (the heads are independent recurrences)
+    tokens = nb * wl.L * len(wl.directions) * passes * (nh / wl.H)
     return {"value": tokens / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{nb} of {wl.B} batches x {wl.H} heads, directions {list(wl.directions)}, "
-                      f"gate+fwd{'+bwd' if wl.backward else ''}{'+conv' if wl.conv else ''}, "
+            "sample": f"{nb} of {wl.B} batches x {nh} of {wl.H} heads (tokens scaled by the head fraction), "
+                      f"directions {list(wl.directions)}, gate+fwd{'+bwd' if wl.backward else ''}{'+conv' if wl.conv else ''}, "
                       f"{passes} passes, {dt:.2f} s wall on {cores} threads"}, dt, tokens
 
 
@@ -334,16 +497,17 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="C2")
+    ap.add_argument("--workload", default="C5")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--grid", type=int, nargs=2, default=None, metavar=("H", "W"),
                     help="patch grid to use instead of the workload's (a reduced copy of a workload, e.g. for a profiler capture)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--family", default="auto", choices=["auto", "fma", "tensor", "mma"])
-    ap.add_argument("--eager", action="store_true", help="time plain stream launches instead of one CUDA graph per step")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the short tokens/s-vs-L sweep over C3, C4 (chunks 32, 64, 128), C5")
+    ap.add_argument("--eager", action="store_true", help="time plain stream launches instead of CUDA-graph replays")
+    ap.add_argument("--min-seconds", type=float, default=1.0, help="device time the repeated K-step region must add up to")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the other workloads (C1 - C4 and the chunk sweep of C4)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     args = ap.parse_args()
 
@@ -353,8 +517,6 @@ def main():
         wl = wl.scaled(chunk=args.chunk)
     if args.grid:
         wl = wl.scaled(name=f"{wl.name}@{args.grid[0]}x{args.grid[1]}", grid_h=args.grid[0], grid_w=args.grid[1])
-    if not wl.backward:
-        wl = wl.scaled(backward=False)
     if args.impl == "reference":
         return run_reference(args, wl)
 
@@ -373,28 +535,46 @@ def main():
     dig.dig_set_impl({"auto": dig.DIG_IMPL_AUTO, "fma": dig.DIG_IMPL_FMA, "tensor": dig.DIG_IMPL_TENSOR, "mma": dig.DIG_IMPL_MMA}[args.family])
     peaks = load_peaks()
     W = max(args.warmup, 3)
+    K = args.steps
+    dt_id = dig.DIG_BF16 if wl.dtype == "bf16" else dig.DIG_F32
+    impl = dig.dig_gla_query_impl(wl.d_k, wl.d_v, wl.chunk, dt_id, int(wl.backward))
 
     blocks = make_blocks(wl, torch, dig)
     tokens_per_step = wl.B * wl.L * len(blocks)
-    th_per_block = wl.B * wl.L * wl.H
 
-    # headline: K steps, kernels launched back to back (one CUDA graph per step unless --eager)
-    sampler = ClockSampler(local)
-    ms_eager = time_steps(blocks, dig, torch, args.steps, W, dist, before_timed=None if not args.eager else sampler.start)
-    ms_graph = None
-    if not args.eager:
-        sampler.start()
-        ms_graph = time_graph_steps(blocks, dig, torch, args.steps, W, dist)
+    # ---- headline: K steps per repetition, repeated until min-seconds of device time have been measured
+    ms_eager = time_steps(blocks, dig, torch, K, W, dist)
+    graph = None if args.eager else capture_step(blocks, dig, torch)
+    launch_mode = "cuda_graph" if graph is not None else "eager"
+    if graph is not None:
+        for _ in range(W):
+            graph.replay()
+    one = (lambda: time_replays(graph, torch, K, dist)) if graph is not None else (lambda: time_steps(blocks, dig, torch, K, 0, dist))
+    first = one()
+    reps = int(min(200, max(3, math.ceil(args.min_seconds * 1e3 / max(first, 1e-3)))))
+    if dist is not None:           # every rank must run the same number of repetitions
+        t = torch.tensor([reps], dtype=torch.int64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        reps = int(t.item())
+    sampler = ClockSampler(local).start()
+    rep_ms = [one() for _ in range(reps)]
     clocks = sampler.stop()
-    ms = ms_graph if ms_graph is not None else ms_eager
-    launch_mode = "cuda_graph" if ms_graph is not None else "eager"
-    # per-kernel times: the same K steps once more with every launch bracketed by two CUDA events
-    ms_events = time_steps(blocks, dig, torch, args.steps, W, dist, before_timed=lambda: dig.dig_profile_enable(True))
-    prof = dig.dig_profile_read()
-    dig.dig_profile_enable(False)
+    ms = float(np.median(rep_ms))
+    value = job_tokens_per_s(tokens_per_step, K, world, ms)
+    step_s = ms * 1e-3 / K
+    timing = {"repetitions": reps, "steps_per_repetition": K, "median_ms": ms, "min_ms": min(rep_ms), "max_ms": max(rep_ms),
+              "timed_seconds_total": sum(rep_ms) * 1e-3,
+              "ms_per_step_x_sm_mhz": (ms / K) * clocks["sm_mhz"] if clocks.get("sm_mhz") else None}
+
+    # forward and backward on their own (same blocks, K steps of plain launches each)
+    parts = {}
+    if wl.backward:
+        for p in ("fwd", "bwd"):
+            parts[p + "_ms_per_step"] = time_steps(blocks, dig, torch, K, 2, dist, part=p) / K
+    # per-kernel times: the same steps once more with every launch bracketed by two CUDA events
+    shares = profile_kernels(blocks, dig, torch, min(K, 10))
     assert dig.dig_last_device_status() == dig.DIG_OK
-    launches = sum(n for n, _ in prof.values())
-    value = job_tokens_per_s(tokens_per_step, args.steps, world, ms)
+    launches_per_step = sum(s["launches"] for s in shares.values()) // min(K, 10)
 
     # end-to-end: pinned host -> device copies of every input, the same calls, device -> host of every result
     h2d = d2h = 0
@@ -402,84 +582,57 @@ def main():
         i, o = b.host_io(torch)
         h2d += i
         d2h += o
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_steps = max(3, min(K, 10))
     ms_e2e = time_steps(blocks, dig, torch, e2e_steps, 3, dist, e2e=True)
     e2e_value = job_tokens_per_s(tokens_per_step, e2e_steps, world, ms_e2e)
 
-    # roofline of the dominant kernel (largest share of device time), from the live event timings
-    fwd_b, bwd_b = bytes_per_token_head(wl)
-    alg_bytes = {"fma_chunk_bwd": bwd_b, "tc_chunk_bwd": bwd_b, "fma_chunk_out": fwd_b, "tc_chunk_out": fwd_b}
-    total_kernel_ms = sum(t for _, t in prof.values())
-    shares = {k: {"launches": n, "ms_per_launch": t / n, "share": t / total_kernel_ms} for k, (n, t) in prof.items()}
-    candidates = [k for k in prof if k in alg_bytes] or list(prof)
-    dom = max(candidates, key=lambda k: prof[k][1])
-    n_dom, t_dom = prof[dom]
-    roofline = None
-    if dom in alg_bytes:
-        achieved = alg_bytes[dom] * th_per_block / (t_dom / n_dom * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get((wl.name, dom)),
-                    "peak_source": peaks["source"],
-                    "algorithmic_bytes_per_launch": alg_bytes[dom] * th_per_block}
-    alg_f, exe_f = flops_per_token_head(wl, wl.chunk)
-    step_s = ms * 1e-3 / args.steps
-    tflops_alg = alg_f * th_per_block * len(blocks) / step_s / 1e12
-    tflops_exe = exe_f * th_per_block * len(blocks) / step_s / 1e12
-    impl = dig.dig_gla_query_impl(wl.d_k, wl.d_v, wl.chunk, dig.DIG_BF16 if wl.dtype == "bf16" else dig.DIG_F32, 1)
+    # rooflines: the whole step, and the kernels with a bandwidth model (the dominant one is the headline object)
+    work = step_work(wl, impl)
+    step_rl = roofline_fracs(work, step_s, peaks)
+    krl = kernel_rooflines(shares, wl, peaks)
+    gla_kernels = [k for k in shares if k in krl and k not in ("gate_logsigmoid", "srem_dwconv3x3")]
+    dom = max(gla_kernels or list(shares), key=lambda k: shares[k]["share"])
+    roofline = dict(krl.get(dom, {}), kernel=dom, share_of_step=shares[dom]["share"]) if dom in krl else None
 
     sweep = {}
     if not args.no_sweep and rank == 0 and world == 1:
-        del blocks
+        del blocks, graph
         torch.cuda.empty_cache()
-        cases = [("C3", {}), ("C4", {}), ("C4_chunk32", {"chunk": 32}), ("C4_chunk128", {"chunk": 128}), ("C5", {})]
-        for name, over in cases:
-            base_wl = CONFIGS[name.split("_")[0]]
-            w2 = base_wl.scaled(directions=(base_wl.directions[0],), conv=False, **over)
-            bl = make_blocks(w2, torch, dig)
-            big = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-            best = None
-            for _ in range(5):
-                big.zero_()      # flush L2 between single-step timings
-                m = time_steps(bl, dig, torch, 1, 1 if best is None else 0, None)
-                best = m if best is None else min(best, m)
-            a2, e2 = flops_per_token_head(w2, w2.chunk)
-            fb, bb = bytes_per_token_head(w2)
-            th = w2.B * w2.L * w2.H
-            fam = dig.dig_gla_query_impl(w2.d_k, w2.d_v, w2.chunk, dig.DIG_BF16, 1)
-            sweep[name] = {"L": w2.L, "B": w2.B, "H": w2.H, "d": w2.d_k, "chunk": w2.chunk, "ms": best,
-                           "kernel_family": {1: "fma", 2: "tensor", 3: "mma"}.get(fam, str(fam)),
-                           "tokens_per_s": w2.B * w2.L / (best * 1e-3),
-                           "tflops_alg": a2 * th / (best * 1e-3) / 1e12, "tflops_exec": e2 * th / (best * 1e-3) / 1e12,
-                           "hbm_frac_of_measured": (fb + bb) * th / (best * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-            del bl, big
-            torch.cuda.empty_cache()
-        sweep["note"] = ("gate + fwd + bwd of one block, first scan direction, L2 flushed before each timing, best of 5; "
-                         "chunk 128 is served by the tensor-core kernels in 64-token tiles")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        for name, base, over in [("C1", "C1", {}), ("C2", "C2", {}), ("C3", "C3", {}), ("C4", "C4", {}),
+                                 ("C4_chunk32", "C4", {"chunk": 32}), ("C4_chunk128", "C4", {"chunk": 128})]:
+            if base == wl.name and not over:
+                continue
+            sweep[name] = sweep_entry(name, CONFIGS[base].scaled(**over), torch, dig, peaks, local, flush)
+        sweep["note"] = ("one whole step of each workload per timing (its scan directions and conv), captured as a CUDA graph; "
+                         "cold = 256 MB written before every timing, warm = back to back; median of 20; roofline from the cold step; "
+                         "the tcgen05 kernels work on 64-token tiles for every requested chunk size (tile_executed)")
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu, _, _ = cpu_baseline(wl)
+        one_thread, _, _ = cpu_baseline(wl, budget_s=8.0, threads=1)
+        cpu["single_thread"] = {"value": one_thread["value"], "sample": one_thread["sample"]}
 
     if rank == 0:
         print(json.dumps({
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": W,
-            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": {dig.DIG_IMPL_TENSOR: "tf32", dig.DIG_IMPL_MMA: "tf32", dig.DIG_IMPL_FMA: "f32"}.get(impl, "f32"), "data": "synthetic",
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": {2: "f16", 3: "tf32", 1: "f32"}.get(impl, "f32"), "data": "synthetic",
             "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "grid": [wl.grid_h, wl.grid_w], "L": wl.L,
-                       "d_k": wl.d_k, "d_v": wl.d_v, "chunk": wl.chunk, "storage": wl.dtype,
+                       "d_k": wl.d_k, "d_v": wl.d_v, "chunk_requested": wl.chunk, "tile_executed": executed_tile(impl, wl.chunk),
+                       "storage": wl.dtype, "operands": "fp16 tiles, fp32 accumulation" if impl == 2 else None,
                        "directions": list(wl.directions), "conv": wl.conv, "blocks_per_step": len(wl.directions),
-                       "launch": launch_mode, "ms_per_step_eager": ms_eager / args.steps,
-                       "ms_per_step_with_kernel_events": ms_events / args.steps,
-                       "kernel_family": {1: "fma", 2: "tensor", 3: "mma"}.get(impl, str(impl)),
-                       "l2": "each block has its own buffers; a step streams several times the 126 MB L2, no flush needed",
-                       "tflops_alg": tflops_alg, "tflops_exec": tflops_exe,
-                       "tensor_frac_of_sustained_bf16_peak_exec": tflops_exe / peaks["bf16_tflops_sustained"]},
+                       "launch": launch_mode, "ms_per_step_eager": ms_eager / K, **parts,
+                       "kernel_family": FAMILY.get(impl, str(impl)),
+                       "l2": "each block has its own buffers; a step streams far more than the 126 MB L2, no flush needed",
+                       "step_roofline": step_rl, "timing": timing},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": ms_e2e / e2e_steps,
                     "copies": "pinned host buffers, two side streams (both PCIe directions overlap the kernels)"},
-            "gpu_launches": launches,
-            "roofline": roofline, "kernels": shares, "cpu_baseline": cpu, "sweep": sweep}))
+            "gpu_launches": launches_per_step * K,
+            "roofline": roofline, "kernel_rooflines": krl, "kernels": shares, "cpu_baseline": cpu, "sweep": sweep}))
     if dist is not None:
         dist.destroy_process_group()
 
