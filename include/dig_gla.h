@@ -38,8 +38,9 @@ typedef enum {
 /* Storage type of q, k, v, out, d_out, dq, dk, dv, x, y, w, bias.  Gates are always fp32.
  *   DIG_F32          fp32 storage, fp32 FMA arithmetic.
  *   DIG_BF16         bf16 storage in and out; products on the tensor cores with operands
- *                    carried at tf32 precision and fp32 accumulation; outputs rounded to
- *                    nearest-even bf16.
+ *                    carried at 11 significant bits (fp16 tiles in the tcgen05 kernels, tf32 in
+ *                    the warp-level ones) and fp32 accumulation; outputs rounded to nearest-even
+ *                    bf16.
  *   DIG_BF16_F32OUT  as DIG_BF16 but out / dq / dk / dv are stored as fp32 (the unrounded
  *                    accumulators).  DIG_BF16 results equal these rounded to bf16, bit for bit. */
 typedef enum { DIG_F32 = 0, DIG_BF16 = 1, DIG_BF16_F32OUT = 2 } dig_dtype;
@@ -49,7 +50,7 @@ typedef enum { DIG_F32 = 0, DIG_BF16 = 1, DIG_BF16_F32OUT = 2 } dig_dtype;
 typedef enum { DIG_ROW_FWD = 0, DIG_ROW_REV = 1, DIG_COL_FWD = 2, DIG_COL_REV = 3 } dig_dir;
 
 /* Which kernel family serves a call.  AUTO picks the tcgen05 tensor-core kernels (TENSOR) when they
- * cover the request (bf16 storage, d_k = d_v = 64, chunks of 64 or 128), else the warp-level
+ * cover the request (bf16 storage, d_k = d_v = 64 or 72, any chunk size), else the warp-level
  * tensor-core kernels (MMA: bf16 storage, any supported head and chunk size that fits shared
  * memory), else the fp32-FMA kernels (fp32 storage, whose products must be fp32-accurate).  Forcing
  * a family that does not cover the request returns DIG_ERR_UNSUPPORTED.  Process-wide; meant for
@@ -80,11 +81,16 @@ dig_status dig_gate_logsigmoid(const void *g, const float *tau_per_head, float *
  * depend on `chunk` beyond rounding.  No 1/sqrt(d) scaling and no normaliser are applied.
  *   q, k, gate: [B][L][H][d_k]; v, out: [B][L][H][d_v]; gate is log(alpha) <= 0, fp32.
  *   d_k, d_v: multiples of 8, 8..128; chunk in {16, 32, 64, 128}; L need not be a multiple of chunk.
- * The tensor-core kernels work on 64-token tiles: with them a request for chunk = 128 is evaluated
- * in 64-token tiles (dig_gla_query_impl tells which family serves a request).
- * The in-chunk decay is formed as exp(+-cumulative gate): the magnitude of the gate summed over
- * one chunk must stay below 80 per channel (true with a wide margin for sigmoid gates with
- * temperature >= 1 at the chunk sizes above); beyond it results may overflow. */
+ * The tcgen05 kernels work on 64-token tiles whatever `chunk` is: a shorter chunk is worked as sub-chunks
+ * of a tile, a longer one as 64 (dig_gla_query_impl tells which family serves a request).
+ * Range of the gates.  The in-chunk decay is formed as exp(+-cumulative gate).  The tcgen05 kernels keep
+ * the decayed operands in fp16 around the centre of a (sub-)chunk: where the gates of a 64-token tile sum
+ * to more than 15.9 in magnitude (any channel) the tile is worked in sub-chunks of 32, 16 or 8 tokens, so
+ * results stay exact for any decay up to 15.9 per 8 consecutive scan positions (log alpha about -2 per
+ * token).  Beyond that the call still completes with finite values, which are not the result, and
+ * dig_last_device_status reports DIG_ERR_RANGE.  The other families form exp(+-sum) in fp32 / tf32: there
+ * the magnitude of the gate summed over one chunk must stay below 80; beyond it results may overflow.
+ * Sigmoid gates with temperature >= 1 are inside both ranges with a wide margin. */
 dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float *gate, void *out,
                        int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
                        int direction, int dtype, void *workspace, size_t workspace_bytes,
@@ -120,7 +126,7 @@ dig_status dig_gla_fwd_static(const void *q, const void *k, const void *v, const
  * print it).  Nothing is saved by the forward call: chunk states are recomputed here.
  *   d_out: [B][L][H][d_v]; dq, dk: [B][L][H][d_k]; dv: [B][L][H][d_v]; dgate: fp32 [B][L][H][d_k].
  * The fp32-FMA and warp-level families cover chunk <= 64 here (shared memory); chunk = 128 is served by
- * the tcgen05 family only (bf16 storage, d_k = d_v = 64, 64-token tiles). */
+ * the tcgen05 family only (bf16 storage, d_k = d_v = 64 or 72, 64-token tiles). */
 dig_status dig_gla_bwd(const void *q, const void *k, const void *v, const float *gate,
                        const void *d_out, void *dq, void *dk, void *dv, float *dgate,
                        int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk,
@@ -224,8 +230,11 @@ dig_status dig_gla_bwd_beta(const void *q, const void *k, const void *v, const f
                             void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* Synchronises `cuda_stream`, then returns and clears the status recorded by device code on the
- * current device: DIG_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last query,
- * DIG_ERR_CUDA if the synchronisation itself failed, DIG_OK otherwise. */
+ * current device since the last query: DIG_ERR_TIMEOUT if a bounded wait inside a kernel expired,
+ * else DIG_ERR_RANGE if some gates decayed faster than the tcgen05 kernels represent (see dig_gla_fwd),
+ * DIG_ERR_CUDA if the synchronisation itself failed, DIG_OK otherwise.  The status is one word per
+ * device, shared by all streams and host threads: with several streams in flight the query tells that
+ * one of the calls since the last query had the condition, not which.  dig_set_impl is process-wide too. */
 dig_status dig_last_device_status(void *cuda_stream);
 
 const char *dig_status_string(int status);

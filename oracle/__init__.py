@@ -247,3 +247,47 @@ def gla_bwd_beta(q, k, v, a, bg, dout, grid_h, grid_w, direction=ROW_FWD, thread
                                            _p(da), _p(db), B, H, grid_h, grid_w, dk, dv_, direction, threads),
            "gla_bwd_beta")
     return dq, dk_, dv, da, db
+
+
+# ---- several scan orders summed (Algorithm 2: bidirectional, Algorithm 3: 4-directional scanning) ----
+def _scan_order(direction: int, grid_h: int, grid_w: int) -> np.ndarray:
+    """Token visited at each position after the re-orderings the algorithms apply to the sequence:
+    nothing, flip, flatten(transpose(reshape2d)), and flip of the transposed sequence."""
+    idx = np.arange(grid_h * grid_w)
+    if direction in (COL_FWD, COL_REV):
+        idx = idx.reshape(grid_h, grid_w).T.reshape(-1)
+    if direction in (ROW_REV, COL_REV):
+        idx = idx[::-1]
+    return np.ascontiguousarray(idx)
+
+
+def gla_fwd_multi(q, k, v, a, grid_h, grid_w, directions, threads=1) -> np.ndarray:
+    """z_out = sum over the listed scan orders of GLA(re-ordered sequence) brought back to the input
+    order, written out as the algorithms do: permute, run the recurrence on the plain sequence, undo
+    the permutation, add."""
+    q, k, v, a = _f64(q), _f64(k), _f64(v), _f64(a)
+    L = grid_h * grid_w
+    out = np.zeros_like(v)
+    for d in directions:
+        p = _scan_order(d, grid_h, grid_w)
+        o = gla_fwd(q[:, p], k[:, p], v[:, p], a[:, p], 1, L, ROW_FWD, threads=threads)
+        back = np.empty_like(o)
+        back[:, p] = o
+        out += back
+    return out
+
+
+def gla_bwd_multi(q, k, v, a, dout, grid_h, grid_w, directions, threads=1):
+    """Gradients of <dout, gla_fwd_multi(...)> with respect to q, k, v and a: the sum over the scan
+    orders of the single-order gradients, each computed on the re-ordered sequence and brought back."""
+    q, k, v, a, dout = _f64(q), _f64(k), _f64(v), _f64(a), _f64(dout)
+    L = grid_h * grid_w
+    tot = [np.zeros_like(q), np.zeros_like(k), np.zeros_like(v), np.zeros_like(a)]
+    for d in directions:
+        p = _scan_order(d, grid_h, grid_w)
+        gs = gla_bwd(q[:, p], k[:, p], v[:, p], a[:, p], dout[:, p], 1, L, ROW_FWD, threads=threads)
+        for t, g_ in zip(tot, gs):
+            back = np.empty_like(g_)
+            back[:, p] = g_
+            t += back
+    return tuple(tot)

@@ -96,3 +96,52 @@ def test_families_are_the_intended_ones():
                 assert dig.dig_gla_query_impl(d, d, chunk, dig.DIG_BF16, 1) == dig.DIG_IMPL_MMA
     finally:
         dig.dig_set_impl(dig.DIG_IMPL_AUTO)
+
+
+def _constant_gate_case(per_token, d=64):
+    from paper_2405_18428_b200 import dig
+    from parity import to_dev
+    wl = _wl(d, 64, grid_h=10, grid_w=20)
+    x = make_inputs(wl, conv=False)
+    gate = np.full(x["q"].shape, per_token, dtype=np.float32)
+    q, k, v, dO = (to_dev(x[n], wl) for n in ("q", "k", "v", "dO"))
+    return wl, x, gate, (q, k, v, torch.from_numpy(gate).cuda(), dO)
+
+
+@pytest.mark.parametrize("d", [64, 72])
+def test_fast_decay_inside_the_range_is_worked_in_sub_chunks(d):
+    """log alpha = -1.9 per token: 64 tokens sum to -122, far beyond what one fp16 tile can centre; the tcgen05
+    kernels fall back to 8-token sub-chunks (8 x 1.9 = 15.2 < 15.9) and still match the oracle."""
+    import oracle
+    from paper_2405_18428_b200 import dig
+    from parity import TOL_BF16, rel_err
+    wl, x, gate, (q, k, v, g, dO) = _constant_gate_case(-1.9, d)
+    out = dig.dig_gla_fwd(q, k, v, g, wl.grid_h, wl.grid_w, 64, 2, f32_out=True)
+    grads = dig.dig_gla_bwd(q, k, v, g, dO, wl.grid_h, wl.grid_w, 64, 2, f32_out=True)
+    torch.cuda.synchronize()
+    assert dig.dig_last_device_status() == dig.DIG_OK
+    a = gate.astype(np.float64)
+    ref = (oracle.gla_fwd(x["q"], x["k"], x["v"], a, wl.grid_h, wl.grid_w, 2),
+           *oracle.gla_bwd(x["q"], x["k"], x["v"], a, x["dO"], wl.grid_h, wl.grid_w, 2))
+    for name, got, want in zip(("out", "dq", "dk", "dv", "dgate"), (out, *grads), ref):
+        got = got.float().cpu().numpy()
+        assert np.isfinite(got).all(), name
+        assert rel_err(got, want) <= TOL_BF16, (name, rel_err(got, want))
+
+
+def test_decay_beyond_the_range_is_reported_not_silent():
+    """log alpha = -3 per token: even 8 tokens sum to -24.  The call must say so through the device status
+    (DIG_ERR_RANGE), return finite numbers, and the status must be cleared by the query."""
+    from paper_2405_18428_b200 import dig
+    wl, x, gate, (q, k, v, g, dO) = _constant_gate_case(-3.0)
+    out = dig.dig_gla_fwd(q, k, v, g, wl.grid_h, wl.grid_w, 64, 0, f32_out=True)
+    torch.cuda.synchronize()
+    assert dig.dig_last_device_status() == dig.DIG_ERR_RANGE
+    assert dig.dig_last_device_status() == dig.DIG_OK
+    assert torch.isfinite(out).all()
+    grads = dig.dig_gla_bwd(q, k, v, g, dO, wl.grid_h, wl.grid_w, 64, 0, f32_out=True)
+    torch.cuda.synchronize()
+    assert dig.dig_last_device_status() == dig.DIG_ERR_RANGE
+    for t in grads:
+        assert torch.isfinite(t).all()
+    assert "range" in dig.status_string(dig.DIG_ERR_RANGE)
