@@ -229,6 +229,26 @@ dig_status dig_gla_bwd_beta(const void *q, const void *k, const void *v, const f
                             int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int direction, int dtype,
                             void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Several scan orders at once (Algorithm 2, bidirectional scanning: GLA(z) + flip(GLA(flip(z))); Algorithm 3,
+ * 4-directional scanning: the row and column orders, forward and flipped, summed):
+ *     out = sum over the directions d in direction_mask of dig_gla_fwd(..., direction = d),
+ * bit d of direction_mask (1 .. 15) selecting dig_dir d, all orders reading the same q, k, v and gate and
+ * writing canonical positions.  dig_gla_bwd_multi returns the gradients of <d_out, out> (the sums of the
+ * single-order gradients).  The orders run one after the other on the stream; each adds its fp32 results
+ * to the same buffers (caller's for DIG_BF16_F32OUT, workspace for DIG_BF16), so the sum is formed in fp32
+ * and rounded to bf16 once.  Served by the tcgen05 kernels only (bf16 storage, d_k = d_v = 64 or 72; else
+ * DIG_ERR_UNSUPPORTED); workspace from dig_gla_multi_workspace_bytes (0 for invalid or unsupported sizes).
+ * Tensors, sizes and the gate range are those of dig_gla_fwd / dig_gla_bwd. */
+size_t dig_gla_multi_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int dtype,
+                                     int backward);
+dig_status dig_gla_fwd_multi(const void *q, const void *k, const void *v, const float *gate, void *out, int B, int H,
+                             int grid_h, int grid_w, int d_k, int d_v, int chunk, unsigned direction_mask, int dtype,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+dig_status dig_gla_bwd_multi(const void *q, const void *k, const void *v, const float *gate, const void *d_out,
+                             void *dq, void *dk, void *dv, float *dgate, int B, int H, int grid_h, int grid_w, int d_k,
+                             int d_v, int chunk, unsigned direction_mask, int dtype, void *workspace,
+                             size_t workspace_bytes, void *cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the status recorded by device code on the
  * current device since the last query: DIG_ERR_TIMEOUT if a bounded wait inside a kernel expired,
  * else DIG_ERR_RANGE if some gates decayed faster than the tcgen05 kernels represent (see dig_gla_fwd),

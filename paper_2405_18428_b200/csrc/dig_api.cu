@@ -391,6 +391,58 @@ dig_status dig_gla_bwd_beta(const void *q, const void *k, const void *v, const f
     return mma_gla_bwd(a);
 }
 
+size_t dig_gla_multi_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int dtype,
+                                     int backward)
+{
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, 0, dtype)) return 0;
+    if (!sweep_supports(d_k, d_v, chunk, dtype)) return 0;
+    return sweep_multi_workspace_bytes(make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, 0), backward != 0, dtype);
+}
+
+dig_status dig_gla_fwd_multi(const void *q, const void *k, const void *v, const float *gate, void *out, int B, int H,
+                             int grid_h, int grid_w, int d_k, int d_v, int chunk, unsigned direction_mask, int dtype,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!q || !k || !v || !gate || !out) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(out)) return DIG_ERR_INVALID_ARG;
+    if (direction_mask == 0 || direction_mask > 15u) return DIG_ERR_INVALID_ARG;
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, 0, dtype)) return DIG_ERR_INVALID_ARG;
+    if (!sweep_supports(d_k, d_v, chunk, dtype)) return DIG_ERR_UNSUPPORTED;
+    const size_t need = dig_gla_multi_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, 0);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    GlaArgs a{};
+    a.q = q; a.k = k; a.v = v; a.gate = gate; a.out = out;
+    a.ws = reinterpret_cast<float *>(workspace);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, 0);
+    a.dtype = dtype;
+    a.stream = (cudaStream_t)cuda_stream;
+    return sweep_gla_fwd_multi(a, direction_mask);
+}
+
+dig_status dig_gla_bwd_multi(const void *q, const void *k, const void *v, const float *gate, const void *d_out,
+                             void *dq, void *dk, void *dv, float *dgate, int B, int H, int grid_h, int grid_w, int d_k,
+                             int d_v, int chunk, unsigned direction_mask, int dtype, void *workspace,
+                             size_t workspace_bytes, void *cuda_stream)
+{
+    if (!q || !k || !v || !gate || !d_out || !dq || !dk || !dv || !dgate) return DIG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(d_out) ||
+        !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(dgate))
+        return DIG_ERR_INVALID_ARG;
+    if (direction_mask == 0 || direction_mask > 15u) return DIG_ERR_INVALID_ARG;
+    if (!valid_geometry(B, H, grid_h, grid_w, d_k, d_v, chunk, 0, dtype)) return DIG_ERR_INVALID_ARG;
+    if (!sweep_supports(d_k, d_v, chunk, dtype)) return DIG_ERR_UNSUPPORTED;
+    const size_t need = dig_gla_multi_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, 1);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DIG_ERR_WORKSPACE;
+    GlaArgs a{};
+    a.q = q; a.k = k; a.v = v; a.gate = gate; a.d_out = d_out;
+    a.dq = dq; a.dk = dk; a.dv = dv; a.dgate = dgate;
+    a.ws = reinterpret_cast<float *>(workspace);
+    a.g = make_geom(B, H, grid_h, grid_w, d_k, d_v, chunk, 0);
+    a.dtype = dtype;
+    a.stream = (cudaStream_t)cuda_stream;
+    return sweep_gla_bwd_multi(a, direction_mask);
+}
+
 dig_status dig_last_device_status(void *cuda_stream)
 {
     if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return DIG_ERR_CUDA;

@@ -85,6 +85,7 @@ struct GlaArgs {
     float *ws;                   // workspace base (fp32 view)
     Geom g;
     int dtype;
+    int accumulate;              // outputs are added to what the (fp32) output buffers hold
     cudaStream_t stream;
 };
 

@@ -41,6 +41,7 @@ struct SweepArgs {
     __half *seg_state16, *slot_s;
     float *slot_g;
     int *status;
+    int accumulate;
     Geom g;
     Plan plan;
 };
@@ -556,7 +557,7 @@ sweep_fwd(const SweepArgs a)
                             if (jc < C::NCH) {
                                 float o[8];
                                 tmem_ld8(lane_base + tmem + aO + 8 * jc, o);
-                                if (inrow) store_out8(out + ro + 8 * jc, o);
+                                if (inrow) store_out8(out + ro + 8 * jc, o, a.accumulate != 0);
                             }
                         }
                     }
@@ -768,7 +769,7 @@ sweep_bwd(const SweepArgs a)
 #pragma unroll
                                     for (int e = 0; e < 8; ++e) a1[e] = fmaf(hh[e], a2[e], a1[e]);
                                 } else if (inrow) {
-                                    store_out8(dv + ro + 8 * jc, a2);
+                                    store_out8(dv + ro + 8 * jc, a2, a.accumulate != 0);
                                 }
                                 {
                                     // q*dq = Qc * (dq accumulator), k*dk = Kc * (dk accumulator): the decay factors cancel
@@ -789,7 +790,7 @@ sweep_bwd(const SweepArgs a)
                                 __syncwarp();           // both halves have read their gates before the table is overwritten
                                 if (inrow) {
                                     if (hf == 0) st8(table + r16 * C::LAMP + 8 * jc, x);        // q*dq - k*dk
-                                    store_out8((hf ? dk : dq) + ro + 8 * jc, a1);
+                                    store_out8((hf ? dk : dq) + ro + 8 * jc, a1, a.accumulate != 0);
                                 }
                             }
                         }
@@ -830,7 +831,7 @@ sweep_bwd(const SweepArgs a)
 #pragma unroll
                     for (int j = 0; j < L::RPS; ++j) {
                         const int ro = r0 + j < nrow ? rowOff[cur * T + r0 + j] : -1;
-                        if (ro >= 0) a.dgate[(size_t)ro + c] = sfx[j] + add;
+                        if (ro >= 0) a.dgate[(size_t)ro + c] = (a.accumulate ? a.dgate[(size_t)ro + c] : 0.f) + (sfx[j] + add);
                     }
                 }
                 cpar ^= 1;
@@ -937,6 +938,7 @@ dig_status run(const GlaArgs &ga)
     a.seg_state = w.seg_state; a.seg_gamma = w.seg_gamma; a.seg_dstate = w.seg_dstate; a.seg_carry = w.seg_carry;
     a.seg_state16 = w.seg_state16; a.slot_s = w.slot_s; a.slot_g = w.slot_g;
     a.status = status;
+    a.accumulate = ga.accumulate;
     a.g = g;
     a.plan = pl;
     const int grid_l = (int)(total < (long long)sms * OCC_L ? total : (long long)sms * OCC_L);
@@ -991,6 +993,86 @@ size_t sweep_workspace_bytes(const Geom &g, bool backward)
     if (sms <= 0) sms = 148;
     const Plan pl = make_plan(g, sms, sweep_per_sm(g.dk, backward));
     return carve(nullptr, g, pl, backward).bytes;
+}
+
+namespace {
+
+// fp32 sums -> bf16 results (round to nearest even), 8 elements per thread.
+__global__ void __launch_bounds__(256) round_to_bf16(const float *__restrict__ src, bf16 *__restrict__ dst, size_t n8)
+{
+    pdl_wait();
+    pdl_launch_dependents();
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n8) return;
+    float f[8];
+    ld8(src + 8 * i, f);
+    store_out8(dst + 8 * i, f);
+}
+dig_status launch_round(const float *src, void *dst, size_t n, cudaStream_t s)
+{
+    const size_t n8 = n / 8;
+    launch_pdl(round_to_bf16, dim3((unsigned)((n8 + 255) / 256)), dim3(256), 0, s, src, (bf16 *)dst, n8);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace
+
+// Several scan orders summed (Algorithm 2 / Algorithm 3): the orders run one after the other, each
+// adding its fp32 results to the same buffers, which are rounded to the storage type once at the end.
+size_t sweep_multi_workspace_bytes(const Geom &g, bool backward, int dtype)
+{
+    size_t n = align256(sweep_workspace_bytes(g, backward));
+    if (dtype == DIG_BF16) {
+        const size_t tok = (size_t)g.B * g.L * g.H;
+        n += backward ? align256(tok * g.dk * 4) * 2 + align256(tok * g.dv * 4) : align256(tok * g.dv * 4);
+    }
+    return n;
+}
+
+dig_status sweep_gla_fwd_multi(const GlaArgs &a0, unsigned mask)
+{
+    GlaArgs a = a0;
+    const size_t tok = (size_t)a.g.B * a.g.L * a.g.H;
+    char *extra = reinterpret_cast<char *>(a0.ws) + align256(sweep_workspace_bytes(a.g, false));
+    const bool narrow = a0.dtype == DIG_BF16;
+    a.dtype = DIG_BF16_F32OUT;
+    if (narrow) a.out = extra;
+    bool first = true;
+    for (int d = 0; d < 4; ++d) {
+        if (!(mask >> d & 1)) continue;
+        a.g.dir = d;
+        a.accumulate = first ? 0 : 1;
+        first = false;
+        const dig_status st = sweep_gla_fwd(a);
+        if (st != DIG_OK) return st;
+    }
+    return narrow ? launch_round(reinterpret_cast<const float *>(extra), a0.out, tok * a.g.dv, a.stream) : DIG_OK;
+}
+
+dig_status sweep_gla_bwd_multi(const GlaArgs &a0, unsigned mask)
+{
+    GlaArgs a = a0;
+    const size_t tok = (size_t)a.g.B * a.g.L * a.g.H;
+    char *extra = reinterpret_cast<char *>(a0.ws) + align256(sweep_workspace_bytes(a.g, true));
+    const bool narrow = a0.dtype == DIG_BF16;
+    a.dtype = DIG_BF16_F32OUT;
+    float *sq = reinterpret_cast<float *>(extra), *sk = reinterpret_cast<float *>(extra + align256(tok * a.g.dk * 4));
+    float *sv = reinterpret_cast<float *>(extra + 2 * align256(tok * a.g.dk * 4));
+    if (narrow) { a.dq = sq; a.dk = sk; a.dv = sv; }
+    bool first = true;
+    for (int d = 0; d < 4; ++d) {
+        if (!(mask >> d & 1)) continue;
+        a.g.dir = d;
+        a.accumulate = first ? 0 : 1;
+        first = false;
+        const dig_status st = sweep_gla_bwd(a);
+        if (st != DIG_OK) return st;
+    }
+    if (!narrow) return DIG_OK;
+    dig_status st;
+    if ((st = launch_round(sq, a0.dq, tok * a.g.dk, a.stream)) != DIG_OK) return st;
+    if ((st = launch_round(sk, a0.dk, tok * a.g.dk, a.stream)) != DIG_OK) return st;
+    return launch_round(sv, a0.dv, tok * a.g.dv, a.stream);
 }
 
 dig_status sweep_gla_fwd(const GlaArgs &a)

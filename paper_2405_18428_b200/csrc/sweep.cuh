@@ -125,9 +125,21 @@ __device__ __forceinline__ void st8(float *p, const float (&f)[8])
     *reinterpret_cast<float4 *>(p) = make_float4(f[0], f[1], f[2], f[3]);
     *reinterpret_cast<float4 *>(p + 4) = make_float4(f[4], f[5], f[6], f[7]);
 }
-// 8 results to global memory in the output storage type.
-__device__ __forceinline__ void store_out8(float *p, const float (&f)[8]) { st8(p, f); }
-__device__ __forceinline__ void store_out8(bf16 *p, const float (&f)[8])
+// 8 results to global memory in the output storage type.  `add`: on top of what is there (fp32
+// outputs only; used when several scan orders are summed into one buffer).
+__device__ __forceinline__ void store_out8(float *p, const float (&f)[8], bool add = false)
+{
+    if (add) {
+        float o[8];
+        ld8(p, o);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o[e] += f[e];
+        st8(p, o);
+    } else {
+        st8(p, f);
+    }
+}
+__device__ __forceinline__ void store_out8(bf16 *p, const float (&f)[8], bool = false)
 {
     uint4 u;
     __nv_bfloat162 t;
@@ -428,5 +440,9 @@ bool sweep_supports(int dk, int dv, int chunk, int dtype);
 size_t sweep_workspace_bytes(const Geom &g, bool backward);
 dig_status sweep_gla_fwd(const GlaArgs &a);
 dig_status sweep_gla_bwd(const GlaArgs &a);
+// Sums over the scan orders of `mask` (bit d = direction d); outputs in the storage type of a.dtype.
+size_t sweep_multi_workspace_bytes(const Geom &g, bool backward, int dtype);
+dig_status sweep_gla_fwd_multi(const GlaArgs &a, unsigned mask);
+dig_status sweep_gla_bwd_multi(const GlaArgs &a, unsigned mask);
 
 }  // namespace dig

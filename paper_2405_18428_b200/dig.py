@@ -25,6 +25,7 @@ DIG_IMPL_AUTO, DIG_IMPL_FMA, DIG_IMPL_TENSOR, DIG_IMPL_MMA = 0, 1, 2, 3
 
 EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig_gate_logsigmoid",
            "dig_gla_fwd", "dig_gla_fwd_static", "dig_gla_bwd", "dig_gla_fwd_state", "dig_gla_bwd_state",
+           "dig_gla_fwd_multi", "dig_gla_bwd_multi", "dig_gla_multi_workspace_bytes",
            "dig_gla_fwd_beta", "dig_gla_bwd_beta", "dig_gla_beta_workspace_bytes", "dig_gla_fwd_outgate", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
            "dig_srem_dwconv_bwd_workspace_bytes", "dig_gla_outgate_fwd", "dig_gla_outgate_bwd",
            "dig_gla_outgate_bwd_workspace_bytes", "dig_last_device_status",
@@ -63,6 +64,12 @@ def lib() -> ctypes.CDLL:
         L.dig_gla_fwd_static.restype = i
         L.dig_gla_bwd.argtypes = [vp] * 9 + [i] * 9 + [vp, sz, vp]
         L.dig_gla_bwd.restype = i
+        L.dig_gla_multi_workspace_bytes.argtypes = [i] * 9
+        L.dig_gla_multi_workspace_bytes.restype = sz
+        L.dig_gla_fwd_multi.argtypes = [vp] * 5 + [i] * 7 + [ctypes.c_uint, i] + [vp, sz, vp]
+        L.dig_gla_fwd_multi.restype = i
+        L.dig_gla_bwd_multi.argtypes = [vp] * 9 + [i] * 7 + [ctypes.c_uint, i] + [vp, sz, vp]
+        L.dig_gla_bwd_multi.restype = i
         L.dig_gla_fwd_outgate.argtypes = [vp] * 7 + [ctypes.c_float, vp, vp] + [i] * 9 + [vp, sz, vp]
         L.dig_gla_fwd_outgate.restype = i
         L.dig_gla_beta_workspace_bytes.argtypes = [i] * 9
@@ -228,6 +235,60 @@ def dig_gla_bwd(q, k, v, gate, d_out, grid_h, grid_w, chunk=64, direction=DIG_RO
                              B, H, grid_h, grid_w, dk, dv, chunk, direction, dtype,
                              workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                              _stream()), "dig_gla_bwd")
+    return dq, dk_, dv_, dgate
+
+
+def _mask(directions) -> int:
+    m = 0
+    for d in directions:
+        m |= 1 << int(d)
+    return m
+
+
+def dig_gla_multi_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, backward) -> int:
+    return lib().dig_gla_multi_workspace_bytes(B, H, grid_h, grid_w, d_k, d_v, chunk, dtype, int(backward))
+
+
+def dig_gla_fwd_multi(q, k, v, gate, grid_h, grid_w, directions, chunk=64, *, f32_out=False, out=None,
+                      workspace=None) -> torch.Tensor:
+    """Sum of dig_gla_fwd over the scan orders in `directions` (an iterable of dig_dir values)."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st = _storage(dtype)
+    if out is None:
+        out = torch.empty((B, L, H, dv), dtype=_out_storage(dtype), device=q.device)
+    need = dig_gla_multi_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 0)
+    workspace = _workspace(workspace, need, q.device)
+    _check(lib().dig_gla_fwd_multi(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"), _dev(v, st, (B, L, H, dv), "v"),
+                                   _dev(gate, torch.float32, q.shape, "gate"),
+                                   _dev(out, _out_storage(dtype), (B, L, H, dv), "out"),
+                                   B, H, grid_h, grid_w, dk, dv, chunk, _mask(directions), dtype,
+                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "dig_gla_fwd_multi")
+    return out
+
+
+def dig_gla_bwd_multi(q, k, v, gate, d_out, grid_h, grid_w, directions, chunk=64, *, f32_out=False, grads=None,
+                      workspace=None):
+    """Gradients of <d_out, dig_gla_fwd_multi(...)>: returns (dq, dk, dv, dgate)."""
+    B, L, H, dk = q.shape
+    dv = v.shape[-1]
+    dtype = _dtype_of(q, f32_out)
+    st, ost = _storage(dtype), _out_storage(dtype)
+    if grads is None:
+        grads = (torch.empty(q.shape, dtype=ost, device=q.device), torch.empty(q.shape, dtype=ost, device=q.device),
+                 torch.empty(v.shape, dtype=ost, device=q.device), torch.empty(q.shape, dtype=torch.float32, device=q.device))
+    dq, dk_, dv_, dgate = grads
+    need = dig_gla_multi_workspace_bytes(B, H, grid_h, grid_w, dk, dv, chunk, dtype, 1)
+    workspace = _workspace(workspace, need, q.device)
+    _check(lib().dig_gla_bwd_multi(_dev(q, st, name="q"), _dev(k, st, q.shape, "k"), _dev(v, st, (B, L, H, dv), "v"),
+                                   _dev(gate, torch.float32, q.shape, "gate"), _dev(d_out, st, v.shape, "d_out"),
+                                   _dev(dq, ost, q.shape, "dq"), _dev(dk_, ost, q.shape, "dk"),
+                                   _dev(dv_, ost, v.shape, "dv"), _dev(dgate, torch.float32, q.shape, "dgate"),
+                                   B, H, grid_h, grid_w, dk, dv, chunk, _mask(directions), dtype,
+                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "dig_gla_bwd_multi")
     return dq, dk_, dv_, dgate
 
 
