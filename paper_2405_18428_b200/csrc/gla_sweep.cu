@@ -197,7 +197,11 @@ sweep_local(const SweepArgs a)
         load_raw<D, NT, BWD, BWD>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
         for (int tile = t0; tile < t1; ++tile) {
             const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
-            if (tid < T) rowOff[nxt * T + tid] = tile + 1 < t1 ? tile_row_offset(g, b, h, D, tile + 1, tid) : -1;
+            if (tid < T) {
+                rowOff[nxt * T + tid] = tile + 1 < t1 ? tile_row_offset(g, b, h, D, tile + 1, tid) : -1;
+                // this kernel's tiles are short: the register prefetch alone does not cover the memory latency
+                if (tile + 2 < t1) prefetch_row<D, BWD, BWD>(a.q, a.k, a.v, a.d_out, a.gate, tile_row_offset(g, b, h, D, tile + 2, tid));
+            }
             write_gates<D, NT, BWD, BWD>(raw, table, rowOff + cur * T);
             __syncthreads();
             float tot_unused;
@@ -292,7 +296,7 @@ seg_scan(float *seg_state, const float *seg_gamma, float *seg_dstate, float *seg
          const float *s_in, float *s_out, const float *ds_out, float *ds_in, int nseg)
 {
     constexpr int NV = (D / 4 + 7) / 8;               // float4 pieces per lane
-    constexpr int NB = 4;                             // segments whose loads are in flight together
+    constexpr int NB = NV <= 2 ? 8 : 4;               // segments whose loads are in flight together
     const int bh = blockIdx.y, c = blockIdx.x * 8 + (threadIdx.x >> 3), l8 = threadIdx.x & 7;
     pdl_wait();
     pdl_launch_dependents();

@@ -233,6 +233,31 @@ __device__ __forceinline__ void load_raw(Raw<Lay<D, NT>::NIT, HQ, HD> &r, const 
     }
 }
 
+// Asks the L2 for one token row of every input tensor (a tile further ahead than the register
+// prefetch reaches, so that the register loads find their lines in the L2).
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" :: "l"(p)); }
+template <int D, bool HQ, bool HD>
+__device__ __forceinline__ void prefetch_row(const bf16 *q, const bf16 *k, const bf16 *v, const bf16 *d_out,
+                                             const float *gate, int row_off)
+{
+    if (row_off < 0) return;
+#pragma unroll
+    for (int b = 0; b < 2 * D; b += 128) {
+        const int e = (b < 2 * D - 16 ? b : 2 * D - 16) / 2;        // the last piece covers the row's end
+        prefetch_l2(k + row_off + e);
+        prefetch_l2(v + row_off + e);
+        if (HQ) prefetch_l2(q + row_off + e);
+        if (HD) prefetch_l2(d_out + row_off + e);
+    }
+    prefetch_l2(k + row_off + D - 8);
+    prefetch_l2(v + row_off + D - 8);
+    if (HQ) prefetch_l2(q + row_off + D - 8);
+    if (HD) prefetch_l2(d_out + row_off + D - 8);
+#pragma unroll
+    for (int b = 0; b < 4 * D; b += 128) prefetch_l2(gate + row_off + b / 4);
+    prefetch_l2(gate + row_off + D - 4);
+}
+
 // Gates of the prefetched tile into the table, in log2 units, zero for rows past the end.
 template <int D, int NT, bool HQ, bool HD>
 __device__ __forceinline__ void write_gates(const Raw<Lay<D, NT>::NIT, HQ, HD> &r, float *table, const int *row_off)
