@@ -136,7 +136,7 @@ def recorded_traffic(kernel, workload):
     if rec.get("source_hash") != source_hash():
         return None
     for r in rec.get("kernels", []):
-        if r["kernel"] == kernel and r["workload"] == workload:
+        if r["kernel"].startswith(kernel) and r["workload"] == workload:
             return r["dram_bytes_per_launch"]
     return None
 

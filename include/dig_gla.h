@@ -11,7 +11,8 @@
  *     (the row-major flattening of the patch grid, i.e. the (B, T, D) sequence of Algorithm 1
  *     split into H heads).  Results are written at canonical positions for every direction.
  *   - Calls only enqueue work on the given stream; they do not synchronise and allocate no
- *     device memory.  Scratch memory is a caller-provided workspace.
+ *     device memory.  Scratch memory is a caller-provided workspace (dig_gla_fwd_static alone
+ *     keeps its scratch in an array of the library image).
  *   - Errors are return codes.  Arguments are validated on the host before any launch; after a
  *     non-zero return the outputs are unspecified.  Nothing traps, aborts or prints.
  */
@@ -102,20 +103,24 @@ dig_status dig_gla_fwd(const void *q, const void *k, const void *v, const float 
  * Who it is for: callers that cannot obtain device memory at call time -- a host application that
  * owns every byte of the GPU and hands plugins only their inputs and outputs, a latency-critical
  * loop in which cudaMalloc's implicit synchronisation is unacceptable, a process whose memory
- * budget was fixed at start-up.  For them the chunk states and decay factors that dig_gla_fwd keeps
+ * budget was fixed at start-up.  For them the segment states and decay factors that dig_gla_fwd keeps
  * in the caller's workspace live in a device array of DIG_GLA_STATIC_SCRATCH_BYTES that is part of
- * the library image: every GPU that loads the library holds that much memory until the process
- * exits.  The call itself allocates and frees nothing, on the host side of CUDA or through torch.
+ * the library image.  A device holds that array from the moment the CUDA runtime loads this part of
+ * the library on it until the process exits: with lazy module loading (the default since CUDA 12)
+ * that moment is the first dig_gla_fwd_static call on the device, whose address look-up triggers the
+ * load and may take a while or fail with DIG_ERR_CUDA; with CUDA_MODULE_LOADING=EAGER it is context
+ * creation.  Make that first call at start-up, outside any stream capture and outside the loop that
+ * must not stall; every later call allocates and frees nothing, on the host side of CUDA or through
+ * torch.
  *
  * Limit: requests for which dig_gla_workspace_bytes(..., backward = 0) exceeds
  * DIG_GLA_STATIC_SCRATCH_BYTES return DIG_ERR_SCRATCH_LIMIT before anything is launched (16 MiB
  * covers e.g. B*H = 48 sequences of 1024 tokens at d_k = d_v = 64, chunk 64).
  *
- * The first call on each device looks up the array's device address (with that device current);
- * make that first call outside any stream capture.  All calls on a device share the one array:
- * it keeps whatever the previous call left there (the kernels overwrite every entry they read,
- * so nothing needs clearing), and two calls whose kernels overlap on the GPU -- different streams,
- * or different host threads -- race on it.  Serialise them on one stream. */
+ * All calls on a device share the one array: it keeps whatever the previous call left there (the
+ * kernels overwrite every entry they read, so nothing needs clearing), and two calls whose kernels
+ * overlap on the GPU -- different streams, or different host threads -- race on it.  Serialise them
+ * on one stream. */
 #define DIG_GLA_STATIC_SCRATCH_BYTES ((size_t)16 << 20)
 dig_status dig_gla_fwd_static(const void *q, const void *k, const void *v, const float *gate,
                               void *out, int B, int H, int grid_h, int grid_w, int d_k, int d_v,
@@ -256,6 +261,12 @@ dig_status dig_gla_bwd_multi(const void *q, const void *k, const void *v, const 
  * device, shared by all streams and host threads: with several streams in flight the query tells that
  * one of the calls since the last query had the condition, not which.  dig_set_impl is process-wide too. */
 dig_status dig_last_device_status(void *cuda_stream);
+
+/* Self-test of the bounded waits (the paper has no counterpart): launches one small kernel whose only
+ * wait can never be satisfied and gives up after limit_us microseconds (1 .. 100000), exactly as the
+ * production kernels' waits do after 0.25 s.  Afterwards dig_last_device_status returns DIG_ERR_TIMEOUT
+ * once; the device and the context stay usable. */
+dig_status dig_selftest_wait_timeout(unsigned limit_us, void *cuda_stream);
 
 const char *dig_status_string(int status);
 

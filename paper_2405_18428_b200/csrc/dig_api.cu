@@ -5,6 +5,7 @@
 
 #include "dig_common.cuh"
 #include "sweep.cuh"
+#include "umma.cuh"
 
 namespace dig {
 
@@ -110,6 +111,19 @@ KernelTimer::KernelTimer(int kernel_id, cudaStream_t s) : slot(-1), stream(s)
 KernelTimer::~KernelTimer()
 {
     if (slot >= 0) cudaEventRecord(g_prof.ev[2 * slot + 1], stream);
+}
+
+// One CTA waits on an mbarrier that nothing ever arrives on, with a short limit: exercises the path a
+// bounded wait takes when it gives up (status word, normal return).
+__global__ void wait_that_expires(int *status, unsigned long long limit_ns)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        umma::mbar_init(&bar, 1);
+        umma::fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) umma::mbar_wait(&bar, 0, status, limit_ns);
 }
 
 int *device_status_ptr()
@@ -454,6 +468,15 @@ dig_status dig_last_device_status(void *cuda_stream)
         return (host & 1) ? DIG_ERR_TIMEOUT : DIG_ERR_RANGE;          // bit 0: a wait expired; bit 1: gates out of range
     }
     return DIG_OK;
+}
+
+dig_status dig_selftest_wait_timeout(unsigned limit_us, void *cuda_stream)
+{
+    if (limit_us == 0 || limit_us > 100000u) return DIG_ERR_INVALID_ARG;
+    int *status = device_status_ptr();
+    if (!status) return DIG_ERR_CUDA;
+    wait_that_expires<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(status, (unsigned long long)limit_us * 1000ull);
+    return cuda_ok(cudaGetLastError());
 }
 
 dig_status dig_profile_enable(int on)

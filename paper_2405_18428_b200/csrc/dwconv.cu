@@ -352,7 +352,9 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
     KernelTimer t(KID_DWCONV, stream);
     // at least as many tiles as CTAs can be resident: the persistent, double-buffered kernel, two or more tiles per CTA
     const long long ntiles = (long long)grid.x * grid.y * grid.z;
-    const int resident = 148 * 3;       // three CTAs of the persistent kernel fit an SM at its register count
+    const int sms = device_sm_count();
+    if (sms <= 0) return DIG_ERR_CUDA;
+    const int resident = sms * 3;       // three CTAs of the persistent kernel fit an SM at its register count
     if (ntiles >= resident && ntiles < (1ll << 31)) {
         const dim3 pgrid((unsigned)(ntiles >= 2 * resident ? resident : (ntiles + 1) / 2));
         switch (dtype) {
@@ -415,7 +417,8 @@ dig_status launch_dwconv_bwd(const void *x, const void *w, const void *dy, void 
         // no more CTAs than stay resident together (three per SM at this kernel's register count), so that
         // their tile loops end together
         const int CHb = dtype == DIG_F32 ? Cfg<float>::CH : Cfg<__nv_bfloat16>::CH;
-        const int nchb = (D + CHb - 1) / CHb, resident = 148 * 3;
+        const int nchb = (D + CHb - 1) / CHb, resident = device_sm_count() * 3;
+        if (resident <= 0) return DIG_ERR_CUDA;
         const int cap = resident / nchb > 0 ? resident / nchb : 1;
         if (nslab > cap) nslab = cap;
     }

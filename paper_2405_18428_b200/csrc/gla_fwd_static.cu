@@ -1,11 +1,13 @@
 // dig_gla_fwd_static: the forward GLA call for callers that cannot allocate device memory.
 //
-// dig_gla_fwd keeps the per-chunk states and decay factors in a workspace the caller allocates.
+// dig_gla_fwd keeps the segment states and decay factors in a workspace the caller allocates.
 // Some callers have no allocator to ask: code that runs where cudaMalloc is forbidden or would
 // stall (a real-time loop, a plugin whose host owns all device memory, a process working under a
 // fixed memory budget).  For them the same scratch lives in a fixed-size array in device global
-// memory that is part of this library's image.  Every GPU that loads the library holds those
-// kScratchBytes until the process exits, whether or not this entry point is ever called.
+// memory that is part of this library's image.  A GPU holds those kScratchBytes from the moment the
+// runtime loads this translation unit's module on it until the process exits: with lazy module
+// loading that is the first call below on the device (the symbol look-up triggers it), with eager
+// loading it is context creation.
 #include <mutex>
 
 #include "dig_common.cuh"
@@ -47,8 +49,8 @@ extern "C" dig_status dig_gla_fwd_static(const void *q, const void *k, const voi
     void *scratch = nullptr;
     const dig_status st = scratch_for_current_device(&scratch);
     if (st != DIG_OK) return st;
-    // The forward kernels write every chunk state and decay factor before reading it, so nothing
-    // in the array has to be cleared between calls.
+    // The forward kernels write every state and decay factor before reading it, so nothing in the
+    // array has to be cleared between calls.
     return dig_gla_fwd(q, k, v, gate, out, B, H, grid_h, grid_w, d_k, d_v, chunk, direction, dtype,
                        scratch, kScratchBytes, cuda_stream);
 }

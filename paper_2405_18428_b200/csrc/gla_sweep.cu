@@ -22,9 +22,10 @@
 // dO Sc^T = dO Sc_local^T + (dO S_segment^T) diag(exp(c) G): two products and one fused multiply-add.
 //
 // Every product is a tcgen05.mma (kind::f16, fp16 operands, fp32 accumulators in tensor memory)
-// issued by one extra warp; the other warps build operand tiles, mask the scores and post-process
-// accumulators.  Token rows of the next tile are prefetched into registers; with 256 worker
-// threads two CTAs share an SM, so one builds while the other's products are in the tensor pipe.
+// issued by thread 0, which otherwise works like the others: all threads build operand tiles, mask
+// the scores and post-process accumulators, phase by phase.  Token rows of the next tile are
+// prefetched into registers; at d = 64 two CTAs of 256 threads share an SM, so one builds while the
+// other's products are in the tensor pipe.
 #include "sweep.cuh"
 
 namespace dig {
@@ -204,8 +205,20 @@ sweep_local(const SweepArgs a)
             }
             write_gates<D, NT, BWD, BWD>(raw, table, rowOff + cur * T);
             __syncthreads();
-            float tot_unused;
-            const bool need = gate_prefix<D, NT>(table, sTot, tot_unused);
+            // the vectors of an undivided tile are written inside the prefix pass (no barrier of their own)
+            const bool whole_ok = pl.sub_max == T;
+            const Vec v0 = vec_of<D>(vecb, iter & 1);
+            float tot_c = 0.f;
+            const bool need = gate_prefix<D, NT>(table, sTot, tot_c, [&](int c, float t) {
+                if (whole_ok) {
+                    const float cv = 0.5f * t;
+                    v0.off[c] = cv;
+                    v0.ec[c] = ex2(cv);
+                    v0.e2c[c] = ex2(t);
+                    if (BWD) v0.aux[c] = ex2(gcum + cv);
+                }
+            });
+            const bool whole = whole_ok && !need;
             int s = pl.sub_max;
             if (need || s < T) {
                 bool bad;
@@ -217,19 +230,23 @@ sweep_local(const SweepArgs a)
                 const int lo = u * s, hi = min(lo + s, T);
                 const Vec vc = vec_of<D>(vecb, iter & 1);
                 if (tid < D) {
-                    const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
-                    const float t = table[(hi - 1) * C::LAMP + tid] - base, cv = 0.5f * t;
-                    vc.off[tid] = base + cv;
-                    vc.ec[tid] = ex2(cv);
-                    vc.e2c[tid] = ex2(t);
+                    float t = tot_c;
+                    if (!whole) {
+                        const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
+                        t = table[(hi - 1) * C::LAMP + tid] - base;
+                        const float cv = 0.5f * t;
+                        vc.off[tid] = base + cv;
+                        vc.ec[tid] = ex2(cv);
+                        vc.e2c[tid] = ex2(t);
+                        if (BWD) vc.aux[tid] = ex2(gcum + cv);  // decay from the segment start to the sub-chunk's centre
+                    }
                     if (BWD) {
-                        vc.aux[tid] = ex2(gcum + cv);           // decay from the segment start to the sub-chunk's centre
                         const size_t slot = ((size_t)(nsub - 1 - u) * g.B * g.H + bh) * pl.ntile + tile;
                         a.slot_g[slot * D + tid] = gcum;
                     }
                     gcum += t;
                 }
-                __syncthreads();
+                if (!whole) __syncthreads();
                 {
                     build_tiles<D, NT, BWD, BWD>(raw, tQ, tK, tV, tG, table, vc.off, rowOff + cur * T, lo, min(hi, nrow));
                     if (BWD) {
@@ -482,8 +499,19 @@ sweep_fwd(const SweepArgs a)
             write_gates<D, NT, true, false>(raw, table, rowOff + cur * T);
             __syncthreads();
             const int my_off = rowOff[cur * T + r16];
-            float tot_unused;
-            const bool need = gate_prefix<D, NT>(table, sTot, tot_unused);
+            // the vectors of an undivided tile are written inside the prefix pass (no barrier of their own)
+            const bool whole_ok = pl.sub_max == T;
+            const Vec v0 = vec_of<D>(vecb, iter & 1);
+            float tot_c = 0.f;
+            const bool need = gate_prefix<D, NT>(table, sTot, tot_c, [&](int c, float t) {
+                if (whole_ok) {
+                    const float cv = 0.5f * t;
+                    v0.off[c] = cv;
+                    v0.ec[c] = ex2(cv);
+                    v0.e2c[c] = ex2(t);
+                }
+            });
+            const bool whole = whole_ok && !need;
             int s = pl.sub_max;
             if (need || s < T) {
                 bool bad;
@@ -494,14 +522,16 @@ sweep_fwd(const SweepArgs a)
             for (int u = 0; u < nsub; ++u, ++iter) {
                 const int lo = u * s, hi = min(lo + s, T);
                 const Vec vc = vec_of<D>(vecb, iter & 1);
-                if (tid < D) {
-                    const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
-                    const float t = table[(hi - 1) * C::LAMP + tid] - base, cv = 0.5f * t;
-                    vc.off[tid] = base + cv;
-                    vc.ec[tid] = ex2(cv);
-                    vc.e2c[tid] = ex2(t);
+                if (!whole) {
+                    if (tid < D) {
+                        const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
+                        const float t = table[(hi - 1) * C::LAMP + tid] - base, cv = 0.5f * t;
+                        vc.off[tid] = base + cv;
+                        vc.ec[tid] = ex2(cv);
+                        vc.e2c[tid] = ex2(t);
+                    }
+                    __syncthreads();
                 }
-                __syncthreads();
                 {
                     build_tiles<D, NT, true, false>(raw, tQ, tK, tV, nullptr, table, vc.off, rowOff + cur * T, lo, min(hi, nrow));
                     write_state_tile<D, NT>(tS, sm, S, vc.ec);                       // Sc = diag(2^c) S
@@ -666,8 +696,20 @@ sweep_bwd(const SweepArgs a)
             const int my_off = rowOff[cur * T + r16];
             // decay since the segment start of the sub-chunk worked first (always slot 0): fetched ahead of its use
             const float g_first = tid < D ? a.slot_g[((size_t)bh * pl.ntile + tile) * D + tid] : 0.f;
-            float tot_unused;
-            const bool need = gate_prefix<D, NT>(table, sTot, tot_unused);
+            // the vectors of an undivided tile are written inside the prefix pass (no barrier of their own)
+            const bool whole_ok = pl.sub_max == T;
+            const Vec v0 = vec_of<D>(vecb, iter & 1);
+            float tot_c = 0.f;
+            const bool need = gate_prefix<D, NT>(table, sTot, tot_c, [&](int c, float t) {
+                if (whole_ok) {
+                    const float cv = 0.5f * t;
+                    v0.off[c] = cv;
+                    v0.ec[c] = ex2(cv);
+                    v0.e2c[c] = ex2(t);
+                    v0.aux[c] = ex2(cv + g_first);
+                }
+            });
+            const bool whole = whole_ok && !need;
             int s = pl.sub_max;
             if (need || s < T) {
                 bool bad;
@@ -679,15 +721,17 @@ sweep_bwd(const SweepArgs a)
                 const int lo = u * s, hi = min(lo + s, T), hiv = min(hi, nrow);
                 const size_t slot = ((size_t)(nsub - 1 - u) * g.B * g.H + bh) * pl.ntile + tile;
                 const Vec vc = vec_of<D>(vecb, iter & 1);
-                if (tid < D) {
-                    const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
-                    const float t = table[(hi - 1) * C::LAMP + tid] - base, cv = 0.5f * t;
-                    vc.off[tid] = base + cv;
-                    vc.ec[tid] = ex2(cv);
-                    vc.e2c[tid] = ex2(t);
-                    vc.aux[tid] = ex2(cv + (u == nsub - 1 ? g_first : a.slot_g[slot * D + tid]));   // exp(c) * decay since the segment start
+                if (!whole) {
+                    if (tid < D) {
+                        const float base = lo ? table[(lo - 1) * C::LAMP + tid] : 0.f;
+                        const float t = table[(hi - 1) * C::LAMP + tid] - base, cv = 0.5f * t;
+                        vc.off[tid] = base + cv;
+                        vc.ec[tid] = ex2(cv);
+                        vc.e2c[tid] = ex2(t);
+                        vc.aux[tid] = ex2(cv + (u == nsub - 1 ? g_first : a.slot_g[slot * D + tid]));   // exp(c) * decay since the segment start
+                    }
+                    __syncthreads();
                 }
-                __syncthreads();
                 {
                     build_tiles<D, NT, true, true>(raw, tQ, tK, tV, tG, table, vc.off, rowOff + cur * T, lo, hiv);
                     write_state_tile<D, NT>(tD, sm, Dst, vc.ec);                    // Dc = diag(2^c) D

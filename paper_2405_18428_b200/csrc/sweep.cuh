@@ -54,7 +54,7 @@ struct Cfg {
     static_assert(BIGM || (NCH % 2 == 0), "heads of at most 64 channels split their state products in two halves");
 };
 
-// Thread roles of a CTA with NT worker threads (plus one warp that issues MMAs and bulk copies).
+// Work split of a CTA of NT threads (thread 0 also issues the MMAs and the bulk copies).
 template <int D, int NT>
 struct Lay {
     using C = Cfg<D>;
@@ -289,12 +289,14 @@ __device__ __forceinline__ Vec vec_of(float *base, int parity)
     return Vec{p, p + D, p + 2 * D, p + 3 * D};
 }
 
-// Turns the table's rows into inclusive prefix sums down the rows (all NT worker threads; the
-// issuing warp takes part in the barriers only).  Returns, uniformly, whether some channel's total
+// Turns the table's rows into inclusive prefix sums down the rows (all NT threads).  Returns, uniformly, whether some channel's total
 // over the tile exceeds kSubLimit in magnitude.  tot_out (threads < D): the channel's total.
-// Contains two barriers; the caller must have placed one after write_gates.
-template <int D, int NT>
-__device__ __forceinline__ bool gate_prefix(float *table, float *sTot, float &tot_out)
+// Contains two barriers; the caller must have placed one after write_gates.  on_total(c, total) runs
+// in the thread that owns channel c before the last barrier: what it writes to shared memory is
+// visible to everyone afterwards (the kernels put the vectors of an undivided tile there, which saves
+// them a barrier of their own).
+template <int D, int NT, typename F>
+__device__ __forceinline__ bool gate_prefix(float *table, float *sTot, float &tot_out, F on_total)
 {
     using L = Lay<D, NT>;
     constexpr int LAMP = Cfg<D>::LAMP;
@@ -326,6 +328,7 @@ __device__ __forceinline__ bool gate_prefix(float *table, float *sTot, float &to
             if (r0 + j < T) table[(r0 + j) * LAMP + c] = a[j] + add;
         tot_out = tot;
         big = seg == 0 && fabsf(tot) > kSubLimit;
+        if (seg == 0) on_total(c, tot);
     }
     return __syncthreads_or(big) != 0;
 }

@@ -139,10 +139,10 @@ __device__ __forceinline__ uint64_t global_ns()
     return t;
 }
 
-// Waits for the phase with the given parity, for at most 0.25 s.  On expiry records the failure in
-// *status and returns false; the caller then skips its remaining work and leaves through the
-// normal exit path (tensor memory is still released).
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status)
+// Waits for the phase with the given parity, for at most limit_ns (0.25 s unless told otherwise).  On
+// expiry records the failure in *status and returns false; the caller then skips its remaining work
+// and leaves through the normal exit path (tensor memory is still released).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status, uint64_t limit_ns = 250000000ull)
 {
     const uint32_t addr = smem_u32(bar);
     uint64_t t0 = 0;
@@ -157,7 +157,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *s
         if ((it & 7) == 7) {
             const uint64_t now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > 250000000ull) {
+            else if (now - t0 > limit_ns) {
                 atomicOr(status, 1);
                 return false;
             }

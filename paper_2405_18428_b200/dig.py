@@ -28,7 +28,7 @@ EXPORTS = ("dig_set_impl", "dig_gla_query_impl", "dig_gla_workspace_bytes", "dig
            "dig_gla_fwd_multi", "dig_gla_bwd_multi", "dig_gla_multi_workspace_bytes",
            "dig_gla_fwd_beta", "dig_gla_bwd_beta", "dig_gla_beta_workspace_bytes", "dig_gla_fwd_outgate", "dig_srem_dwconv", "dig_srem_dwconv_bwd",
            "dig_srem_dwconv_bwd_workspace_bytes", "dig_gla_outgate_fwd", "dig_gla_outgate_bwd",
-           "dig_gla_outgate_bwd_workspace_bytes", "dig_last_device_status",
+           "dig_gla_outgate_bwd_workspace_bytes", "dig_last_device_status", "dig_selftest_wait_timeout",
            "dig_status_string", "dig_profile_enable", "dig_profile_kernels", "dig_profile_read")
 
 _lib = None
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.dig_gla_outgate_bwd.restype = i
         L.dig_last_device_status.argtypes = [vp]
         L.dig_last_device_status.restype = i
+        L.dig_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp]
+        L.dig_selftest_wait_timeout.restype = i
         L.dig_status_string.argtypes = [i]
         L.dig_status_string.restype = ctypes.c_char_p
         L.dig_profile_enable.argtypes = [i]
@@ -337,6 +339,11 @@ def dig_srem_dwconv_bwd(x, w, dy, grid_h, grid_w, direction=DIG_ROW_FWD, *, with
 
 def dig_last_device_status() -> int:
     return lib().dig_last_device_status(_stream())
+
+
+def dig_selftest_wait_timeout(limit_us: int = 1000) -> None:
+    """Launches the kernel whose only wait expires after limit_us; dig_last_device_status then reports it."""
+    _check(lib().dig_selftest_wait_timeout(int(limit_us), _stream()), "dig_selftest_wait_timeout")
 
 
 def dig_profile_enable(on: bool) -> None:

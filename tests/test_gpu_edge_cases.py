@@ -145,3 +145,14 @@ def test_decay_beyond_the_range_is_reported_not_silent():
     for t in grads:
         assert torch.isfinite(t).all()
     assert "range" in dig.status_string(dig.DIG_ERR_RANGE)
+
+
+def test_a_wait_that_nothing_satisfies_expires_and_is_reported_once():
+    """Every wait inside the kernels is bounded.  A dedicated kernel waits 2 ms on a barrier nobody arrives
+    on: the device status must say so exactly once, and the library must keep working afterwards."""
+    from paper_2405_18428_b200 import dig
+    assert dig.dig_last_device_status() == dig.DIG_OK
+    dig.dig_selftest_wait_timeout(2000)
+    assert dig.dig_last_device_status() == dig.DIG_ERR_TIMEOUT
+    assert dig.dig_last_device_status() == dig.DIG_OK
+    check_workload(_wl(64, 64), 0)
