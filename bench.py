@@ -434,6 +434,56 @@ def sweep_entry(name, wl, torch, dig, peaks, local, flush, reps=20):
     return res
 
 
+def multi_direction_entry(wl, torch, dig, flush, reps=20):
+    """Sums over the four scan orders (Algorithm 3) of one workload: the library's entry points, which add
+    every order's fp32 results into one set of buffers, against four single-order calls plus torch adds."""
+    from paper_2405_18428_b200.inputs import make_inputs
+    x = make_inputs(wl, conv=False)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(torch.bfloat16)
+    q, k, v, g, dO = (dev(x[n]) for n in ("q", "k", "v", "g", "dO"))
+    gate = dig.dig_gate_logsigmoid(g, x["tau"])
+    dirs = (0, 1, 2, 3)
+    dt = dig.DIG_BF16
+    ws1 = torch.empty(dig.dig_gla_workspace_bytes(wl.B, wl.H, wl.grid_h, wl.grid_w, wl.d_k, wl.d_v, wl.chunk, dt, 1), dtype=torch.uint8, device="cuda")
+    wsm = torch.empty(dig.dig_gla_multi_workspace_bytes(wl.B, wl.H, wl.grid_h, wl.grid_w, wl.d_k, wl.d_v, wl.chunk, dt, 1), dtype=torch.uint8, device="cuda")
+    outs = [torch.empty_like(v) for _ in dirs]
+    grads = [(torch.empty_like(q), torch.empty_like(q), torch.empty_like(v), torch.empty(q.shape, dtype=torch.float32, device="cuda")) for _ in dirs]
+    out_m = torch.empty_like(v)
+    grads_m = (torch.empty_like(q), torch.empty_like(q), torch.empty_like(v), torch.empty(q.shape, dtype=torch.float32, device="cuda"))
+
+    def separate():
+        for i, d in enumerate(dirs):
+            dig.dig_gla_fwd(q, k, v, gate, wl.grid_h, wl.grid_w, wl.chunk, d, out=outs[i], workspace=ws1)
+            dig.dig_gla_bwd(q, k, v, gate, dO, wl.grid_h, wl.grid_w, wl.chunk, d, grads=grads[i], workspace=ws1)
+        o = outs[0] + outs[1] + outs[2] + outs[3]
+        gs = [grads[0][j] + grads[1][j] + grads[2][j] + grads[3][j] for j in range(4)]
+        return o, gs
+
+    def fused():
+        dig.dig_gla_fwd_multi(q, k, v, gate, wl.grid_h, wl.grid_w, dirs, wl.chunk, out=out_m, workspace=wsm)
+        dig.dig_gla_bwd_multi(q, k, v, gate, dO, wl.grid_h, wl.grid_w, dirs, wl.chunk, grads=grads_m, workspace=wsm)
+
+    for _ in range(3):
+        separate()
+        fused()
+    torch.cuda.synchronize()
+    th = wl.B * wl.L * wl.H
+    fwd_b, bwd_b = bytes_per_token_head(wl)
+    d = wl.d_k
+    # output bytes per (token, head) with d = d_k = d_v, bf16 results and an fp32 gate gradient:
+    #   separate: 4 orders x 12d stored, then the adds read 4 x 12d and store 12d            -> 108 d
+    #   entry points: fp32 sums of out, dq, dk, dv (16d): stored once, read + stored 3 times, read once
+    #   more and rounded to 8d; the gate gradient (4d) stored once, read + stored 3 times      -> 164 d
+    sep_out, fus_out = th * 108 * d, th * 164 * d
+    return {"workload": wl.name, "directions": list(dirs),
+            "four_calls_plus_adds": median_single(separate, torch, reps, flush),
+            "multi_entry_points": median_single(fused, torch, reps, flush),
+            "output_bytes_model": {"four_calls_plus_adds": sep_out, "multi_entry_points": fus_out,
+                                   "inputs_each": 4 * th * (fwd_b + bwd_b),
+                                   "note": "both read q, k, v, dO and the gates once per order; the entry points form the sums in fp32 "
+                                           "and round once, at the price of fp32 read-add-store traffic on the outputs"}}
+
+
 def cpu_baseline(wl, budget_s=16.0, threads=None):
     """The fp64 oracle, as it stands, on a bounded sample of the workload: whole (batch, head)
     pairs, every scan direction of the workload, gate + fwd + bwd (+ conv on those batches)."""
@@ -604,6 +654,7 @@ def main():
             if base == wl.name and not over:
                 continue
             sweep[name] = sweep_entry(name, CONFIGS[base].scaled(**over), torch, dig, peaks, local, flush)
+        sweep["multi"] = multi_direction_entry(CONFIGS["C2"], torch, dig, flush)
         sweep["note"] = ("one whole step of each workload per timing (its scan directions and conv), captured as a CUDA graph; "
                          "cold = 256 MB written before every timing, warm = back to back; median of 20; roofline from the cold step; "
                          "the tcgen05 kernels work on 64-token tiles for every requested chunk size (tile_executed)")
