@@ -119,11 +119,11 @@ __device__ __forceinline__ void issue_state_product(uint32_t tmem_acc, const cha
     using C = Cfg<D>;
     const uint32_t a = smem_u32(tA), b = smem_u32(tB);
     if constexpr (C::BIGM) {
-        issue<128, C::NACC, true, true>(tmem_acc, a, C::CHT, b, C::CHT, T / 16, false);
+        issue<128, C::NACC, true, true, T / 16, C::CHT, C::CHT>(tmem_acc, a, b, false);
     } else {
         constexpr int HCH = C::NCH / 2;
-        issue<64, D / 2, true, true>(tmem_acc, a, C::CHT, b, C::CHT, T / 16, false);
-        issue<64, D / 2, true, true>(tmem_acc + (16u << 16), a, C::CHT, b + HCH * C::CHT, C::CHT, T / 16, false);
+        issue<64, D / 2, true, true, T / 16, C::CHT, C::CHT>(tmem_acc, a, b, false);
+        issue<64, D / 2, true, true, T / 16, C::CHT, C::CHT>(tmem_acc + (16u << 16), a, b + HCH * C::CHT, false);
     }
 }
 
@@ -172,6 +172,7 @@ sweep_local(const SweepArgs a)
     constexpr uint32_t aU = 0, aW = C::BIGM ? C::NACC : D / 2;
 
     const int tid = threadIdx.x, lane = tid & 31;
+    constexpr int kIssuer = NT - 32;        // lane 0 of the last warp issues the MMAs (warps 0 and 1 carry the per-channel work)
     cta_setup(ctl, 1, SM::tmem_cols, smem, SM::kTilesPad);
     const uint32_t tmem = ctl->tmem_base, lane_base = (uint32_t)(32 * ((tid >> 5) & 3)) << 16;
     const Geom &g = a.g;
@@ -257,7 +258,7 @@ sweep_local(const SweepArgs a)
                 }
                 tc_fence_before_sync();
                 SYNC_OR_DIE();
-                if (tid == 0) {
+                if (tid == kIssuer) {
                     tc_fence_after_sync();
                     issue_state_product<D>(tmem + aU, tK, tV);                   // Kc^T V
                     if (BWD) issue_state_product<D>(tmem + aW, tQ, tG);         // Qc^T dO
@@ -458,6 +459,7 @@ sweep_fwd(const SweepArgs a)
     static_assert(aO + C::NACC <= SM::tmem_cols, "tensor memory");
 
     const int tid = threadIdx.x, lane = tid & 31, q4 = (tid >> 5) & 3, cg = tid >> 7, hf = lane >> 4;
+    constexpr int kIssuer = NT - 32;        // lane 0 of the last warp issues the MMAs (warps 0 and 1 carry the per-channel work)
     const int r16 = 16 * q4 + (lane & 15);
     cta_setup(ctl, 1, SM::tmem_cols, smem, SM::kTiles);
     const uint32_t tmem = ctl->tmem_base, lane_base = (uint32_t)(32 * q4) << 16;
@@ -539,11 +541,11 @@ sweep_fwd(const SweepArgs a)
                 }
                 tc_fence_before_sync();
                 SYNC_OR_DIE();
-                if (tid == 0) {
+                if (tid == kIssuer) {
                     tc_fence_after_sync();
-                    issue<64, 64, false, false>(tmem + aP, smem_u32(tQ), C::CHT, smem_u32(tK), C::CHT, C::KS, false);   // Qc Kc^T
+                    issue<64, 64, false, false, C::KS, C::CHT, C::CHT>(tmem + aP, smem_u32(tQ), smem_u32(tK), false);   // Qc Kc^T
                     mma_commit(&ctl->bar[0]);
-                    issue<64, D, false, true>(tmem + aO, smem_u32(tQ), C::CHT, smem_u32(tS), C::CHS, C::KS, false);     // Qc Sc
+                    issue<64, D, false, true, C::KS, C::CHT, C::CHS>(tmem + aO, smem_u32(tQ), smem_u32(tS), false);     // Qc Sc
                 }
                 {
                     if (u == nsub - 1 && tile + 1 < t1)
@@ -572,9 +574,9 @@ sweep_fwd(const SweepArgs a)
                 }
                 tc_fence_before_sync();
                 SYNC_OR_DIE();
-                if (tid == 0) {
+                if (tid == kIssuer) {
                     tc_fence_after_sync();
-                    issue<64, D, false, true>(tmem + aO, smem_u32(tP), C::CHT, smem_u32(tV), C::CHT, T / 16, true);     // + P V
+                    issue<64, D, false, true, T / 16, C::CHT, C::CHT>(tmem + aO, smem_u32(tP), smem_u32(tV), true);     // + P V
                     issue_state_product<D>(tmem + aU, tK, tV);                                                         // Kc^T V
                     mma_commit(&ctl->bar[0]);
                 }
@@ -639,6 +641,7 @@ sweep_bwd(const SweepArgs a)
     static_assert(aV + C::NACC <= SM::tmem_cols, "tensor memory");
 
     const int tid = threadIdx.x, lane = tid & 31, q4 = (tid >> 5) & 3, cg = tid >> 7, hf = lane >> 4;
+    constexpr int kIssuer = NT - 32;        // lane 0 of the last warp issues the MMAs (warps 0 and 1 carry the per-channel work)
     const int r16 = 16 * q4 + (lane & 15);
     cta_setup(ctl, 2, SM::tmem_cols, smem, SM::kTiles);
     const uint32_t tmem = ctl->tmem_base, lane_base = (uint32_t)(32 * q4) << 16;
@@ -676,7 +679,7 @@ sweep_bwd(const SweepArgs a)
             __syncthreads();
             load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
         }
-        if (tid == 0) {
+        if (tid == kIssuer) {
             // the zero-start state of the sub-chunk worked first (always slot 0 of its tile) and, once per
             // segment, the state entering the segment; later sub-chunks' states are fetched as soon as the
             // products of the one before are done
@@ -739,18 +742,18 @@ sweep_bwd(const SweepArgs a)
                 }
                 tc_fence_before_sync();
                 SYNC_OR_DIE();
-                if (tid == 0) {
+                if (tid == kIssuer) {
                     ok = mbar_wait(barS, par, a.status);          // both state tiles have landed
                     tc_fence_after_sync();
                     const uint32_t sQ = smem_u32(tQ), sK = smem_u32(tK), sV = smem_u32(tV), sG = smem_u32(tG);
                     const uint32_t sS = smem_u32(tS), sI = smem_u32(tI), sD = smem_u32(tD);
-                    issue<64, 64, false, false>(tmem + aP, sQ, C::CHT, sK, C::CHT, C::KS, false);             // Qc Kc^T
-                    issue<64, 64, false, false>(tmem + aP + kHi, sG, C::CHT, sV, C::CHT, C::KS, false);       // dO V^T
+                    issue<64, 64, false, false, C::KS, C::CHT, C::CHT>(tmem + aP, sQ, sK, false);             // Qc Kc^T
+                    issue<64, 64, false, false, C::KS, C::CHT, C::CHT>(tmem + aP + kHi, sG, sV, false);       // dO V^T
                     mma_commit(barG1);
-                    issue<64, D, false, false>(tmem + aQK, sG, C::CHT, sS, C::CHS, C::KS, false);             // dO Sc_local^T
-                    issue<64, D, false, false>(tmem + aV, sG, C::CHT, sI, C::CHS, C::KS, false);              // dO S_segment^T
-                    issue<64, D, false, false>(tmem + aQK + kHi, sV, C::CHT, sD, C::CHS, C::KS, false);       // V Dc^T
-                    issue<64, D, false, true>(tmem + aV + kHi, sK, C::CHT, sD, C::CHS, C::KS, false);         // Kc Dc
+                    issue<64, D, false, false, C::KS, C::CHT, C::CHS>(tmem + aQK, sG, sS, false);             // dO Sc_local^T
+                    issue<64, D, false, false, C::KS, C::CHT, C::CHS>(tmem + aV, sG, sI, false);              // dO S_segment^T
+                    issue<64, D, false, false, C::KS, C::CHT, C::CHS>(tmem + aQK + kHi, sV, sD, false);       // V Dc^T
+                    issue<64, D, false, true, C::KS, C::CHT, C::CHS>(tmem + aV + kHi, sK, sD, false);         // Kc Dc
                 }
                 {
                     // the raw rows are spent: the next tile's gates (needed first) start now, its q, k, v, dO rows
@@ -781,13 +784,13 @@ sweep_bwd(const SweepArgs a)
                 }
                 tc_fence_before_sync();
                 SYNC_OR_DIE();
-                if (tid == 0) {
+                if (tid == kIssuer) {
                     tc_fence_after_sync();
                     const uint32_t sQ = smem_u32(tQ), sK = smem_u32(tK), sG = smem_u32(tG);
                     const uint32_t sP = smem_u32(tP), sdP = smem_u32(tdP);
-                    issue<64, D, false, true>(tmem + aQK, sdP, C::CHT, sK, C::CHT, T / 16, true);             // + dP Kc
-                    issue<64, D, true, true>(tmem + aQK + kHi, sdP, C::CHT, sQ, C::CHT, T / 16, true);        // + dP^T Qc
-                    issue<64, D, true, true>(tmem + aV + kHi, sP, C::CHT, sG, C::CHT, T / 16, true);          // + P^T dO
+                    issue<64, D, false, true, T / 16, C::CHT, C::CHT>(tmem + aQK, sdP, sK, true);             // + dP Kc
+                    issue<64, D, true, true, T / 16, C::CHT, C::CHT>(tmem + aQK + kHi, sdP, sQ, true);        // + dP^T Qc
+                    issue<64, D, true, true, T / 16, C::CHT, C::CHT>(tmem + aV + kHi, sP, sG, true);          // + P^T dO
                     issue_state_product<D>(tmem + aP, tQ, tG);                                                // Qc^T dO
                     mma_commit(barG1);
                 }
@@ -795,7 +798,7 @@ sweep_bwd(const SweepArgs a)
                     ok = wait_all(barG1, 1, a.status);
                     if (ok) {
                         tc_fence_after_sync();
-                        if (tid == 0 && (u > 0 || tile > t0)) {
+                        if (tid == kIssuer && (u > 0 || tile > t0)) {
                             // every product has completed: fetch the next sub-chunk's zero-start state
                             const size_t nslot = u > 0 ? slot + (size_t)g.B * g.H * pl.ntile : (size_t)bh * pl.ntile + (tile - 1);
                             const char *src = reinterpret_cast<const char *>(a.slot_s + nslot * (D * D));
@@ -888,7 +891,7 @@ sweep_bwd(const SweepArgs a)
         }
     }
 die:
-    if (!ok && tid == 0) mbar_wait(barS, par, a.status);      // let bulk copies in flight land
+    if (!ok && tid == kIssuer) mbar_wait(barS, par, a.status);      // let bulk copies in flight land
     cta_teardown(ctl, SM::tmem_cols);
 }
 

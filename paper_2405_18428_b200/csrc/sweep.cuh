@@ -158,21 +158,22 @@ __device__ __forceinline__ void store_out8(bf16 *p, const float (&f)[8], bool = 
 __device__ __forceinline__ uint64_t kdesc(uint32_t saddr, uint32_t ch) { return make_desc(saddr, ch, 128, 0); }
 __device__ __forceinline__ uint64_t mdesc(uint32_t saddr, uint32_t ch) { return make_desc(saddr, 128, ch, 0); }
 
-// D[tmem] (+)= A * B over `ksteps` steps of 16 along the contraction.  a / b: shared-memory address
+// D[tmem] (+)= A * B over KSTEPS steps of 16 along the contraction.  a / b: shared-memory address
 // of the first element the product uses (a row or chunk offset selects a slice), ach / bch: chunk
-// strides of the tiles.
-template <int M, int N, bool A_MN, bool B_MN>
-__device__ __forceinline__ void issue(uint32_t d_tmem, uint32_t a, uint32_t ach, uint32_t b, uint32_t bch, int ksteps,
-                                      bool accumulate)
+// strides of the tiles (compile-time, so every descriptor is the first one plus a constant in its
+// low word: shared-memory addresses stay below 2^18, the address field cannot carry into the next).
+template <int M, int N, bool A_MN, bool B_MN, int KSTEPS, uint32_t ACH, uint32_t BCH>
+__device__ __forceinline__ void issue(uint32_t d_tmem, uint32_t a, uint32_t b, bool accumulate)
 {
     static_assert((M == 64 && N % 8 == 0) || (M == 128 && N % 16 == 0), "instruction shape");
     constexpr uint32_t idesc = idesc_f16(M, N, A_MN, B_MN);
-    uint64_t da = A_MN ? mdesc(a, ach) : kdesc(a, ach), db = B_MN ? mdesc(b, bch) : kdesc(b, bch);
-    const uint64_t sa = A_MN ? 16u : (2u * ach) >> 4, sb = B_MN ? 16u : (2u * bch) >> 4;
-    for (int kk = 0; kk < ksteps; ++kk) {
-        mma_f16(d_tmem, da, db, idesc, accumulate || kk > 0);
-        da += sa;
-        db += sb;
+    const uint64_t da = A_MN ? mdesc(a, ACH) : kdesc(a, ACH), db = B_MN ? mdesc(b, BCH) : kdesc(b, BCH);
+    constexpr uint32_t sa = A_MN ? 16u : (2u * ACH) >> 4, sb = B_MN ? 16u : (2u * BCH) >> 4;
+    const uint32_t alo = (uint32_t)da, ahi = (uint32_t)(da >> 32), blo = (uint32_t)db, bhi = (uint32_t)(db >> 32);
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+        const uint64_t xa = ((uint64_t)ahi << 32) | (alo + kk * sa), xb = ((uint64_t)bhi << 32) | (blo + kk * sb);
+        mma_f16(d_tmem, xa, xb, idesc, accumulate || kk > 0);
     }
 }
 
