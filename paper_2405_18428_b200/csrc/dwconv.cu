@@ -3,6 +3,8 @@
 // coalesced loads; each thread then owns 8 channels of one tile column and walks down the rows.
 // The scan order the residual stream is in (`dir`) only permutes the filter taps:
 // reverse orders see the filter rotated by 180 degrees, column orders see it transposed.
+#include <type_traits>
+
 #include "dig_common.cuh"
 
 namespace dig {
@@ -120,58 +122,73 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
     }
 }
 
-// The same convolution for grids with several tiles per resident CTA: a persistent CTA walks over tiles
-// (x fastest, then y, batch, channel block) and fills the halo tile of its next tile with cp.async into a
-// second buffer while it computes the current one, so the load latency is paid once per CTA, not once
-// per tile.  Out-of-grid pixels and channels are zero-filled by the copy itself (source size 0).
+// The same convolution for grids that fill the machine: a CTA walks down a strip of TX pixel columns and
+// CH channels, row by row.  Input rows (TX + 2 pixels with the halo) arrive through cp.async in a ring of
+// kRing rows, kRing - 1 rows ahead of the arithmetic, so every input row is fetched once per strip, widened
+// once per thread and feeds the three output rows around it from registers (acc[r % 3] belongs to output
+// row r).  Out-of-grid pixels and channels are zero-filled by the copy itself (source size 0).  One barrier
+// per row: the slot refilled after the barrier of row r is the one row r - 1 was read from.
+// Strip s = ((channel block * B + batch) * strips_x + strip column) * nseg + row segment; a row segment
+// covers seg_rows output rows (plus one halo row on either side).
+constexpr int kRing = 6;
+
 template <typename T, typename TO>
 __global__ void __launch_bounds__(Cfg<T>::kThreads, 3)
-srem_dwconv3x3_stream(const T *__restrict__ x, const T *__restrict__ w, const T *__restrict__ bias,
-                      TO *__restrict__ y, int B, int gh, int gw, int D, int dir, int tiles_x, int tiles_y, int ntiles)
+srem_dwconv3x3_strip(const T *__restrict__ x, const T *__restrict__ w, const T *__restrict__ bias,
+                     TO *__restrict__ y, int B, int gh, int gw, int D, int dir, int strips_x, int nseg, int seg_rows,
+                     int nstrips)
 {
     constexpr int CH = Cfg<T>::CH, kLanes = Cfg<T>::kLanes, kConvThreads = Cfg<T>::kThreads;
     constexpr int kPieces = (int)sizeof(Vec8<T>) / 16;
-    __shared__ Vec8<T> tile[2][TY + 2][TX + 2][kLanes];
+    constexpr int kRowVecs = (TX + 2) * kLanes;                  // 16/32-byte vectors of one input row of the strip
+    constexpr int kFill = (kRowVecs + kConvThreads - 1) / kConvThreads;
+    __shared__ Vec8<T> ring[kRing][TX + 2][kLanes];
     const int lane = threadIdx.x % kLanes, col = threadIdx.x / kLanes;
     pdl_wait();
     pdl_launch_dependents();
-    auto decode = [&](int t, int &b, int &chb, int &y0, int &x0) {
-        const int per_img = tiles_x * tiles_y, z = t / per_img, r = t - z * per_img;
-        chb = z / B;
-        b = z - chb * B;
-        y0 = (r / tiles_x) * TY;
-        x0 = (r % tiles_x) * TX;
-    };
-    auto fill = [&](int t, int buf) {
-        int b, chb, y0, x0;
-        decode(t, b, chb, y0, x0);
-        const T *xb = x + (size_t)b * gh * gw * D;
-        for (int idx = threadIdx.x; idx < (TY + 2) * (TX + 2) * kLanes; idx += kConvThreads) {
-            const int l = idx % kLanes, pix = idx / kLanes;
-            const int tx = pix % (TX + 2), ty = pix / (TX + 2);
-            const int gy = y0 + ty - 1, gx = x0 + tx - 1, c = chb * CH + l * VEC;
-            const bool in = gy >= 0 && gy < gh && gx >= 0 && gx < gw && c < D;
-            const char *src = reinterpret_cast<const char *>(in ? xb + ((size_t)gy * gw + gx) * D + c : x);
-            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&tile[buf][ty][tx][l]);
-#pragma unroll
-            for (int p = 0; p < kPieces; ++p)
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 16 * p), "l"(src + (in ? 16 * p : 0)),
-                             "r"(in ? 16 : 0) : "memory");
-        }
-    };
-    int t = blockIdx.x, cur_chb = -1;
-    if (t < ntiles) fill(t, 0);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    // with the loads off the critical path the kernel is bound by instruction issue: the taps are kept as
-    // fp32 in registers and every input row is read and widened once for the three output rows it feeds
+    int cur_chb = -1;
     float wf[3][3][8], bs[8];
-    for (int buf = 0; t < ntiles; t += gridDim.x, buf ^= 1) {
-        if (t + (int)gridDim.x < ntiles) fill(t + gridDim.x, buf ^ 1);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        int b, chb, y0, x0;
-        decode(t, b, chb, y0, x0);
+    for (int s = blockIdx.x; s < nstrips; s += gridDim.x) {
+        const int sg = s % nseg, s1 = s / nseg, sx = s1 % strips_x, s2 = s1 / strips_x, b = s2 % B, chb = s2 / B;
+        const int x0 = sx * TX, ys = sg * seg_rows, ye = min(ys + seg_rows, gh), nr = ye - ys + 2;
         const int ch = chb * CH + lane * VEC;
-        const bool ch_ok = ch < D;
+        const bool ch_ok = ch < D, out_ok = ch_ok && x0 + col < gw;
+        const T *xb = x + (size_t)b * gh * gw * D;
+        // this thread's vectors of an input row: pixel column, validity and offsets stay the same for every row
+        int f_off[kFill];
+        uint32_t f_dst[kFill];
+        bool f_ok[kFill];
+#pragma unroll
+        for (int i = 0; i < kFill; ++i) {
+            const int idx = (int)threadIdx.x + i * kConvThreads, l = idx % kLanes, tx = idx / kLanes;
+            const int gx = x0 + tx - 1, c = chb * CH + l * VEC;
+            f_ok[i] = idx < kRowVecs && gx >= 0 && gx < gw && c < D;
+            f_off[i] = f_ok[i] ? gx * D + c : 0;
+            f_dst[i] = idx < kRowVecs ? (uint32_t)__cvta_generic_to_shared(&ring[0][tx][l]) : 0u;
+        }
+        auto fill = [&](int rr) {       // input row rr of the strip (image row ys - 1 + rr) into its ring slot
+            const int gy = ys - 1 + rr;
+            const bool row_ok = gy >= 0 && gy < gh;
+            const T *row = xb + (size_t)(row_ok ? gy : 0) * gw * D;
+            const uint32_t slot = (uint32_t)(rr % kRing) * (uint32_t)sizeof(ring[0]);
+#pragma unroll
+            for (int i = 0; i < kFill; ++i) {
+                if (i + 1 < kFill || (int)threadIdx.x + i * kConvThreads < kRowVecs) {
+                    const bool in = row_ok && f_ok[i];
+                    const char *src = reinterpret_cast<const char *>(in ? row + f_off[i] : x);
+#pragma unroll
+                    for (int p = 0; p < kPieces; ++p)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(f_dst[i] + slot + 16 * p),
+                                     "l"(src + (in ? 16 * p : 0)), "r"(in ? 16 : 0) : "memory");
+                }
+            }
+        };
+        __syncthreads();                // the previous strip's last rows have been read
+#pragma unroll
+        for (int i = 0; i < kRing - 1; ++i) {
+            if (i < nr) fill(i);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
         if (chb != cur_chb) {            // uniform over the CTA: the taps of this channel block, re-oriented
             cur_chb = chb;
 #pragma unroll
@@ -187,36 +204,47 @@ srem_dwconv3x3_stream(const T *__restrict__ x, const T *__restrict__ w, const T 
             for (int i = 0; i < 8; ++i) bs[i] = 0.f;
             if (bias != nullptr && ch_ok) Vec8<T>::load(bias + ch).unpack(bs);
         }
-        asm volatile("cp.async.wait_group 1;" ::: "memory");      // everything but the newest group: this tile has landed
-        __syncthreads();
-        if (ch_ok && x0 + col < gw) {
-            // acc[r % 3] belongs to output row r; tile row rr (0 = the halo row above) feeds output rows rr - u,
-            // u = 0..2, and completes output row rr - 2
-            float acc[3][8];
+        float acc[3][8];
 #pragma unroll
-            for (int rr = 0; rr < TY + 2; ++rr) {
-                if (rr < TY) {
+        for (int r = 0; r < 3; ++r)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[rr % 3][i] = bs[i];
-                }
-                float xv[3][8];
+            for (int i = 0; i < 8; ++i) acc[r][i] = 0.f;
+        TO *yrow = y + (((size_t)b * gh + ys) * gw + x0 + col) * D + ch;     // output row completed next
+        // One input row: PH = rr % 3 is a compile-time constant so that the accumulators stay in registers.
+        // Row rr starts output row rr (of the segment), feeds rr - 1 and completes rr - 2.  The rows before the
+        // first and after the last output row accumulate into registers that are re-initialised or dropped.
+        auto step = [&](int rr, auto ph_tag) {
+            constexpr int PH = decltype(ph_tag)::value;
+            asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 2) : "memory");      // row rr has landed
+            __syncthreads();
+            if (rr + kRing - 1 < nr) fill(rr + kRing - 1);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            float xv[3][8];
+            const int slot = rr % kRing;
 #pragma unroll
-                for (int v = 0; v < 3; ++v) tile[buf][rr][col + v][lane].unpack(xv[v]);
+            for (int v = 0; v < 3; ++v) ring[slot][col + v][lane].unpack(xv[v]);
 #pragma unroll
-                for (int u = 0; u < 3; ++u) {
-                    const int ty = rr - u;
-                    if (ty >= 0 && ty < TY) {
+            for (int i = 0; i < 8; ++i) acc[PH][i] = bs[i];
 #pragma unroll
-                        for (int v = 0; v < 3; ++v)
+            for (int u = 0; u < 3; ++u) {
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) acc[ty % 3][i] = fmaf(wf[u][v][i], xv[v][i], acc[ty % 3][i]);
+                for (int v = 0; v < 3; ++v)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        float &a = acc[(PH + 3 - u) % 3][i];
+                        a = fmaf(wf[u][v][i], xv[v][i], a);
                     }
-                }
-                const int done = rr - 2;
-                if (done >= 0 && y0 + done < gh) store8(y + (((size_t)b * gh + y0 + done) * gw + x0 + col) * D + ch, acc[done % 3]);
             }
+            if (rr >= 2) {
+                if (out_ok) store8(yrow, acc[(PH + 1) % 3]);
+                yrow += (size_t)gw * D;
+            }
+        };
+        for (int rr = 0; rr < nr; rr += 3) {
+            step(rr, std::integral_constant<int, 0>{});
+            if (rr + 1 < nr) step(rr + 1, std::integral_constant<int, 1>{});
+            if (rr + 2 < nr) step(rr + 2, std::integral_constant<int, 2>{});
         }
-        __syncthreads();                 // this buffer is refilled during the next iteration
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
@@ -350,27 +378,37 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
     const dim3 grid((gw + TX - 1) / TX, (gh + TY - 1) / TY, B * nchb);
     if (grid.y > 65535 || (size_t)B * nchb > 65535) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_DWCONV, stream);
-    // at least as many tiles as CTAs can be resident: the persistent, double-buffered kernel, two or more tiles per CTA
+    // grids with at least one tile per resident CTA: strips of TX columns walked row by row, cut into row
+    // segments so that about three CTAs per SM (what the kernel's register count lets share an SM) have work
     const long long ntiles = (long long)grid.x * grid.y * grid.z;
     const int sms = device_sm_count();
     if (sms <= 0) return DIG_ERR_CUDA;
-    const int resident = sms * 3;       // three CTAs of the persistent kernel fit an SM at its register count
+    const int resident = sms * 3;
     if (ntiles >= resident && ntiles < (1ll << 31)) {
-        const dim3 pgrid((unsigned)(ntiles >= 2 * resident ? resident : (ntiles + 1) / 2));
+        const long long cols = (long long)grid.x * B * nchb;        // strips before the cut into row segments
+        int nseg = (int)(resident / cols);                          // one wave of CTAs where the strips allow it
+        if (nseg < 1) nseg = 1;
+        if (nseg > (gh + 7) / 8) nseg = (gh + 7) / 8;               // segments of at least 8 rows (two halo rows each)
+        const int seg_rows = (gh + nseg - 1) / nseg;
+        nseg = (gh + seg_rows - 1) / seg_rows;
+        const long long nstrips = cols * nseg;
+        if (nstrips >= (1ll << 31)) return DIG_ERR_UNSUPPORTED;
+        const dim3 pgrid((unsigned)(nstrips < resident ? nstrips : resident));
         switch (dtype) {
             case DIG_F32:
-                launch_pdl(srem_dwconv3x3_stream<float, float>, pgrid, dim3(Cfg<float>::kThreads), 0, stream, (const float *)x,
-                           (const float *)w, (const float *)bias, (float *)y, B, gh, gw, D, dir, (int)grid.x, (int)grid.y, (int)ntiles);
+                launch_pdl(srem_dwconv3x3_strip<float, float>, pgrid, dim3(Cfg<float>::kThreads), 0, stream, (const float *)x,
+                           (const float *)w, (const float *)bias, (float *)y, B, gh, gw, D, dir, (int)grid.x, nseg, seg_rows,
+                           (int)nstrips);
                 break;
             case DIG_BF16:
-                launch_pdl(srem_dwconv3x3_stream<__nv_bfloat16, __nv_bfloat16>, pgrid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
+                launch_pdl(srem_dwconv3x3_strip<__nv_bfloat16, __nv_bfloat16>, pgrid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
                            (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias, (__nv_bfloat16 *)y, B, gh,
-                           gw, D, dir, (int)grid.x, (int)grid.y, (int)ntiles);
+                           gw, D, dir, (int)grid.x, nseg, seg_rows, (int)nstrips);
                 break;
             case DIG_BF16_F32OUT:
-                launch_pdl(srem_dwconv3x3_stream<__nv_bfloat16, float>, pgrid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
+                launch_pdl(srem_dwconv3x3_strip<__nv_bfloat16, float>, pgrid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
                            (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, (const __nv_bfloat16 *)bias, (float *)y, B, gh, gw, D,
-                           dir, (int)grid.x, (int)grid.y, (int)ntiles);
+                           dir, (int)grid.x, nseg, seg_rows, (int)nstrips);
                 break;
             default: return DIG_ERR_INVALID_ARG;
         }
