@@ -1,6 +1,9 @@
 // extern "C" entry points: argument validation, kernel-family choice, launches.
 #include <atomic>
 #include <cstring>
+#include <map>
+#include <mutex>
+#include <utility>
 #include <vector>
 
 #include "dig_common.cuh"
@@ -144,6 +147,20 @@ int device_sm_count()
         cached[dev].store(n);
     }
     return n;
+}
+
+dig_status ensure_dynamic_smem(const void *kernel, size_t bytes)
+{
+    static std::mutex mu;
+    static std::map<std::pair<const void *, int>, size_t> granted;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DIG_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    size_t &have = granted[std::make_pair(kernel, dev)];
+    if (bytes <= have) return DIG_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return DIG_ERR_CUDA;
+    have = bytes;
+    return DIG_OK;
 }
 
 }  // namespace dig

@@ -132,14 +132,17 @@ size_t mma_beta_workspace_bytes(const Geom &g, bool backward);
 dig_status launch_state_scan_fwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tf32 = false);
 dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t s, const StateIO &sio, bool tf32 = false);
 // Scans with the value-channel gate (row-major states, tf32-rounded results) and the cross-chunk part of its gradient.
-dig_status launch_state_scan_fwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s);
-dig_status launch_state_scan_bwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s);
+dig_status launch_state_scan_fwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s, bool tf32);
+dig_status launch_state_scan_bwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s, bool tf32);
 dig_status launch_beta_carry(float *dbgate, float *xtot, const Geom &g, cudaStream_t s);
 
 // Device status word (bounded waits report here).
 int *device_status_ptr();
 // Streaming multiprocessors of the current device (cached per device), 0 on error.
 int device_sm_count();
+// Raises a kernel's dynamic shared memory limit to at least `bytes`; the driver is asked only when the
+// value grows (remembered per kernel and device).
+dig_status ensure_dynamic_smem(const void *kernel, size_t bytes);
 
 // Optional per-kernel timing (dig_profile_*): when enabled, every launch site brackets its
 // kernel with two CUDA events on the launching stream.

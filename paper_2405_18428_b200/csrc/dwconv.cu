@@ -124,16 +124,17 @@ srem_dwconv3x3(const T *__restrict__ x, const T *__restrict__ w, const T *__rest
 
 // The same convolution for grids that fill the machine: a CTA walks down a strip of TX pixel columns and
 // CH channels, row by row.  Input rows (TX + 2 pixels with the halo) arrive through cp.async in a ring of
-// kRing rows, kRing - 1 rows ahead of the arithmetic, so every input row is fetched once per strip, widened
-// once per thread and feeds the three output rows around it from registers (acc[r % 3] belongs to output
-// row r).  Out-of-grid pixels and channels are zero-filled by the copy itself (source size 0).  One barrier
+// kRing rows, kRing - 1 rows ahead of the arithmetic, so every input row is fetched once per strip.  A thread
+// owns 4 channels of two neighbouring pixel columns: it widens the four pixels around them once per row and
+// feeds the three output rows around that row from registers (acc[r % 3] belongs to output row r); at this
+// register count four CTAs share an SM.  Out-of-grid pixels and channels are zero-filled by the copy itself (source size 0).  One barrier
 // per row: the slot refilled after the barrier of row r is the one row r - 1 was read from.
 // Strip s = ((channel block * B + batch) * strips_x + strip column) * nseg + row segment; a row segment
 // covers seg_rows output rows (plus one halo row on either side).
 constexpr int kRing = 6;
 
 template <typename T, typename TO>
-__global__ void __launch_bounds__(Cfg<T>::kThreads, 3)
+__global__ void __launch_bounds__(Cfg<T>::kThreads, 4)
 srem_dwconv3x3_strip(const T *__restrict__ x, const T *__restrict__ w, const T *__restrict__ bias,
                      TO *__restrict__ y, int B, int gh, int gw, int D, int dir, int strips_x, int nseg, int seg_rows,
                      int nstrips)
@@ -142,17 +143,19 @@ srem_dwconv3x3_strip(const T *__restrict__ x, const T *__restrict__ w, const T *
     constexpr int kPieces = (int)sizeof(Vec8<T>) / 16;
     constexpr int kRowVecs = (TX + 2) * kLanes;                  // 16/32-byte vectors of one input row of the strip
     constexpr int kFill = (kRowVecs + kConvThreads - 1) / kConvThreads;
+    constexpr int kQuads = CH / 4;                                // 4-channel groups of a pixel
+    static_assert(kQuads * (TX / 2) == kConvThreads, "one thread per (column pair, channel quad)");
     __shared__ Vec8<T> ring[kRing][TX + 2][kLanes];
-    const int lane = threadIdx.x % kLanes, col = threadIdx.x / kLanes;
+    const int quad = threadIdx.x % kQuads, c0 = 2 * (threadIdx.x / kQuads);     // first of the thread's two columns
     pdl_wait();
     pdl_launch_dependents();
     int cur_chb = -1;
-    float wf[3][3][8], bs[8];
+    float wf[3][3][4], bs[4];
     for (int s = blockIdx.x; s < nstrips; s += gridDim.x) {
         const int sg = s % nseg, s1 = s / nseg, sx = s1 % strips_x, s2 = s1 / strips_x, b = s2 % B, chb = s2 / B;
         const int x0 = sx * TX, ys = sg * seg_rows, ye = min(ys + seg_rows, gh), nr = ye - ys + 2;
-        const int ch = chb * CH + lane * VEC;
-        const bool ch_ok = ch < D, out_ok = ch_ok && x0 + col < gw;
+        const int ch = chb * CH + quad * 4;
+        const bool ch_ok = ch < D, ok0 = ch_ok && x0 + c0 < gw, ok1 = ch_ok && x0 + c0 + 1 < gw;
         const T *xb = x + (size_t)b * gh * gw * D;
         // this thread's vectors of an input row: pixel column, validity and offsets stay the same for every row
         int f_off[kFill];
@@ -198,18 +201,18 @@ srem_dwconv3x3_strip(const T *__restrict__ x, const T *__restrict__ w, const T *
                     int su = u, sv = v;
                     if (dir & 2) { su = v; sv = u; }
                     if (dir & 1) { su = 2 - su; sv = 2 - sv; }
-                    (ch_ok ? Vec8<T>::load(w + (size_t)(su * 3 + sv) * D + ch) : Vec8<T>::zero()).unpack(wf[u][v]);
+                    const float4 t = ch_ok ? load4(w + (size_t)(su * 3 + sv) * D + ch) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    wf[u][v][0] = t.x; wf[u][v][1] = t.y; wf[u][v][2] = t.z; wf[u][v][3] = t.w;
                 }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) bs[i] = 0.f;
-            if (bias != nullptr && ch_ok) Vec8<T>::load(bias + ch).unpack(bs);
+            const float4 t = (bias != nullptr && ch_ok) ? load4(bias + ch) : make_float4(0.f, 0.f, 0.f, 0.f);
+            bs[0] = t.x; bs[1] = t.y; bs[2] = t.z; bs[3] = t.w;
         }
-        float acc[3][8];
+        float acc[3][2][4];
 #pragma unroll
         for (int r = 0; r < 3; ++r)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[r][i] = 0.f;
-        TO *yrow = y + (((size_t)b * gh + ys) * gw + x0 + col) * D + ch;     // output row completed next
+            for (int i = 0; i < 4; ++i) acc[r][0][i] = acc[r][1][i] = 0.f;
+        TO *yrow = y + (((size_t)b * gh + ys) * gw + x0 + c0) * D + ch;      // output row completed next
         // One input row: PH = rr % 3 is a compile-time constant so that the accumulators stay in registers.
         // Row rr starts output row rr (of the segment), feeds rr - 1 and completes rr - 2.  The rows before the
         // first and after the last output row accumulate into registers that are re-initialised or dropped.
@@ -219,24 +222,32 @@ srem_dwconv3x3_strip(const T *__restrict__ x, const T *__restrict__ w, const T *
             __syncthreads();
             if (rr + kRing - 1 < nr) fill(rr + kRing - 1);
             asm volatile("cp.async.commit_group;" ::: "memory");
-            float xv[3][8];
-            const int slot = rr % kRing;
+            float xv[4][4];
+            const T *rowp = reinterpret_cast<const T *>(&ring[rr % kRing][0][0]) + quad * 4;     // [TX + 2][CH] elements
 #pragma unroll
-            for (int v = 0; v < 3; ++v) ring[slot][col + v][lane].unpack(xv[v]);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[PH][i] = bs[i];
-#pragma unroll
-            for (int u = 0; u < 3; ++u) {
-#pragma unroll
-                for (int v = 0; v < 3; ++v)
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float &a = acc[(PH + 3 - u) % 3][i];
-                        a = fmaf(wf[u][v][i], xv[v][i], a);
-                    }
+            for (int v = 0; v < 4; ++v) {
+                const float4 t = load4(rowp + (c0 + v) * CH);
+                xv[v][0] = t.x; xv[v][1] = t.y; xv[v][2] = t.z; xv[v][3] = t.w;
             }
+#pragma unroll
+            for (int p = 0; p < 2; ++p)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[PH][p][i] = bs[i];
+#pragma unroll
+            for (int u = 0; u < 3; ++u)
+#pragma unroll
+                for (int p = 0; p < 2; ++p)
+#pragma unroll
+                    for (int v = 0; v < 3; ++v)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            float &a = acc[(PH + 3 - u) % 3][p][i];
+                            a = fmaf(wf[u][v][i], xv[p + v][i], a);
+                        }
             if (rr >= 2) {
-                if (out_ok) store8(yrow, acc[(PH + 1) % 3]);
+                const float (&r0)[4] = acc[(PH + 1) % 3][0], (&r1)[4] = acc[(PH + 1) % 3][1];
+                if (ok0) store4(yrow, make_float4(r0[0], r0[1], r0[2], r0[3]));
+                if (ok1) store4(yrow + D, make_float4(r1[0], r1[1], r1[2], r1[3]));
                 yrow += (size_t)gw * D;
             }
         };
@@ -379,11 +390,11 @@ dig_status launch_dwconv(const void *x, const void *w, const void *bias, void *y
     if (grid.y > 65535 || (size_t)B * nchb > 65535) return DIG_ERR_UNSUPPORTED;
     KernelTimer t(KID_DWCONV, stream);
     // grids with at least one tile per resident CTA: strips of TX columns walked row by row, cut into row
-    // segments so that about three CTAs per SM (what the kernel's register count lets share an SM) have work
+    // segments so that about four CTAs per SM (what the kernel's register count lets share an SM) have work
     const long long ntiles = (long long)grid.x * grid.y * grid.z;
     const int sms = device_sm_count();
     if (sms <= 0) return DIG_ERR_CUDA;
-    const int resident = sms * 3;
+    const int resident = sms * 4;
     if (ntiles >= resident && ntiles < (1ll << 31)) {
         const long long cols = (long long)grid.x * B * nchb;        // strips before the cut into row segments
         int nseg = (int)(resident / cols);                          // one wave of CTAs where the strips allow it

@@ -448,7 +448,7 @@ template <typename K>
 dig_status set_smem(K kernel, size_t bytes)
 {
     if (bytes > kMaxSmem) return DIG_ERR_UNSUPPORTED;
-    return cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    return ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), bytes);
 }
 
 template <typename T, typename TO>

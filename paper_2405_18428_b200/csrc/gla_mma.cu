@@ -7,18 +7,24 @@
 // through mma.sync.m16n8k8 (tf32 operands, fp32 accumulation) with fragments read straight from
 // padded fp32 tiles in shared memory, so any multiple of 8 works as a contraction length and any
 // multiple of 16 (after zero padding) as an output extent.  Operands are rounded to tf32 when the
-// tiles are filled.
+// tiles are filled.  Requests in fp32 storage (served here only with the value-channel gate) keep full
+// fp32 tiles instead and split every operand at fragment load into a tf32 head and a tf32 tail,
+// x = hi + lo: three products hi*hi + lo*hi + hi*lo per fragment pair leave errors of order 2^-21,
+// the accuracy fp32 storage is held to.
 //
 // Notation per chunk (rows j = 0..C-1 in scan order, zero rows past the end of the sequence):
 //   Lam_j = inclusive prefix sum of the gates, gamma = exp(Lam_{C-1}),
 //   Qt = q*exp(Lam), Kt = k*exp(-Lam), Kh = k*exp(Lam_{C-1}-Lam),
 //   S = state entering the chunk, Dg = diag(gamma) * dL/d(state leaving the chunk); the scan kernels
 //   leave both rounded to tf32 in the workspace.
+#include <type_traits>
+
 #include "dig_common.cuh"
 
 namespace dig {
 namespace {
 
+using bf16 = __nv_bfloat16;
 constexpr int kThreads = 512, kWarps = kThreads / 32;
 constexpr int kMaxNB = 8;                    // 8-column fragments per warp tile: up to 64 columns
 
@@ -64,6 +70,16 @@ __device__ __forceinline__ float tf32r(float x)
     return __uint_as_float(u);
 }
 
+// Rounding of a tile element: none when the operands are split at fragment load (PR).
+template <bool PR>
+__device__ __forceinline__ float rnd(float x) { return PR ? x : tf32r(x); }
+// x = hi + lo with hi the tf32 truncation of x (what the tensor core reads of an fp32 register anyway).
+__device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo)
+{
+    hi = __float_as_uint(x) & 0xffffe000u;
+    lo = __float_as_uint(x - __uint_as_float(hi));
+}
+
 __device__ __forceinline__ void mma8(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
     asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -75,7 +91,7 @@ __device__ __forceinline__ void mma8(float (&c)[4], const uint32_t (&a)[4], uint
 // A(m, k) = A[m*sam + k*sak], B(k, n) = Bm[k*sbk + n*sbn]; k0, k1 multiples of 8.
 // Fragment layout of m16n8k8: with g = lane / 4, t = lane % 4 a lane holds A(g | g+8, t | t+4),
 // B(t | t+4, g) and the results C(g | g+8, 2t | 2t+1).
-template <int NB>
+template <bool PR, int NB>
 __device__ __forceinline__ void warp_mma(float (&acc)[NB][4], const float *A, int sam, int sak, int r0,
                                          const float *Bm, int sbk, int sbn, int c0, int nbw, int k0, int k1)
 {
@@ -84,17 +100,27 @@ __device__ __forceinline__ void warp_mma(float (&acc)[NB][4], const float *A, in
     const float *pb = Bm + (t + k0) * sbk + (c0 + g) * sbn;
 #pragma unroll 2
     for (int k = k0; k < k1; k += 8) {
-        uint32_t a[4];
-        a[0] = __float_as_uint(pa[0]);
-        a[1] = __float_as_uint(pa[8 * sam]);
-        a[2] = __float_as_uint(pa[4 * sak]);
-        a[3] = __float_as_uint(pa[8 * sam + 4 * sak]);
+        const float af[4] = {pa[0], pa[8 * sam], pa[4 * sak], pa[8 * sam + 4 * sak]};
+        uint32_t a[4], al[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (PR) split_tf32(af[i], a[i], al[i]);
+            else a[i] = __float_as_uint(af[i]);
+        }
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb)
             if (nb < nbw) {
-                const uint32_t b0 = __float_as_uint(pb[8 * nb * sbn]);
-                const uint32_t b1 = __float_as_uint(pb[4 * sbk + 8 * nb * sbn]);
-                mma8(acc[nb], a, b0, b1);
+                const float bf0 = pb[8 * nb * sbn], bf1 = pb[4 * sbk + 8 * nb * sbn];
+                if (PR) {
+                    uint32_t b0, b1, b0l, b1l;
+                    split_tf32(bf0, b0, b0l);
+                    split_tf32(bf1, b1, b1l);
+                    mma8(acc[nb], al, b0, b1);          // the small terms first
+                    mma8(acc[nb], a, b0l, b1l);
+                    mma8(acc[nb], a, b0, b1);
+                } else {
+                    mma8(acc[nb], a, __float_as_uint(bf0), __float_as_uint(bf1));
+                }
             }
         pa += 8 * sak;
         pb += 8 * sbk;
@@ -215,6 +241,10 @@ __device__ __forceinline__ void load_gates(float *dst, int ld, const float *gate
         else *reinterpret_cast<float4 *>(dst + j * ld + c) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
+__device__ __forceinline__ void load_rows(float *dst, int ld, const float *src, const int *sRow, int C, int d, int dp)
+{
+    load_gates(dst, ld, src, sRow, C, d, dp);       // fp32 rows travel like the gates
+}
 // A [dk][dv] state of the workspace (rounded to tf32 by the scan kernels) -> [dk][ld] tile.
 __device__ __forceinline__ void load_state(float *dst, int ld, const float *src, int dk, int dv)
 {
@@ -255,6 +285,7 @@ __device__ __forceinline__ void prefix_gates(float *lam, int ld, int C, int dkp,
 }
 // In place: sQ (raw q) -> Qt = q*exp(Lam), sK (raw k) -> Kt = k*exp(-Lam), or with sLast given
 // -> Kh = k*exp(Lam_{C-1}-Lam); rounded to tf32.  Either tile may be null.
+template <bool PR>
 __device__ __forceinline__ void scale_qk(float *sQ, float *sK, const float *sLam, const float *sLast, int ldk, int C, int dp)
 {
     const int per_row = dp >> 2;
@@ -264,7 +295,7 @@ __device__ __forceinline__ void scale_qk(float *sQ, float *sK, const float *sLam
         if (sQ) {
             const float4 x = *reinterpret_cast<const float4 *>(sQ + j * ldk + c);
             *reinterpret_cast<float4 *>(sQ + j * ldk + c) = make_float4(
-                tf32r(x.x * __expf(lam.x)), tf32r(x.y * __expf(lam.y)), tf32r(x.z * __expf(lam.z)), tf32r(x.w * __expf(lam.w)));
+                rnd<PR>(x.x * __expf(lam.x)), rnd<PR>(x.y * __expf(lam.y)), rnd<PR>(x.z * __expf(lam.z)), rnd<PR>(x.w * __expf(lam.w)));
         }
         if (sK) {
             float4 e = make_float4(-lam.x, -lam.y, -lam.z, -lam.w);
@@ -274,14 +305,14 @@ __device__ __forceinline__ void scale_qk(float *sQ, float *sK, const float *sLam
             }
             const float4 x = *reinterpret_cast<const float4 *>(sK + j * ldk + c);
             *reinterpret_cast<float4 *>(sK + j * ldk + c) = make_float4(
-                tf32r(x.x * __expf(e.x)), tf32r(x.y * __expf(e.y)), tf32r(x.z * __expf(e.z)), tf32r(x.w * __expf(e.w)));
+                rnd<PR>(x.x * __expf(e.x)), rnd<PR>(x.y * __expf(e.y)), rnd<PR>(x.z * __expf(e.z)), rnd<PR>(x.w * __expf(e.w)));
         }
     }
 }
 
 // sP[t][s] = A_t . B_s for s <= t, 0 above the diagonal, rounded to tf32 (A, B: [C][ld] tiles, contraction
 // over the first K columns).  The diagonal has weight 1: the token's own k^T v enters undecayed.
-template <int NB>
+template <int NB, bool PR>
 __device__ __forceinline__ void masked_scores(float *sP, int ldp, const float *A, const float *Bm, int ld, int C, int K)
 {
     const Tiling tl(C, C);
@@ -292,9 +323,9 @@ __device__ __forceinline__ void masked_scores(float *sP, int ldp, const float *A
         if (nbt <= 0) continue;
         float acc[NB][4];
         zero(acc);
-        if (c0 <= r0 + 15) warp_mma(acc, A, ld, 1, r0, Bm, 1, ld, c0, nbt, 0, K);
+        if (c0 <= r0 + 15) warp_mma<PR>(acc, A, ld, 1, r0, Bm, 1, ld, c0, nbt, 0, K);
         for_pairs(acc, r0, c0, nbt, [&](int t, int s, float v0, float v1) {
-            *reinterpret_cast<float2 *>(sP + t * ldp + s) = make_float2(s <= t ? tf32r(v0) : 0.f, s + 1 <= t ? tf32r(v1) : 0.f);
+            *reinterpret_cast<float2 *>(sP + t * ldp + s) = make_float2(s <= t ? rnd<PR>(v0) : 0.f, s + 1 <= t ? rnd<PR>(v1) : 0.f);
         });
     }
 }
@@ -303,13 +334,13 @@ __device__ __forceinline__ void masked_scores(float *sP, int ldp, const float *A
 // U = Kh^T V (and, for the backward pass, W = Qt^T dO); gamma = exp(Lam_{C-1}).
 // BETA: with the value-channel gate the value side mirrors the key side: M = prefix sums of log(beta),
 // gamma_v = exp(M_{C-1}), U = Kh^T Vh with Vh = v*exp(M_{C-1}-M), W = Qt^T G with G = dO*exp(M).
-template <bool BWD, typename DM, bool BETA>
+template <bool BWD, typename DM, bool BETA, typename TI>
 __global__ void __launch_bounds__(kThreads)
-mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
-                const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate,
-                const __nv_bfloat16 *__restrict__ d_out, float *__restrict__ states, float *__restrict__ gamma,
+mma_chunk_state(const TI *__restrict__ q, const TI *__restrict__ k, const TI *__restrict__ v, const float *__restrict__ gate,
+                const TI *__restrict__ d_out, float *__restrict__ states, float *__restrict__ gamma,
                 float *__restrict__ dstates, BetaDev bd, Geom g)
 {
+    constexpr bool PR = std::is_same<TI, float>::value;
     extern __shared__ __align__(16) float smem[];
     __shared__ int sRow[128];
     const DM dm(g);
@@ -343,10 +374,10 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
     if (BETA) prefix_gates(sM, ldv, C, dvp, sMlast, sSegV);
     const size_t chunk_id = (size_t)bh * g.N + chunk;
     for (int c = threadIdx.x; c < dk; c += kThreads) gamma[chunk_id * dk + c] = __expf(sLast[c]);
-    scale_qk(BWD ? sQ : nullptr, sX, sLam, sLast, ldk, C, dkp);
+    scale_qk<PR>(BWD ? sQ : nullptr, sX, sLam, sLast, ldk, C, dkp);
     if (BETA) {
         for (int e = threadIdx.x; e < dv; e += kThreads) bd.gamma_v[chunk_id * dv + e] = __expf(sMlast[e]);
-        scale_qk(BWD ? sG : nullptr, sV, sM, sMlast, ldv, C, dvp);      // G = dO*exp(M), Vh = v*exp(M_{C-1}-M)
+        scale_qk<PR>(BWD ? sG : nullptr, sV, sM, sMlast, ldv, C, dvp);      // G = dO*exp(M), Vh = v*exp(M_{C-1}-M)
     }
     __syncthreads();
     constexpr int NB = frag_bound(pad16(DM::kDK), DM::kDV);
@@ -360,13 +391,13 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
         if (nbt <= 0) continue;
         float acc[NB][4];
         zero(acc);
-        warp_mma(acc, sX, 1, ldk, r0, sV, ldv, 1, c0, nbt, 0, C);           // sum_t Kh[t][c] V[t][e]
+        warp_mma<PR>(acc, sX, 1, ldk, r0, sV, ldv, 1, c0, nbt, 0, C);           // sum_t Kh[t][c] V[t][e]
         for_pairs(acc, r0, c0, nbt, [&](int c, int e, float v0, float v1) {
             if (c < dk && e < dv) store2(U + c * dv + e, v0, v1);
         });
         if (BWD) {
             zero(acc);
-            warp_mma(acc, sQ, 1, ldk, r0, sG, ldv, 1, c0, nbt, 0, C);       // sum_t Qt[t][c] dO[t][e]
+            warp_mma<PR>(acc, sQ, 1, ldk, r0, sG, ldv, 1, c0, nbt, 0, C);       // sum_t Qt[t][c] dO[t][e]
             for_pairs(acc, r0, c0, nbt, [&](int c, int e, float v0, float v1) {
                 if (c < dk && e < dv) store2(W + c * dv + e, v0, v1);
             });
@@ -377,12 +408,12 @@ mma_chunk_state(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__rest
 // ---- kernel 3: outputs ------------------------------------------------------------------------------
 // out = tril(Qt Kt^T) V + Qt S
 // BETA: out = exp(M) * (tril(Qt Kt^T) Vt + Qt S) with Vt = v*exp(-M).
-template <typename TO, typename DM, bool BETA>
+template <typename TO, typename DM, bool BETA, typename TI>
 __global__ void __launch_bounds__(kThreads)
-mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
-              const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate, const float *__restrict__ states,
-              TO *__restrict__ out, BetaDev bd, Geom g)
+mma_chunk_out(const TI *__restrict__ q, const TI *__restrict__ k, const TI *__restrict__ v, const float *__restrict__ gate,
+              const float *__restrict__ states, TO *__restrict__ out, BetaDev bd, Geom g)
 {
+    constexpr bool PR = std::is_same<TI, float>::value;
     extern __shared__ __align__(16) float smem[];
     __shared__ int sRow[128];
     const DM dm(g);
@@ -413,10 +444,10 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     __syncthreads();
     prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
     if (BETA) prefix_gates(sM, ldv, C, dv, sMlast, sSegV);
-    scale_qk(sQ, sK, sLam, nullptr, ldk, C, dk);
-    if (BETA) scale_qk(nullptr, sV, sM, nullptr, ldv, C, dv);           // Vt = v*exp(-M)
+    scale_qk<PR>(sQ, sK, sLam, nullptr, ldk, C, dk);
+    if (BETA) scale_qk<PR>(nullptr, sV, sM, nullptr, ldv, C, dv);           // Vt = v*exp(-M)
     __syncthreads();
-    masked_scores<frag_bound(DM::kC, DM::kC)>(sP, ldp, sQ, sK, ldk, C, dk);
+    masked_scores<frag_bound(DM::kC, DM::kC), PR>(sP, ldp, sQ, sK, ldk, C, dk);
     __syncthreads();
     constexpr int NB = frag_bound(DM::kC, DM::kDV);
     const Tiling tl(C, dv);
@@ -427,8 +458,8 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
         if (nbt <= 0) continue;
         float acc[NB][4];
         zero(acc);
-        warp_mma(acc, sP, ldp, 1, r0, sV, ldv, 1, c0, nbt, 0, r0 + 16);     // columns past the diagonal are zero
-        warp_mma(acc, sQ, ldk, 1, r0, sS, ldv, 1, c0, nbt, 0, dk);
+        warp_mma<PR>(acc, sP, ldp, 1, r0, sV, ldv, 1, c0, nbt, 0, r0 + 16);     // columns past the diagonal are zero
+        warp_mma<PR>(acc, sQ, ldk, 1, r0, sS, ldv, 1, c0, nbt, 0, dk);
         for_pairs(acc, r0, c0, nbt, [&](int j, int e, float v0, float v1) {
             const int row = sRow[j];
             if (BETA) {
@@ -452,14 +483,14 @@ mma_chunk_out(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
 //   dbgate_j = sum_{r >= j} (o*dO - v*dv)_r  with  o*dO = (P Vt + Qt S)*G  and  v*dv = Vt*(dv accumulator)
 // (the unscaled output P Vt + Qt S is recomputed here, two more products, rather than read back in
 // storage precision), summed here inside the chunk; the chunk total goes to xtot for the cross-chunk part.
-template <typename TO, typename DM, bool BETA>
+template <typename TO, typename DM, bool BETA, typename TI>
 __global__ void __launch_bounds__(kThreads)
-mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
-              const __nv_bfloat16 *__restrict__ v, const float *__restrict__ gate,
-              const __nv_bfloat16 *__restrict__ d_out, const float *__restrict__ states,
+mma_chunk_bwd(const TI *__restrict__ q, const TI *__restrict__ k, const TI *__restrict__ v, const float *__restrict__ gate,
+              const TI *__restrict__ d_out, const float *__restrict__ states,
               const float *__restrict__ dstates, const float *__restrict__ carry, TO *__restrict__ dq,
               TO *__restrict__ dk_out, TO *__restrict__ dv_out, float *__restrict__ dgate, BetaDev bd, Geom g)
 {
+    constexpr bool PR = std::is_same<TI, float>::value;
     extern __shared__ __align__(16) float smem[];
     __shared__ int sRow[128];
     const DM dm(g);
@@ -496,11 +527,11 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
     __syncthreads();
     prefix_gates(sLam, ldk, C, dkp, sLast, sSeg);
     if (BETA) prefix_gates(sM, ldv, C, dv, sMlast, sSegV);
-    scale_qk(sQ, sK, sLam, nullptr, ldk, C, dk);
-    if (BETA) scale_qk(sG, sV, sM, nullptr, ldv, C, dv);                // G = dO*exp(M), Vt = v*exp(-M)
+    scale_qk<PR>(sQ, sK, sLam, nullptr, ldk, C, dk);
+    if (BETA) scale_qk<PR>(sG, sV, sM, nullptr, ldv, C, dv);                // G = dO*exp(M), Vt = v*exp(-M)
     __syncthreads();
-    masked_scores<frag_bound(DM::kC, DM::kC)>(sP, ldp, sQ, sK, ldk, C, dk);
-    masked_scores<frag_bound(DM::kC, DM::kC)>(sdP, ldp, sG, sV, ldv, C, dv);
+    masked_scores<frag_bound(DM::kC, DM::kC), PR>(sP, ldp, sQ, sK, ldk, C, dk);
+    masked_scores<frag_bound(DM::kC, DM::kC), PR>(sdP, ldp, sG, sV, ldv, C, dv);
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gi = lane >> 2, ti = lane & 3;
     {
@@ -513,14 +544,14 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
             if (nbt <= 0) continue;
             float acc[NB][4];
             zero(acc);
-            warp_mma(acc, sP, 1, ldp, r0, sG, ldv, 1, c0, nbt, r0, C);
-            warp_mma(acc, sK, ldk, 1, r0, sD, ldv, 1, c0, nbt, 0, dk);
+            warp_mma<PR>(acc, sP, 1, ldp, r0, sG, ldv, 1, c0, nbt, r0, C);
+            warp_mma<PR>(acc, sK, ldk, 1, r0, sD, ldv, 1, c0, nbt, 0, dk);
             if (BETA) {
                 // unscaled output of the same tile, then x = o*dO - v*dv = (P Vt + Qt S)*G - Vt*(dv accumulator)
                 float oh[NB][4];
                 zero(oh);
-                warp_mma(oh, sP, ldp, 1, r0, sV, ldv, 1, c0, nbt, 0, r0 + 16);
-                warp_mma(oh, sQ, ldk, 1, r0, sS, ldv, 1, c0, nbt, 0, dk);
+                warp_mma<PR>(oh, sP, ldp, 1, r0, sV, ldv, 1, c0, nbt, 0, r0 + 16);
+                warp_mma<PR>(oh, sQ, ldk, 1, r0, sS, ldv, 1, c0, nbt, 0, dk);
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb)
                     if (nb < nbt) {
@@ -560,8 +591,8 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
             if (nbt <= 0) continue;
             float acc[NB][4], xq[NB][4];
             zero(acc);
-            warp_mma(acc, sdP, ldp, 1, r0, sK, ldk, 1, c0, nbt, 0, r0 + 16);          // sum_{s <= t} dP[t][s] Kt[s][c]
-            warp_mma(acc, sG, ldv, 1, r0, sS, 1, ldv, c0, nbt, 0, dv);                // sum_e dO[t][e] S[c][e]
+            warp_mma<PR>(acc, sdP, ldp, 1, r0, sK, ldk, 1, c0, nbt, 0, r0 + 16);          // sum_{s <= t} dP[t][s] Kt[s][c]
+            warp_mma<PR>(acc, sG, ldv, 1, r0, sS, 1, ldv, c0, nbt, 0, dv);                // sum_e dO[t][e] S[c][e]
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb)
                 if (nb < nbt) {
@@ -580,8 +611,8 @@ mma_chunk_bwd(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restri
                 }
             });
             zero(acc);
-            warp_mma(acc, sdP, 1, ldp, r0, sQ, ldk, 1, c0, nbt, r0, C);               // sum_{t >= s} dP[t][s] Qt[t][c]
-            warp_mma(acc, sV, ldv, 1, r0, sD, 1, ldv, c0, nbt, 0, dv);                // sum_e V[s][e] Dg[c][e]
+            warp_mma<PR>(acc, sdP, 1, ldp, r0, sQ, ldk, 1, c0, nbt, r0, C);               // sum_{t >= s} dP[t][s] Qt[t][c]
+            warp_mma<PR>(acc, sV, ldv, 1, r0, sD, 1, ldv, c0, nbt, 0, dv);                // sum_e V[s][e] Dg[c][e]
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb)
                 if (nb < nbt) {
@@ -677,10 +708,8 @@ template <typename K>
 dig_status set_smem(K kernel, size_t bytes)
 {
     if (bytes > kMaxSmem) return DIG_ERR_UNSUPPORTED;
-    return cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    return ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), bytes);
 }
-
-using bf16 = __nv_bfloat16;
 
 // The value-channel gate keeps two more blocks behind the common workspace: gamma_v and, for the
 // backward pass, the chunk totals of o*do - v*dv, both [B*H][N][d_v].
@@ -699,61 +728,63 @@ BetaDev beta_dev(const GlaArgs &a, const Workspace &w, bool backward)
     return bd;
 }
 
-template <typename TO, typename DM, bool BETA>
+template <typename TO, typename DM, bool BETA, typename TI = bf16>
 dig_status fwd_dims(const GlaArgs &a)
 {
+    constexpr bool kRound = !std::is_same<TI, float>::value;     // states rounded to tf32 by the scans
     const Geom &g = a.g;
     const Workspace w = carve_workspace(a.ws, g, false);
     const BetaDev bd = beta_dev(a, w, false);
     const dim3 grid(g.N, g.B * g.H);
     dig_status st;
-    auto k1 = mma_chunk_state<false, DM, BETA>;
+    auto k1 = mma_chunk_state<false, DM, BETA, TI>;
     if ((st = set_smem(k1, smem_state(g, false, BETA))) != DIG_OK) return st;
-    auto k3 = mma_chunk_out<TO, DM, BETA>;
+    auto k3 = mma_chunk_out<TO, DM, BETA, TI>;
     if ((st = set_smem(k3, smem_out(g, BETA))) != DIG_OK) return st;
     {
         KernelTimer t(KID_MMA_STATE, a.stream);
-        k1<<<grid, kThreads, smem_state(g, false, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
+        k1<<<grid, kThreads, smem_state(g, false, BETA), a.stream>>>((const TI *)a.q, (const TI *)a.k, (const TI *)a.v,
                                                                     a.gate, nullptr, w.states, w.gamma, nullptr, bd, g);
     }
-    if (BETA) st = launch_state_scan_fwd_beta(w, bd.gamma_v, g, a.stream);
-    else st = launch_state_scan_fwd(w, g, a.stream, a.sio, true);
+    if (BETA) st = launch_state_scan_fwd_beta(w, bd.gamma_v, g, a.stream, kRound);
+    else st = launch_state_scan_fwd(w, g, a.stream, a.sio, kRound);
     if (st != DIG_OK) return st;
     KernelTimer t(KID_MMA_OUT, a.stream);
-    k3<<<grid, kThreads, smem_out(g, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
+    k3<<<grid, kThreads, smem_out(g, BETA), a.stream>>>((const TI *)a.q, (const TI *)a.k, (const TI *)a.v, a.gate,
                                                         w.states, (TO *)a.out, bd, g);
     return cuda_ok(cudaGetLastError());
 }
 
-template <typename TO, typename DM, bool BETA>
+template <typename TO, typename DM, bool BETA, typename TI = bf16>
 dig_status bwd_dims(const GlaArgs &a)
 {
+    constexpr bool kRound = !std::is_same<TI, float>::value;
     const Geom &g = a.g;
     const Workspace w = carve_workspace(a.ws, g, true);
     const BetaDev bd = beta_dev(a, w, true);
     const dim3 grid(g.N, g.B * g.H);
     dig_status st;
-    auto k1 = mma_chunk_state<true, DM, BETA>;
+    auto k1 = mma_chunk_state<true, DM, BETA, TI>;
     if ((st = set_smem(k1, smem_state(g, true, BETA))) != DIG_OK) return st;
-    auto k4 = mma_chunk_bwd<TO, DM, BETA>;
+    auto k4 = mma_chunk_bwd<TO, DM, BETA, TI>;
     if ((st = set_smem(k4, smem_bwd(g, BETA))) != DIG_OK) return st;
     {
         KernelTimer t(KID_MMA_STATE, a.stream);
-        k1<<<grid, kThreads, smem_state(g, true, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v,
-                                                                   a.gate, (const bf16 *)a.d_out, w.states, w.gamma, w.dstates,
+        k1<<<grid, kThreads, smem_state(g, true, BETA), a.stream>>>((const TI *)a.q, (const TI *)a.k, (const TI *)a.v,
+                                                                   a.gate, (const TI *)a.d_out, w.states, w.gamma, w.dstates,
                                                                    bd, g);
     }
     if (BETA) {
-        if ((st = launch_state_scan_fwd_beta(w, bd.gamma_v, g, a.stream)) != DIG_OK) return st;
-        if ((st = launch_state_scan_bwd_beta(w, bd.gamma_v, g, a.stream)) != DIG_OK) return st;
+        if ((st = launch_state_scan_fwd_beta(w, bd.gamma_v, g, a.stream, kRound)) != DIG_OK) return st;
+        if ((st = launch_state_scan_bwd_beta(w, bd.gamma_v, g, a.stream, kRound)) != DIG_OK) return st;
     } else {
-        if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, true)) != DIG_OK) return st;
-        if ((st = launch_state_scan_bwd(w, g, a.stream, a.sio, true)) != DIG_OK) return st;
+        if ((st = launch_state_scan_fwd(w, g, a.stream, a.sio, kRound)) != DIG_OK) return st;
+        if ((st = launch_state_scan_bwd(w, g, a.stream, a.sio, kRound)) != DIG_OK) return st;
     }
     {
         KernelTimer t(KID_MMA_BWD, a.stream);
-        k4<<<grid, kThreads, smem_bwd(g, BETA), a.stream>>>((const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, a.gate,
-                                                            (const bf16 *)a.d_out, w.states, w.dstates, w.carry, (TO *)a.dq,
+        k4<<<grid, kThreads, smem_bwd(g, BETA), a.stream>>>((const TI *)a.q, (const TI *)a.k, (const TI *)a.v, a.gate,
+                                                            (const TI *)a.d_out, w.states, w.dstates, w.carry, (TO *)a.dq,
                                                             (TO *)a.dk, (TO *)a.dv, a.dgate, bd, g);
     }
     if (cudaGetLastError() != cudaSuccess) return DIG_ERR_CUDA;
@@ -786,7 +817,7 @@ dig_status bwd_typed(const GlaArgs &a)
 
 bool mma_supports(int dk, int dv, int chunk, int dtype, bool backward, bool beta)
 {
-    if (dtype == DIG_F32) return false;      // one tf32 pass is not fp32-accurate
+    if (dtype == DIG_F32 && !beta) return false;      // fp32 storage: only the full gate is served here (split operands)
     Geom g{};
     g.dk = dk; g.dv = dv; g.C = chunk;
     if (backward) return smem_bwd(g, beta) <= kMaxSmem && smem_state(g, true, beta) <= kMaxSmem;
@@ -803,6 +834,7 @@ dig_status mma_gla_fwd(const GlaArgs &a)
     const bool beta = a.bio.bgate != nullptr;
     if (a.dtype == DIG_BF16) return beta ? fwd_typed<__nv_bfloat16, true>(a) : fwd_typed<__nv_bfloat16, false>(a);
     if (a.dtype == DIG_BF16_F32OUT) return beta ? fwd_typed<float, true>(a) : fwd_typed<float, false>(a);
+    if (a.dtype == DIG_F32 && beta) return fwd_dims<float, AnyDims, true, float>(a);
     return DIG_ERR_UNSUPPORTED;
 }
 
@@ -811,6 +843,7 @@ dig_status mma_gla_bwd(const GlaArgs &a)
     const bool beta = a.bio.bgate != nullptr;
     if (a.dtype == DIG_BF16) return beta ? bwd_typed<__nv_bfloat16, true>(a) : bwd_typed<__nv_bfloat16, false>(a);
     if (a.dtype == DIG_BF16_F32OUT) return beta ? bwd_typed<float, true>(a) : bwd_typed<float, false>(a);
+    if (a.dtype == DIG_F32 && beta) return bwd_dims<float, AnyDims, true, float>(a);
     return DIG_ERR_UNSUPPORTED;
 }
 

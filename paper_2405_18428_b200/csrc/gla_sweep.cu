@@ -171,7 +171,7 @@ sweep_local(const SweepArgs a)
     Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 3 * T);
     constexpr uint32_t aU = 0, aW = C::BIGM ? C::NACC : D / 2;
 
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x;
     constexpr int kIssuer = NT - 32;        // lane 0 of the last warp issues the MMAs (warps 0 and 1 carry the per-channel work)
     cta_setup(ctl, 1, SM::tmem_cols, smem, SM::kTilesPad);
     const uint32_t tmem = ctl->tmem_base, lane_base = (uint32_t)(32 * ((tid >> 5) & 3)) << 16;
@@ -301,7 +301,7 @@ die:
 }
 
 // =================================================================================================
-// seg_scan: the recurrence over segment ends, one sequence per blockIdx.y, 8 state rows per block,
+// seg_scan: the recurrence over segment ends, one sequence per blockIdx.x, 8 state rows per block,
 // 8 lanes per row.  Forward: seg_state[s] (state a segment leaves from a zero start) becomes the
 // state entering segment s.  Backward flavour: seg_dstate[s] (the segment's own contribution)
 // becomes the gradient with respect to the state leaving segment s, seg_carry the gate-gradient
@@ -315,7 +315,7 @@ seg_scan(float *seg_state, const float *seg_gamma, float *seg_dstate, float *seg
 {
     constexpr int NV = (D / 4 + 7) / 8;               // float4 pieces per lane
     constexpr int NB = NV <= 2 ? 8 : 4;               // segments whose loads are in flight together
-    const int bh = blockIdx.y, c = blockIdx.x * 8 + (threadIdx.x >> 3), l8 = threadIdx.x & 7;
+    const int bh = blockIdx.x, c = blockIdx.y * 8 + (threadIdx.x >> 3), l8 = threadIdx.x & 7;
     pdl_wait();
     pdl_launch_dependents();
     float4 s[NV];
@@ -965,7 +965,7 @@ int sweep_per_sm(int d, bool backward)
 template <typename K>
 dig_status set_smem(K kern, size_t bytes)
 {
-    return cuda_ok(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    return ensure_dynamic_smem(reinterpret_cast<const void *>(kern), bytes);
 }
 
 template <int D, bool BWD>
@@ -1006,7 +1006,7 @@ dig_status run(const GlaArgs &ga)
     {
         auto kern = seg_scan<D, BWD>;
         KernelTimer t(KID_SW_SCAN, ga.stream);
-        launch_pdl(kern, dim3(D / 8, g.B * g.H), dim3(64), 0, ga.stream, w.seg_state, (const float *)w.seg_gamma, w.seg_dstate,
+        launch_pdl(kern, dim3(g.B * g.H, D / 8), dim3(64), 0, ga.stream, w.seg_state, (const float *)w.seg_gamma, w.seg_dstate,
                    w.seg_carry, w.seg_state16, ga.sio.s_in, ga.sio.s_out, ga.sio.ds_out, ga.sio.ds_in, pl.nseg);
         if ((st = cuda_ok(cudaGetLastError())) != DIG_OK) return st;
     }

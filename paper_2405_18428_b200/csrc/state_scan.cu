@@ -198,10 +198,10 @@ state_scan_bwd(const float *__restrict__ states, float *__restrict__ dstates,
 // ---- the same scans with the value-channel gate (full gate G = alpha^T beta of Eq. gate_gla) ---------
 // The state decays along its rows by gamma (key channels) and along its columns by gamma_v (value
 // channels): S_[i+1] = diag(gamma_i) S_[i] diag(gamma_v_i) + U_i, and the mirror image for D.  Row-major
-// states only (warp-MMA family); stored states and diag(gamma) D diag(gamma_v) are rounded to tf32.
+// states only (warp-MMA family); with `tf32` the stored states and diag(gamma) D diag(gamma_v) are rounded to tf32.
 __global__ void __launch_bounds__(kScanThreads)
 state_scan_fwd_beta(float *__restrict__ states, const float *__restrict__ gamma, const float *__restrict__ gamma_v,
-                    float *__restrict__ s_final, int N, int dk, int dv)
+                    float *__restrict__ s_final, int N, int dk, int dv, bool tf32)
 {
     const int e4 = blockIdx.x * kScanThreads + threadIdx.x;
     if (e4 * 4 >= dk * dv) return;
@@ -225,7 +225,7 @@ state_scan_fwd_beta(float *__restrict__ states, const float *__restrict__ gamma,
 #pragma unroll
         for (int j = 0; j < kAhead; ++j) {
             if (i + j < N) {
-                st[(size_t)(i + j) * sstride] = round4_tf32(run);
+                st[(size_t)(i + j) * sstride] = tf32 ? round4_tf32(run) : run;
                 run.x = fmaf(g[j].x, run.x, u[j].x);
                 run.y = fmaf(g[j].y, run.y, u[j].y);
                 run.z = fmaf(g[j].z, run.z, u[j].z);
@@ -238,7 +238,7 @@ state_scan_fwd_beta(float *__restrict__ states, const float *__restrict__ gamma,
 
 __global__ void __launch_bounds__(32 * kRowsPerBlock)
 state_scan_bwd_beta(const float *__restrict__ states, float *__restrict__ dstates, const float *__restrict__ gamma,
-                    const float *__restrict__ gamma_v, float *__restrict__ carry, int N, int dk, int dv)
+                    const float *__restrict__ gamma_v, float *__restrict__ carry, int N, int dk, int dv, bool tf32)
 {
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * kRowsPerBlock + (threadIdx.x >> 5);
@@ -277,7 +277,7 @@ state_scan_bwd_beta(const float *__restrict__ states, float *__restrict__ dstate
 #pragma unroll
             for (int r = 0; r < kMaxPerLane; ++r) {
                 const int e = lane + 32 * r;
-                if (e < dv) D[(size_t)ch * sstride + e] = round_tf32(g[j][r] * run[r]);
+                if (e < dv) D[(size_t)ch * sstride + e] = tf32 ? round_tf32(g[j][r] * run[r]) : g[j][r] * run[r];
                 dot = fmaf(sn[j][r], run[r], dot);
                 run[r] = fmaf(g[j][r], run[r], w[j][r]);
             }
@@ -364,19 +364,19 @@ dig_status launch_state_scan_bwd(const Workspace &w, const Geom &g, cudaStream_t
     return cuda_ok(cudaGetLastError());
 }
 
-dig_status launch_state_scan_fwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s)
+dig_status launch_state_scan_fwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s, bool tf32)
 {
     const dim3 grid((g.dk * g.dv / 4 + kScanThreads - 1) / kScanThreads, g.B * g.H);
     KernelTimer t(KID_SCAN_FWD, s);
-    state_scan_fwd_beta<<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, gamma_v, w.sfinal, g.N, g.dk, g.dv);
+    state_scan_fwd_beta<<<grid, kScanThreads, 0, s>>>(w.states, w.gamma, gamma_v, w.sfinal, g.N, g.dk, g.dv, tf32);
     return cuda_ok(cudaGetLastError());
 }
 
-dig_status launch_state_scan_bwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s)
+dig_status launch_state_scan_bwd_beta(const Workspace &w, const float *gamma_v, const Geom &g, cudaStream_t s, bool tf32)
 {
     const dim3 grid((g.dk + kRowsPerBlock - 1) / kRowsPerBlock, g.B * g.H);
     KernelTimer t(KID_SCAN_BWD, s);
-    state_scan_bwd_beta<<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, gamma_v, w.carry, g.N, g.dk, g.dv);
+    state_scan_bwd_beta<<<grid, 32 * kRowsPerBlock, 0, s>>>(w.states, w.dstates, w.gamma, gamma_v, w.carry, g.N, g.dk, g.dv, tf32);
     return cuda_ok(cudaGetLastError());
 }
 
