@@ -220,8 +220,10 @@ dig_status dig_gla_fwd_outgate(const void *q, const void *k, const void *v, cons
  *   S_t = diag(exp(gate_t)) S_{t-1} diag(exp(bgate_t)) + k_t^T v_t,   out_t = q_t S_t,
  * bgate = log(beta) <= 0, fp32 [B][L][H][d_v]; everything else as in dig_gla_fwd / dig_gla_bwd.
  * dig_gla_bwd_beta returns dbgate (fp32 [B][L][H][d_v]) beside the other gradients.
- * Served by the warp-level tensor-core kernels only: bf16 storage (DIG_F32 returns DIG_ERR_UNSUPPORTED),
- * any supported head and chunk size that fits shared memory.  The workspace is larger than that of
+ * Served by the warp-level tensor-core kernels, for every dtype: with bf16 storage the operands are rounded
+ * to tf32 (results within 2e-2 of RMS like dig_gla_fwd), with DIG_F32 every operand is split into two tf32
+ * parts and the products are exact to about 2^-21 (results within 1e-4 of RMS, the fp32 bound).  Any
+ * supported head and chunk size that fits shared memory.  The workspace is larger than that of
  * dig_gla_fwd / dig_gla_bwd: dig_gla_beta_workspace_bytes (0 for invalid or unsupported sizes).  The same
  * bound of 80 on the magnitude of a gate summed over one chunk applies to bgate. */
 size_t dig_gla_beta_workspace_bytes(int B, int H, int grid_h, int grid_w, int d_k, int d_v, int chunk, int dtype,

@@ -6,7 +6,7 @@ import torch
 
 import oracle
 from paper_2405_18428_b200.inputs import CONFIGS, Workload, make_inputs, round_to_bf16
-from parity import TOL_BF16, oracle_threads, rel_err, to_dev
+from parity import TOL_BF16, TOL_F32, oracle_threads, rel_err, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -15,7 +15,9 @@ def _run(wl, direction, seed, tau_v=8.0):
     from paper_2405_18428_b200 import dig
     x = make_inputs(wl, conv=False)
     rng = np.random.default_rng(seed)
-    gb = round_to_bf16(rng.standard_normal((wl.B, wl.grid_h * wl.grid_w, wl.H, wl.d_v)).astype(np.float32))
+    gb = rng.standard_normal((wl.B, wl.grid_h * wl.grid_w, wl.H, wl.d_v)).astype(np.float32)
+    if wl.dtype == "bf16":
+        gb = round_to_bf16(gb)
     a = oracle.gate(x["g"], x["tau"])
     bg = oracle.gate(gb, np.full(wl.H, tau_v, dtype=np.float32))          # log(beta) = logsigmoid / tau
     thr = oracle_threads()
@@ -24,6 +26,16 @@ def _run(wl, direction, seed, tau_v=8.0):
     q, k, v, g, dO = (to_dev(x[n], wl) for n in ("q", "k", "v", "g", "dO"))
     gate = dig.dig_gate_logsigmoid(g, x["tau"])
     bgate = dig.dig_gate_logsigmoid(to_dev(gb, wl), np.full(wl.H, tau_v, dtype=np.float32))
+    if wl.dtype == "f32":
+        # fp32 storage: one pass, held to the fp32 bound (the kernels split every operand into two tf32 parts)
+        out = dig.dig_gla_fwd_beta(q, k, v, gate, bgate, wl.grid_h, wl.grid_w, wl.chunk, direction)
+        grads = dig.dig_gla_bwd_beta(q, k, v, gate, bgate, dO, wl.grid_h, wl.grid_w, wl.chunk, direction)
+        torch.cuda.synchronize()
+        assert dig.dig_last_device_status() == dig.DIG_OK
+        assert all(t.dtype == torch.float32 for t in (out, *grads))
+        errs = {n: rel_err(t.cpu().numpy(), r) for n, t, r in zip(("out", "dq", "dk", "dv", "dgate", "dbgate"), (out, *grads), (ro, *rg))}
+        assert all(np.isfinite(e) and e <= TOL_F32 for e in errs.values()), errs
+        return errs
     res = {}
     for f32_out in (True, False):
         out = dig.dig_gla_fwd_beta(q, k, v, gate, bgate, wl.grid_h, wl.grid_w, wl.chunk, direction, f32_out=f32_out)
@@ -88,8 +100,21 @@ def test_beta_one_equals_the_alpha_only_entry_point():
         assert rel_err(x1.cpu().numpy(), x2.cpu().numpy().astype("float64")) <= TOL_BF16
 
 
-def test_fp32_storage_is_refused():
+@pytest.mark.parametrize("direction", [0, 1, 2, 3])
+def test_fp32_storage_small_ragged_all_directions(direction):
+    wl = Workload("beta32", B=2, H=3, grid_h=7, grid_w=9, d_k=24, d_v=40, chunk=16, dtype="f32", backward=True,
+                  tau=(16.0, 2.0, 1.0), seed=35)
+    print(_run(wl, direction, 10 + direction))
+
+
+@pytest.mark.parametrize("d,chunk", [(64, 64), (72, 64), (64, 32)])
+def test_fp32_storage_head_and_chunk_sizes(d, chunk):
+    wl = Workload("beta32", B=1, H=2, grid_h=20, grid_w=13, d_k=d, d_v=d, chunk=chunk, dtype="f32", backward=True,
+                  tau=(16.0, 4.0), seed=36)
+    print(_run(wl, 1, 7))
+
+
+def test_fp32_storage_alpha_only_stays_with_the_fma_family():
+    """Without the value-channel gate, fp32 storage is served by the fp32 FMA kernels."""
     from paper_2405_18428_b200 import dig
-    q = torch.zeros(1, 16, 1, 8, device="cuda")
-    with pytest.raises(dig.DigError):
-        dig.dig_gla_fwd_beta(q, q, q, q, q, 4, 4, 16, 0)
+    assert dig.dig_gla_query_impl(64, 64, 64, dig.DIG_F32, 1) == dig.DIG_IMPL_FMA
