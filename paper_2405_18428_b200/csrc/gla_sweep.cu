@@ -152,7 +152,7 @@ struct LocalSmem {
     static constexpr int kTilesPad = kTiles;
     static_assert(!C::BIGM || 16 * C::CHT <= 2 * C::TILE_T, "an M = 128 operand must stay inside the tile area");
     static constexpr int kFloats = T * C::LAMP + L::NSEG * D + 8 * D;
-    static constexpr size_t bytes = kTilesPad + kFloats * 4 + 3 * T * 4 + sizeof(Ctl);
+    static constexpr size_t bytes = kTilesPad + kFloats * 4 + 4 * T * 4 + sizeof(Ctl);
     static constexpr uint32_t tmem_cols = C::BIGM ? (BWD ? 256 : 128) : (BWD ? 64 : 32);
 };
 
@@ -168,7 +168,7 @@ sweep_local(const SweepArgs a)
     float *table = reinterpret_cast<float *>(smem + SM::kTilesPad);
     float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D;
     int *rowOff = reinterpret_cast<int *>(vecb + 8 * D);
-    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 3 * T);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 4 * T);
     constexpr uint32_t aU = 0, aW = C::BIGM ? C::NACC : D / 2;
 
     const int tid = threadIdx.x;
@@ -198,7 +198,7 @@ sweep_local(const SweepArgs a)
         __syncthreads();
         load_raw<D, NT, BWD, BWD>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
         for (int tile = t0; tile < t1; ++tile) {
-            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
+            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) & 3;
             if (tid < T) {
                 rowOff[nxt * T + tid] = tile + 1 < t1 ? tile_row_offset(g, b, h, D, tile + 1, tid) : -1;
                 // this kernel's tiles are short: the register prefetch alone does not cover the memory latency
@@ -437,7 +437,7 @@ struct FwdSmem {
     using L = Lay<D, NT>;
     static constexpr int kTiles = 3 * C::TILE_T + C::TILE_S + C::TILE_P;      // tQ tK tV tS tP
     static constexpr int kFloats = T * C::LAMP + L::NSEG * D + 8 * D;
-    static constexpr size_t bytes = kTiles + kFloats * 4 + 3 * T * 4 + sizeof(Ctl);
+    static constexpr size_t bytes = kTiles + kFloats * 4 + 4 * T * 4 + sizeof(Ctl);
     static constexpr uint32_t tmem_cols = C::BIGM ? 256 : 128;
 };
 
@@ -453,7 +453,7 @@ sweep_fwd(const SweepArgs a)
     float *table = reinterpret_cast<float *>(smem + SM::kTiles);
     float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D;
     int *rowOff = reinterpret_cast<int *>(vecb + 8 * D);
-    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 3 * T);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 4 * T);
     // the state product is issued after the scores have been read and reuses their columns
     constexpr uint32_t aP = 0, aO = C::BIGM ? C::NACC : 64, aU = aP;
     static_assert(aO + C::NACC <= SM::tmem_cols, "tensor memory");
@@ -496,7 +496,7 @@ sweep_fwd(const SweepArgs a)
             load_raw<D, NT, true, false>(raw, a.q, a.k, a.v, nullptr, a.gate, rowOff + cur * T);
         }
         for (int tile = t0; tile < t1; ++tile) {
-            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
+            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) & 3;
             if (tid < T) rowOff[nxt * T + tid] = tile + 1 < t1 ? tile_row_offset(g, b, h, D, tile + 1, tid) : -1;
             write_gates<D, NT, true, false>(raw, table, rowOff + cur * T);
             __syncthreads();
@@ -617,7 +617,7 @@ struct BwdSmem {
     using L = Lay<D, NT>;
     static constexpr int kTiles = 4 * C::TILE_T + 3 * C::TILE_S + 2 * C::TILE_P;      // tQ tK tV tG | tS tI tD | tP tdP
     static constexpr int kFloats = T * C::LAMP + L::NSEG * D + 8 * D + 2 * D;
-    static constexpr size_t bytes = kTiles + kFloats * 4 + 3 * T * 4 + sizeof(Ctl);
+    static constexpr size_t bytes = kTiles + kFloats * 4 + 4 * T * 4 + sizeof(Ctl);
     static constexpr uint32_t tmem_cols = 256;
 };
 
@@ -635,7 +635,7 @@ sweep_bwd(const SweepArgs a)
     float *table = reinterpret_cast<float *>(smem + SM::kTiles);
     float *sTot = table + T * C::LAMP, *vecb = sTot + L::NSEG * D, *sCarry = vecb + 8 * D;
     int *rowOff = reinterpret_cast<int *>(sCarry + 2 * D);
-    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 3 * T);
+    Ctl *ctl = reinterpret_cast<Ctl *>(rowOff + 4 * T);
     constexpr uint32_t W0 = C::BIGM ? C::NACC : 64;
     constexpr uint32_t aP = 0, aQK = W0, aV = W0 + C::NACC, kHi = 16u << 16;
     static_assert(aV + C::NACC <= SM::tmem_cols, "tensor memory");
@@ -657,16 +657,15 @@ sweep_bwd(const SweepArgs a)
     const int total = g.B * g.H * pl.nseg;
     TO *dq = reinterpret_cast<TO *>(a.dq), *dk = reinterpret_cast<TO *>(a.dk), *dv = reinterpret_cast<TO *>(a.dv);
 
-    {
-        const int sid = blockIdx.x;
-        if (sid < total) {
-            const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg, b = bh / g.H, h = bh - b * g.H;
-            const int t1 = min(sg * pl.G + pl.G, pl.ntile);
-            if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, t1 - 1, tid);
-            __syncthreads();
-            load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
-        }
-    }
+    // the first tile's rows are inputs of the call: their loads need not wait for the scan kernel
+    auto prime = [&](int sid) {
+        const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg, b = bh / g.H, h = bh - b * g.H;
+        const int t1 = min(sg * pl.G + pl.G, pl.ntile);
+        if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, t1 - 1, tid);
+        __syncthreads();
+        load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
+    };
+    if ((int)blockIdx.x < total) prime(blockIdx.x);
     pdl_wait();
     pdl_launch_dependents();
     for (int sid = blockIdx.x; sid < total; sid += gridDim.x) {
@@ -674,11 +673,7 @@ sweep_bwd(const SweepArgs a)
         const int t0 = sg * pl.G, t1 = min(t0 + pl.G, pl.ntile);
         load_state<D, NT>(a.seg_dstate + (size_t)sid * D * D, sm, Dst);
         if (tid < D) sCarry[cpar * D + tid] = a.seg_carry[(size_t)sid * D + tid];
-        if (sid != (int)blockIdx.x) {
-            if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, t1 - 1, tid);
-            __syncthreads();
-            load_raw<D, NT, true, true>(raw, a.q, a.k, a.v, a.d_out, a.gate, rowOff + cur * T);
-        }
+        if (sid != (int)blockIdx.x) prime(sid);
         if (tid == kIssuer) {
             // the zero-start state of the sub-chunk worked first (always slot 0 of its tile) and, once per
             // segment, the state entering the segment; later sub-chunks' states are fetched as soon as the
@@ -692,7 +687,7 @@ sweep_bwd(const SweepArgs a)
             }
         }
         for (int tile = t1 - 1; tile >= t0; --tile) {
-            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) % 3;
+            const int nrow = min(T, g.L - tile * T), nxt = (cur + 1) & 3;
             if (tid < T) rowOff[nxt * T + tid] = tile > t0 ? tile_row_offset(g, b, h, D, tile - 1, tid) : -1;
             write_gates<D, NT, true, true>(raw, table, rowOff + cur * T);
             __syncthreads();
