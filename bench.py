@@ -484,6 +484,85 @@ def multi_direction_entry(wl, torch, dig, flush, reps=20):
                                            "and round once, at the price of fp32 read-add-store traffic on the outputs"}}
 
 
+def next_rows_entry(torch, dig, peaks, flush, reps=20):
+    """The operators beyond the timed step, each timed alone (median of `reps` single calls, L2 flushed before
+    each): conv backward, output gate forward / backward, the full gate alpha^T beta forward + backward, and a
+    forward pass cut in two pieces that hand the state over.  Algorithmic bytes are the tensors each one must
+    read and write once (bf16 tensors, fp32 gates and parameter gradients neglected)."""
+    from paper_2405_18428_b200.inputs import CONFIGS, make_inputs
+    out = {}
+    hbm = peaks["hbm_gbs"]
+
+    def entry(run, alg_bytes, extra=None):
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize()
+        t = median_single(run, torch, reps, flush)
+        gbs = alg_bytes / (t["median_ms"] * 1e-3) / 1e9
+        e = {**t, "algorithmic_bytes": alg_bytes, "achieved_gbs": gbs, "hbm_frac": gbs / hbm, "peak_source": peaks["source"]}
+        if extra:
+            e.update(extra)
+        return e
+
+    # conv backward and output gate on the shape of the largest config (16384 tokens x 1152 channels)
+    wl = CONFIGS["C5"]
+    D = wl.H * wl.d_v
+    n = wl.B * wl.L * D
+    g = torch.Generator(device="cuda").manual_seed(5)
+    x = torch.randn(wl.B, wl.L, D, device="cuda", generator=g).to(torch.bfloat16)
+    dy = torch.randn(wl.B, wl.L, D, device="cuda", generator=g).to(torch.bfloat16)
+    w = (torch.randn(3, 3, D, device="cuda", generator=g) / 3).to(torch.bfloat16)
+    out["conv_backward"] = entry(lambda: dig.dig_srem_dwconv_bwd(x, w, dy, wl.grid_h, wl.grid_w, 0),
+                                 6 * n, {"shape": [wl.B, wl.grid_h, wl.grid_w, D], "bytes_model": "x, dy read, dx written: 6 B per element"})
+    o = x.view(wl.B, wl.L, wl.H, wl.d_v)
+    r = dy.view(wl.B, wl.L, wl.H, wl.d_v)
+    dz = torch.randn(wl.B, wl.L, wl.H, wl.d_v, device="cuda", generator=g).to(torch.bfloat16)
+    ln_w = torch.ones(wl.d_v, device="cuda")
+    ln_b = torch.zeros(wl.d_v, device="cuda")
+    out["output_gate_forward"] = entry(lambda: dig.dig_gla_outgate_fwd(o, r, ln_w, ln_b), 6 * n,
+                                       {"shape": [wl.B, wl.L, wl.H, wl.d_v], "bytes_model": "o, r read, z written: 6 B per element"})
+    out["output_gate_backward"] = entry(lambda: dig.dig_gla_outgate_bwd(o, r, dz, ln_w, ln_b), 10 * n,
+                                        {"shape": [wl.B, wl.L, wl.H, wl.d_v], "bytes_model": "o, r, dz read, d_o, d_r written: 10 B per element"})
+    del x, dy, w, o, r, dz
+    torch.cuda.empty_cache()
+
+    # the full gate (served by the warp-level tensor-core family) and the state hand-over, on the 4096-token config
+    wl = CONFIGS["C3"]
+    xin = make_inputs(wl, conv=False)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(torch.bfloat16)
+    q, k, v, gg, dO = (dev(xin[m]) for m in ("q", "k", "v", "g", "dO"))
+    gate = dig.dig_gate_logsigmoid(gg, xin["tau"])
+    bgate = dig.dig_gate_logsigmoid(dev(xin["g"][..., ::-1]), xin["tau"])       # d_k = d_v here: the key gate's logits, channels reversed
+    th = wl.B * wl.L * wl.H
+    fwd_b, bwd_b = bytes_per_token_head(wl)
+    beta_bytes = th * (fwd_b + bwd_b + 4 * wl.d_v * 3)        # bgate read by both passes, dbgate written
+
+    def beta():
+        dig.dig_gla_fwd_beta(q, k, v, gate, bgate, wl.grid_h, wl.grid_w, wl.chunk, 0)
+        dig.dig_gla_bwd_beta(q, k, v, gate, bgate, dO, wl.grid_h, wl.grid_w, wl.chunk, 0)
+
+    def alpha_only():
+        dig.dig_gla_fwd(q, k, v, gate, wl.grid_h, wl.grid_w, wl.chunk, 0)
+        dig.dig_gla_bwd(q, k, v, gate, dO, wl.grid_h, wl.grid_w, wl.chunk, 0)
+
+    out["full_gate_fwd_bwd"] = entry(beta, beta_bytes, {"workload": wl.name, "kernel_family": "mma", "tokens_per_s": None})
+    out["full_gate_fwd_bwd"]["tokens_per_s"] = wl.B * wl.L / (out["full_gate_fwd_bwd"]["median_ms"] * 1e-3)
+    out["full_gate_fwd_bwd"]["alpha_only_same_config"] = entry(alpha_only, th * (fwd_b + bwd_b), {"kernel_family": "tensor"})
+
+    # forward pass of the first and the second half of the rows of the grid, the state of the first handed to the second
+    half = wl.grid_h // 2
+    Lh = half * wl.grid_w
+    parts = [tuple(t[:, :Lh].contiguous() for t in (q, k, v, gate)), tuple(t[:, Lh:].contiguous() for t in (q, k, v, gate))]
+
+    def two_pieces():
+        _, s = dig.dig_gla_fwd_state(*parts[0], None, half, wl.grid_w, wl.chunk, 0, want_s_out=True)
+        dig.dig_gla_fwd_state(*parts[1], s, wl.grid_h - half, wl.grid_w, wl.chunk, 0, want_s_out=False)
+
+    out["state_handover_forward"] = entry(two_pieces, th * fwd_b, {"workload": wl.name, "pieces": 2})
+    out["state_handover_forward"]["one_call"] = entry(lambda: dig.dig_gla_fwd(q, k, v, gate, wl.grid_h, wl.grid_w, wl.chunk, 0), th * fwd_b)
+    return out
+
+
 def cpu_baseline(wl, budget_s=16.0, threads=None):
     """The fp64 oracle, as it stands, on a bounded sample of the workload: whole (batch, head)
     pairs, every scan direction of the workload, gate + fwd + bwd (+ conv on those batches)."""
@@ -655,6 +734,7 @@ def main():
                 continue
             sweep[name] = sweep_entry(name, CONFIGS[base].scaled(**over), torch, dig, peaks, local, flush)
         sweep["multi"] = multi_direction_entry(CONFIGS["C2"], torch, dig, flush)
+        sweep["next_rows"] = next_rows_entry(torch, dig, peaks, flush)
         sweep["note"] = ("one whole step of each workload per timing (its scan directions and conv), captured as a CUDA graph; "
                          "cold = 256 MB written before every timing, warm = back to back; median of 20; roofline from the cold step; "
                          "the tcgen05 kernels work on 64-token tiles for every requested chunk size (tile_executed)")

@@ -1,9 +1,9 @@
 // Output gate of the GLA layer (Eq. attn_gla, the line that forms Y_t before the projection W_O):
 //     z = Swish(r) (.) LN(o)      per (token, head) row of d_v values,
 // and its reverse mode.  Elementwise plus two row reductions, so bandwidth-bound: a row is held by 8
-// (d_v <= 64) or 16 lanes of a warp with 8 consecutive values each (16-byte loads of bf16, 2 x 16 of
-// fp32), the row statistics come from shuffles inside that lane group, every tensor is read once and
-// written once.  The affine gradients are summed per CTA in registers and shared memory and then
+// (d_v <= 64), 9 (d_v = 72: three rows per warp, five lanes idle) or 16 lanes of a warp with 8
+// consecutive values each (16-byte loads of bf16, 2 x 16 of fp32), the row statistics come from
+// shuffles inside that lane group, every tensor is read once and written once.  The affine gradients are summed per CTA in registers and shared memory and then
 // across CTAs by a second kernel in a fixed order.
 #include "dig_common.cuh"
 
@@ -14,7 +14,7 @@ constexpr int kThreads = 256;
 // Grid caps (measured): the reverse kernel does best with as many CTAs as stay resident together, three
 // per SM at its register count, so that the grid-stride loops end together and not in a ragged last
 // wave; the forward kernel does best with eight per SM.
-constexpr int kSMs = 148, kFwdPerSM = 8, kBwdPerSM = 3;
+constexpr int kFwdPerSM = 8, kBwdPerSM = 3;
 
 __device__ __forceinline__ void load8(const float *p, float (&f)[8])
 {
@@ -47,28 +47,56 @@ __device__ __forceinline__ void store8(__nv_bfloat16 *p, const float (&f)[8])
     *reinterpret_cast<uint4 *>(p) = u;
 }
 
-template <int LPR> __device__ __forceinline__ float group_sum(float x)
+// Thread -> (row slot of the CTA, lane of the row's group): 32 / LPR rows per warp.
+template <int LPR>
+struct RowMap {
+    static constexpr int kRowsPerWarp = 32 / LPR, kRows = (kThreads / 32) * kRowsPerWarp;
+    int lane, slot, gbase;      // lane in the group, row slot, first warp lane of the group
+    bool valid;                 // false for the warp's left-over lanes when LPR is not a power of two
+    __device__ __forceinline__ RowMap()
+    {
+        const int l = threadIdx.x & 31, grp = l / LPR;
+        lane = l - grp * LPR;
+        gbase = grp * LPR;
+        valid = grp < kRowsPerWarp;
+        slot = (threadIdx.x >> 5) * kRowsPerWarp + (valid ? grp : 0);
+    }
+};
+// Sum over the row's lane group, returned to all of its lanes.  Power-of-two groups: butterfly.  Nine
+// lanes: the ninth is folded into the first, a butterfly over the first eight, then a broadcast.
+template <int LPR> __device__ __forceinline__ float group_sum(float x, const RowMap<LPR> &m)
 {
+    if ((LPR & (LPR - 1)) == 0) {
 #pragma unroll
-    for (int m = LPR / 2; m >= 1; m >>= 1) x += __shfl_xor_sync(0xffffffffu, x, m);
-    return x;
+        for (int k = LPR / 2; k >= 1; k >>= 1) x += __shfl_xor_sync(0xffffffffu, x, k);
+        return x;
+    }
+    static_assert((LPR & (LPR - 1)) == 0 || LPR == 9, "lane groups of a power of two or of nine");
+    const float y = __shfl_sync(0xffffffffu, x, min(m.gbase + 8, 31));
+    if (m.lane == 0) x += y;
+#pragma unroll
+    for (int k = 4; k >= 1; k >>= 1) {
+        const float t = __shfl_sync(0xffffffffu, x, min(m.gbase + ((m.lane ^ k) & 7), 31));
+        if (m.lane < 8) x += t;
+    }
+    return __shfl_sync(0xffffffffu, x, m.gbase);
 }
 
 // Normalised row n = (o - mean) * rstd of the lane's 8 columns (zero where the lane holds none).
 template <int LPR> __device__ __forceinline__ float normalise(const float (&o)[8], bool has, float inv_d, float eps,
-                                                               float (&n)[8])
+                                                               float (&n)[8], const RowMap<LPR> &m)
 {
     float s = 0.f;
 #pragma unroll
     for (int e = 0; e < 8; ++e) s += o[e];
-    const float mean = group_sum<LPR>(s) * inv_d;
+    const float mean = group_sum<LPR>(s, m) * inv_d;
     float v = 0.f;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         n[e] = has ? o[e] - mean : 0.f;
         v = fmaf(n[e], n[e], v);
     }
-    const float rstd = rsqrtf(group_sum<LPR>(v) * inv_d + eps);
+    const float rstd = rsqrtf(group_sum<LPR>(v, m) * inv_d + eps);
 #pragma unroll
     for (int e = 0; e < 8; ++e) n[e] *= rstd;
     return rstd;
@@ -84,9 +112,10 @@ __global__ void __launch_bounds__(kThreads)
 outgate_fwd(const TA *o, const TR *__restrict__ r, const float *__restrict__ ln_w,
             const float *__restrict__ ln_b, TZ *z, long long rows, int dv, float eps)
 {
-    constexpr int kRows = kThreads / LPR;
-    const int lane = threadIdx.x % LPR, slot = threadIdx.x / LPR, col = lane * 8;
-    const bool has_col = col < dv;
+    constexpr int kRows = RowMap<LPR>::kRows;
+    const RowMap<LPR> rm;
+    const int slot = rm.slot, col = rm.lane * 8;
+    const bool has_col = rm.valid && col < dv;
     const float inv_d = 1.f / (float)dv;
     float w[8], b[8];
 #pragma unroll
@@ -104,7 +133,7 @@ outgate_fwd(const TA *o, const TR *__restrict__ r, const float *__restrict__ ln_
             load8(o + row * dv + col, ov);
             load8(r + row * dv + col, rv);
         }
-        normalise<LPR>(ov, has, inv_d, eps, n);
+        normalise<LPR>(ov, has, inv_d, eps, n, rm);
         float out[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) out[e] = rv[e] * sigmoidf(rv[e]) * fmaf(n[e], w[e], b[e]);
@@ -118,10 +147,11 @@ outgate_bwd(const TI *__restrict__ o, const TI *__restrict__ r, const TI *__rest
             const float *__restrict__ ln_w, const float *__restrict__ ln_b, TO *__restrict__ d_o,
             TO *__restrict__ d_r, float *__restrict__ partial, long long rows, int dv, float eps)
 {
-    constexpr int kRows = kThreads / LPR;
+    constexpr int kRows = RowMap<LPR>::kRows;
     __shared__ float red[kRows][2][LPR * 8];
-    const int lane = threadIdx.x % LPR, slot = threadIdx.x / LPR, col = lane * 8;
-    const bool has_col = col < dv;
+    const RowMap<LPR> rm;
+    const int slot = rm.slot, col = rm.lane * 8;
+    const bool has_col = rm.valid && col < dv;
     const float inv_d = 1.f / (float)dv;
     float w[8], b[8], aw[8], ab[8];
 #pragma unroll
@@ -141,7 +171,7 @@ outgate_bwd(const TI *__restrict__ o, const TI *__restrict__ r, const TI *__rest
             load8(r + row * dv + col, rv);
             load8(dz + row * dv + col, gv);
         }
-        const float rstd = normalise<LPR>(ov, has, inv_d, eps, n);
+        const float rstd = normalise<LPR>(ov, has, inv_d, eps, n, rm);
         float dr[8], dn[8], s1 = 0.f, s2 = 0.f;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
@@ -155,7 +185,7 @@ outgate_bwd(const TI *__restrict__ o, const TI *__restrict__ r, const TI *__rest
             s1 += dn[e];
             s2 = fmaf(dn[e], n[e], s2);
         }
-        const float m1 = group_sum<LPR>(s1) * inv_d, m2 = group_sum<LPR>(s2) * inv_d;
+        const float m1 = group_sum<LPR>(s1, rm) * inv_d, m2 = group_sum<LPR>(s2, rm) * inv_d;
         float dov[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) dov[e] = rstd * (dn[e] - m1 - n[e] * m2);
@@ -165,10 +195,12 @@ outgate_bwd(const TI *__restrict__ o, const TI *__restrict__ r, const TI *__rest
         }
     }
     if (partial == nullptr) return;
+    if (rm.valid) {
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        red[slot][0][col + e] = aw[e];
-        red[slot][1][col + e] = ab[e];
+        for (int e = 0; e < 8; ++e) {
+            red[slot][0][col + e] = aw[e];
+            red[slot][1][col + e] = ab[e];
+        }
     }
     __syncthreads();
     // partial[cta][2][dv]
@@ -199,10 +231,14 @@ outgate_affine_sum(const float *__restrict__ partial, float *__restrict__ dln_w,
     }
 }
 
+// lanes per row for a row length
+int lanes_for(int dv) { return dv <= 64 ? 8 : dv == 72 ? 9 : 16; }
 int grid_for(long long rows, int lpr, int per_sm = kBwdPerSM)
 {
-    const int kMaxCtas = kSMs * per_sm;
-    const long long per = kThreads / lpr, need = (rows + per - 1) / per;
+    int sms = device_sm_count();
+    if (sms <= 0) sms = 148;            // sizing call without a device: the count the launch will most likely see
+    const int kMaxCtas = sms * per_sm;
+    const long long per = (kThreads / 32) * (32 / lpr), need = (rows + per - 1) / per;
     return (int)(need < kMaxCtas ? need : kMaxCtas);
 }
 
@@ -212,6 +248,9 @@ void fwd_dispatch3(const void *o, const void *r, const float *w, const float *b,
 {
     if (dv <= 64)
         launch_pdl(outgate_fwd<TA, TR, TZ, 8>, dim3(grid_for(rows, 8, kFwdPerSM)), dim3(kThreads), 0, stream, (const TA *)o,
+                   (const TR *)r, w, b, (TZ *)z, rows, dv, eps);
+    else if (dv == 72)
+        launch_pdl(outgate_fwd<TA, TR, TZ, 9>, dim3(grid_for(rows, 9, kFwdPerSM)), dim3(kThreads), 0, stream, (const TA *)o,
                    (const TR *)r, w, b, (TZ *)z, rows, dv, eps);
     else
         launch_pdl(outgate_fwd<TA, TR, TZ, 16>, dim3(grid_for(rows, 16, kFwdPerSM)), dim3(kThreads), 0, stream, (const TA *)o,
@@ -231,6 +270,9 @@ void bwd_dispatch(const void *o, const void *r, const void *dz, const float *w, 
     if (dv <= 64)
         launch_pdl(outgate_bwd<TI, TO, 8>, dim3(grid_for(rows, 8)), dim3(kThreads), 0, stream, (const TI *)o,
                    (const TI *)r, (const TI *)dz, w, b, (TO *)d_o, (TO *)d_r, partial, rows, dv, eps);
+    else if (dv == 72)
+        launch_pdl(outgate_bwd<TI, TO, 9>, dim3(grid_for(rows, 9)), dim3(kThreads), 0, stream, (const TI *)o,
+                   (const TI *)r, (const TI *)dz, w, b, (TO *)d_o, (TO *)d_r, partial, rows, dv, eps);
     else
         launch_pdl(outgate_bwd<TI, TO, 16>, dim3(grid_for(rows, 16)), dim3(kThreads), 0, stream, (const TI *)o,
                    (const TI *)r, (const TI *)dz, w, b, (TO *)d_o, (TO *)d_r, partial, rows, dv, eps);
@@ -240,7 +282,7 @@ void bwd_dispatch(const void *o, const void *r, const void *dz, const float *w, 
 
 size_t outgate_bwd_workspace_bytes(long long rows, int dv)
 {
-    return (size_t)grid_for(rows, dv <= 64 ? 8 : 16) * 2 * (size_t)dv * sizeof(float);
+    return (size_t)grid_for(rows, lanes_for(dv)) * 2 * (size_t)dv * sizeof(float);
 }
 
 dig_status launch_outgate_fwd(const void *o, const void *r, const float *ln_w, const float *ln_b, void *z,
@@ -281,7 +323,7 @@ dig_status launch_outgate_bwd(const void *o, const void *r, const void *dz, cons
     if (!affine) return DIG_OK;
     KernelTimer t(KID_OUTGATE, stream);
     launch_pdl(outgate_affine_sum, dim3((2 * dv + 255) / 256), dim3(256), 0, stream, (const float *)partial, dln_w,
-               dln_b, grid_for(rows, dv <= 64 ? 8 : 16), dv);
+               dln_b, grid_for(rows, lanes_for(dv)), dv);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -149,7 +149,14 @@ def test_conv_bwd_rejects_short_workspace():
 
 @pytest.mark.parametrize("dtype,direction,bias", [("f32", 1, True), ("bf16", 2, True), ("bf16", 3, False)])
 def test_conv_many_tiles_per_cta(dtype, direction, bias):
-    """3 x 96 x 96 pixels x 136 channels: 1728 tiles, which selects the persistent double-buffered kernel
-    (ragged last channel block, every scan order's tap permutation, bf16 and fp32 storage and output)."""
+    """3 x 96 x 96 pixels x 136 channels: 1728 tiles, which selects the strip-walking kernel (8 row segments
+    per strip, ragged last channel block, every scan order's tap permutation, bf16 and fp32 storage and output)."""
     _conv_case(3, 96, 96, 136, dtype, direction, bias=bias, seed=9)
     _conv_bwd_case(3, 96, 96, 136, dtype, direction, with_bias=bias, seed=9)      # dx runs through the same kernel
+
+
+@pytest.mark.parametrize("dtype,direction", [("bf16", 0), ("f32", 3)])
+def test_conv_strips_ragged_and_persistent(dtype, direction):
+    """16 x 45 x 100 pixels x 264 channels: 13 strips per image row of which the last is 4 columns wide, a last
+    channel block of 8 channels, and more strips (624) than CTAs stay resident, so some CTAs walk two strips."""
+    _conv_case(16, 45, 100, 264, dtype, direction, bias=True, seed=11)
