@@ -263,88 +263,144 @@ srem_dwconv3x3_strip(const T *__restrict__ x, const T *__restrict__ w, const T *
 // ---- reverse mode: filter and bias gradients ------------------------------------------------------
 // dw'[u][v][c] = sum over pixels of dy[i][j][c] * x[i+u-1][j+v-1][c] (zero outside the grid), computed
 // in canonical taps and written to the stored tap the scan order maps (u, v) to; dbias = sum of dy.
-// Same tiling as the forward kernel: a CTA stages the halo tile of x and the tile of dy of TY x TX pixels
-// and one block of channels in shared memory; a thread owns 8 channels of one tile column and adds the
-// nine products of its TY pixels to 72 + 8 accumulators.  CTA y of a channel block takes the tiles
-// y, y + gridDim.y, ... in that order, then the CTA's column threads are summed in shared memory and
-// one partial sum per CTA is written; a second kernel adds the partial sums in a fixed order, so the
-// result does not depend on scheduling.
+// Same walk as the forward strip kernel: a CTA goes down strips of TX pixel columns and CH channels row
+// by row, rows of x (with the halo) and of dy arriving through cp.async rings.  A thread owns 4 channels
+// of two neighbouring columns: input row r meets the dy rows r, r - 1, r - 2 (kept in registers, g[r % 3]
+// is dy row r) in the taps u = 0, 1, 2 and adds 72 products to its 36 + 4 accumulators.  CTA y of a
+// channel block takes the strips y, y + gridDim.y, ... in that order; then the CTA's column pairs are
+// summed through shared memory and one partial sum per CTA is written; a second kernel adds the partial
+// sums in a fixed order, so the result does not depend on scheduling.  The dy rows a CTA reads are those
+// of its own row segment only (segments share halo rows of x, not output rows).
 constexpr int kWgPixels = 128;       // pixels per partial sum (sizes the workspace)
 
 template <typename T>
-__global__ void __launch_bounds__(Cfg<T>::kThreads)
+__global__ void __launch_bounds__(Cfg<T>::kThreads, 4)
 srem_dwconv_wgrad(const T *__restrict__ x, const T *__restrict__ dy, float *__restrict__ partial,
-                  int B, int gh, int gw, int D, int dir)
+                  int B, int gh, int gw, int D, int dir, int strips_x, int nseg, int seg_rows, int nstrips)
 {
     constexpr int CH = Cfg<T>::CH, kLanes = Cfg<T>::kLanes, kConvThreads = Cfg<T>::kThreads;
-    // halo tile of x and tile of dy; the same memory later holds the per-warp sums [warps][10][CH]
-    constexpr int kHalo = (TY + 2) * (TX + 2) * kLanes, kInner = TY * TX * kLanes, kWarps = kConvThreads / 32;
-    constexpr size_t kBytes = sizeof(Vec8<T>) * (kHalo + kInner) > sizeof(float) * kWarps * 10 * CH
-                                  ? sizeof(Vec8<T>) * (kHalo + kInner) : sizeof(float) * kWarps * 10 * CH;
-    __shared__ __align__(16) char sm[kBytes];
-    Vec8<T> (*tile)[TX + 2][kLanes] = reinterpret_cast<Vec8<T> (*)[TX + 2][kLanes]>(sm);
-    Vec8<T> (*gtile)[TX][kLanes] = reinterpret_cast<Vec8<T> (*)[TX][kLanes]>(sm + sizeof(Vec8<T>) * kHalo);
-    const int lane = threadIdx.x % kLanes, col = threadIdx.x / kLanes;
-    const int tiles_x = (gw + TX - 1) / TX, tiles_y = (gh + TY - 1) / TY, ntiles = B * tiles_x * tiles_y;
+    constexpr int kPieces = (int)sizeof(Vec8<T>) / 16, kQuads = CH / 4, kWarps = kConvThreads / 32;
+    constexpr int kRowX = (TX + 2) * kLanes, kRowG = TX * kLanes, kRowVecs = kRowX + kRowG;
+    constexpr int kFill = (kRowVecs + kConvThreads - 1) / kConvThreads;
+    // rings of x rows and dy rows; the same memory later holds the per-warp sums [warps][10][CH]
+    constexpr size_t kRingBytes = sizeof(Vec8<T>) * kRing * kRowVecs, kRedBytes = sizeof(float) * kWarps * 10 * CH;
+    __shared__ __align__(16) char sm[kRingBytes > kRedBytes ? kRingBytes : kRedBytes];
+    Vec8<T> (*xring)[TX + 2][kLanes] = reinterpret_cast<Vec8<T> (*)[TX + 2][kLanes]>(sm);
+    Vec8<T> (*gring)[TX][kLanes] = reinterpret_cast<Vec8<T> (*)[TX][kLanes]>(sm + sizeof(Vec8<T>) * kRing * kRowX);
+    const int quad = threadIdx.x % kQuads, c0 = 2 * (threadIdx.x / kQuads);
+    const int chb = blockIdx.x;
     pdl_wait();
     pdl_launch_dependents();
-    float acc[10][8];
+    float acc[3][3][4], accb[4];
 #pragma unroll
-    for (int k = 0; k < 10; ++k)
+    for (int u = 0; u < 3; ++u)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[k][i] = 0.f;
-    for (int t = blockIdx.y; t < ntiles; t += gridDim.y) {
-        const int b = t / (tiles_x * tiles_y), r = t - b * (tiles_x * tiles_y);
-        const int y0 = (r / tiles_x) * TY, x0 = (r % tiles_x) * TX;
-        const size_t img = (size_t)b * gh * gw;
-        __syncthreads();                 // the previous tile has been consumed
-        for (int idx = threadIdx.x; idx < (TY + 2) * (TX + 2) * kLanes; idx += kConvThreads) {
-            const int l = idx % kLanes, pix = idx / kLanes;
-            const int tx = pix % (TX + 2), ty = pix / (TX + 2);
-            const int gy = y0 + ty - 1, gx = x0 + tx - 1, c = blockIdx.x * CH + l * VEC;
-            Vec8<T> v = Vec8<T>::zero();
-            if (gy >= 0 && gy < gh && gx >= 0 && gx < gw && c < D) v = Vec8<T>::load(x + (img + (size_t)gy * gw + gx) * D + c);
-            tile[ty][tx][l] = v;
+        for (int v = 0; v < 3; ++v)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[u][v][i] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) accb[i] = 0.f;
+    for (int s = blockIdx.y; s < nstrips; s += gridDim.y) {
+        const int sg = s % nseg, s1 = s / nseg, sx = s1 % strips_x, b = s1 / strips_x;
+        const int x0 = sx * TX, ys = sg * seg_rows, ye = min(ys + seg_rows, gh), nr = ye - ys + 2;
+        const T *xb = x + (size_t)b * gh * gw * D, *gb = dy + (size_t)b * gh * gw * D;
+        // this thread's vectors of a row pair (x row with halo, then dy row): columns and offsets stay the same
+        int f_off[kFill];
+        uint32_t f_dst[kFill];
+        bool f_ok[kFill], f_isx[kFill];
+#pragma unroll
+        for (int i = 0; i < kFill; ++i) {
+            const int idx = (int)threadIdx.x + i * kConvThreads;
+            const bool isx = idx < kRowX;
+            const int j = isx ? idx : idx - kRowX, l = j % kLanes, tx = j / kLanes;
+            const int gx = isx ? x0 + tx - 1 : x0 + tx, c = chb * CH + l * VEC;
+            f_isx[i] = isx;
+            f_ok[i] = idx < kRowVecs && gx >= 0 && gx < gw && c < D;
+            f_off[i] = f_ok[i] ? gx * D + c : 0;
+            f_dst[i] = idx >= kRowVecs ? 0u
+                       : isx ? (uint32_t)__cvta_generic_to_shared(&xring[0][tx][l]) : (uint32_t)__cvta_generic_to_shared(&gring[0][tx][l]);
         }
-        for (int idx = threadIdx.x; idx < TY * TX * kLanes; idx += kConvThreads) {
-            const int l = idx % kLanes, pix = idx / kLanes;
-            const int tx = pix % TX, ty = pix / TX;
-            const int gy = y0 + ty, gx = x0 + tx, c = blockIdx.x * CH + l * VEC;
-            Vec8<T> v = Vec8<T>::zero();         // pixels outside the grid contribute nothing
-            if (gy < gh && gx < gw && c < D) v = Vec8<T>::load(dy + (img + (size_t)gy * gw + gx) * D + c);
-            gtile[ty][tx][l] = v;
+        auto fill = [&](int rr) {       // x row rr of the strip (image row ys - 1 + rr) and dy row rr (image row ys + rr)
+            const int gyx = ys - 1 + rr, gyg = ys + rr;
+            const bool okx = gyx >= 0 && gyx < gh, okg = gyg < ye;
+            const T *rowx = xb + (size_t)(okx ? gyx : 0) * gw * D, *rowg = gb + (size_t)(okg ? gyg : 0) * gw * D;
+            const uint32_t slx = (uint32_t)(rr % kRing) * (uint32_t)sizeof(xring[0]), slg = (uint32_t)(rr % kRing) * (uint32_t)sizeof(gring[0]);
+#pragma unroll
+            for (int i = 0; i < kFill; ++i) {
+                if (i + 1 < kFill || (int)threadIdx.x + i * kConvThreads < kRowVecs) {
+                    const bool in = f_ok[i] && (f_isx[i] ? okx : okg);
+                    const char *src = reinterpret_cast<const char *>(in ? (f_isx[i] ? rowx : rowg) + f_off[i] : x);
+                    const uint32_t dst = f_dst[i] + (f_isx[i] ? slx : slg);
+#pragma unroll
+                    for (int p = 0; p < kPieces; ++p)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 16 * p), "l"(src + (in ? 16 * p : 0)),
+                                     "r"(in ? 16 : 0) : "memory");
+                }
+            }
+        };
+        __syncthreads();                // the previous strip's last rows have been read
+#pragma unroll
+        for (int i = 0; i < kRing - 1; ++i) {
+            if (i < nr) fill(i);
+            asm volatile("cp.async.commit_group;" ::: "memory");
         }
-        __syncthreads();
+        float g[3][2][4];
 #pragma unroll
-        for (int ty = 0; ty < TY; ++ty) {
-            float g[8];
-            gtile[ty][col][lane].unpack(g);
+        for (int r = 0; r < 3; ++r)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[9][e] += g[e];
+            for (int i = 0; i < 4; ++i) g[r][0][i] = g[r][1][i] = 0.f;
+        // One row: PH = rr % 3 is a compile-time constant so that the dy rows stay in registers.
+        auto step = [&](int rr, auto ph_tag) {
+            constexpr int PH = decltype(ph_tag)::value;
+            asm volatile("cp.async.wait_group %0;" ::"n"(kRing - 2) : "memory");      // rows rr have landed
+            __syncthreads();
+            if (rr + kRing - 1 < nr) fill(rr + kRing - 1);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            float xv[4][4];
+            const T *rowp = reinterpret_cast<const T *>(&xring[rr % kRing][0][0]) + quad * 4;
+            const T *rowg = reinterpret_cast<const T *>(&gring[rr % kRing][0][0]) + quad * 4;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const float4 t = load4(rowp + (c0 + v) * CH);
+                xv[v][0] = t.x; xv[v][1] = t.y; xv[v][2] = t.z; xv[v][3] = t.w;
+            }
+#pragma unroll
+            for (int p = 0; p < 2; ++p) {
+                const float4 t = load4(rowg + (c0 + p) * CH);       // zero past the segment's last row and past the grid
+                g[PH][p][0] = t.x; g[PH][p][1] = t.y; g[PH][p][2] = t.z; g[PH][p][3] = t.w;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) accb[i] += g[PH][p][i];
+            }
 #pragma unroll
             for (int u = 0; u < 3; ++u)
 #pragma unroll
-                for (int v = 0; v < 3; ++v) {
-                    float xv[8];
-                    tile[ty + u][col + v][lane].unpack(xv);
+                for (int p = 0; p < 2; ++p)
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[u * 3 + v][e] = fmaf(g[e], xv[e], acc[u * 3 + v][e]);
-                }
+                    for (int v = 0; v < 3; ++v)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            acc[u][v][i] = fmaf(g[(PH + 3 - u) % 3][p][i], xv[p + v][i], acc[u][v][i]);
+        };
+        for (int rr = 0; rr < nr; rr += 3) {
+            step(rr, std::integral_constant<int, 0>{});
+            if (rr + 1 < nr) step(rr + 1, std::integral_constant<int, 1>{});
+            if (rr + 2 < nr) step(rr + 2, std::integral_constant<int, 2>{});
         }
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
-    // sum over the tile columns: the columns a warp holds by shuffles (a warp is 32 / kLanes columns of all
-    // lanes), the warps through shared memory
+    // sum over the column pairs: those a warp holds by shuffles (a warp is 32 / kQuads column pairs of all
+    // quads), the warps through shared memory
     float *red = reinterpret_cast<float *>(sm);
     const int warp = threadIdx.x >> 5;
 #pragma unroll
     for (int k = 0; k < 10; ++k)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            float v = acc[k][e];
+        for (int e = 0; e < 4; ++e) {
+            float v = k < 9 ? acc[k / 3][k % 3][e] : accb[e];
 #pragma unroll
-            for (int m = kLanes; m < 32; m <<= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
-            if ((threadIdx.x & 31) < kLanes) red[(warp * 10 + k) * CH + lane * VEC + e] = v;
+            for (int m = kQuads; m < 32; m <<= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+            if ((threadIdx.x & 31) < kQuads) red[(warp * 10 + k) * CH + quad * 4 + e] = v;
         }
     __syncthreads();
     // partial[part][k][D]: k = stored tap index 0..8, 9 = bias
@@ -365,16 +421,20 @@ srem_dwconv_wgrad(const T *__restrict__ x, const T *__restrict__ dy, float *__re
     }
 }
 
+// One warp per output value: its lanes add every 32nd partial sum, then a butterfly (a fixed order).
 __global__ void __launch_bounds__(256)
 srem_dwconv_wgrad_sum(const float *__restrict__ partial, float *__restrict__ dw, float *__restrict__ dbias,
                       int nslab, int D)
 {
     pdl_wait();
     pdl_launch_dependents();
-    const int idx = blockIdx.x * 256 + threadIdx.x;
-    if (idx >= 10 * D) return;
+    const int idx = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (idx >= 10 * D) return;          // uniform over the warp
     float sum = 0.f;
-    for (int s = 0; s < nslab; ++s) sum += partial[(size_t)s * 10 * D + idx];
+    for (int s = lane; s < nslab; s += 32) sum += partial[(size_t)s * 10 * D + idx];
+#pragma unroll
+    for (int k = 16; k >= 1; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
+    if (lane != 0) return;
     if (idx < 9 * D) dw[idx] = sum;
     else if (dbias != nullptr) dbias[idx - 9 * D] = sum;
 }
@@ -458,36 +518,41 @@ dig_status launch_dwconv_bwd(const void *x, const void *w, const void *dy, void 
 {
     dig_status st = launch_dwconv(dy, w, nullptr, dx, B, gh, gw, D, dir ^ 1, dtype, stream);
     if (st != DIG_OK) return st;
-    // one partial sum per CTA row; never more rows than tiles, never more than the workspace holds
-    const int npix = B * gh * gw, ntiles = B * ((gh + TY - 1) / TY) * ((gw + TX - 1) / TX);
-    int nslab = (npix + kWgPixels - 1) / kWgPixels;
-    if (nslab > ntiles) nslab = ntiles;
-    {
-        // no more CTAs than stay resident together (three per SM at this kernel's register count), so that
-        // their tile loops end together
-        const int CHb = dtype == DIG_F32 ? Cfg<float>::CH : Cfg<__nv_bfloat16>::CH;
-        const int nchb = (D + CHb - 1) / CHb, resident = device_sm_count() * 3;
-        if (resident <= 0) return DIG_ERR_CUDA;
-        const int cap = resident / nchb > 0 ? resident / nchb : 1;
-        if (nslab > cap) nslab = cap;
-    }
-    if (nslab > 65535) return DIG_ERR_UNSUPPORTED;
+    // One partial sum per CTA row.  No more CTA rows than stay resident together (four CTAs per SM at this
+    // kernel's register count) so that their strip loops end together, never more than the workspace holds;
+    // strips are cut into row segments until every CTA row has one.
+    const int CHb = dtype == DIG_F32 ? Cfg<float>::CH : Cfg<__nv_bfloat16>::CH;
+    const int nchb = (D + CHb - 1) / CHb, resident = device_sm_count() * 4;
+    if (resident <= 0) return DIG_ERR_CUDA;
+    const long long npix = (long long)B * gh * gw;
+    long long nslab = (npix + kWgPixels - 1) / kWgPixels;
+    const int cap = resident / nchb > 0 ? resident / nchb : 1;
+    if (nslab > cap) nslab = cap;
+    const int strips_x = (gw + TX - 1) / TX;
+    const long long base = (long long)B * strips_x;
+    int nseg = (int)(nslab / base);                                 // rounded down: no CTA row gets a second strip while others have one
+    if (nseg > (gh + 7) / 8) nseg = (gh + 7) / 8;                   // segments of at least 8 rows
+    if (nseg < 1) nseg = 1;
+    const int seg_rows = (gh + nseg - 1) / nseg;
+    nseg = (gh + seg_rows - 1) / seg_rows;
+    const long long nstrips = base * nseg;
+    if (nslab > nstrips) nslab = nstrips;
+    if (nslab > 65535 || nstrips >= (1ll << 31)) return DIG_ERR_UNSUPPORTED;
     {
         KernelTimer t(KID_DWCONV_WGRAD, stream);
-        if (dtype == DIG_F32) {
-            const dim3 grid((D + Cfg<float>::CH - 1) / Cfg<float>::CH, nslab);
-            launch_pdl(srem_dwconv_wgrad<float>, grid, dim3(Cfg<float>::kThreads), 0, stream,
-                       (const float *)x, (const float *)dy, partial, B, gh, gw, D, dir);
-        } else {
-            const dim3 grid((D + Cfg<__nv_bfloat16>::CH - 1) / Cfg<__nv_bfloat16>::CH, nslab);
+        const dim3 grid(nchb, (unsigned)nslab);
+        if (dtype == DIG_F32)
+            launch_pdl(srem_dwconv_wgrad<float>, grid, dim3(Cfg<float>::kThreads), 0, stream, (const float *)x, (const float *)dy,
+                       partial, B, gh, gw, D, dir, strips_x, nseg, seg_rows, (int)nstrips);
+        else
             launch_pdl(srem_dwconv_wgrad<__nv_bfloat16>, grid, dim3(Cfg<__nv_bfloat16>::kThreads), 0, stream,
-                       (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)dy, partial, B, gh, gw, D, dir);
-        }
+                       (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)dy, partial, B, gh, gw, D, dir, strips_x, nseg, seg_rows,
+                       (int)nstrips);
     }
     if (cudaGetLastError() != cudaSuccess) return DIG_ERR_CUDA;
     KernelTimer t(KID_DWCONV_WGRAD, stream);
-    launch_pdl(srem_dwconv_wgrad_sum, dim3((10 * D + 255) / 256), dim3(256), 0, stream, (const float *)partial, dw, dbias,
-               nslab, D);
+    launch_pdl(srem_dwconv_wgrad_sum, dim3((10 * D + 7) / 8), dim3(256), 0, stream, (const float *)partial, dw, dbias,
+               (int)nslab, D);
     return cuda_ok(cudaGetLastError());
 }
 

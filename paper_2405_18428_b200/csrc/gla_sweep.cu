@@ -22,7 +22,7 @@
 // dO Sc^T = dO Sc_local^T + (dO S_segment^T) diag(exp(c) G): two products and one fused multiply-add.
 //
 // Every product is a tcgen05.mma (kind::f16, fp16 operands, fp32 accumulators in tensor memory)
-// issued by thread 0, which otherwise works like the others: all threads build operand tiles, mask
+// issued by lane 0 of the last warp, which otherwise works like the others: all threads build operand tiles, mask
 // the scores and post-process accumulators, phase by phase.  Token rows of the next tile are
 // prefetched into registers; at d = 64 two CTAs of 256 threads share an SM, so one builds while the
 // other's products are in the tensor pipe.

@@ -102,7 +102,8 @@ template <int LPR> __device__ __forceinline__ float normalise(const float (&o)[8
     return rstd;
 }
 
-__device__ __forceinline__ float sigmoidf(float r) { return 1.f / (1.f + __expf(-r)); }
+// 1 / (1 + e^-r) with the fast exponential and the fast reciprocal (2 ulp each; e^-r = inf gives 0)
+__device__ __forceinline__ float sigmoidf(float r) { return __fdividef(1.f, 1.f + __expf(-r)); }
 
 // TA: type of o (the GLA output: input storage type when it comes from memory written by a caller, output
 // storage type when it comes straight from the forward pass), TR: type of r, TZ: type of z.  o and z may
@@ -214,16 +215,21 @@ outgate_bwd(const TI *__restrict__ o, const TI *__restrict__ r, const TI *__rest
     }
 }
 
+// One warp per parameter: its lanes add every 32nd partial sum, then a butterfly (a fixed order, so the
+// result does not depend on scheduling).
 __global__ void __launch_bounds__(256)
 outgate_affine_sum(const float *__restrict__ partial, float *__restrict__ dln_w, float *__restrict__ dln_b,
                    int nctas, int dv)
 {
     pdl_wait();
     pdl_launch_dependents();
-    const int idx = blockIdx.x * 256 + threadIdx.x;
-    if (idx >= 2 * dv) return;
+    const int idx = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (idx >= 2 * dv) return;          // uniform over the warp
     float sum = 0.f;
-    for (int s = 0; s < nctas; ++s) sum += partial[(size_t)s * 2 * dv + idx];
+    for (int s = lane; s < nctas; s += 32) sum += partial[(size_t)s * 2 * dv + idx];
+#pragma unroll
+    for (int k = 16; k >= 1; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
+    if (lane != 0) return;
     if (idx < dv) {
         if (dln_w != nullptr) dln_w[idx] = sum;
     } else if (dln_b != nullptr) {
@@ -322,7 +328,7 @@ dig_status launch_outgate_bwd(const void *o, const void *r, const void *dz, cons
     if (cudaGetLastError() != cudaSuccess) return DIG_ERR_CUDA;
     if (!affine) return DIG_OK;
     KernelTimer t(KID_OUTGATE, stream);
-    launch_pdl(outgate_affine_sum, dim3((2 * dv + 255) / 256), dim3(256), 0, stream, (const float *)partial, dln_w,
+    launch_pdl(outgate_affine_sum, dim3((2 * dv + 7) / 8), dim3(256), 0, stream, (const float *)partial, dln_w,
                dln_b, grid_for(rows, lanes_for(dv)), dv);
     return cuda_ok(cudaGetLastError());
 }

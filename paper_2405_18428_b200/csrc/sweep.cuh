@@ -54,7 +54,7 @@ struct Cfg {
     static_assert(BIGM || (NCH % 2 == 0), "heads of at most 64 channels split their state products in two halves");
 };
 
-// Work split of a CTA of NT threads (thread 0 also issues the MMAs and the bulk copies).
+// Work split of a CTA of NT threads (lane 0 of the last warp also issues the MMAs and the bulk copies).
 template <int D, int NT>
 struct Lay {
     using C = Cfg<D>;
