@@ -160,3 +160,12 @@ def test_conv_strips_ragged_and_persistent(dtype, direction):
     """16 x 45 x 100 pixels x 264 channels: 13 strips per image row of which the last is 4 columns wide, a last
     channel block of 8 channels, and more strips (624) than CTAs stay resident, so some CTAs walk two strips."""
     _conv_case(16, 45, 100, 264, dtype, direction, bias=True, seed=11)
+    _conv_bwd_case(16, 45, 100, 264, dtype, direction, with_bias=True, seed=11)      # dx by the same kernel, dw by the strip walk of x and dy
+
+
+@pytest.mark.parametrize("gh,gw", [(2, 2048), (1, 4100), (300, 9)])
+def test_conv_strips_flat_and_narrow_grids(gh, gw):
+    """Grids of one or two rows (a strip is then only halo rows plus them) and grids narrower than two strips,
+    large enough in the other extent to select the strip-walking kernels."""
+    _conv_case(8, gh, gw, 136, "bf16", 2, bias=True, seed=12)
+    _conv_bwd_case(8, gh, gw, 136, "bf16", 1, with_bias=True, seed=12)
