@@ -733,6 +733,10 @@ def main():
             if base == wl.name and not over:
                 continue
             sweep[name] = sweep_entry(name, CONFIGS[base].scaled(**over), torch, dig, peaks, local, flush)
+        # many short sequences (a training batch at 256 x 256 pixels): more sequences than resident CTAs, so sequences
+        # are not cut into segments and the forward pass is the forward sweep alone
+        sweep["many_sequences"] = sweep_entry("many_sequences", CONFIGS["C2"].scaled(name="B128_L256", B=128, grid_h=16, grid_w=16, directions=(0,), conv=False),
+                                              torch, dig, peaks, local, flush)
         sweep["multi"] = multi_direction_entry(CONFIGS["C2"], torch, dig, flush)
         sweep["next_rows"] = next_rows_entry(torch, dig, peaks, flush)
         sweep["note"] = ("one whole step of each workload per timing (its scan directions and conv), captured as a CUDA graph; "

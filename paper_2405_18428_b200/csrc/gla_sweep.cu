@@ -11,6 +11,9 @@
 //                          contribution to the state gradient
 //             seg_scan     forward over the states, backward over the state gradients, gate-gradient carry
 //             sweep_bwd    per segment in reverse: dq, dk, dv, dgate with the state gradient on chip
+// With at least as many sequences as CTAs stay resident the sequences are not cut (one segment each):
+// the forward pass is then sweep_fwd alone, started from the start state, and the backward pass runs a
+// local sweep that only stores the per-chunk states.
 // Per (sub-)chunk, with Lam the cumulative gate inside it, c = Lam_end / 2 per channel,
 //   Qc = q exp(Lam - c), Kc = k exp(c - Lam), Sc = diag(exp(c)) S_in, Dc = diag(exp(c)) D_out:
 //   P   = tril(Qc Kc^T)                         dP = tril(dO V^T)
@@ -41,6 +44,8 @@ struct SweepArgs {
     float *seg_state, *seg_gamma, *seg_dstate, *seg_carry;
     __half *seg_state16, *slot_s;
     float *slot_g;
+    const float *s_in;      // forward pass with uncut sequences: the start state ([B*H][d][d], may be null) ...
+    float *s_out;           // ... and where the final state goes (may be null)
     int *status;
     int accumulate;
     Geom g;
@@ -156,10 +161,14 @@ struct LocalSmem {
     static constexpr uint32_t tmem_cols = C::BIGM ? (BWD ? 256 : 128) : (BWD ? 64 : 32);
 };
 
-template <int D, int NT, bool BWD, int OCC>
+// SLOTS: also store, per (sub-)chunk, the zero-start state and the decay since the segment start (what the
+// backward sweep reads).  The backward flavour (BWD) always does and adds the segment's contribution to the
+// state gradient; a backward pass over uncut sequences needs only the stored states (BWD = false, SLOTS = true).
+template <int D, int NT, bool BWD, int OCC, bool SLOTS = BWD>
 __global__ void __launch_bounds__(NT, OCC)
 sweep_local(const SweepArgs a)
 {
+    static_assert(SLOTS || !BWD, "the backward flavour stores the per-chunk states");
     using C = Cfg<D>;
     using L = Lay<D, NT>;
     using SM = LocalSmem<D, NT, BWD>;
@@ -241,7 +250,7 @@ sweep_local(const SweepArgs a)
                         vc.e2c[tid] = ex2(t);
                         if (BWD) vc.aux[tid] = ex2(gcum + cv);  // decay from the segment start to the sub-chunk's centre
                     }
-                    if (BWD) {
+                    if (SLOTS) {
                         const size_t slot = ((size_t)(nsub - 1 - u) * g.B * g.H + bh) * pl.ntile + tile;
                         a.slot_g[slot * D + tid] = gcum;
                     }
@@ -250,7 +259,7 @@ sweep_local(const SweepArgs a)
                 if (!whole) __syncthreads();
                 {
                     build_tiles<D, NT, BWD, BWD>(raw, tQ, tK, tV, tG, table, vc.off, rowOff + cur * T, lo, min(hi, nrow));
-                    if (BWD) {
+                    if (SLOTS) {
                         const size_t slot = ((size_t)(nsub - 1 - u) * g.B * g.H + bh) * pl.ntile + tile;
                         write_state_slot<D, NT>(a.slot_s + slot * (D * D), sm, S, vc.ec);
                     }
@@ -474,7 +483,9 @@ sweep_fwd(const SweepArgs a)
     const int total = g.B * g.H * pl.nseg;
     TO *out = reinterpret_cast<TO *>(a.out);
 
-    // the first tile's rows are inputs of the call: their loads need not wait for the scan kernel
+    // The first tile's rows are inputs of the call: their loads need not wait for the scan kernel (whose own
+    // wait covered whatever produced them).  Uncut sequences have no kernel in front that has waited: wait first.
+    if (pl.nseg == 1) pdl_wait();
     {
         const int sid = blockIdx.x;
         if (sid < total) {
@@ -489,7 +500,8 @@ sweep_fwd(const SweepArgs a)
     for (int sid = blockIdx.x; sid < total; sid += gridDim.x) {
         const int bh = sid / pl.nseg, sg = sid - bh * pl.nseg, b = bh / g.H, h = bh - b * g.H;
         const int t0 = sg * pl.G, t1 = min(t0 + pl.G, pl.ntile);
-        load_state<D, NT>(a.seg_state + (size_t)sid * D * D, sm, S);
+        if (pl.nseg == 1) load_state<D, NT>(a.s_in ? a.s_in + (size_t)sid * D * D : nullptr, sm, S);      // uncut: no scan ran
+        else load_state<D, NT>(a.seg_state + (size_t)sid * D * D, sm, S);
         if (sid != (int)blockIdx.x) {
             if (tid < T) rowOff[cur * T + tid] = tile_row_offset(g, b, h, D, t0, tid);
             __syncthreads();
@@ -603,6 +615,7 @@ sweep_fwd(const SweepArgs a)
             }
             cur = nxt;
         }
+        if (pl.nseg == 1 && a.s_out) store_state<D, NT>(a.s_out + (size_t)sid * D * D, sm, S);
     }
 die:
     cta_teardown(ctl, SM::tmem_cols);
@@ -904,7 +917,10 @@ struct Shape<72> {
     static constexpr int NT_LOCAL_F = 640, NT_LOCAL_B = 640, NT_FWD = 640, NT_BWD = 640, OCC = 1;
 };
 
-Plan make_plan(const Geom &g, int sms, int per_sm)
+// A forward pass whose sequences are not cut (one segment each) runs the forward sweep alone, from the
+// start state: no local sweep, no scan.  Cut sequences pay for the local sweep as well, about 0.7 of a
+// forward sweep; the backward pass needs the local sweep (the per-tile states) in either case.
+Plan make_plan(const Geom &g, int sms, int per_sm, bool backward)
 {
     Plan p;
     p.ntile = (g.L + T - 1) / T;
@@ -915,7 +931,8 @@ Plan make_plan(const Geom &g, int sms, int per_sm)
     for (int G = p.ntile; G >= 1; --G) {
         const int nseg = (p.ntile + G - 1) / G;
         const long long rounds = (bh * nseg + slots - 1) / slots;
-        const long long cost = rounds * (G + 1);          // a segment costs about one tile of fill and drain
+        long long cost = rounds * (G + 1) * 10;             // a segment costs about one tile of fill and drain
+        if (!backward && nseg > 1) cost += cost * 7 / 10;
         if (best < 0 || cost < best) {
             best = cost;
             p.G = G;
@@ -973,7 +990,7 @@ dig_status run(const GlaArgs &ga)
     const int sms = device_sm_count();
     int *status = device_status_ptr();
     if (!status || sms <= 0) return DIG_ERR_CUDA;
-    const Plan pl = make_plan(g, sms, OCC_M);
+    const Plan pl = make_plan(g, sms, OCC_M, BWD);
     const SweepWs w = carve(reinterpret_cast<char *>(ga.ws), g, pl, BWD);
     const long long total = (long long)g.B * g.H * pl.nseg;
     if (total > (1ll << 30) || (long long)g.B * g.L * g.H * D >= (1ll << 31)) return DIG_ERR_UNSUPPORTED;     // 31-bit row offsets
@@ -989,8 +1006,21 @@ dig_status run(const GlaArgs &ga)
     a.plan = pl;
     const int grid_l = (int)(total < (long long)sms * OCC_L ? total : (long long)sms * OCC_L);
     const int grid_m = (int)(total < (long long)sms * OCC_M ? total : (long long)sms * OCC_M);
+    a.s_in = ga.sio.s_in;
+    a.s_out = ga.sio.s_out;
+    const bool sweep_only = !BWD && pl.nseg == 1;      // uncut sequences: the forward sweep starts from the start state itself
     dig_status st;
-    {
+    // backward pass over uncut sequences whose start-state gradient is not asked for: the segment's own
+    // contribution to the state gradient is never used, the local sweep only has to store the states
+    const bool states_only = BWD && pl.nseg == 1 && ga.sio.ds_in == nullptr;
+    if (states_only) {
+        auto kern = sweep_local<D, SH::NT_LOCAL_F, false, OCC_L, true>;
+        constexpr size_t smem = LocalSmem<D, SH::NT_LOCAL_F, false>::bytes;
+        if ((st = set_smem(kern, smem)) != DIG_OK) return st;
+        KernelTimer t(KID_SW_LOCAL, ga.stream);
+        launch_pdl(kern, dim3(grid_l), dim3(SH::NT_LOCAL_F), smem, ga.stream, a);
+        if ((st = cuda_ok(cudaGetLastError())) != DIG_OK) return st;
+    } else if (!sweep_only) {
         auto kern = sweep_local<D, NT_L, BWD, OCC_L>;
         constexpr size_t smem = LocalSmem<D, NT_L, BWD>::bytes;
         if ((st = set_smem(kern, smem)) != DIG_OK) return st;
@@ -998,7 +1028,7 @@ dig_status run(const GlaArgs &ga)
         launch_pdl(kern, dim3(grid_l), dim3(NT_L), smem, ga.stream, a);
         if ((st = cuda_ok(cudaGetLastError())) != DIG_OK) return st;
     }
-    {
+    if (!sweep_only) {
         auto kern = seg_scan<D, BWD>;
         KernelTimer t(KID_SW_SCAN, ga.stream);
         launch_pdl(kern, dim3(g.B * g.H, D / 8), dim3(64), 0, ga.stream, w.seg_state, (const float *)w.seg_gamma, w.seg_dstate,
@@ -1037,7 +1067,7 @@ size_t sweep_workspace_bytes(const Geom &g, bool backward)
 {
     int sms = device_sm_count();
     if (sms <= 0) sms = 148;
-    const Plan pl = make_plan(g, sms, sweep_per_sm(g.dk, backward));
+    const Plan pl = make_plan(g, sms, sweep_per_sm(g.dk, backward), backward);
     return carve(nullptr, g, pl, backward).bytes;
 }
 

@@ -47,6 +47,26 @@ def test_tensor_family(direction):
     print(_run(wl, direction, 1))
 
 
+@pytest.mark.parametrize("d,B,H,direction", [(64, 20, 16, 2), (72, 10, 16, 1), (64, 1, 2, 0)])
+def test_tensor_family_uncut_sequences(d, B, H, direction):
+    """More sequences than CTAs stay resident (or a single tile per sequence): the forward pass then runs
+    the forward sweep alone, which takes the start state as its entry state and writes the final state."""
+    g = (8, 24) if B > 1 else (4, 9)
+    wl = Workload("st1", B=B, H=H, grid_h=g[0], grid_w=g[1], d_k=d, d_v=d, chunk=64, dtype="bf16", backward=True,
+                  tau=(16.0, 4.0), seed=25)
+    print(_run(wl, direction, 6))
+
+
+@pytest.mark.parametrize("d,B,H,direction", [(64, 20, 16, 3), (72, 10, 16, 0)])
+def test_plain_entry_points_on_uncut_sequences(d, B, H, direction):
+    """The same regime through dig_gla_fwd / dig_gla_bwd: the backward pass then runs the local sweep that
+    only stores the per-chunk states (nothing asks for the gradient of a start state)."""
+    from parity import check_workload
+    wl = Workload("st2", B=B, H=H, grid_h=8, grid_w=24, d_k=d, d_v=d, chunk=64, dtype="bf16", backward=True,
+                  tau=(16.0, 4.0), seed=26)
+    print(check_workload(wl, direction))
+
+
 @pytest.mark.parametrize("direction", [1, 2])
 def test_mma_family(direction):
     wl = Workload("st", B=1, H=2, grid_h=9, grid_w=10, d_k=72, d_v=72, chunk=64, dtype="bf16", backward=True,
